@@ -1,0 +1,336 @@
+/*
+ * CPU oracle for the SMaLL layer definitions (arXiv 2303.04769).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what each
+ * layer computes.  It is used by the tests, by the smoke check and by the
+ * benchmark's CPU-baseline leg, and by nothing else; the CUDA library neither
+ * includes nor links it and shares no code with it.
+ *
+ * Conventions: tensors are dense NCHW float32 (the "natural" layout, before the
+ * paper's blocked layout of Section 4.4 is applied); filters are [K][C][FH][FW];
+ * every sum is carried in double and rounded to float once; bias is added in
+ * double before that rounding; ReLU follows the rounding.  Padding (which the
+ * paper leaves to "code surrounding the kernels", Section 4.2.1) is read as
+ * zero padding for the FMA layers and as "ignored positions" for pooling.
+ *
+ * Two independent statements of the arithmetic live here on purpose:
+ *   - so_conv2d / so_dwconv2d / so_pool2d / so_relu / so_fc: the per-output
+ *     definitions of Section 3.2 (classes of layers);
+ *   - so_abstract_layer: Algorithm 1 (the abstract layer loop nest) with its
+ *     blocking parameters, taken in the paper's loop order, for any
+ *     (F_H, F_W, F_C, S_H, S_W, S_C, K, G) of Section 3.1 and Table 1.
+ * The tests check each against the other, and both against brute force,
+ * library routines and closed forms.
+ *
+ * Parity unpinned: nothing (every exported routine has at least one pin in
+ * tests/test_oracle_*.py).  Accuracy of trained networks is not computed here.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define SO_EXPORT __attribute__((visibility("default")))
+
+/* ---- Section 3.1.2: output extent of a sliding window, with floor division and explicit pads.
+ * With both pads zero this is the paper's O = (I - F) / S + 1. */
+SO_EXPORT int so_out_size(int I, int F, int S, int pad_before, int pad_after) {
+    int span = I + pad_before + pad_after - F;
+    if (I < 1 || F < 1 || S < 1 || span < 0) return 0;
+    return span / S + 1;
+}
+
+/* "same" padding: O = ceil(I / S); the total pad is what the last window needs, the smaller half first. */
+SO_EXPORT void so_same_pad(int I, int F, int S, int *O, int *before, int *after) {
+    int o = (I + S - 1) / S;
+    int total = (o - 1) * S + F - I;
+    if (total < 0) total = 0;
+    *O = o;
+    *before = total / 2;
+    *after = total - total / 2;
+}
+
+/* Section 3.1.2: number of groups produced by sliding the window over channels, and O_C = K * G. */
+SO_EXPORT int so_groups(int I_C, int F_C, int S_C) { return (I_C - F_C) / S_C + 1; }
+SO_EXPORT int so_out_channels(int K, int G) { return K * G; }
+
+/* Section 5.3: float model memory = 4 bytes x (parameters + largest input/output buffer pair + model input). */
+SO_EXPORT double so_model_memory_mib(long params, long largest_in_out_pair, long model_input) {
+    return 4.0 * (double)(params + largest_in_out_pair + model_input) / 1048576.0;
+}
+
+/* ---- Section 4.4 / Figure 2: blocked layout.  Fastest to slowest: Cb channels, width, height,
+ * channel blocks; the batch is the added outermost dimension (Section 3.1.1). */
+SO_EXPORT long so_blk_index(int n, int c, int h, int w, int C, int H, int W, int Cb) {
+    long blocks = (C + Cb - 1) / Cb;
+    long blk = c / Cb, lane = c % Cb;
+    return ((((long)n * blocks + blk) * H + h) * W + w) * Cb + lane;
+}
+
+SO_EXPORT long so_blk_elems(int N, int C, int H, int W, int Cb) {
+    long blocks = (C + Cb - 1) / Cb;
+    return (long)N * blocks * Cb * H * W;
+}
+
+SO_EXPORT void so_pack(const float *nchw, float *blk, int N, int C, int H, int W, int Cb) {
+    long total = so_blk_elems(N, C, H, W, Cb);
+    for (long i = 0; i < total; ++i) blk[i] = 0.0f; /* pad lanes hold +0 */
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w)
+                    blk[so_blk_index(n, c, h, w, C, H, W, Cb)] = nchw[(((long)n * C + c) * H + h) * W + w];
+}
+
+SO_EXPORT void so_unpack(const float *blk, float *nchw, int N, int C, int H, int W, int Cb) {
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w)
+                    nchw[(((long)n * C + c) * H + h) * W + w] = blk[so_blk_index(n, c, h, w, C, H, W, Cb)];
+}
+
+static inline float so_finish(double acc, int relu) {
+    float r = (float)acc;
+    if (relu) r = r > 0.0f ? r : 0.0f;
+    return r;
+}
+
+/* ---- Full channel reduction (Section 3.2 item 4, Table 1 row 4): convolution, incl. 1x1.
+ * out[n,k,oh,ow] = bias[k] + sum_{c,x,y} in[n,c,oh*S+x-pt,ow*S+y-pl] * w[k,c,x,y]  (no filter flip);
+ * reads outside the plane are 0.  accumulate != 0 adds the previous content of out (the kernel's
+ * LOAD phase of Algorithm 2 picking up an existing partial result). */
+SO_EXPORT void so_conv2d(const float *in, const float *w, const float *bias, float *out,
+                         int N, int C, int K, int H, int W, int FH, int FW, int S,
+                         int pt, int pb, int pl, int pr, int relu, int accumulate) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k)
+            for (int oh = 0; oh < OH; ++oh)
+                for (int ow = 0; ow < OW; ++ow) {
+                    double acc = bias ? (double)bias[k] : 0.0;
+                    for (int c = 0; c < C; ++c)
+                        for (int x = 0; x < FH; ++x) {
+                            int ih = oh * S + x - pt;
+                            if (ih < 0 || ih >= H) continue;
+                            for (int y = 0; y < FW; ++y) {
+                                int iw = ow * S + y - pl;
+                                if (iw < 0 || iw >= W) continue;
+                                acc += (double)in[(((long)n * C + c) * H + ih) * W + iw] *
+                                       (double)w[(((long)k * C + c) * FH + x) * FW + y];
+                            }
+                        }
+                    long o = (((long)n * K + k) * OH + oh) * OW + ow;
+                    if (accumulate) acc += (double)out[o];
+                    out[o] = so_finish(acc, relu);
+                }
+}
+
+/* Same sums with a float accumulator, in the same loop order: only used to report a second CPU timing. */
+SO_EXPORT void so_conv2d_f32acc(const float *in, const float *w, const float *bias, float *out,
+                                int N, int C, int K, int H, int W, int FH, int FW, int S,
+                                int pt, int pb, int pl, int pr, int relu, int accumulate) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k)
+            for (int oh = 0; oh < OH; ++oh)
+                for (int ow = 0; ow < OW; ++ow) {
+                    float acc = bias ? bias[k] : 0.0f;
+                    for (int c = 0; c < C; ++c)
+                        for (int x = 0; x < FH; ++x) {
+                            int ih = oh * S + x - pt;
+                            if (ih < 0 || ih >= H) continue;
+                            for (int y = 0; y < FW; ++y) {
+                                int iw = ow * S + y - pl;
+                                if (iw < 0 || iw >= W) continue;
+                                acc += in[(((long)n * C + c) * H + ih) * W + iw] *
+                                       w[(((long)k * C + c) * FH + x) * FW + y];
+                            }
+                        }
+                    long o = (((long)n * K + k) * OH + oh) * OW + ow;
+                    if (accumulate) acc += out[o];
+                    out[o] = so_finish((double)acc, relu);
+                }
+}
+
+/* ---- Single channel reduction with weights (Section 3.2 item 2; Table 1 row 2: F_C = 1, K = 1,
+ * G = I_C): depthwise convolution, one FHxFW filter per channel, w is [C][FH][FW]. */
+SO_EXPORT void so_dwconv2d(const float *in, const float *w, const float *bias, float *out,
+                           int N, int C, int H, int W, int FH, int FW, int S,
+                           int pt, int pb, int pl, int pr, int relu) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int oh = 0; oh < OH; ++oh)
+                for (int ow = 0; ow < OW; ++ow) {
+                    double acc = bias ? (double)bias[c] : 0.0;
+                    for (int x = 0; x < FH; ++x) {
+                        int ih = oh * S + x - pt;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int y = 0; y < FW; ++y) {
+                            int iw = ow * S + y - pl;
+                            if (iw < 0 || iw >= W) continue;
+                            acc += (double)in[(((long)n * C + c) * H + ih) * W + iw] *
+                                   (double)w[((long)c * FH + x) * FW + y];
+                        }
+                    }
+                    out[(((long)n * C + c) * OH + oh) * OW + ow] = so_finish(acc, relu);
+                }
+}
+
+/* ---- Single channel reduction without weights: pooling.  mode 0 = max, 1 = average.
+ * Max: the window is scanned row by row and a later element replaces the best only when strictly
+ * greater, so the first maximum wins; idx (optional) receives ih*W+iw of the winner.  Padded
+ * positions never take part: they cannot win the max and are left out of the mean's sum and count. */
+SO_EXPORT void so_pool2d(const float *in, float *out, int32_t *idx,
+                         int N, int C, int H, int W, int FH, int FW, int S,
+                         int pt, int pb, int pl, int pr, int mode) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c) {
+            const float *plane = in + ((long)n * C + c) * H * W;
+            for (int oh = 0; oh < OH; ++oh)
+                for (int ow = 0; ow < OW; ++ow) {
+                    long o = (((long)n * C + c) * OH + oh) * OW + ow;
+                    int have = 0, best_i = -1, count = 0;
+                    float best = 0.0f;
+                    double sum = 0.0;
+                    for (int x = 0; x < FH; ++x) {
+                        int ih = oh * S + x - pt;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int y = 0; y < FW; ++y) {
+                            int iw = ow * S + y - pl;
+                            if (iw < 0 || iw >= W) continue;
+                            float v = plane[(long)ih * W + iw];
+                            if (!have || v > best) { best = v; best_i = ih * W + iw; have = 1; }
+                            sum += (double)v;
+                            ++count;
+                        }
+                    }
+                    if (mode == 0) {
+                        out[o] = have ? best : 0.0f;
+                        if (idx) idx[o] = best_i;
+                    } else {
+                        out[o] = count ? (float)(sum / (double)count) : 0.0f;
+                    }
+                }
+        }
+}
+
+/* ---- Single element reductions (Section 3.2 item 1): ReLU = Max with zero (Table 2); addition. */
+SO_EXPORT void so_relu(const float *in, float *out, long n) {
+    for (long i = 0; i < n; ++i) out[i] = in[i] > 0.0f ? in[i] : 0.0f;
+}
+
+SO_EXPORT void so_add(const float *a, const float *b, float *out, long n, int relu) {
+    for (long i = 0; i < n; ++i) out[i] = so_finish((double)a[i] + (double)b[i], relu);
+}
+
+/* ---- Full reduction (Section 3.2 item 5): the flattened input [N][J] times a J x K filter bank,
+ * stored as w[K][J] with J in (c, h, w) order. */
+SO_EXPORT void so_fc(const float *in, const float *w, const float *bias, float *out,
+                     int N, int J, int K, int relu) {
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k) {
+            double acc = bias ? (double)bias[k] : 0.0;
+            for (int j = 0; j < J; ++j) acc += (double)in[(long)n * J + j] * (double)w[(long)k * J + j];
+            out[(long)n * K + k] = so_finish(acc, relu);
+        }
+}
+
+/* ---- Algorithm 1: the abstract layer loop nest, for one image, in the paper's loop order.
+ *
+ * Section 3.1: the window F_H x F_W x F_C slides with strides S_H, S_W over the plane and S_C over
+ * channels; G = (I_C - F_C)/S_C + 1 groups, K filters per group, O_C = K*G.  Output channel g*K + k
+ * reduces input channels g*S_C .. g*S_C + F_C - 1 with filter W[g][k] (Section 3.1.3: the filter
+ * tensor is F_H x F_W x F_C x K x G; stored here as [G][K][F_C][F_H][F_W]).  No padding: this is the
+ * paper's definition as printed.
+ *
+ * Blocking (Section 4.1): g in steps of G_b, k in steps of K_b, the channel reduction in steps of
+ * F_Cb, output columns in steps of O_Wb; the innermost six loops are the kernel, which updates an
+ * O_Wb x G_b x K_b tile in three phases (Section 4.2.1): LOAD the tile, COMPUTE, STORE it back.
+ * The first F_C block starts the tile at `init` (0 for FMA layers, -inf for max pooling, 0 for ReLU);
+ * later blocks pick up the stored partial result.
+ *
+ * op 0: FMA  (tile += I * W)        op 1: MAX (tile = max(tile, I), W unused, may be NULL)
+ * The running tile is kept in double; `out` is float and receives the final values only. */
+SO_EXPORT int so_abstract_layer(const float *in, const float *w, float *out,
+                                int I_C, int I_H, int I_W,
+                                int F_H, int F_W, int F_C, int S_H, int S_W, int S_C, int K,
+                                int G_b, int K_b, int F_Cb, int O_Wb, int op, double init) {
+    if (F_C < 1 || S_C < 1 || (I_C - F_C) % S_C != 0) return -1;
+    int G = so_groups(I_C, F_C, S_C);
+    int O_H = so_out_size(I_H, F_H, S_H, 0, 0), O_W = so_out_size(I_W, F_W, S_W, 0, 0);
+    int O_C = so_out_channels(K, G);
+    if (O_H < 1 || O_W < 1 || G < 1) return -1;
+    if (G_b < 1 || K_b < 1 || F_Cb < 1 || O_Wb < 1) return -1;
+    long osz = (long)O_C * O_H * O_W;
+    double *partial = (double *)malloc(sizeof(double) * (size_t)osz); /* O between F_C blocks */
+    double *tile = (double *)malloc(sizeof(double) * (size_t)O_Wb * G_b * K_b);
+    if (!partial || !tile) { free(partial); free(tile); return -2; }
+
+    for (int g = 0; g < G; g += G_b)
+        for (int k = 0; k < K; k += K_b)
+            for (int i = 0; i < F_C; i += F_Cb)
+                for (int j = 0; j < O_H; ++j)
+                    for (int l = 0; l < O_W; l += O_Wb) {
+                        int nl = O_W - l < O_Wb ? O_W - l : O_Wb;
+                        int ng = G - g < G_b ? G - g : G_b;
+                        int nk = K - k < K_b ? K - k : K_b;
+                        int ni = F_C - i < F_Cb ? F_C - i : F_Cb;
+                        /* LOAD phase */
+                        for (int ll = 0; ll < nl; ++ll)
+                            for (int gg = 0; gg < ng; ++gg)
+                                for (int kk = 0; kk < nk; ++kk) {
+                                    long oc = (long)(g + gg) * K + (k + kk);
+                                    tile[((long)ll * G_b + gg) * K_b + kk] =
+                                        i == 0 ? init : partial[(oc * O_H + j) * O_W + (l + ll)];
+                                }
+                        /* COMPUTE phase: the kernel loops */
+                        for (int x = 0; x < F_H; ++x)
+                            for (int y = 0; y < F_W; ++y)
+                                for (int ii = 0; ii < ni; ++ii)
+                                    for (int ll = 0; ll < nl; ++ll)
+                                        for (int gg = 0; gg < ng; ++gg)
+                                            for (int kk = 0; kk < nk; ++kk) {
+                                                int c = (g + gg) * S_C + (i + ii);
+                                                int ih = j * S_H + x, iw = (l + ll) * S_W + y;
+                                                double v = (double)in[((long)c * I_H + ih) * I_W + iw];
+                                                double *t = &tile[((long)ll * G_b + gg) * K_b + kk];
+                                                if (op == 0) {
+                                                    long wi = (((((long)(g + gg) * K + (k + kk)) * F_C + (i + ii)) * F_H + x) * F_W + y);
+                                                    *t += v * (double)w[wi];
+                                                } else {
+                                                    if (v > *t) *t = v;
+                                                }
+                                            }
+                        /* STORE phase */
+                        for (int ll = 0; ll < nl; ++ll)
+                            for (int gg = 0; gg < ng; ++gg)
+                                for (int kk = 0; kk < nk; ++kk) {
+                                    long oc = (long)(g + gg) * K + (k + kk);
+                                    partial[(oc * O_H + j) * O_W + (l + ll)] = tile[((long)ll * G_b + gg) * K_b + kk];
+                                }
+                    }
+    for (long o = 0; o < osz; ++o) out[o] = (float)partial[o];
+    free(partial);
+    free(tile);
+    return 0;
+}
+
+SO_EXPORT int so_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
