@@ -1,0 +1,218 @@
+/*
+ * small.h - C ABI of a B200 (sm_100a) implementation of the SMaLL layer set
+ * (arXiv 2303.04769): one loop-nest family specialised per layer by its
+ * dimensions, every layer reading and writing the same blocked-channel layout
+ * so that no layer reformats data.
+ *
+ * GENERAL CONVENTIONS
+ *
+ * Blocked layout (paper Section 4.4, Figure 2).  An activation tensor with N
+ * images, C channels and an H x W plane is stored as
+ *     float[N][ceil(C / Cb)][H][W][Cb]          Cb = small_channel_block() = 32
+ * channels fastest, then width, height, channel block, image.  Channels C ..
+ * ceil(C/Cb)*Cb - 1 of the last block ("pad lanes") are +0.0f: small_pack writes
+ * them so and every layer keeps them so.  Input and output of every layer use
+ * this one layout (the paper's premise); only small_pack / small_unpack touch
+ * NCHW.
+ *
+ * Pointers.  Unless a parameter says "host", every pointer is a DEVICE pointer
+ * on the context's device, 16-byte aligned, to memory the CALLER owns and keeps
+ * alive until the work queued on `stream` has finished.  The library allocates
+ * no device memory in any layer call.  Input and output ranges must not overlap
+ * unless the function says so.
+ *
+ * Streams and errors.  `stream` is a cudaStream_t passed as void* (NULL = the
+ * default stream).  Calls only enqueue work.  Every function returns a
+ * small_status; argument errors are found on the host before anything is
+ * launched (nothing is enqueued when the result is not SMALL_OK).  A CUDA
+ * launch failure gives SMALL_ERR_CUDA and keeps the CUDA code for
+ * small_last_cuda_error().  Device-side pipeline waits are bounded; one that
+ * runs out records SMALL_ERR_TIMEOUT in a status word read by
+ * small_device_status().
+ *
+ * Layer parameters are the paper's (Section 3.1): input channels C (I_C),
+ * filters / output channels K, plane H x W (I_H, I_W), window FH x FW (F_H,
+ * F_W), one stride for both plane dimensions (S_H = S_W), plus explicit zero
+ * padding on the four sides, which the paper leaves to the code around its
+ * kernels (Section 4.2.1).  Output extent: O = floor((I + pad_a + pad_b - F) /
+ * stride) + 1, which is Section 3.1.2's formula when the pads are zero.
+ */
+#ifndef SMALL_H
+#define SMALL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct small_ctx small_ctx; /* opaque; one per device; not thread-safe */
+
+typedef enum {
+    SMALL_OK = 0,
+    SMALL_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, unknown flag or mode */
+    SMALL_ERR_SHAPE = 2,       /* a dimension < 1, an empty output, pad >= window, size overflow */
+    SMALL_ERR_ALIGN = 3,       /* a device pointer is not 16-byte aligned */
+    SMALL_ERR_OVERLAP = 4,     /* input and output ranges overlap where that is not allowed */
+    SMALL_ERR_WORKSPACE = 5,   /* workspace too small or a slot id out of range */
+    SMALL_ERR_UNSUPPORTED = 6, /* valid request outside what the kernels cover */
+    SMALL_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed */
+    SMALL_ERR_TIMEOUT = 8,     /* a bounded device-side wait ran out */
+    SMALL_ERR_NOT_INIT = 9     /* ctx is NULL or was shut down */
+} small_status;
+
+/* flags for the weighted layers and small_add */
+enum {
+    SMALL_RELU = 1u,       /* out = max(out, 0) after bias (Table 2: ReLU = Max), fused in the epilogue */
+    SMALL_ACCUMULATE = 2u, /* out = out_previous + result (+ bias): the LOAD phase of the paper's kernel
+                              (Algorithm 2) picking up an existing partial result; used for residual joins */
+    SMALL_MATH_FP32 = 0u << 4,   /* FP32 FMA on CUDA cores, FP32 accumulate */
+    SMALL_MATH_TF32 = 1u << 4,   /* TF32 tensor-core products, FP32 accumulate */
+    SMALL_MATH_3XTF32 = 2u << 4, /* three TF32 products per term (hi*hi + hi*lo + lo*hi), FP32 accumulate */
+    SMALL_MATH_MASK = 3u << 4
+};
+
+enum { SMALL_POOL_MAX = 0, SMALL_POOL_AVG = 1 };
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Creates the context for CUDA device `device` (makes it current, loads the driver entry point
+ * used to encode tensor maps, allocates a 256-byte device status block - the only device
+ * allocation the library ever makes).  *ctx receives the handle.  Errors: INVALID_ARG, CUDA,
+ * UNSUPPORTED (the device is not compute capability 10.x). */
+int small_init(int device, small_ctx **ctx);
+/* Frees the context.  Work still queued on any stream must have finished. */
+int small_shutdown(small_ctx *ctx);
+/* Cb, the channel block of the blocked layout (Section 4.4: a machine-specific parameter). 32 here:
+ * one 128-byte line per pixel and block, the width of a warp and of the tensor-core swizzle row. */
+int small_channel_block(void);
+/* Number of floats of a blocked tensor: N * ceil(C/Cb)*Cb * H * W; 0 if a dimension is < 1. */
+size_t small_packed_elems(int N, int C, int H, int W);
+/* floor((I + pad_before + pad_after - F) / stride) + 1, or 0 when that window does not fit (Section 3.1.2). */
+int small_out_size(int I, int F, int stride, int pad_before, int pad_after);
+const char *small_strerror(int status);
+/* Last cudaError_t / CUresult seen by this context (0 if none). */
+int small_last_cuda_error(small_ctx *ctx);
+/* Synchronises `stream`, then reads and clears the device status word: *status is SMALL_OK or
+ * SMALL_ERR_TIMEOUT (a tensor-core pipeline wait gave up; the affected outputs are undefined). */
+int small_device_status(small_ctx *ctx, int *status, void *stream);
+
+/* ---- layout (Section 4.4) ------------------------------------------------------------------ */
+
+/* NCHW float[N][C][H][W] -> blocked; pad lanes are written as +0.  Bit-exact move. */
+int small_pack(small_ctx *ctx, const float *nchw, float *blk, int N, int C, int H, int W, void *stream);
+/* blocked -> NCHW, dropping pad lanes.  Bit-exact move. */
+int small_unpack(small_ctx *ctx, const float *blk, float *nchw, int N, int C, int H, int W, void *stream);
+
+/* ---- filters: packed once, off the timed path (Section 4.4: the filter tensor has its own blocked
+ * layout).  The packed layouts are private to the library; `math` is SMALL_MATH_FP32/TF32/3XTF32 and
+ * decides which copies the packed buffer holds (FP32 always; TF32-rounded K-major tiles for the two
+ * tensor-core modes; the low-order residual tiles for 3XTF32).  A layer call may use any math mode
+ * whose copies the buffer holds, i.e. any mode <= the one it was packed for. */
+size_t small_conv_weight_elems(int C, int K, int FH, int FW, unsigned math);
+/* w_kcrs: device float[K][C][FH][FW].  w_blk: device, small_conv_weight_elems floats. */
+int small_pack_conv_weights(small_ctx *ctx, const float *w_kcrs, float *w_blk, int C, int K, int FH, int FW,
+                            unsigned math, void *stream);
+size_t small_dw_weight_elems(int C, int FH, int FW);
+/* w_crs: device float[C][FH][FW] (one filter per channel: Table 1, single channel reduction). */
+int small_pack_dw_weights(small_ctx *ctx, const float *w_crs, float *w_blk, int C, int FH, int FW, void *stream);
+size_t small_fc_weight_elems(int J, int K);
+/* w_kj: device float[K][J]. */
+int small_pack_fc_weights(small_ctx *ctx, const float *w_kj, float *w_blk, int J, int K, void *stream);
+
+/* ---- layers -------------------------------------------------------------------------------- */
+
+/* Full channel reduction (Section 3.2 item 4; Table 1: F_C = I_C, K = O_C, G = 1): standard and 1x1
+ * convolution, cross-correlation form, zero padding, with the bias / accumulate / ReLU epilogue:
+ *   out[n,k,oh,ow] = [out[n,k,oh,ow] +] bias[k] + sum_{c,x,y} in[n,c,oh*s+x-pad_t,ow*s+y-pad_l] * w[k,c,x,y]
+ * in: blocked [N][C][H][W]; out: blocked [N][K][OH][OW]; bias: K floats or NULL.
+ * flags: SMALL_RELU | SMALL_ACCUMULATE | one SMALL_MATH_*.  The tensor-core modes apply to the shapes
+ * small_conv2d_uses_tensor_cores accepts (stride 1, padded row within the kernel's tile); any other shape
+ * runs the FP32 kernel (tighter accuracy, no error).
+ * Errors: NOT_INIT, INVALID_ARG, SHAPE (dims < 1, empty output, pad >= window), ALIGN, OVERLAP,
+ * UNSUPPORTED (window so large that one input tile exceeds shared memory). */
+int small_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
+                 int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                 int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
+/* 1 if small_conv2d would run this shape on the tensor cores under a tensor-core math mode, else 0. */
+int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                                   int pad_t, int pad_b, int pad_l, int pad_r);
+
+/* Single channel reduction with weights (Section 3.2 item 2; Table 1: F_C = 1, K = 1, G = I_C):
+ * depthwise convolution, one FH x FW filter per channel, + bias[c], optional ReLU.
+ * flags: SMALL_RELU (a math mode is accepted and ignored: FP32 FMA; the layer is bandwidth-bound). */
+int small_dwconv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
+                   int N, int C, int H, int W, int FH, int FW, int stride,
+                   int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
+
+/* Single channel reduction without weights: max or average pooling (Section 3.2 item 2; Table 2).
+ * Padded positions are ignored (never the max; excluded from the mean's sum and count).
+ * Max: the window is scanned row by row and the first maximum wins; idx (NULL, or a blocked int32 tensor
+ * of the output's shape, max mode only) receives ih*W + iw of the winner.  Pad lanes: value 0, index 0. */
+int small_pool2d(small_ctx *ctx, const float *in, float *out, int32_t *idx,
+                 int N, int C, int H, int W, int FH, int FW, int stride,
+                 int pad_t, int pad_b, int pad_l, int pad_r, int mode, void *stream);
+
+/* Single element reduction (Section 3.2 item 1; Table 2: ReLU = Max): out = in > 0 ? in : +0.
+ * out may equal in (in place); any other overlap is an error. */
+int small_relu(small_ctx *ctx, const float *in, float *out, int N, int C, int H, int W, void *stream);
+
+/* Single element reduction "addition" (Section 3.2 item 1): out = a + b, then ReLU if SMALL_RELU.
+ * out may equal a or b. */
+int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N, int C, int H, int W,
+              unsigned flags, void *stream);
+
+/* Full reduction (Section 3.2 item 5; Table 1 row 5): out[n,k] = bias[k] + sum_j in[n,j] * w[k,j].
+ * in: blocked [N][J][1][1]; out: blocked [N][K][1][1].  (A full reduction over an H x W plane is
+ * small_conv2d with FH = H, FW = W, as long as that window fits the kernel's shared-memory tile.)
+ * flags: SMALL_RELU (a math mode is accepted and ignored). */
+int small_fc(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
+             int N, int J, int K, unsigned flags, void *stream);
+
+/* ---- networks (Section 5.3: layers share intermediate buffers; Section 5.4: end-to-end inference) -- */
+
+enum { SMALL_OP_CONV = 0, SMALL_OP_DWCONV = 1, SMALL_OP_POOL = 2, SMALL_OP_RELU = 3, SMALL_OP_ADD = 4, SMALL_OP_FC = 5 };
+enum { SMALL_SLOT_INPUT = -1, SMALL_SLOT_OUTPUT = -2 }; /* the caller's in_blk / out_blk */
+
+typedef struct small_layer {
+    int op;                 /* SMALL_OP_* */
+    int C, K;               /* input / output channels (K ignored for DWCONV, POOL, RELU, ADD; C = J for FC) */
+    int H, W;               /* input plane (1 x 1 for FC) */
+    int FH, FW, stride;     /* window and stride (CONV, DWCONV, POOL) */
+    int pad_t, pad_b, pad_l, pad_r;
+    unsigned flags;         /* SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_* as the op allows */
+    int pool_mode;          /* SMALL_POOL_* */
+    const float *w_blk;     /* packed filters (device) or NULL */
+    const float *bias;      /* device or NULL */
+    int src, dst;           /* slot ids >= 0, or SMALL_SLOT_INPUT / SMALL_SLOT_OUTPUT */
+    int src2;               /* second operand of ADD; ignored otherwise */
+} small_layer;
+
+/* Bytes of workspace for `layers` at batch N: slot s is as large as the largest tensor any layer reads
+ * from or writes to it, rounded up to 256 bytes; slots are laid out back to back.  0 on invalid input. */
+size_t small_net_workspace_bytes(const small_layer *layers, int n_layers, int N);
+/* Runs the layers in order on `stream`.  layers: HOST array.  in_blk: blocked network input (read by
+ * layers whose src is SMALL_SLOT_INPUT); out_blk: receives what is written to SMALL_SLOT_OUTPUT.
+ * workspace: device, 256-byte aligned.  No data is reformatted between layers.  Every layer is
+ * validated before the first launch. */
+int small_run_net(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
+                  const float *in_blk, float *out_blk, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Extra device bytes small_run_net_host needs beyond small_net_workspace_bytes: staging for the NCHW
+ * input and output and their blocked forms. */
+size_t small_net_host_staging_bytes(int N, int C, int H, int W, int outC, int outH, int outW);
+/* End-to-end convenience: in_nchw_host (HOST, float[N][C][H][W]) is copied to the device, packed, run
+ * through the layers, unpacked and copied to out_nchw_host (HOST, float[N][outC][outH][outW]).  Pinned
+ * host memory makes the copies asynchronous.  workspace: device, 256-byte aligned, at least
+ * small_net_workspace_bytes + small_net_host_staging_bytes.  Returns after enqueuing; synchronise
+ * `stream` before reading the result. */
+int small_run_net_host(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
+                       const float *in_nchw_host, int C, int H, int W,
+                       float *out_nchw_host, int outC, int outH, int outW,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SMALL_H */

@@ -1,0 +1,78 @@
+// Shared host-side declarations of the library: context, launch checks, argument validation.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+#include "small.h"
+
+#define SMALL_CB 32          // channel block of the blocked layout (floats): one 128-byte line
+#define SMALL_API extern "C" __attribute__((visibility("default")))
+
+struct small_ctx {
+    int device;
+    int last_cuda;           // last cudaError_t / CUresult seen
+    int *dev_status;         // device status word (timeouts of bounded waits)
+    void *encode_tiled;      // cuTensorMapEncodeTiled, resolved through the runtime
+    int sm_count;
+    size_t max_smem_optin;
+};
+
+namespace small {
+
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline int blocks_of(int C) { return (C + SMALL_CB - 1) / SMALL_CB; }
+static inline size_t packed_elems(int N, int C, int H, int W) {
+    if (N < 1 || C < 1 || H < 1 || W < 1) return 0;
+    return (size_t)N * blocks_of(C) * SMALL_CB * (size_t)H * W;
+}
+static inline int out_size(int I, int F, int S, int pa, int pb) {
+    if (I < 1 || F < 1 || S < 1) return 0;
+    int span = I + pa + pb - F;
+    if (span < 0) return 0;
+    return span / S + 1;
+}
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
+    uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+static inline int check_launch(small_ctx *ctx) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
+    return SMALL_OK;
+}
+
+// Geometry of one windowed layer, validated once on the host and passed to kernels by value.
+struct Geom {
+    int N, C, K, H, W, FH, FW, S, pt, pb, pl, pr, OH, OW;
+    int CB, KB;   // channel blocks of input and output
+};
+
+// Fills g and returns SMALL_OK, or the status that describes what is wrong.
+int make_geom(Geom &g, int N, int C, int K, int H, int W, int FH, int FW, int S, int pt, int pb, int pl, int pr);
+
+// ---- kernel launchers (each in its own .cu); all return a small_status ----
+int launch_pack(small_ctx *, const float *nchw, float *blk, int N, int C, int H, int W, cudaStream_t);
+int launch_unpack(small_ctx *, const float *blk, float *nchw, int N, int C, int H, int W, cudaStream_t);
+int launch_pack_conv_weights(small_ctx *, const float *w, float *wb, int C, int K, int FH, int FW, unsigned math, cudaStream_t);
+int launch_pack_dw_weights(small_ctx *, const float *w, float *wb, int C, int FH, int FW, cudaStream_t);
+int launch_pack_fc_weights(small_ctx *, const float *w, float *wb, int J, int K, cudaStream_t);
+int launch_relu(small_ctx *, const float *in, float *out, size_t n, cudaStream_t);
+int launch_add(small_ctx *, const float *a, const float *b, float *out, size_t n, bool relu, cudaStream_t);
+int launch_pool(small_ctx *, const float *in, float *out, int32_t *idx, const Geom &, int mode, cudaStream_t);
+int launch_dwconv(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
+int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, float *out, int N, int J, int K, bool relu, cudaStream_t);
+int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
+                     bool relu, bool accumulate, cudaStream_t);
+// tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32
+bool conv_tc_supported(const Geom &);
+int launch_conv_tc(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
+                   const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t);
+
+// Sizes (in floats) of the sections of a packed convolution filter buffer.
+size_t conv_w_fp32_elems(int C, int K, int FH, int FW);   // [KB][CB][FH][FW][32 ci][32 ko]
+size_t conv_w_tc_elems(int C, int K, int FH, int FW);     // [CB][FH*FW][KB*32][32 ci]
+
+}  // namespace small
