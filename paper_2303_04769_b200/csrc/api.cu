@@ -1,0 +1,282 @@
+// C ABI of the library: context, argument validation and dispatch.  Every step of a layer runs in the
+// kernels of the neighbouring .cu files; this file only checks arguments and launches.
+#include <cstdio>
+#include <cstring>
+#include <initializer_list>
+#include <new>
+
+#include "common.cuh"
+
+namespace small {
+
+int make_geom(Geom &g, int N, int C, int K, int H, int W, int FH, int FW, int S, int pt, int pb, int pl, int pr) {
+    if (N < 1 || C < 1 || K < 1 || H < 1 || W < 1 || FH < 1 || FW < 1 || S < 1) return SMALL_ERR_SHAPE;
+    if (pt < 0 || pb < 0 || pl < 0 || pr < 0) return SMALL_ERR_SHAPE;
+    if (pt >= FH || pb >= FH || pl >= FW || pr >= FW) return SMALL_ERR_SHAPE;  // a window never lies wholly in the pad
+    int OH = out_size(H, FH, S, pt, pb), OW = out_size(W, FW, S, pl, pr);
+    if (OH < 1 || OW < 1) return SMALL_ERR_SHAPE;
+    // 32-bit index arithmetic inside a plane, 64-bit across planes: keep planes and rows well inside int range
+    if ((long long)H * W > (1ll << 24) || (long long)N * blocks_of(C) > (1ll << 30) || (long long)N * blocks_of(K) > (1ll << 30))
+        return SMALL_ERR_SHAPE;
+    g = Geom{N, C, K, H, W, FH, FW, S, pt, pb, pl, pr, OH, OW, blocks_of(C), blocks_of(K)};
+    return SMALL_OK;
+}
+
+size_t conv_w_fp32_elems(int C, int K, int FH, int FW) {
+    return (size_t)blocks_of(K) * blocks_of(C) * FH * FW * SMALL_CB * SMALL_CB;
+}
+size_t conv_w_tc_elems(int C, int K, int FH, int FW) {
+    return (size_t)blocks_of(C) * FH * FW * blocks_of(K) * SMALL_CB * SMALL_CB;
+}
+
+static int check_ptrs(std::initializer_list<const void *> required, std::initializer_list<const void *> optional = {}) {
+    for (const void *p : required) {
+        if (!p) return SMALL_ERR_INVALID_ARG;
+        if (!aligned16(p)) return SMALL_ERR_ALIGN;
+    }
+    for (const void *p : optional)
+        if (p && !aligned16(p)) return SMALL_ERR_ALIGN;
+    return SMALL_OK;
+}
+
+static unsigned math_of(unsigned flags) { return flags & SMALL_MATH_MASK; }
+static bool math_valid(unsigned m) { return m == SMALL_MATH_FP32 || m == SMALL_MATH_TF32 || m == SMALL_MATH_3XTF32; }
+
+}  // namespace small
+
+using namespace small;
+
+SMALL_API int small_channel_block(void) { return SMALL_CB; }
+SMALL_API size_t small_packed_elems(int N, int C, int H, int W) { return packed_elems(N, C, H, W); }
+SMALL_API int small_out_size(int I, int F, int stride, int pa, int pb) {
+    if (pa < 0 || pb < 0) return 0;
+    return out_size(I, F, stride, pa, pb);
+}
+
+SMALL_API const char *small_strerror(int s) {
+    switch (s) {
+        case SMALL_OK: return "ok";
+        case SMALL_ERR_INVALID_ARG: return "invalid argument (null pointer, unknown flag or mode)";
+        case SMALL_ERR_SHAPE: return "invalid shape (dimension < 1, empty output, pad >= window, or too large)";
+        case SMALL_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case SMALL_ERR_OVERLAP: return "input and output ranges overlap";
+        case SMALL_ERR_WORKSPACE: return "workspace too small or slot id out of range";
+        case SMALL_ERR_UNSUPPORTED: return "request outside what the kernels cover";
+        case SMALL_ERR_CUDA: return "CUDA call failed (see small_last_cuda_error)";
+        case SMALL_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        case SMALL_ERR_NOT_INIT: return "context is null or shut down";
+        default: return "unknown status";
+    }
+}
+
+SMALL_API int small_init(int device, small_ctx **out) {
+    if (!out) return SMALL_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) return SMALL_ERR_CUDA;
+    if (device < 0 || device >= count) return SMALL_ERR_INVALID_ARG;
+    if ((e = cudaSetDevice(device)) != cudaSuccess) return SMALL_ERR_CUDA;
+    small_ctx *c = new (std::nothrow) small_ctx();
+    if (!c) return SMALL_ERR_INVALID_ARG;
+    c->device = device;
+    c->last_cuda = 0;
+    c->encode_tiled = nullptr;
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, device)) != cudaSuccess) { delete c; return SMALL_ERR_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    c->max_smem_optin = prop.sharedMemPerBlockOptin;
+    if (prop.major != 10) { delete c; return SMALL_ERR_UNSUPPORTED; }  // kernels are built for sm_100a only
+    void *block = nullptr;
+    if ((e = cudaMalloc(&block, 256)) != cudaSuccess) { delete c; return SMALL_ERR_CUDA; }
+    cudaMemset(block, 0, 256);
+    c->dev_status = static_cast<int *>(block);
+    cudaDriverEntryPointQueryResult q;
+    void *fn = nullptr;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+        cudaFree(block);
+        delete c;
+        return SMALL_ERR_CUDA;
+    }
+    c->encode_tiled = fn;
+    *out = c;
+    return SMALL_OK;
+}
+
+SMALL_API int small_shutdown(small_ctx *ctx) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    cudaSetDevice(ctx->device);
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
+    delete ctx;
+    return SMALL_OK;
+}
+
+SMALL_API int small_last_cuda_error(small_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+SMALL_API int small_device_status(small_ctx *ctx, int *status, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (!status) return SMALL_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int host = 0;
+    cudaError_t e = cudaMemcpyAsync(&host, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->dev_status, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
+    *status = host;
+    return SMALL_OK;
+}
+
+// ---- layout ----
+SMALL_API int small_pack(small_ctx *ctx, const float *nchw, float *blk, int N, int C, int H, int W, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({nchw, blk})) return s;
+    if (N < 1 || C < 1 || H < 1 || W < 1 || (long long)H * W > (1ll << 24)) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(nchw, sizeof(float) * (size_t)N * C * H * W, blk, sizeof(float) * packed_elems(N, C, H, W))) return SMALL_ERR_OVERLAP;
+    return launch_pack(ctx, nchw, blk, N, C, H, W, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_unpack(small_ctx *ctx, const float *blk, float *nchw, int N, int C, int H, int W, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({nchw, blk})) return s;
+    if (N < 1 || C < 1 || H < 1 || W < 1 || (long long)H * W > (1ll << 24)) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(nchw, sizeof(float) * (size_t)N * C * H * W, blk, sizeof(float) * packed_elems(N, C, H, W))) return SMALL_ERR_OVERLAP;
+    return launch_unpack(ctx, blk, nchw, N, C, H, W, static_cast<cudaStream_t>(stream));
+}
+
+// ---- filters ----
+SMALL_API size_t small_conv_weight_elems(int C, int K, int FH, int FW, unsigned math) {
+    if (C < 1 || K < 1 || FH < 1 || FW < 1 || !math_valid(math)) return 0;
+    size_t n = conv_w_fp32_elems(C, K, FH, FW);
+    if (math != SMALL_MATH_FP32) n += conv_w_tc_elems(C, K, FH, FW);
+    if (math == SMALL_MATH_3XTF32) n += conv_w_tc_elems(C, K, FH, FW);
+    return n;
+}
+
+SMALL_API int small_pack_conv_weights(small_ctx *ctx, const float *w, float *wb, int C, int K, int FH, int FW,
+                                      unsigned math, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (!math_valid(math)) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({w, wb})) return s;
+    if (C < 1 || K < 1 || FH < 1 || FW < 1) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(w, sizeof(float) * (size_t)K * C * FH * FW, wb, sizeof(float) * small_conv_weight_elems(C, K, FH, FW, math)))
+        return SMALL_ERR_OVERLAP;
+    return launch_pack_conv_weights(ctx, w, wb, C, K, FH, FW, math, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API size_t small_dw_weight_elems(int C, int FH, int FW) {
+    if (C < 1 || FH < 1 || FW < 1) return 0;
+    return (size_t)blocks_of(C) * FH * FW * SMALL_CB;
+}
+
+SMALL_API int small_pack_dw_weights(small_ctx *ctx, const float *w, float *wb, int C, int FH, int FW, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({w, wb})) return s;
+    if (C < 1 || FH < 1 || FW < 1) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(w, sizeof(float) * (size_t)C * FH * FW, wb, sizeof(float) * small_dw_weight_elems(C, FH, FW))) return SMALL_ERR_OVERLAP;
+    return launch_pack_dw_weights(ctx, w, wb, C, FH, FW, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API size_t small_fc_weight_elems(int J, int K) {
+    if (J < 1 || K < 1) return 0;
+    return (size_t)blocks_of(K) * blocks_of(J) * SMALL_CB * SMALL_CB;
+}
+
+SMALL_API int small_pack_fc_weights(small_ctx *ctx, const float *w, float *wb, int J, int K, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({w, wb})) return s;
+    if (J < 1 || K < 1) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(w, sizeof(float) * (size_t)K * J, wb, sizeof(float) * small_fc_weight_elems(J, K))) return SMALL_ERR_OVERLAP;
+    return launch_pack_fc_weights(ctx, w, wb, J, K, static_cast<cudaStream_t>(stream));
+}
+
+// ---- layers ----
+SMALL_API int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                                             int pt, int pb, int pl, int pr) {
+    Geom g;
+    if (make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr) != SMALL_OK) return 0;
+    return conv_tc_supported(g) ? 1 : 0;
+}
+
+SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
+                           int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                           int pt, int pb, int pl, int pr, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    unsigned math = math_of(flags);
+    if (!math_valid(math)) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, w, out}, {bias})) return s;
+    Geom g;
+    if (int s = make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr)) return s;
+    if (ranges_overlap(in, sizeof(float) * packed_elems(N, C, H, W), out, sizeof(float) * packed_elems(N, K, g.OH, g.OW)))
+        return SMALL_ERR_OVERLAP;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    bool relu = flags & SMALL_RELU, acc = flags & SMALL_ACCUMULATE;
+    if (math != SMALL_MATH_FP32 && conv_tc_supported(g)) {
+        const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);
+        const float *w_lo = w_hi + conv_w_tc_elems(C, K, FH, FW);
+        return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, relu, acc, math, st);
+    }
+    return launch_conv_fp32(ctx, in, w, bias, out, g, relu, acc, st);
+}
+
+SMALL_API int small_dwconv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
+                             int N, int C, int H, int W, int FH, int FW, int stride,
+                             int pt, int pb, int pl, int pr, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    if (!math_valid(math_of(flags))) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, w, out}, {bias})) return s;
+    Geom g;
+    if (int s = make_geom(g, N, C, C, H, W, FH, FW, stride, pt, pb, pl, pr)) return s;
+    if (ranges_overlap(in, sizeof(float) * packed_elems(N, C, H, W), out, sizeof(float) * packed_elems(N, C, g.OH, g.OW)))
+        return SMALL_ERR_OVERLAP;
+    return launch_dwconv(ctx, in, w, bias, out, g, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_pool2d(small_ctx *ctx, const float *in, float *out, int32_t *idx,
+                           int N, int C, int H, int W, int FH, int FW, int stride,
+                           int pt, int pb, int pl, int pr, int mode, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (mode != SMALL_POOL_MAX && mode != SMALL_POOL_AVG) return SMALL_ERR_INVALID_ARG;
+    if (idx && mode != SMALL_POOL_MAX) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, out}, {idx})) return s;
+    Geom g;
+    if (int s = make_geom(g, N, C, C, H, W, FH, FW, stride, pt, pb, pl, pr)) return s;
+    size_t in_b = sizeof(float) * packed_elems(N, C, H, W), out_b = sizeof(float) * packed_elems(N, C, g.OH, g.OW);
+    if (ranges_overlap(in, in_b, out, out_b)) return SMALL_ERR_OVERLAP;
+    if (idx && (ranges_overlap(in, in_b, idx, out_b) || ranges_overlap(out, out_b, idx, out_b))) return SMALL_ERR_OVERLAP;
+    return launch_pool(ctx, in, out, idx, g, mode, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_relu(small_ctx *ctx, const float *in, float *out, int N, int C, int H, int W, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({in, out})) return s;
+    size_t n = packed_elems(N, C, H, W);
+    if (n == 0) return SMALL_ERR_SHAPE;
+    if (in != out && ranges_overlap(in, n * sizeof(float), out, n * sizeof(float))) return SMALL_ERR_OVERLAP;
+    return launch_relu(ctx, in, out, n, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N, int C, int H, int W,
+                        unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~SMALL_RELU) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({a, b, out})) return s;
+    size_t n = packed_elems(N, C, H, W);
+    if (n == 0) return SMALL_ERR_SHAPE;
+    if (a != out && ranges_overlap(a, n * sizeof(float), out, n * sizeof(float))) return SMALL_ERR_OVERLAP;
+    if (b != out && ranges_overlap(b, n * sizeof(float), out, n * sizeof(float))) return SMALL_ERR_OVERLAP;
+    return launch_add(ctx, a, b, out, n, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_fc(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
+                       int N, int J, int K, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    if (!math_valid(math_of(flags))) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, w, out}, {bias})) return s;
+    if (N < 1 || J < 1 || K < 1 || (long long)N * blocks_of(J) > (1ll << 30) || (long long)N * blocks_of(K) > (1ll << 30)) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(in, sizeof(float) * packed_elems(N, J, 1, 1), out, sizeof(float) * packed_elems(N, K, 1, 1))) return SMALL_ERR_OVERLAP;
+    return launch_fc(ctx, in, w, bias, out, N, J, K, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
+}
