@@ -1,0 +1,66 @@
+// Single element reductions (paper Section 3.2 item 1): ReLU (the Max kernel against zero) and addition.
+// Bandwidth-bound: 128-bit loads and stores over the channel block, several independent loads in flight per thread.
+#include "common.cuh"
+
+namespace small {
+
+__device__ __forceinline__ float relu1(float v) { return v > 0.0f ? v : 0.0f; }   // -0 and negatives -> +0
+__device__ __forceinline__ float4 relu4(float4 v) { return make_float4(relu1(v.x), relu1(v.y), relu1(v.z), relu1(v.w)); }
+
+template <int UNROLL>
+__global__ void __launch_bounds__(256) relu_kernel(const float4 *__restrict__ in, float4 *__restrict__ out, size_t n4) {
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+    for (; i + (UNROLL - 1) * stride < n4; i += UNROLL * stride) {
+        float4 v[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) v[u] = __ldcs(in + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) __stcs(out + i + u * stride, relu4(v[u]));
+    }
+    for (; i < n4; i += stride) __stcs(out + i, relu4(__ldcs(in + i)));
+}
+
+template <int UNROLL>
+__global__ void __launch_bounds__(256) add_kernel(const float4 *__restrict__ a, const float4 *__restrict__ b,
+                                                  float4 *__restrict__ out, size_t n4, bool relu) {
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+    for (; i + (UNROLL - 1) * stride < n4; i += UNROLL * stride) {
+        float4 x[UNROLL], y[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) { x[u] = __ldcs(a + i + u * stride); y[u] = __ldcs(b + i + u * stride); }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            float4 r = make_float4(x[u].x + y[u].x, x[u].y + y[u].y, x[u].z + y[u].z, x[u].w + y[u].w);
+            __stcs(out + i + u * stride, relu ? relu4(r) : r);
+        }
+    }
+    for (; i < n4; i += stride) {
+        float4 x = __ldcs(a + i), y = __ldcs(b + i);
+        float4 r = make_float4(x.x + y.x, x.y + y.y, x.z + y.z, x.w + y.w);
+        __stcs(out + i, relu ? relu4(r) : r);
+    }
+}
+
+static int stream_grid(small_ctx *ctx, size_t n4, int unroll) {
+    size_t want = (n4 + 256ull * unroll - 1) / (256ull * unroll);
+    size_t cap = (size_t)ctx->sm_count * 8;      // 8 resident CTAs of 256 threads per SM
+    if (want < 1) want = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+int launch_relu(small_ctx *ctx, const float *in, float *out, size_t n, cudaStream_t st) {
+    size_t n4 = n / 4;   // a blocked tensor is a whole number of 32-float lines
+    relu_kernel<4><<<stream_grid(ctx, n4, 4), 256, 0, st>>>(reinterpret_cast<const float4 *>(in), reinterpret_cast<float4 *>(out), n4);
+    return check_launch(ctx);
+}
+
+int launch_add(small_ctx *ctx, const float *a, const float *b, float *out, size_t n, bool relu, cudaStream_t st) {
+    size_t n4 = n / 4;
+    add_kernel<4><<<stream_grid(ctx, n4, 4), 256, 0, st>>>(reinterpret_cast<const float4 *>(a), reinterpret_cast<const float4 *>(b),
+                                                         reinterpret_cast<float4 *>(out), n4, relu);
+    return check_launch(ctx);
+}
+
+}  // namespace small
