@@ -1,0 +1,177 @@
+// Networks: a list of layer descriptors run in order over caller-provided slots of one workspace (paper Section 5.3:
+// layers share intermediate buffers; Section 4.4: every layer reads and writes the same layout, so nothing is
+// reformatted between layers).
+#include <vector>
+
+#include "common.cuh"
+
+namespace small {
+
+struct SlotPlan {
+    std::vector<size_t> bytes;    // per slot
+    std::vector<size_t> offset;   // per slot, 256-byte aligned
+    size_t total = 0;
+};
+
+static size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+// Output shape of a layer; false if the descriptor is malformed.
+static bool layer_out_shape(const small_layer &L, int N, int &oc, int &oh, int &ow) {
+    Geom g;
+    switch (L.op) {
+        case SMALL_OP_CONV:
+            if (make_geom(g, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r)) return false;
+            oc = L.K; oh = g.OH; ow = g.OW; return true;
+        case SMALL_OP_DWCONV:
+        case SMALL_OP_POOL:
+            if (make_geom(g, N, L.C, L.C, L.H, L.W, L.FH, L.FW, L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r)) return false;
+            oc = L.C; oh = g.OH; ow = g.OW; return true;
+        case SMALL_OP_RELU:
+        case SMALL_OP_ADD:
+            if (L.C < 1 || L.H < 1 || L.W < 1) return false;
+            oc = L.C; oh = L.H; ow = L.W; return true;
+        case SMALL_OP_FC:
+            if (L.C < 1 || L.K < 1 || L.H != 1 || L.W != 1) return false;
+            oc = L.K; oh = 1; ow = 1; return true;
+        default: return false;
+    }
+}
+
+static bool plan_slots(const small_layer *layers, int n_layers, int N, SlotPlan &plan) {
+    if (!layers || n_layers < 1 || N < 1) return false;
+    auto need = [&](int slot, size_t bytes) {
+        if (slot < 0) return slot == SMALL_SLOT_INPUT || slot == SMALL_SLOT_OUTPUT;
+        if (slot > 4096) return false;
+        if ((size_t)slot >= plan.bytes.size()) plan.bytes.resize(slot + 1, 0);
+        if (plan.bytes[slot] < bytes) plan.bytes[slot] = bytes;
+        return true;
+    };
+    for (int i = 0; i < n_layers; ++i) {
+        const small_layer &L = layers[i];
+        int oc, oh, ow;
+        if (!layer_out_shape(L, N, oc, oh, ow)) return false;
+        size_t in_b = sizeof(float) * packed_elems(N, L.C, L.H, L.W), out_b = sizeof(float) * packed_elems(N, oc, oh, ow);
+        if (!need(L.src, in_b) || !need(L.dst, out_b)) return false;
+        if (L.op == SMALL_OP_ADD && !need(L.src2, in_b)) return false;
+        if (L.dst == SMALL_SLOT_INPUT) return false;
+    }
+    plan.offset.resize(plan.bytes.size());
+    size_t off = 0;
+    for (size_t s = 0; s < plan.bytes.size(); ++s) { plan.offset[s] = off; off += round256(plan.bytes[s]); }
+    plan.total = off;
+    return true;
+}
+
+}  // namespace small
+
+using namespace small;
+
+SMALL_API size_t small_net_workspace_bytes(const small_layer *layers, int n_layers, int N) {
+    SlotPlan plan;
+    if (!plan_slots(layers, n_layers, N, plan)) return 0;
+    return plan.total;
+}
+
+SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
+                            const float *in_blk, float *out_blk, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (!layers || !in_blk || !out_blk) return SMALL_ERR_INVALID_ARG;
+    if (!aligned16(in_blk) || !aligned16(out_blk) || (workspace && ((uintptr_t)workspace & 255u))) return SMALL_ERR_ALIGN;
+    SlotPlan plan;
+    if (!plan_slots(layers, n_layers, N, plan)) return SMALL_ERR_SHAPE;
+    if (plan.total > workspace_bytes || (plan.total && !workspace)) return SMALL_ERR_WORKSPACE;
+    char *base = static_cast<char *>(workspace);
+    auto rd = [&](int slot) -> const float * {
+        if (slot == SMALL_SLOT_INPUT) return in_blk;
+        if (slot == SMALL_SLOT_OUTPUT) return out_blk;
+        return reinterpret_cast<const float *>(base + plan.offset[slot]);
+    };
+    auto wr = [&](int slot) -> float * {
+        if (slot == SMALL_SLOT_OUTPUT) return out_blk;
+        return reinterpret_cast<float *>(base + plan.offset[slot]);
+    };
+    // validate every layer before the first launch: weights present where needed, flags known
+    for (int i = 0; i < n_layers; ++i) {
+        const small_layer &L = layers[i];
+        bool weighted = L.op == SMALL_OP_CONV || L.op == SMALL_OP_DWCONV || L.op == SMALL_OP_FC;
+        if (weighted && !L.w_blk) return SMALL_ERR_INVALID_ARG;
+        if (weighted && (!aligned16(L.w_blk) || (L.bias && !aligned16(L.bias)))) return SMALL_ERR_ALIGN;
+        unsigned allowed = L.op == SMALL_OP_CONV ? (SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_MASK)
+                         : (L.op == SMALL_OP_DWCONV || L.op == SMALL_OP_FC) ? (SMALL_RELU | SMALL_MATH_MASK)
+                         : L.op == SMALL_OP_ADD ? SMALL_RELU : 0u;
+        if (L.flags & ~allowed) return SMALL_ERR_INVALID_ARG;
+        if ((L.flags & SMALL_MATH_MASK) == SMALL_MATH_MASK) return SMALL_ERR_INVALID_ARG;
+        if (L.op == SMALL_OP_POOL && L.pool_mode != SMALL_POOL_MAX && L.pool_mode != SMALL_POOL_AVG) return SMALL_ERR_INVALID_ARG;
+        if (L.src == L.dst && L.op != SMALL_OP_RELU && L.op != SMALL_OP_ADD) return SMALL_ERR_OVERLAP;
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        const small_layer &L = layers[i];
+        int s = SMALL_OK;
+        switch (L.op) {
+            case SMALL_OP_CONV:
+                s = small_conv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
+                                 L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
+                break;
+            case SMALL_OP_DWCONV:
+                s = small_dwconv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.H, L.W, L.FH, L.FW, L.stride,
+                                   L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
+                break;
+            case SMALL_OP_POOL:
+                s = small_pool2d(ctx, rd(L.src), wr(L.dst), nullptr, N, L.C, L.H, L.W, L.FH, L.FW, L.stride,
+                                 L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.pool_mode, stream);
+                break;
+            case SMALL_OP_RELU:
+                s = small_relu(ctx, rd(L.src), wr(L.dst), N, L.C, L.H, L.W, stream);
+                break;
+            case SMALL_OP_ADD:
+                s = small_add(ctx, rd(L.src), rd(L.src2), wr(L.dst), N, L.C, L.H, L.W, L.flags, stream);
+                break;
+            case SMALL_OP_FC:
+                s = small_fc(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.flags, stream);
+                break;
+        }
+        if (s != SMALL_OK) return s;
+    }
+    return SMALL_OK;
+}
+
+SMALL_API size_t small_net_host_staging_bytes(int N, int C, int H, int W, int outC, int outH, int outW) {
+    if (N < 1 || C < 1 || H < 1 || W < 1 || outC < 1 || outH < 1 || outW < 1) return 0;
+    return round256(sizeof(float) * (size_t)N * C * H * W) + round256(sizeof(float) * packed_elems(N, C, H, W)) +
+           round256(sizeof(float) * packed_elems(N, outC, outH, outW)) + round256(sizeof(float) * (size_t)N * outC * outH * outW);
+}
+
+SMALL_API int small_run_net_host(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
+                                 const float *in_host, int C, int H, int W,
+                                 float *out_host, int outC, int outH, int outW,
+                                 void *workspace, size_t workspace_bytes, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (!layers || !in_host || !out_host || !workspace) return SMALL_ERR_INVALID_ARG;
+    if ((uintptr_t)workspace & 255u) return SMALL_ERR_ALIGN;
+    {   // the layer list must be well formed even when it needs no slot
+        SlotPlan plan;
+        if (!plan_slots(layers, n_layers, N, plan)) return SMALL_ERR_SHAPE;
+    }
+    size_t net_b = small_net_workspace_bytes(layers, n_layers, N);
+    size_t stage_b = small_net_host_staging_bytes(N, C, H, W, outC, outH, outW);
+    if (stage_b == 0) return SMALL_ERR_SHAPE;
+    if (net_b + stage_b > workspace_bytes) return SMALL_ERR_WORKSPACE;
+    // the last layer must produce the declared output shape
+    int oc, oh, ow;
+    if (!layer_out_shape(layers[n_layers - 1], N, oc, oh, ow) || oc != outC || oh != outH || ow != outW) return SMALL_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *p = static_cast<char *>(workspace) + net_b;
+    size_t in_nchw_b = sizeof(float) * (size_t)N * C * H * W, out_nchw_b = sizeof(float) * (size_t)N * outC * outH * outW;
+    float *d_in_nchw = reinterpret_cast<float *>(p); p += round256(in_nchw_b);
+    float *d_in_blk = reinterpret_cast<float *>(p); p += round256(sizeof(float) * packed_elems(N, C, H, W));
+    float *d_out_blk = reinterpret_cast<float *>(p); p += round256(sizeof(float) * packed_elems(N, outC, outH, outW));
+    float *d_out_nchw = reinterpret_cast<float *>(p);
+    cudaError_t e = cudaMemcpyAsync(d_in_nchw, in_host, in_nchw_b, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
+    if (int s = small_pack(ctx, d_in_nchw, d_in_blk, N, C, H, W, stream)) return s;
+    if (int s = small_run_net(ctx, layers, n_layers, N, d_in_blk, d_out_blk, workspace, net_b, stream)) return s;
+    if (int s = small_unpack(ctx, d_out_blk, d_out_nchw, N, outC, outH, outW, stream)) return s;
+    e = cudaMemcpyAsync(out_host, d_out_nchw, out_nchw_b, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
+    return SMALL_OK;
+}

@@ -1,0 +1,135 @@
+"""Turns a layer list (dicts with op / src / dst / C / K / FH / FW / stride / pad / relu / accumulate / pool) into
+the small_layer descriptors of small_run_net: packs the filters once through the library, assigns named tensors
+to workspace slots and allocates the workspace with torch.  Host-side bookkeeping only."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+def assign_slots(layers):
+    """Greedy slot reuse by liveness: a tensor's slot is free again after its last reader; a layer never writes
+    the slot it reads (only accumulate updates its destination in place).  'in' / 'out' are the caller's."""
+    last_use = {}
+    for i, L in enumerate(layers):
+        last_use[L["src"]] = i
+        if L.get("accumulate"):
+            last_use[L["dst"]] = i
+    slot_of, free, n_slots = {"in": B.SLOT_INPUT, "out": B.SLOT_OUTPUT}, [], 0
+    for i, L in enumerate(layers):
+        dst = L["dst"]
+        if dst not in slot_of:
+            if free:
+                slot_of[dst] = free.pop(0)
+            else:
+                slot_of[dst] = n_slots
+                n_slots += 1
+        name = L["src"]
+        if last_use.get(name) == i and slot_of.get(name, -1) >= 0 and name != dst:
+            free.append(slot_of[name])
+    return slot_of, n_slots
+
+
+class Net:
+    """A network resident on the device: packed filters, descriptors and workspace."""
+
+    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda"):
+        self.ctx = ctx
+        self.N = net["batch"] if batch is None else batch
+        self.in_shape = tuple(net["input"])
+        self.math = B.MATH[math]
+        self.keep = []            # device tensors the descriptors point into
+        slot_of, _ = assign_slots(net["layers"])
+        self.slot_of = slot_of
+        dims = {"in": self.in_shape}
+        descs = []
+        self.layer_rows = []
+        for L, (w, b) in zip(net["layers"], params):
+            c, h, wd = dims[L["src"]]
+            fh, fw = L["FH"], L["FW"]
+            if L["op"] == "pool" and fh == 0:
+                fh, fw = h, wd
+            pt, pb, pl, pr = L["pad"]
+            d = B.small_layer()
+            d.C, d.K, d.H, d.W, d.FH, d.FW, d.stride = L["C"], L["K"], h, wd, fh, fw, L["stride"]
+            d.pad_t, d.pad_b, d.pad_l, d.pad_r = pt, pb, pl, pr
+            d.src, d.dst, d.src2 = slot_of[L["src"]], slot_of[L["dst"]], 0
+            flags = (B.RELU if L["relu"] else 0) | (B.ACCUMULATE if L.get("accumulate") else 0)
+            wt = None if w is None else torch.from_numpy(w).to(device)
+            bt = None if b is None else torch.from_numpy(b).to(device)
+            oh, ow = B.small_out_size(h, fh, L["stride"], pt, pb), B.small_out_size(wd, fw, L["stride"], pl, pr)
+            if L["op"] == "conv":
+                d.op = B.OP_CONV
+                flags |= self.math
+                wb = torch.empty(B.small_conv_weight_elems(L["C"], L["K"], fh, fw, self.math), device=device)
+                B.small_pack_conv_weights(ctx, wt, wb, L["C"], L["K"], fh, fw, self.math)
+            elif L["op"] == "dwconv":
+                d.op = B.OP_DWCONV
+                wb = torch.empty(B.small_dw_weight_elems(L["C"], fh, fw), device=device)
+                B.small_pack_dw_weights(ctx, wt, wb, L["C"], fh, fw)
+            elif L["op"] == "pool":
+                d.op = B.OP_POOL
+                d.pool_mode = B.POOL_MAX if L["pool"] == "max" else B.POOL_AVG
+                wb = None
+            elif L["op"] == "fc":
+                d.op = B.OP_FC
+                wb = torch.empty(B.small_fc_weight_elems(L["C"], L["K"]), device=device)
+                B.small_pack_fc_weights(ctx, wt, wb, L["C"], L["K"])
+                oh = ow = 1
+            else:
+                raise ValueError(L["op"])
+            d.flags = flags
+            d.w_blk = None if wb is None else wb.data_ptr()
+            d.bias = None if bt is None else bt.data_ptr()
+            self.keep += [wb, bt, wt]
+            dims[L["dst"]] = (L["K"], oh, ow)
+            self.layer_rows.append(dict(name=L["name"], op=L["op"], C=L["C"], K=L["K"], H=h, W=wd, FH=fh, FW=fw,
+                                        stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=L["dst"]))
+            descs.append(d)
+        torch.cuda.synchronize()
+        self.dims = dims
+        self.out_shape = dims["out"]
+        self.layers = (B.small_layer * len(descs))(*descs)
+        self.ws_bytes = B.small_net_workspace_bytes(self.layers, self.N)
+        c, h, w = self.in_shape
+        oc, oh, ow = self.out_shape
+        self.stage_bytes = B.small_net_host_staging_bytes(self.N, c, h, w, oc, oh, ow)
+        self.workspace = torch.empty(self.ws_bytes + self.stage_bytes + 256, dtype=torch.uint8, device=device)
+        assert self.workspace.data_ptr() % 256 == 0
+        self.out_blk = torch.empty(B.small_packed_elems(self.N, oc, oh, ow), device=device)
+
+    def run(self, in_blk, out_blk=None, stream=None, n_layers=None):
+        """Runs all layers (or the first n_layers, to inspect an intermediate)."""
+        out_blk = self.out_blk if out_blk is None else out_blk
+        layers = self.layers if n_layers is None else (B.small_layer * n_layers)(*self.layers[:n_layers])
+        B.small_run_net(self.ctx, layers, self.N, in_blk, out_blk, self.workspace, self.ws_bytes, stream)
+        return out_blk
+
+    def run_host(self, in_host, out_host, stream=None):
+        c, h, w = self.in_shape
+        oc, oh, ow = self.out_shape
+        B.small_run_net_host(self.ctx, self.layers, self.N, in_host, c, h, w, out_host, oc, oh, ow,
+                             self.workspace, self.ws_bytes + self.stage_bytes, stream)
+
+    def slot_offsets(self):
+        """Byte offset of every slot, by the library's rule: sizes rounded up to 256 bytes, back to back."""
+        sizes = {}
+        for L, row in zip(self.layers, self.layer_rows):
+            if L.src >= 0:
+                sizes[L.src] = max(sizes.get(L.src, 0), 4 * B.small_packed_elems(self.N, L.C, L.H, L.W))
+            if L.dst >= 0:
+                sizes[L.dst] = max(sizes.get(L.dst, 0), 4 * B.small_packed_elems(self.N, row["K"], row["OH"], row["OW"]))
+        offs, off = {}, 0
+        for s in range(max(sizes) + 1 if sizes else 0):
+            offs[s] = off
+            off += ((sizes.get(s, 0) + 255) // 256) * 256
+        return offs
+
+    def slot_tensor(self, name):
+        """View of a named intermediate inside the workspace (valid right after the layer that wrote it)."""
+        slot = self.slot_of[name]
+        c, h, w = self.dims[name]
+        n = B.small_packed_elems(self.N, c, h, w)
+        off = self.slot_offsets()[slot]
+        return self.workspace[off:off + 4 * n].view(torch.float32)
