@@ -1,0 +1,432 @@
+"""Benchmark of the SMaLL layer set on B200.
+
+python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--math fp32|tf32|3xtf32] [--no-sweep]
+
+One step = one pass of the 8-layer residual CNN (batch 256 per GPU) through small_run_net, inputs resident in HBM.
+The JSON line also carries the end-to-end figure from host buffers (small_run_net_host), the per-kernel roofline
+of the dominant kernel, the GPU-scale layer sweep (GFLOP/s and fraction of each layer's roofline) and the CPU
+oracle timed on the host cores.  `--impl reference` times the CPU oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from synth import configs
+
+WORKLOAD = "residual_cnn"          # the 8-layer residual CNN, batch 256
+METRIC, UNIT = "inferences_per_sec", "inferences/s"
+FLUSH_BYTES = 256 << 20            # larger than the 126 MB L2
+TOL = {"fp32": 1e-5, "tf32": 2e-3, "3xtf32": 1e-5}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                    sm_max_mhz=p.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
+
+
+def mode_peak_tflops(mode, peaks, sm_count=148):
+    """Peak of the arithmetic a convolution runs in: TF32 tensor = half the measured BF16 burst (nominal ratio);
+    3xTF32 = a third of that; FP32 = SMs x 128 lanes x 2 x max SM clock."""
+    if mode == "tf32":
+        return peaks["bf16_burst"] * 0.5
+    if mode == "3xtf32":
+        return peaks["bf16_burst"] * 0.5 / 3.0
+    return sm_count * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+
+
+def layer_work(row, N, accumulate=False):
+    """Algorithmic FLOPs and bytes of one layer from its logical dimensions (each tensor moved once, 4-byte floats)."""
+    C, K, H, W, FH, FW, OH, OW = (row[k] for k in ("C", "K", "H", "W", "FH", "FW", "OH", "OW"))
+    if row["op"] == "conv":
+        fl = 2.0 * N * OH * OW * K * C * FH * FW
+        by = 4.0 * (N * C * H * W + N * K * OH * OW * (2 if accumulate else 1) + K * C * FH * FW + K)
+    elif row["op"] == "dwconv":
+        fl = 2.0 * N * OH * OW * C * FH * FW
+        by = 4.0 * (N * C * (H * W + OH * OW) + C * FH * FW + C)
+    elif row["op"] == "pool":
+        fl = 1.0 * N * C * OH * OW * FH * FW
+        by = 4.0 * N * C * (H * W + OH * OW)
+    elif row["op"] == "fc":
+        fl = 2.0 * N * C * K
+        by = 4.0 * (N * C + N * K + C * K + K)
+    else:
+        fl, by = 0.0, 8.0 * N * C * H * W
+    return fl, by
+
+
+class ClockSampler:
+    """nvidia-smi sampled every 100 ms while the timed region runs (reading only; nothing is set)."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                mhz.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(mhz)}
+
+
+def dist_env(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def max_over_ranks(value, world, device=None):
+    """The slowest rank's time: all-reduce MAX over the job (NCCL on GPUs, gloo in the CPU tests)."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value, world, device=None):
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def whole_job_throughput(units_local, ms_local, world, device=None):
+    """Units all ranks processed / the slowest rank's time.  Images are independent, so ranks share nothing."""
+    units = sum_over_ranks(units_local, world, device)
+    ms = max_over_ranks(ms_local, world, device)
+    return units / (ms * 1e-3), ms
+
+
+# ------------------------------------------------------------------------------------------- CPU oracle legs
+def time_oracle_net(batch_cap, target_s=12.0):
+    """The oracle as it stands on the host cores: a bounded sample of the workload's batch."""
+    import oracle
+    from oracle import nets
+    net = configs.NETWORKS[WORKLOAD]()
+    params = configs.make_params(net)
+    probe = 8
+    x = configs.make_input(net, probe)
+    t0 = time.perf_counter()
+    nets.run_net(net, params, x)
+    dt = time.perf_counter() - t0
+    n = int(max(probe, min(batch_cap, probe * target_s / max(dt, 1e-6))))
+    x = configs.make_input(net, n)
+    t0 = time.perf_counter()
+    nets.run_net(net, params, x)
+    dt = time.perf_counter() - t0
+    return n / dt, n, dt, oracle.num_threads()
+
+
+def reference_arm(args):
+    rank, world, _ = dist_env(args.gpus)
+    if rank != 0:
+        return
+    net = configs.NETWORKS[WORKLOAD]()
+    times, n_used, cores = [], 0, 0
+    for i in range(args.warmup + args.steps):
+        ips, n_used, dt, cores = time_oracle_net(net["batch"], target_s=6.0)
+        if i >= args.warmup:
+            times.append(n_used / ips)
+    ms = 1e3 * sum(times) / len(times)
+    value = n_used / (ms * 1e-3)
+    sample = f"{n_used} of {net['batch']} images per step, double accumulation, OpenMP"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64 accumulate over f32 data", "data": "synthetic",
+            "config": {"workload": f"{WORKLOAD}: 8-layer residual CNN, 3x32x32 input, batch {net['batch']}", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------- GPU legs
+def gpu_main(args):
+    import torch
+    from paper_2303_04769_b200 import binding as B
+    from paper_2303_04769_b200 import build as lib_build
+    from paper_2303_04769_b200.net import Net
+
+    rank, world, local = dist_env(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        lib_build.build()
+    if world > 1:
+        dist.barrier()
+    ctx = B.small_init(local)
+    peaks = load_peaks()
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+
+    net = configs.NETWORKS[WORKLOAD]()
+    N = net["batch"]
+    params = configs.make_params(net)
+    gnet = Net(ctx, net, params, math=args.math, device=dev)
+    c, h, w = gnet.in_shape
+    oc, oh, ow = gnet.out_shape
+    # rotating input sets, seeded and distinct per rank and slot
+    R = 4
+    host_in = [torch.from_numpy(configs.make_input(net, N, seed=20230304 + 17 * rank + r)).pin_memory() for r in range(R)]
+    in_blk = []
+    for r in range(R):
+        blk = torch.empty(B.small_packed_elems(N, c, h, w), device=dev)
+        B.small_pack(ctx, host_in[r].to(dev), blk, N, c, h, w)
+        in_blk.append(blk)
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    host_out = torch.empty((N, oc, oh, ow)).pin_memory()
+    torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for i in range(warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        evs = []
+        for i in range(steps):
+            flush.zero_()                      # evict L2 between steps
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(i)
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in evs) / steps
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms_dev = timed(lambda i: gnet.run(in_blk[i % R]), args.steps, args.warmup)
+    ms_e2e = timed(lambda i: gnet.run_host(host_in[i % R], host_out), args.steps, args.warmup)
+    clocks = sampler.stop() if sampler else None
+    value, ms = whole_job_throughput(N, ms_dev, world, dev)
+    e2e_value, _ = whole_job_throughput(N, ms_e2e, world, dev)
+    status = B.small_device_status(ctx)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- per-kernel timing of the same network, one launch at a time on the same stream
+    def time_launch(fn, reps=20, warm=3):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return min(ts), statistics.median(ts)
+
+    gnet.run(in_blk[0])
+    layer_table = []
+    by_kernel = {}
+    for i, (row, L) in enumerate(zip(gnet.layer_rows, net["layers"])):
+        # accumulate layers update their destination in place; values drift over repetitions but the work does not
+        tmin, tmed = time_launch(lambda i=i: gnet.run_layer(i, in_blk[0]))
+        fl, by = layer_work(row, N, L.get("accumulate", False))
+        kern = row["op"]
+        if row["op"] == "conv":
+            tc = args.math != "fp32" and B.small_conv2d_uses_tensor_cores(N, row["C"], row["K"], row["H"], row["W"], row["FH"], row["FW"],
+                                                                           row["stride"], row["pad"])
+            kern = f"conv_{args.math}_tensor" if tc else "conv_fp32_cuda_core"
+        layer_table.append({"layer": row["name"], "kernel": kern, "us": round(tmed * 1e3, 2), "gflops": round(fl / tmed / 1e6, 1),
+                            "gbs": round(by / tmed / 1e6, 1)})
+        k = by_kernel.setdefault(kern, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
+        k["ms"] += tmed; k["flops"] += fl; k["bytes"] += by; k["launches"] += 1
+    dom_name, dom = max(by_kernel.items(), key=lambda kv: kv[1]["ms"])
+    if dom_name.startswith("conv"):
+        mode = "fp32" if dom_name.endswith("cuda_core") else args.math
+        peak = mode_peak_tflops(mode, peaks, sm_count)
+        ach = dom["flops"] / (dom["ms"] * 1e-3) / 1e12
+        roofline = {"bound": "alu" if mode == "fp32" else "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                    "frac": ach / peak, "traffic": None, "kernel": dom_name, "launches_per_step": dom["launches"],
+                    "peak_source": f"{peaks['source']}: " + ("SMs x 128 x 2 x max SM clock" if mode == "fp32" else "BF16 burst x 0.5 (TF32)" + (" / 3" if mode == "3xtf32" else ""))}
+    else:
+        ach = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                    "traffic": None, "kernel": dom_name, "launches_per_step": dom["launches"], "peak_source": peaks["source"]}
+
+    sweep = None if (args.no_sweep or world > 1) else run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch)
+
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        ips, n_used, dt, cores = time_oracle_net(N)
+        cpu = {"value": ips, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{n_used} of {N} images, one pass, {dt:.1f} s, double accumulation, OpenMP"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": {"fp32": "f32", "tf32": "tf32 products, f32 accumulate", "3xtf32": "3xtf32 products, f32 accumulate"}[args.math],
+            "data": "synthetic",
+            "config": {"workload": f"{WORKLOAD}: 8-layer residual CNN, 3x32x32 input, batch {N} per GPU (configs[1])",
+                       "math": args.math, "tolerance_rel_l2": TOL[args.math], "l2": "flushed between steps (256 MB write)",
+                       "inputs": f"{R} rotating seeded input sets", "parallelism": f"batch shards x{world}, no collective"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * N * c * h * w, "d2h_bytes_per_step": 4 * N * oc * oh * ow,
+                    "ms_per_step": ms_e2e},
+            "gpu_launches": len(gnet.layer_rows) * args.steps,
+            "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu, "device_status": status,
+            "kernels": {k: {"launches_per_step": v["launches"], "ms": round(v["ms"], 4),
+                            "share": round(v["ms"] / sum(x["ms"] for x in by_kernel.values()), 3)} for k, v in by_kernel.items()},
+            "layers": layer_table, "sweep": sweep}
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    B.small_shutdown(ctx)
+
+
+def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
+    """GPU-scale layer sweep, batch 128: each layer timed alone over rotating buffer sets that together exceed L2;
+    GFLOP/s, GB/s and the fraction of the layer's roofline = max(FLOPs / peak of its math mode, bytes / HBM)."""
+    import synth
+    N = configs.SWEEP_BATCH
+    rows = []
+    for C, HW in configs.SWEEP_SIZES:
+        elems = B.small_packed_elems(N, C, HW, HW)
+        sets = max(2, min(6, int((1 << 30) // (8 * elems)) or 2))   # in + out per set, about 1 GB in total
+        host = synth.uniform((N, C, HW, HW), -1.0, 1.0, 500 + C)
+        nchw = torch.from_numpy(host).to(dev)
+        ins, outs = [], []
+        for s in range(sets):
+            blk = torch.empty(elems, device=dev)
+            B.small_pack(ctx, nchw, blk, N, C, HW, HW)
+            ins.append(blk)
+            outs.append(torch.empty(elems, device=dev))
+        del nchw
+        bias = torch.from_numpy(synth.uniform((C,), -1.0, 1.0, 600 + C)).to(dev)
+        state = {"i": 0}
+
+        def rot():
+            state["i"] = (state["i"] + 1) % sets
+            return ins[state["i"]], outs[state["i"]]
+
+        def record(kind, mode, fl, by, tmin, tmed, bound_mode):
+            t_roof = max(fl / (mode_peak_tflops(bound_mode, peaks, sm_count) * 1e12) if fl and bound_mode else 0.0, by / (peaks["hbm_gbs"] * 1e9))
+            rows.append({"layer": kind, "C": C, "HW": HW, "mode": mode, "us_min": round(tmin * 1e3, 2), "us_med": round(tmed * 1e3, 2),
+                         "gflops": round(fl / tmed / 1e6, 1), "gbs": round(by / tmed / 1e6, 1),
+                         "roofline_us": round(t_roof * 1e6, 2), "frac": round(t_roof / (tmed * 1e-3), 4)})
+
+        for F, pad, kind in ((3, (1, 1, 1, 1), "conv3x3"), (1, (0, 0, 0, 0), "conv1x1")):
+            w = torch.from_numpy(synth.uniform((C, C, F, F), -1.0, 1.0, 700 + C + F)).to(dev)
+            wb = torch.empty(B.small_conv_weight_elems(C, C, F, F, B.MATH_3XTF32), device=dev)
+            B.small_pack_conv_weights(ctx, w, wb, C, C, F, F, B.MATH_3XTF32)
+            fl = 2.0 * N * HW * HW * C * C * F * F
+            by = 4.0 * (2 * N * C * HW * HW + C * C * F * F + C)
+            uses_tc = B.small_conv2d_uses_tensor_cores(N, C, C, HW, HW, F, F, 1, pad)
+            for mode in ("fp32", "tf32", "3xtf32"):
+                if mode != "fp32" and not uses_tc:
+                    continue
+                def call(mode=mode):
+                    a, o = rot()
+                    B.small_conv2d(ctx, a, wb, bias, o, N, C, C, HW, HW, F, F, 1, pad, B.RELU | B.MATH[mode])
+                reps = 5 if mode == "fp32" and F == 3 else 20
+                tmin, tmed = time_launch(call, reps=reps, warm=2)
+                record(kind, mode, fl, by, tmin, tmed, mode)
+            del w, wb
+        wdw = torch.from_numpy(synth.uniform((C, 3, 3), -1.0, 1.0, 800 + C)).to(dev)
+        wdb = torch.empty(B.small_dw_weight_elems(C, 3, 3), device=dev)
+        B.small_pack_dw_weights(ctx, wdw, wdb, C, 3, 3)
+
+        def dw():
+            a, o = rot()
+            B.small_dwconv2d(ctx, a, wdb, bias, o, N, C, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU)
+        tmin, tmed = time_launch(dw)
+        record("dw3x3", "fp32", 2.0 * N * HW * HW * C * 9, 4.0 * (2 * N * C * HW * HW + 10 * C), tmin, tmed, None)
+        OHW = (HW - 2) // 2 + 1
+
+        def mp():
+            a, o = rot()
+            B.small_pool2d(ctx, a, o, None, N, C, HW, HW, 2, 2, 2, (0, 0, 0, 0), B.POOL_MAX)
+        tmin, tmed = time_launch(mp)
+        record("maxpool2x2", "fp32", 0.0, 4.0 * N * C * (HW * HW + OHW * OHW), tmin, tmed, None)
+
+        def rl():
+            a, o = rot()
+            B.small_relu(ctx, a, o, N, C, HW, HW)
+        tmin, tmed = time_launch(rl)
+        record("relu", "fp32", 0.0, 8.0 * N * C * HW * HW, tmin, tmed, None)
+        del ins, outs
+        torch.cuda.empty_cache()
+    return {"batch": N, "buffers": "rotating input/output sets of about 1 GB per size (larger than L2)", "rows": rows}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--math", default="fp32", choices=["fp32", "tf32", "3xtf32"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        gpu_main(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -112,6 +112,30 @@ class Net:
         B.small_run_net_host(self.ctx, self.layers, self.N, in_host, c, h, w, out_host, oc, oh, ow,
                              self.workspace, self.ws_bytes + self.stage_bytes, stream)
 
+    def slot_ptr(self, slot, in_blk, out_blk):
+        if slot == B.SLOT_INPUT:
+            return in_blk.data_ptr()
+        if slot == B.SLOT_OUTPUT:
+            return out_blk.data_ptr()
+        return self.workspace.data_ptr() + self.slot_offsets()[slot]
+
+    def run_layer(self, i, in_blk, out_blk=None, stream=None):
+        """Launches layer i alone through its own entry point, on the same buffers small_run_net would use."""
+        out_blk = self.out_blk if out_blk is None else out_blk
+        L, N = self.layers[i], self.N
+        src, dst = self.slot_ptr(L.src, in_blk, out_blk), self.slot_ptr(L.dst, in_blk, out_blk)
+        pad = (L.pad_t, L.pad_b, L.pad_l, L.pad_r)
+        if L.op == B.OP_CONV:
+            B.small_conv2d(self.ctx, src, L.w_blk, L.bias, dst, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride, pad, L.flags, stream)
+        elif L.op == B.OP_DWCONV:
+            B.small_dwconv2d(self.ctx, src, L.w_blk, L.bias, dst, N, L.C, L.H, L.W, L.FH, L.FW, L.stride, pad, L.flags, stream)
+        elif L.op == B.OP_POOL:
+            B.small_pool2d(self.ctx, src, dst, None, N, L.C, L.H, L.W, L.FH, L.FW, L.stride, pad, L.pool_mode, stream)
+        elif L.op == B.OP_FC:
+            B.small_fc(self.ctx, src, L.w_blk, L.bias, dst, N, L.C, L.K, L.flags, stream)
+        else:
+            raise ValueError(L.op)
+
     def slot_offsets(self):
         """Byte offset of every slot, by the library's rule: sizes rounded up to 256 bytes, back to back."""
         sizes = {}
