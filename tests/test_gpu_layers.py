@@ -201,3 +201,52 @@ def test_argument_errors_launch_nothing():
     assert L.small_relu(c, x.data_ptr(), x.data_ptr() + 64, 1, 32, 4, 4, st) == 4   # partial overlap
     torch.cuda.synchronize()
     assert B.small_device_status(c) == 0
+
+
+CONV_TC_CASES = [  # N, C, K, H, W, FH, FW, pad  (stride 1: the shapes the tensor-core kernel takes)
+    (1, 16, 16, 32, 32, 3, 3, (1, 1, 1, 1)),       # the single-conv workload
+    (2, 64, 64, 56, 56, 3, 3, (1, 1, 1, 1)),       # sweep shapes at small batch: row tiles of one image
+    (3, 128, 128, 28, 28, 3, 3, (1, 1, 1, 1)),
+    (5, 256, 256, 14, 14, 3, 3, (1, 1, 1, 1)),     # several images per strip, two filter tiles
+    (19, 512, 512, 7, 7, 3, 3, (1, 1, 1, 1)),      # ragged last strip (19 = 2 x 8 + 3 images)
+    (2, 64, 64, 56, 56, 1, 1, (0, 0, 0, 0)),
+    (23, 512, 512, 7, 7, 1, 1, (0, 0, 0, 0)),
+    (3, 64, 64, 25, 5, 1, 1, (0, 0, 0, 0)),
+    (2, 3, 16, 32, 32, 3, 3, (1, 1, 1, 1)),        # few input channels: the rest of the block is zero
+    (2, 70, 45, 9, 11, 3, 3, (1, 1, 1, 1)),        # ragged channel counts
+    (2, 33, 200, 17, 19, 5, 3, (2, 1, 0, 2)),      # asymmetric pads, rectangular window, ragged filter tile
+    (1, 40, 40, 17, 17, 2, 2, (0, 1, 1, 0)),
+    (3, 32, 32, 40, 200, 3, 3, (1, 1, 1, 1)),      # wide rows
+    (4, 32, 64, 6, 6, 3, 3, (2, 0, 0, 2)),
+    (1, 96, 32, 6, 6, 6, 6, (0, 0, 0, 0)),         # full reduction as a full-window convolution
+    (2, 32, 32, 3, 300, 1, 1, (0, 0, 0, 0)),       # row wider than the kernel's tile: runs the FP32 kernel instead
+]
+
+
+@pytest.mark.parametrize("case", CONV_TC_CASES)
+def test_conv_tf32_tensor_cores(case):
+    N, C, K, H, W, FH, FW, pad = case
+    x, w, b = rnd((N, C, H, W), 16), rnd((K, C, FH, FW), 17), rnd((K,), 18)
+    wb = torch.empty(B.small_conv_weight_elems(C, K, FH, FW, B.MATH_TF32), device="cuda")
+    B.small_pack_conv_weights(ctx(), dev(w), wb, C, K, FH, FW, B.MATH_TF32)
+    bx = to_blk(x)
+    ref = oracle.conv2d(x, w, b, 1, pad, relu=True)
+    OH, OW = ref.shape[2:]
+    uses = B.small_conv2d_uses_tensor_cores(N, C, K, H, W, FH, FW, 1, pad)
+    assert uses == (W + max(pad[2], pad[3]) <= 256)
+    out = new_blk(N, K, OH, OW)
+    B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, 1, pad, B.RELU | B.MATH_TF32)
+    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    assert B.small_device_status(ctx()) == 0
+    assert err <= 2e-3, err
+    if uses:
+        assert err > 1e-7     # TF32 products: not the FP32 kernel in disguise
+    assert pad_lanes_are_zero(out, N, K, OH, OW)
+    prev = rnd((N, K, OH, OW), 19)
+    acc = to_blk(prev)
+    B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, 1, pad, B.ACCUMULATE | B.MATH_TF32)
+    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, 1, pad, accumulate_into=prev)) <= 2e-3
+    # deterministic: the same launch twice gives the same bits
+    out2 = new_blk(N, K, OH, OW)
+    B.small_conv2d(ctx(), bx, wb, dev(b), out2, N, C, K, H, W, FH, FW, 1, pad, B.RELU | B.MATH_TF32)
+    assert torch.equal(out.view(torch.int32), out2.view(torch.int32))
