@@ -264,17 +264,19 @@ def gpu_main(args):
         return
 
     # ---- per-kernel timing of the same network, one launch at a time on the same stream
-    def time_launch(fn, reps=20, warm=3):
+    def time_launch(fn, reps=20, warm=3, inner=1):
+        """Device time of one launch: `inner` back-to-back launches between two events, minimum and median over `reps`."""
         for _ in range(warm):
             fn()
         ts = []
         for _ in range(reps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            fn()
+            for _ in range(inner):
+                fn()
             e1.record()
             e1.synchronize()
-            ts.append(e0.elapsed_time(e1))
+            ts.append(e0.elapsed_time(e1) / inner)
         return min(ts), statistics.median(ts)
 
     gnet.run(in_blk[0])
@@ -282,7 +284,7 @@ def gpu_main(args):
     by_kernel = {}
     for i, (row, L) in enumerate(zip(gnet.layer_rows, net["layers"])):
         # accumulate layers update their destination in place; values drift over repetitions but the work does not
-        tmin, tmed = time_launch(lambda i=i: gnet.run_layer(i, in_blk[0]))
+        tmin, tmed = time_launch(lambda i=i: gnet.run_layer(i, in_blk[0]), inner=10)
         fl, by = layer_work(row, N, L.get("accumulate", False))
         kern = row["op"]
         if row["op"] == "conv":
@@ -379,8 +381,8 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
                 def call(mode=mode):
                     a, o = rot()
                     B.small_conv2d(ctx, a, wb, bias, o, N, C, C, HW, HW, F, F, 1, pad, B.RELU | B.MATH[mode])
-                reps = 5 if mode == "fp32" and F == 3 else 20
-                tmin, tmed = time_launch(call, reps=reps, warm=2)
+                slow = mode == "fp32" and F == 3
+                tmin, tmed = time_launch(call, reps=5 if slow else 20, warm=2, inner=1 if slow else 10)
                 record(kind, mode, fl, by, tmin, tmed, mode)
             del w, wb
         wdw = torch.from_numpy(synth.uniform((C, 3, 3), -1.0, 1.0, 800 + C)).to(dev)
@@ -390,20 +392,20 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
         def dw():
             a, o = rot()
             B.small_dwconv2d(ctx, a, wdb, bias, o, N, C, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU)
-        tmin, tmed = time_launch(dw)
+        tmin, tmed = time_launch(dw, inner=10)
         record("dw3x3", "fp32", 2.0 * N * HW * HW * C * 9, 4.0 * (2 * N * C * HW * HW + 10 * C), tmin, tmed, None)
         OHW = (HW - 2) // 2 + 1
 
         def mp():
             a, o = rot()
             B.small_pool2d(ctx, a, o, None, N, C, HW, HW, 2, 2, 2, (0, 0, 0, 0), B.POOL_MAX)
-        tmin, tmed = time_launch(mp)
+        tmin, tmed = time_launch(mp, inner=10)
         record("maxpool2x2", "fp32", 0.0, 4.0 * N * C * (HW * HW + OHW * OHW), tmin, tmed, None)
 
         def rl():
             a, o = rot()
             B.small_relu(ctx, a, o, N, C, HW, HW)
-        tmin, tmed = time_launch(rl)
+        tmin, tmed = time_launch(rl, inner=10)
         record("relu", "fp32", 0.0, 8.0 * N * C * HW * HW, tmin, tmed, None)
         del ins, outs
         torch.cuda.empty_cache()
@@ -413,8 +415,8 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--math", default="fp32", choices=["fp32", "tf32", "3xtf32"])
     ap.add_argument("--no-sweep", action="store_true")

@@ -126,15 +126,16 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 }
 
 // Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows 128 bytes apart, groups of 8 rows 1024
-// bytes apart.  `addr` is the 128-byte-aligned row start plus the 32-byte K step; the base-offset field carries the
-// row phase of a start that is not on a 1024-byte boundary.
+// bytes apart.  `addr` is the 128-byte-aligned row start plus the 32-byte K step.  The tensor core, like TMA, takes
+// the swizzle phase from the absolute shared-memory address (bits 7-9 select the XOR applied to the 16-byte chunk
+// index), so a start that is not on a 1024-byte boundary - every shifted tap - reads the strip exactly as TMA wrote
+// it and the descriptor's base-offset field stays 0 (checked on the device: a non-zero value permutes the chunks).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     uint64_t d = 0;
     d |= (uint64_t)((addr & 0x3FFFFu) >> 4);            // start address
     d |= (uint64_t)1 << 16;                              // leading byte offset (unused with this swizzle)
     d |= (uint64_t)(1024u >> 4) << 32;                   // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
-    d |= (uint64_t)((addr >> 7) & 7u) << 49;             // base offset
     d |= (uint64_t)2 << 61;                              // 128-byte swizzle
     return d;
 }
