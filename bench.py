@@ -412,6 +412,60 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
     return {"batch": N, "buffers": "rotating input/output sets of about 1 GB per size (larger than L2)", "rows": rows}
 
 
+def single_layer(args):
+    """--layer KIND:C:HW[:BATCH]: one sweep layer, a few launches, for profiler captures (ncu -k ... -c ...)."""
+    import torch
+    import synth
+    from paper_2303_04769_b200 import binding as B
+    parts = args.layer.split(":")
+    kind, C, HW = parts[0], int(parts[1]), int(parts[2])
+    N = int(parts[3]) if len(parts) > 3 else configs.SWEEP_BATCH
+    dev = torch.device("cuda", 0)
+    ctx = B.small_init(0)
+    elems = B.small_packed_elems(N, C, HW, HW)
+    x = torch.empty(elems, device=dev)
+    B.small_pack(ctx, torch.from_numpy(synth.uniform((N, C, HW, HW), -1.0, 1.0, 500 + C)).to(dev), x, N, C, HW, HW)
+    y = torch.empty(elems, device=dev)
+    bias = torch.from_numpy(synth.uniform((C,), -1.0, 1.0, 600 + C)).to(dev)
+    if kind in ("conv3x3", "conv1x1"):
+        F, pad = (3, (1, 1, 1, 1)) if kind == "conv3x3" else (1, (0, 0, 0, 0))
+        w = torch.from_numpy(synth.uniform((C, C, F, F), -1.0, 1.0, 700 + C + F)).to(dev)
+        wb = torch.empty(B.small_conv_weight_elems(C, C, F, F, B.MATH_3XTF32), device=dev)
+        B.small_pack_conv_weights(ctx, w, wb, C, C, F, F, B.MATH_3XTF32)
+        fn = lambda: B.small_conv2d(ctx, x, wb, bias, y, N, C, C, HW, HW, F, F, 1, pad, B.RELU | B.MATH[args.math])
+        fl, by = 2.0 * N * HW * HW * C * C * F * F, 4.0 * (2 * N * C * HW * HW + C * C * F * F + C)
+    elif kind == "dw3x3":
+        w = torch.from_numpy(synth.uniform((C, 3, 3), -1.0, 1.0, 800 + C)).to(dev)
+        wb = torch.empty(B.small_dw_weight_elems(C, 3, 3), device=dev)
+        B.small_pack_dw_weights(ctx, w, wb, C, 3, 3)
+        fn = lambda: B.small_dwconv2d(ctx, x, wb, bias, y, N, C, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU)
+        fl, by = 2.0 * N * HW * HW * C * 9, 4.0 * (2 * N * C * HW * HW + 10 * C)
+    elif kind == "maxpool2x2":
+        fn = lambda: B.small_pool2d(ctx, x, y, None, N, C, HW, HW, 2, 2, 2, (0, 0, 0, 0), B.POOL_MAX)
+        OHW = (HW - 2) // 2 + 1
+        fl, by = 0.0, 4.0 * N * C * (HW * HW + OHW * OHW)
+    elif kind == "relu":
+        fn = lambda: B.small_relu(ctx, x, y, N, C, HW, HW)
+        fl, by = 0.0, 8.0 * N * C * HW * HW
+    else:
+        raise SystemExit(f"unknown layer kind {kind}")
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    ts = []
+    for i in range(args.warmup + args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        if i >= args.warmup:
+            ts.append(e0.elapsed_time(e1))
+    t = statistics.median(ts)
+    print(json.dumps({"layer": kind, "C": C, "HW": HW, "batch": N, "math": args.math, "us_med": t * 1e3, "us_min": min(ts) * 1e3,
+                      "gflops": fl / t / 1e6, "gbs": by / t / 1e6, "algorithmic_bytes": by, "flops": fl,
+                      "device_status": B.small_device_status(ctx)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -421,10 +475,13 @@ def main():
     ap.add_argument("--math", default="fp32", choices=["fp32", "tf32", "3xtf32"])
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--layer", default=None, help="KIND:C:HW[:BATCH] - run one sweep layer only (for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.layer:
+        single_layer(args)
+    elif args.impl == "reference":
         reference_arm(args)
     else:
         gpu_main(args)

@@ -347,7 +347,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------- host side
 size_t ctrl_bytes(int BN) { return 16 * kAStages + 16 * kMaxBStages + 8 + 16 + (size_t)BN * 4; }
 
-TcPlan make_plan(const Geom &g, size_t max_smem) {
+// Plan for at most `max_chunks` accumulator chunks per CTA; ok = false when the shape does not fit.
+TcPlan make_plan_chunks(const Geom &g, size_t max_smem, int max_chunks) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;
@@ -362,11 +363,11 @@ TcPlan make_plan(const Geom &g, size_t max_smem) {
     p.n_tiles = ceil_div(Kp, p.BN);
     const long long pv = (long long)p.Hq * p.Wq;
     int a0max;
-    if (2 * pv <= kMaxChunks * 128 && p.Hq <= 256) {
-        p.nn = (int)((kMaxChunks * 128) / pv);
+    if (2 * pv <= max_chunks * 128 && p.Hq <= 256) {
+        // several whole images per strip
+        p.nn = (int)((max_chunks * 128) / pv);
         if (p.nn > 256) p.nn = 256;
         if (p.nn > g.N) p.nn = g.N;
-        if (p.nn < 1) return p;
         p.chunks = ceil_div((int)(p.nn * pv), 128);
         p.total_chunks = p.chunks; p.tiles_img = 1;
         p.Rs = p.Hq;
@@ -375,9 +376,10 @@ TcPlan make_plan(const Geom &g, size_t max_smem) {
         p.strip_px = p.nn * p.Rs * p.Wq;
         a0max = 0;   // with one image per strip the kernel's row-tile formulas describe the same geometry (q0 = 0)
     } else {
+        // row tiles of one image: runs of chunks * 128 pixels of the flattened padded plane
         p.nn = 1;
         p.total_chunks = ceil_div(g.OH * p.Wq, 128);
-        p.chunks = p.total_chunks < kMaxChunks ? p.total_chunks : kMaxChunks;
+        p.chunks = p.total_chunks < max_chunks ? p.total_chunks : max_chunks;
         p.tiles_img = ceil_div(p.total_chunks, p.chunks);
         p.Rs = (p.Wq - 1 + p.chunks * 128 - 1) / p.Wq + 1 + g.FH - 1;
         if (p.Rs > 256) return p;
@@ -402,6 +404,16 @@ TcPlan make_plan(const Geom &g, size_t max_smem) {
     p.smem_bytes = (uint32_t)(fixed + (size_t)p.b_stages * p.b_stage_bytes);
     if ((long long)p.m_tiles * p.n_tiles > 0x7fffffffLL) return p;
     p.ok = true;
+    return p;
+}
+
+// The largest tile that fits shared memory (wide rows or tall windows leave room for fewer chunks).
+TcPlan make_plan(const Geom &g, size_t max_smem) {
+    TcPlan p{};
+    for (int chunks = kMaxChunks; chunks >= 1; --chunks) {
+        p = make_plan_chunks(g, max_smem, chunks);
+        if (p.ok) break;
+    }
     return p;
 }
 
