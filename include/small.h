@@ -212,6 +212,28 @@ int small_run_net_host(small_ctx *ctx, const small_layer *layers, int n_layers, 
                        float *out_nchw_host, int outC, int outH, int outW,
                        void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- for callers that cannot allocate device memory (the paper has no counterpart to this entry point) ---- */
+
+/* Size in bytes (32 MiB) of the workspace array built into the library image.  Every GPU that loads the library
+ * holds that much device memory until the process exits. */
+size_t small_static_workspace_bytes(void);
+/* small_run_net with the intermediate buffers taken from that built-in array instead of a caller workspace, for
+ * callers that have no device memory to give and may not allocate any: a process whose device memory was handed
+ * in full to another allocator, or a request path on which an allocation's possible device-wide synchronisation
+ * is not acceptable.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine); the
+ * caller still passes the blocked input and output.  Arguments, validation and results are those of
+ * small_run_net.  Extra errors: SMALL_ERR_WORKSPACE when small_net_workspace_bytes(layers, n_layers, N) exceeds
+ * small_static_workspace_bytes() (nothing is launched; use small_run_net with your own workspace, or a smaller
+ * batch); SMALL_ERR_UNSUPPORTED for a device index of 64 or more.
+ * First call on a device: looks up the array's device address (made with that device current, restored
+ * afterwards).  Make that first call before starting any stream capture.
+ * Sharing: all calls on a device use the same array, and it keeps what the last call left there.  No call
+ * depends on that content (each layer overwrites its whole output before it is read), but two calls whose work
+ * overlaps on the GPU - different streams, or one stream per thread - race on the array: order them, e.g. by
+ * issuing them on one stream. */
+int small_run_net_static(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
+                         const float *in_blk, float *out_blk, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,7 +29,7 @@ EXPORTS = [
     "small_pack_conv_weights", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
     "small_relu", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
-    "small_net_host_staging_bytes", "small_run_net_host",
+    "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
 ]
 
 
@@ -94,6 +94,9 @@ def lib():
     L.small_net_host_staging_bytes.argtypes = [I] * 7
     L.small_net_host_staging_bytes.restype = Z
     L.small_run_net_host.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, I, I, I, P, I, I, I, P, Z, P]
+    L.small_static_workspace_bytes.argtypes = []
+    L.small_static_workspace_bytes.restype = Z
+    L.small_run_net_static.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, P, P]
     _lib = L
     return L
 
@@ -233,3 +236,13 @@ def small_run_net_host(ctx, layers, N, in_host, C, H, W, out_host, outC, outH, o
     """in_host / out_host: CPU tensors (pinned for asynchronous copies)."""
     _check(lib().small_run_net_host(ctx, layers, len(layers), N, _ptr(in_host), C, H, W, _ptr(out_host), outC, outH, outW,
                                     _ptr(workspace), workspace_bytes, _stream(stream)), "small_run_net_host")
+
+
+def small_static_workspace_bytes():
+    return lib().small_static_workspace_bytes()
+
+
+def small_run_net_static(ctx, layers, N, in_blk, out_blk, stream=None):
+    """small_run_net on the library's built-in workspace: no device allocation by the call (see include/small.h)."""
+    _check(lib().small_run_net_static(ctx, layers, len(layers), N, _ptr(in_blk), _ptr(out_blk), _stream(stream)),
+           "small_run_net_static")

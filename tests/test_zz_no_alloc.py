@@ -1,0 +1,46 @@
+"""small_run_net_static - the network runner for callers that cannot allocate device memory (their memory belongs
+to another allocator, or an allocation's device-wide stall is not acceptable where they call from) - must give
+exactly what small_run_net gives with a caller workspace.  Collected last on purpose (file name), so a run that
+stops at the first failure has already run every other test.  Passes alone in a fresh process and after the others."""
+import numpy as np
+import pytest
+import torch
+
+from synth import configs
+from paper_2303_04769_b200 import binding as B
+from paper_2303_04769_b200.net import Net
+from gpu_util import ctx, to_blk, from_blk, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_workspace_matches_caller_workspace_twice_in_a_row():
+    batch = 8
+    net = configs.kws_cnn(batch=batch)
+    gnet = Net(ctx(), net, configs.make_params(net))
+    assert 0 < gnet.ws_bytes <= B.small_static_workspace_bytes() == 32 << 20
+    oc, oh, ow = gnet.out_shape
+    for call, seed in enumerate((11, 12)):          # two calls in a row, different inputs: the second one finds
+        x = configs.make_input(net, batch, seed=seed)   # the first one's leftovers in the shared array
+        in_blk = to_blk(x)
+        want = gnet.run(in_blk).clone()                                  # existing entry point, caller's workspace
+        got = torch.full_like(want, float("nan"))
+        B.small_run_net_static(ctx(), gnet.layers, batch, in_blk, got)   # new entry point, built-in workspace
+        torch.cuda.synchronize()
+        a, b = from_blk(got, batch, oc, oh, ow), from_blk(want, batch, oc, oh, ow)
+        assert np.isfinite(a).all()
+        assert rel_l2(a, b) <= 1e-5, (call, rel_l2(a, b))   # the tolerance of the FP32 parity tests; same kernels, so equal
+    assert B.small_device_status(ctx()) == 0
+
+
+def test_static_workspace_rejects_what_does_not_fit():
+    net = configs.residual_cnn(batch=256)               # three 32 MiB activation slots: too large for the array
+    gnet = Net(ctx(), net, configs.make_params(net))
+    assert gnet.ws_bytes > B.small_static_workspace_bytes()
+    x = torch.zeros(B.small_packed_elems(256, 3, 32, 32), device="cuda")
+    out = torch.full((B.small_packed_elems(256, 10, 1, 1),), 7.0, device="cuda")
+    with pytest.raises(B.SmallError) as e:
+        B.small_run_net_static(ctx(), gnet.layers, 256, x, out)
+    assert e.value.status == 5                          # SMALL_ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())                     # nothing was launched
