@@ -20,9 +20,12 @@
 // operand: rows 128 bytes apart, start address (q + x*Wq + y) * 128.  Columns ow >= OW of each row are computed and
 // dropped.  Small planes put several whole images in one strip the same way (image pitch Hq = H + max(pad_t, pad_b)).
 //
-// Roles: warp 0 = TMA producer for input strips, warp 2 = TMA producer for filter tiles, warp 1 = MMA issuer (one
-// elected thread each), warps 4-7 = epilogue.  Every mbarrier wait is bounded; on expiry the kernel records
-// SMALL_ERR_TIMEOUT in the context's status word, lets its in-flight copies land, frees tensor memory and returns.
+// Persistent CTAs (one per SM) walk the tile list with stride gridDim.x.  Roles: warp 0 = TMA producer for input
+// strips, warp 2 = TMA producer for filter tiles, warp 1 = MMA issuer (one elected thread each), warps 4-7 = epilogue.
+// The producers run ahead across tiles; the epilogue hands each 128-pixel accumulator chunk back to the MMA issuer as
+// soon as it has been read out of tensor memory, so the next tile's MMAs overlap the current tile's stores.
+// Every mbarrier wait is bounded; on expiry the kernel records SMALL_ERR_TIMEOUT in the context's status word, lets
+// its in-flight copies land, frees tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -36,6 +39,7 @@ constexpr int kMaxChunks = 4;          // 128-pixel accumulator chunks per CTA
 constexpr int kAStages = 2;
 constexpr int kMaxBStages = 8;
 constexpr uint32_t kWaitIters = 1u << 24;   // bounded spin: try_wait itself suspends for a while per call
+constexpr int kCtrlBarrierBytes = 16 * kAStages + 16 * kMaxBStages + 8 + 8 * kMaxChunks;   // all mbarriers
 
 struct TcPlan {
     int OH, OW, Wq, Hq;
@@ -56,7 +60,7 @@ struct TcPlan {
 struct TcArgs {
     const float *bias; float *out; int *status;
     int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
-    int nn, chunks, total_chunks, tiles_img, n_tiles, BN, Rs, strip_px, tail_px;
+    int nn, chunks, total_chunks, tiles_img, m_tiles, n_tiles, BN, Rs, strip_px, tail_px;
     int tmem_cols, b_stages;
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     int relu, accumulate;
@@ -162,6 +166,40 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 }
 
 // ---------------------------------------------------------------------------------------------- kernel
+struct Tile { int n_tile, n0, q0, row0, a0, chunks; };
+
+__device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
+    Tile r;
+    r.n_tile = t % a.n_tiles;
+    const int m_tile = t / a.n_tiles;
+    if (a.nn == 1) {
+        r.n0 = m_tile / a.tiles_img;
+        const int ti = m_tile - r.n0 * a.tiles_img;
+        const int c0 = ti * a.chunks;
+        r.chunks = min(a.chunks, a.total_chunks - c0);
+        r.q0 = c0 * 128;
+        r.row0 = r.q0 / a.Wq;
+        r.a0 = r.q0 - r.row0 * a.Wq;
+    } else {
+        r.n0 = m_tile * a.nn;
+        r.q0 = 0; r.row0 = 0; r.a0 = 0;
+        r.chunks = a.chunks;
+    }
+    return r;
+}
+
+__device__ __forceinline__ void st_global_v8(float *p, const float *v) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+__device__ __forceinline__ void ld_global_v8(const float *p, float *v) {
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -171,40 +209,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t b_base = a_base + kAStages * a.a_stage_bytes;
     const uint32_t ctrl = b_base + a.b_stages * a.b_stage_bytes;
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
-    // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias tile
+    // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias for all filters
     const uint32_t bar_a_full = ctrl, bar_a_empty = ctrl + 8 * kAStages;
     const uint32_t bar_b_full = ctrl + 16 * kAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
     const uint32_t bar_acc = bar_b_empty + 8 * kMaxBStages;
-    const uint32_t ctrl_words = (16 * kAStages + 16 * kMaxBStages + 8) / 4;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr) + ctrl_words;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr) + ctrl_words + 1;
-    float *bias_s = reinterpret_cast<float *>(ctrl_ptr) + ctrl_words + 4;
+    const uint32_t bar_chunk_free = bar_acc + 8;                 // kMaxChunks barriers
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
+    float *bias_s = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tile = blockIdx.x % a.n_tiles;
-    const int m_tile = blockIdx.x / a.n_tiles;
-
-    // tile geometry
-    int n0, q0, row0, a0, chunks_t;
-    if (a.nn == 1) {
-        n0 = m_tile / a.tiles_img;
-        const int ti = m_tile % a.tiles_img;
-        const int c0 = ti * a.chunks;
-        chunks_t = min(a.chunks, a.total_chunks - c0);
-        q0 = c0 * 128;
-        row0 = q0 / a.Wq;
-        a0 = q0 - row0 * a.Wq;
-    } else {
-        n0 = m_tile * a.nn;
-        q0 = 0; row0 = 0; a0 = 0;
-        chunks_t = a.chunks;
-    }
     const int T = a.FH * a.FW;
+    const int total_tiles = a.m_tiles * a.n_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, 1); }
         for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, 1); }
         mbar_init(bar_acc, 1);
+        for (int c = 0; c < kMaxChunks; ++c) mbar_init(bar_chunk_free + 8 * c, 4);   // one arrival per epilogue warp
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -213,10 +235,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         float4 *tail = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + (size_t)a.strip_px * 128);
         for (int i = threadIdx.x; i < a.tail_px * 8; i += kThreads) tail[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    for (int i = threadIdx.x; i < a.BN; i += kThreads) {
-        const int k = n_tile * a.BN + i;
-        bias_s[i] = (a.bias && k < a.K) ? a.bias[k] : 0.0f;
-    }
+    for (int i = threadIdx.x; i < a.KB * 32; i += kThreads) bias_s[i] = (a.bias && i < a.K) ? a.bias[i] : 0.0f;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy zeros visible to the tensor core
     if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), (uint32_t)a.tmem_cols);
     tc_fence_before();
@@ -225,36 +244,44 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 0 && lane == 0) {
-        // ---- input strips: one box per channel block
+        // ---- input strips: one box per (tile, channel block)
         uint32_t armed_mask = 0, last_parity[kAStages] = {0, 0};
         bool alive = true;
-        for (int cb = 0; cb < a.CB && alive; ++cb) {
-            const int s = cb % kAStages;
-            const uint32_t use = cb / kAStages;
-            if (use > 0) alive = mbar_wait(bar_a_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
-            if (!alive) break;
-            mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
-            tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, -a.pl, row0 - a.pt, cb, n0);
-            armed_mask |= 1u << s;
-            last_parity[s] = use & 1;
+        uint32_t ia = 0;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+            const Tile tl = decode_tile(a, t);
+            for (int cb = 0; cb < a.CB && alive; ++cb, ++ia) {
+                const int s = ia % kAStages;
+                const uint32_t use = ia / kAStages;
+                if (use > 0) alive = mbar_wait(bar_a_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
+                if (!alive) break;
+                mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
+                tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, -a.pl, tl.row0 - a.pt, cb, tl.n0);
+                armed_mask |= 1u << s;
+                last_parity[s] = use & 1;
+            }
         }
         if (!alive)   // let copies that are still in flight land before the CTA exits
             for (int s = 0; s < kAStages; ++s)
                 if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_a_full + 8 * s, last_parity[s]); ++it) {}
     } else if (warp == 2 && lane == 0) {
-        // ---- filter tiles: BN rows x 128 bytes per (channel block, tap)
+        // ---- filter tiles: BN rows x 128 bytes per (tile, channel block, tap)
         uint32_t armed_mask = 0, last_parity[kMaxBStages] = {};
         bool alive = true;
-        const int total = a.CB * T;
-        for (int i = 0; i < total && alive; ++i) {
-            const int s = i % a.b_stages;
-            const uint32_t use = i / a.b_stages;
-            if (use > 0) alive = mbar_wait(bar_b_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
-            if (!alive) break;
-            mbar_expect_tx(bar_b_full + 8 * s, a.b_stage_bytes);
-            tma_load_4d(b_base + s * a.b_stage_bytes, &map_b, bar_b_full + 8 * s, 0, n_tile * a.BN, i % T, i / T);
-            armed_mask |= 1u << s;
-            last_parity[s] = use & 1;
+        uint32_t ib = 0;
+        const int per_tile = a.CB * T;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+            const int n_tile = t % a.n_tiles;
+            for (int i = 0; i < per_tile && alive; ++i, ++ib) {
+                const int s = ib % a.b_stages;
+                const uint32_t use = ib / a.b_stages;
+                if (use > 0) alive = mbar_wait(bar_b_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
+                if (!alive) break;
+                mbar_expect_tx(bar_b_full + 8 * s, a.b_stage_bytes);
+                tma_load_4d(b_base + s * a.b_stage_bytes, &map_b, bar_b_full + 8 * s, 0, n_tile * a.BN, i % T, i / T);
+                armed_mask |= 1u << s;
+                last_parity[s] = use & 1;
+            }
         }
         if (!alive)
             for (int s = 0; s < a.b_stages; ++s)
@@ -263,74 +290,107 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ---- MMA issue
         const uint32_t idesc = instr_desc(a.BN);
         bool alive = true;
-        int bi = 0;
-        for (int cb = 0; cb < a.CB && alive; ++cb) {
-            const int sa = cb % kAStages;
-            alive = mbar_wait(bar_a_full + 8 * sa, (cb / kAStages) & 1, abort_flag, a.status);
-            if (!alive) break;
-            const uint32_t a_stage = a_base + sa * a.a_stage_bytes;
-            for (int tap = 0; tap < T && alive; ++tap, ++bi) {
-                const int sb = bi % a.b_stages;
-                alive = mbar_wait(bar_b_full + 8 * sb, (bi / a.b_stages) & 1, abort_flag, a.status);
+        uint32_t ia = 0, ib = 0, it = 0;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x, ++it) {
+            const Tile tl = decode_tile(a, t);
+            for (int cb = 0; cb < a.CB && alive; ++cb, ++ia) {
+                const int sa = ia % kAStages;
+                alive = mbar_wait(bar_a_full + 8 * sa, (ia / kAStages) & 1, abort_flag, a.status);
                 if (!alive) break;
-                tc_fence_after();
-                const int x = tap / a.FW, y = tap - x * a.FW;
-                const uint32_t a_tap = a_stage + (uint32_t)(a0 + x * a.Wq + y) * 128u;
-                const uint32_t b_stage = b_base + sb * a.b_stage_bytes;
-                for (int c = 0; c < chunks_t; ++c) {
+                const uint32_t a_stage = a_base + sa * a.a_stage_bytes;
+                for (int tap = 0; tap < T && alive; ++tap, ++ib) {
+                    const int sb = ib % a.b_stages;
+                    alive = mbar_wait(bar_b_full + 8 * sb, (ib / a.b_stages) & 1, abort_flag, a.status);
+                    if (!alive) break;
+                    tc_fence_after();
+                    const int x = tap / a.FW, y = tap - x * a.FW;
+                    const uint32_t a_tap = a_stage + (uint32_t)(tl.a0 + x * a.Wq + y) * 128u;
+                    const uint32_t b_stage = b_base + sb * a.b_stage_bytes;
+                    for (int c = 0; c < tl.chunks && alive; ++c) {
+                        if (it > 0 && cb == 0 && tap == 0) {   // the previous tile's values of this chunk must have left tensor memory
+                            alive = mbar_wait(bar_chunk_free + 8 * c, (it - 1) & 1, abort_flag, a.status);
+                            if (!alive) break;
+                            tc_fence_after();
+                        }
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        mma_tf32(tmem + (uint32_t)(c * a.BN), smem_desc(a_tap + (uint32_t)c * (128u * 128u) + k * 32u),
-                                 smem_desc(b_stage + k * 32u), idesc, (cb | tap | k) != 0);
+                        for (int k = 0; k < 4; ++k) {
+                            mma_tf32(tmem + (uint32_t)(c * a.BN), smem_desc(a_tap + (uint32_t)c * (128u * 128u) + k * 32u),
+                                     smem_desc(b_stage + k * 32u), idesc, (cb | tap | k) != 0);
+                        }
                     }
+                    if (alive) mma_commit(bar_b_empty + 8 * sb);     // filter stage reusable once these MMAs have read it
                 }
-                mma_commit(bar_b_empty + 8 * sb);     // filter stage reusable once these MMAs have read it
+                if (alive) mma_commit(bar_a_empty + 8 * sa);
             }
-            if (alive) mma_commit(bar_a_empty + 8 * sa);
+            if (alive) mma_commit(bar_acc);
         }
-        if (alive) mma_commit(bar_acc);
     } else if (warp >= 4) {
         // ---- epilogue: each warp owns the 32 tensor-memory lanes of its quarter; thread = one pixel of a chunk
-        const bool alive = mbar_wait(bar_acc, 0, abort_flag, a.status);
-        tc_fence_after();
-        if (alive) {
-            const int quarter = warp & 3;
-            const int row = quarter * 32 + lane;
-            const int kb0 = n_tile * (a.BN / 32);
-            for (int c = 0; c < chunks_t; ++c) {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        bool alive = true;
+        uint32_t it = 0;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x, ++it) {
+            const Tile tl = decode_tile(a, t);
+            alive = mbar_wait(bar_acc, it & 1, abort_flag, a.status);
+            if (!alive) break;
+            tc_fence_after();
+            const int kb0 = tl.n_tile * (a.BN / 32);
+            // every chunk slot is handed back each tile (also the ones this tile did not use), so that the MMA issuer's
+            // wait on a slot always refers to the previous tile
+            for (int c = 0; c < kMaxChunks; ++c) {
+                if (c >= tl.chunks) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_chunk_free + 8 * c);
+                    continue;
+                }
                 const int q = c * 128 + row;
                 bool valid;
                 int n, oh, ow;
                 if (a.nn == 1) {
-                    const int qq = q0 + q;
-                    oh = qq / a.Wq; ow = qq - oh * a.Wq; n = n0;
+                    const int qq = tl.q0 + q;
+                    oh = qq / a.Wq; ow = qq - oh * a.Wq; n = tl.n0;
                     valid = oh < a.OH && ow < a.OW;
                 } else {
                     const int pv = a.Hq * a.Wq;
                     const int img = q / pv, rem = q - img * pv;
-                    oh = rem / a.Wq; ow = rem - oh * a.Wq; n = n0 + img;
+                    oh = rem / a.Wq; ow = rem - oh * a.Wq; n = tl.n0 + img;
                     valid = img < a.nn && n < a.N && oh < a.OH && ow < a.OW;
                 }
-                for (int j = 0; j < a.BN / 32; ++j) {
+                const int nj = a.BN / 32;
+                for (int j = 0; j < nj; ++j) {
                     float v[32];
                     tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * a.BN + j * 32), v);
+                    if (j == nj - 1) {   // the chunk's values are in registers: give the slot back before storing
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_chunk_free + 8 * c);
+                    }
                     const int kb = kb0 + j;
                     if (!valid || kb >= a.KB) continue;
-                    float4 *dst = reinterpret_cast<float4 *>(a.out + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow) * 32);
-                    const float *bs = bias_s + j * 32;
+                    float *dst = a.out + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow) * 32;
+                    const float *bs = bias_s + kb * 32;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float4 r = make_float4(v[4 * i] + bs[4 * i], v[4 * i + 1] + bs[4 * i + 1], v[4 * i + 2] + bs[4 * i + 2], v[4 * i + 3] + bs[4 * i + 3]);
-                        if (a.accumulate) { const float4 p = dst[i]; r.x += p.x; r.y += p.y; r.z += p.z; r.w += p.w; }
-                        if (a.relu) { r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f); r.z = fmaxf(r.z, 0.f); r.w = fmaxf(r.w, 0.f); }
-                        const int k = kb * 32 + 4 * i;   // pad lanes of the last filter block stay +0
-                        if (k + 3 >= a.K) {
-                            if (k + 0 >= a.K) r.x = 0.f;
-                            if (k + 1 >= a.K) r.y = 0.f;
-                            if (k + 2 >= a.K) r.z = 0.f;
-                            if (k + 3 >= a.K) r.w = 0.f;
+                    for (int i = 0; i < 4; ++i) {
+                        float r[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) r[e] = v[8 * i + e] + bs[8 * i + e];
+                        if (a.accumulate) {
+                            float p[8];
+                            ld_global_v8(dst + 8 * i, p);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) r[e] += p[e];
                         }
-                        dst[i] = r;
+                        if (a.relu) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) r[e] = fmaxf(r[e], 0.f);
+                        }
+                        const int k = kb * 32 + 8 * i;   // pad lanes of the last filter block stay +0
+                        if (k + 7 >= a.K) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) if (k + e >= a.K) r[e] = 0.f;
+                        }
+                        st_global_v8(dst + 8 * i, r);
                     }
                 }
             }
@@ -345,10 +405,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 // ---------------------------------------------------------------------------------------------- host side
-size_t ctrl_bytes(int BN) { return 16 * kAStages + 16 * kMaxBStages + 8 + 16 + (size_t)BN * 4; }
+size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4; }
 
-// Plan for at most `max_chunks` accumulator chunks per CTA; ok = false when the shape does not fit.
-TcPlan make_plan_chunks(const Geom &g, size_t max_smem, int max_chunks) {
+// Plan for at most `max_chunks` accumulator chunks per tile and filter tiles of `BN`; ok = false when it does not fit.
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_chunks, int BN) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;
@@ -359,12 +419,12 @@ TcPlan make_plan_chunks(const Geom &g, size_t max_smem, int max_chunks) {
     p.Hq = g.H + padh;
     if (p.Wq > 256 || g.FH * g.FW > 64) return p;
     const int Kp = g.KB * 32;
-    p.BN = Kp <= 128 ? Kp : 128;
+    p.BN = BN < Kp ? BN : Kp;
     p.n_tiles = ceil_div(Kp, p.BN);
     const long long pv = (long long)p.Hq * p.Wq;
     int a0max;
-    if (2 * pv <= max_chunks * 128 && p.Hq <= 256) {
-        // several whole images per strip
+    if (pv <= max_chunks * 128 && p.Hq <= 256) {
+        // whole images per strip: as many as fill the chunks (at least one)
         p.nn = (int)((max_chunks * 128) / pv);
         if (p.nn > 256) p.nn = 256;
         if (p.nn > g.N) p.nn = g.N;
@@ -379,7 +439,8 @@ TcPlan make_plan_chunks(const Geom &g, size_t max_smem, int max_chunks) {
         // row tiles of one image: runs of chunks * 128 pixels of the flattened padded plane
         p.nn = 1;
         p.total_chunks = ceil_div(g.OH * p.Wq, 128);
-        p.chunks = p.total_chunks < max_chunks ? p.total_chunks : max_chunks;
+        const int tiles = ceil_div(p.total_chunks, max_chunks);
+        p.chunks = ceil_div(p.total_chunks, tiles);              // balanced: 7 chunks -> 4 + 3, not 4 + 4 slots
         p.tiles_img = ceil_div(p.total_chunks, p.chunks);
         p.Rs = (p.Wq - 1 + p.chunks * 128 - 1) / p.Wq + 1 + g.FH - 1;
         if (p.Rs > 256) return p;
@@ -397,7 +458,7 @@ TcPlan make_plan_chunks(const Geom &g, size_t max_smem, int max_chunks) {
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols <<= 1;
     if (p.tmem_cols > 512) return p;
-    const size_t fixed = 1024 + (size_t)kAStages * p.a_stage_bytes + ctrl_bytes(p.BN);
+    const size_t fixed = 1024 + (size_t)kAStages * p.a_stage_bytes + ctrl_bytes(g.KB);
     if (fixed + 2 * (size_t)p.b_stage_bytes > max_smem) return p;
     size_t room = (max_smem - fixed) / p.b_stage_bytes;
     p.b_stages = (int)(room < (size_t)kMaxBStages ? room : kMaxBStages);
@@ -407,14 +468,36 @@ TcPlan make_plan_chunks(const Geom &g, size_t max_smem, int max_chunks) {
     return p;
 }
 
-// The largest tile that fits shared memory (wide rows or tall windows leave room for fewer chunks).
-TcPlan make_plan(const Geom &g, size_t max_smem) {
-    TcPlan p{};
-    for (int chunks = kMaxChunks; chunks >= 1; --chunks) {
-        p = make_plan_chunks(g, max_smem, chunks);
-        if (p.ok) break;
-    }
-    return p;
+// Estimated cycles of the whole layer under a plan: the slower of MMA issue and L2 -> shared-memory traffic per tile,
+// plus a fixed hand-over cost, times the tiles the busiest SM gets.
+double plan_cost(const TcPlan &p, const Geom &g, int sms) {
+    const double steps = (double)g.CB * g.FH * g.FW;
+    const double avg_chunks = p.nn == 1 ? (double)p.total_chunks / p.tiles_img : (double)p.chunks;
+    const double mma = avg_chunks * steps * 4.0 * (p.BN / 2.0 < 16.0 ? 16.0 : p.BN / 2.0);
+    const double bytes = (double)g.CB * p.strip_px * 128.0 + steps * p.b_stage_bytes + avg_chunks * 128.0 * p.BN * 4.0;
+    const double mem = bytes / 24.0;                 // bytes per clock one SM can expect from L2 when all SMs pull
+    const double starve = p.b_stages < 4 ? 1.15 : 1.0;   // few filter stages in flight: the MMA issuer waits on L2 latency
+    const double tile = (mma > mem ? mma : mem) * starve + 2500.0;
+    const double tiles = (double)p.m_tiles * p.n_tiles;
+    const double per_sm = tiles <= sms ? 1.0 : tiles / sms;
+    const double waves = per_sm < 4.0 ? (double)(long long)(per_sm + 0.999) : per_sm;   // few tiles per SM: whole waves
+    return waves * tile;
+}
+
+// The cheapest plan over the tile shapes that fit (wide rows or tall windows leave room for fewer chunks).
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms) {
+    TcPlan best{};
+    double best_cost = 0.0;
+    const int bns[3] = {128, 64, 32};
+    for (int chunks = kMaxChunks; chunks >= 1; --chunks)
+        for (int b = 0; b < 3; ++b) {
+            if (b > 0 && bns[b] >= g.KB * 32) continue;      // same as the previous candidate
+            TcPlan p = make_plan_with(g, max_smem, chunks, bns[b]);
+            if (!p.ok) continue;
+            const double c = plan_cost(p, g, sms);
+            if (!best.ok || c < best_cost) { best = p; best_cost = c; }
+        }
+    return best;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -424,13 +507,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 }  // namespace
 
 bool conv_tc_supported(const Geom &g) {
-    return make_plan(g, 227 * 1024).ok;
+    return make_plan(g, 227 * 1024, 148).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &g, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
     (void)w_lo; (void)mode;
-    TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024);
+    TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_a, map_b;
@@ -459,14 +542,16 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.bias = bias; a.out = out; a.status = ctx->dev_status;
     a.N = g.N; a.K = g.K; a.KB = g.KB; a.CB = g.CB; a.OH = g.OH; a.OW = g.OW; a.Wq = p.Wq; a.Hq = p.Hq;
     a.FH = g.FH; a.FW = g.FW; a.pt = g.pt; a.pl = g.pl;
-    a.nn = p.nn; a.chunks = p.chunks; a.total_chunks = p.total_chunks; a.tiles_img = p.tiles_img; a.n_tiles = p.n_tiles;
+    a.nn = p.nn; a.chunks = p.chunks; a.total_chunks = p.total_chunks; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
     a.BN = p.BN; a.Rs = p.Rs; a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.tmem_cols = p.tmem_cols; a.b_stages = p.b_stages;
     a.a_stage_bytes = p.a_stage_bytes; a.b_stage_bytes = p.b_stage_bytes;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.relu = relu; a.accumulate = accumulate;
     cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
-    conv_tc_kernel<<<(unsigned)(p.m_tiles * p.n_tiles), kThreads, p.smem_bytes, st>>>(map_a, map_b, a);
+    const long long tiles = (long long)p.m_tiles * p.n_tiles;
+    const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
+    conv_tc_kernel<<<grid, kThreads, p.smem_bytes, st>>>(map_a, map_b, a);
     return check_launch(ctx);
 }
 
