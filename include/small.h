@@ -98,6 +98,14 @@ int small_last_cuda_error(small_ctx *ctx);
  * SMALL_ERR_TIMEOUT (a tensor-core pipeline wait gave up; the affected outputs are undefined). */
 int small_device_status(small_ctx *ctx, int *status, void *stream);
 
+/* Measures the dense TF32 tensor-core rate of this device: every SM issues `iters` x 4 back-to-back
+ * tcgen05.mma kind::tf32 of shape 128 x n x 8 (n = 64, 128 or 256) on operands resident in shared memory.
+ * cycles_dev: device buffer of one 64-bit word per SM (receives each SM's cycle count).  *tflops: whole-device rate
+ * from CUDA events; *cycles_per_mma: SM 0's cycles per MMA instruction.  Synchronises `stream`.  This is the
+ * measured denominator of the tensor-bound rooflines (the paper has no counterpart: its kernels are CPU SIMD). */
+int small_measure_tf32_peak(small_ctx *ctx, int n, int iters, long long *cycles_dev, double *tflops,
+                            double *cycles_per_mma, void *stream);
+
 /* ---- layout (Section 4.4) ------------------------------------------------------------------ */
 
 /* NCHW float[N][C][H][W] -> blocked; pad lanes are written as +0.  Bit-exact move. */

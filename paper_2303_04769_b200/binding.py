@@ -25,7 +25,7 @@ MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
 EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
-    "small_last_cuda_error", "small_device_status", "small_pack", "small_unpack", "small_conv_weight_elems",
+    "small_last_cuda_error", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
     "small_relu", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
@@ -94,6 +94,7 @@ def lib():
     L.small_net_host_staging_bytes.argtypes = [I] * 7
     L.small_net_host_staging_bytes.restype = Z
     L.small_run_net_host.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, I, I, I, P, I, I, I, P, Z, P]
+    L.small_measure_tf32_peak.argtypes = [P, I, I, P, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), P]
     L.small_static_workspace_bytes.argtypes = []
     L.small_static_workspace_bytes.restype = Z
     L.small_run_net_static.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, P, P]
@@ -246,3 +247,13 @@ def small_run_net_static(ctx, layers, N, in_blk, out_blk, stream=None):
     """small_run_net on the library's built-in workspace: no device allocation by the call (see include/small.h)."""
     _check(lib().small_run_net_static(ctx, layers, len(layers), N, _ptr(in_blk), _ptr(out_blk), _stream(stream)),
            "small_run_net_static")
+
+
+def small_measure_tf32_peak(ctx, n=128, iters=4096, stream=None):
+    """(TFLOP/s of the whole device, cycles per 128 x n x 8 MMA) from the library's issue-rate probe."""
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    cycles = torch.zeros(sms, dtype=torch.int64, device="cuda")
+    tf, cpm = ctypes.c_double(0), ctypes.c_double(0)
+    _check(lib().small_measure_tf32_peak(ctx, n, iters, _ptr(cycles), ctypes.byref(tf), ctypes.byref(cpm), _stream(stream)),
+           "small_measure_tf32_peak")
+    return tf.value, cpm.value

@@ -1,31 +1,38 @@
 // Full channel reduction on the tensor cores (paper Section 3.2 item 4; Algorithms 1 and 2) for stride-1 windows:
 // an implicit GEMM straight from the blocked layout, with no im2col buffer and no reformatting (Section 4.4).
 //
-//   D[pixel, k] = sum over (channel block cb, tap (x,y), 32 channels ci)  A[pixel + shift(x,y), ci] * B[k, ci]
+//   D[k, pixel] = sum over (channel block cb, tap (x,y), 32 channels ci)  W[k, ci] * X[pixel + shift(x,y), ci]
 //
 // How the paper's loop nest maps onto the SM:
-//   k block loop (parallel)        -> N tiles of BN filters, one CTA per (pixel tile, N tile)
+//   k block loop (parallel)        -> filter tiles of 128 (the MMA's M rows), one tile = (pixel tile, filter tile)
 //   i loop over F_C in F_Cb steps  -> cb loop over 32-channel blocks: one TMA box of the input per block
 //   x, y kernel loops              -> taps: the SAME shared-memory strip is re-read with a shifted start address
 //   ii loop                        -> four K=8 TF32 MMAs per 32-channel block (tcgen05.mma kind::tf32)
-//   O_wb x K_b register tile       -> 128-pixel x BN accumulator chunks in tensor memory (up to 4 per CTA)
+//   O_wb x K_b register tile       -> 128 filters x up to 256 pixels per accumulator slot in tensor memory, 2 slots
 //   LOAD / STORE phases            -> epilogue: tensor memory -> registers, + bias, (+ previous output), ReLU, store
+//
+// Filters are the MMA's M operand and pixels its N operand because the pipe only runs at full rate for N = 256
+// (measured with this library's issue probe: 128 cycles per 128x256x8 MMA, but about 119 cycles for any N <= 224),
+// and a layer always has hundreds of pixels while it may have only 64 or 128 filters.  As a bonus the accumulator
+// comes out as [filter][pixel]: a warp holds 32 consecutive filters of one pixel = one 128-byte line of the blocked
+// output, so every store is fully coalesced.
 //
 // The strip.  A blocked input plane is [H][W][32 floats]: one pixel and channel block = one 128-byte row, the K-major
 // operand row of a TF32 MMA with the 128-byte swizzle.  TMA copies a box of Rs rows x Wq pixels (starting at column
 // -pad_l, row -pad_t of the tile, out-of-range elements filled with zeros = the padding) densely into shared memory.
 // With the row pitch Wq = W + max(pad_l, pad_r), the right padding of one row and the left padding of the next are the
 // same zero pixels, so the strip is the zero-padded image flattened to one pixel sequence, and output pixel q (also
-// numbered with pitch Wq) needs strip pixel q + x*Wq + y for tap (x, y).  Any 128 consecutive q form a valid MMA A
+// numbered with pitch Wq) needs strip pixel q + x*Wq + y for tap (x, y).  Any run of consecutive q is a valid MMA
 // operand: rows 128 bytes apart, start address (q + x*Wq + y) * 128.  Columns ow >= OW of each row are computed and
 // dropped.  Small planes put several whole images in one strip the same way (image pitch Hq = H + max(pad_t, pad_b)).
 //
 // Persistent CTAs (one per SM) walk the tile list with stride gridDim.x.  Roles: warp 0 = TMA producer for input
-// strips, warp 2 = TMA producer for filter tiles, warp 1 = MMA issuer (one elected thread each), warps 4-7 = epilogue.
-// The producers run ahead across tiles; the epilogue hands each 128-pixel accumulator chunk back to the MMA issuer as
-// soon as it has been read out of tensor memory, so the next tile's MMAs overlap the current tile's stores.
-// Every mbarrier wait is bounded; on expiry the kernel records SMALL_ERR_TIMEOUT in the context's status word, lets
-// its in-flight copies land, frees tensor memory and returns.
+// strips, warp 2 = TMA producer for filter tiles, warp 1 = MMA issuer (one elected thread each), warps 4-7 = epilogue
+// (warp q owns filters 32q..32q+31 of the tile).  The producers run ahead across tiles; accumulator slots are handed
+// back to the MMA issuer as soon as the epilogue has read them out of tensor memory, so the next tile's MMAs overlap
+// the current tile's stores (one-slot tiles alternate between the two slots).  Every mbarrier wait is bounded; on
+// expiry the kernel records SMALL_ERR_TIMEOUT in the context's status word, lets its in-flight copies land, frees
+// tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -35,34 +42,36 @@ namespace small {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kMaxChunks = 4;          // 128-pixel accumulator chunks per CTA
+constexpr int kSlots = 2;              // accumulator slots of 256 tensor-memory columns
+constexpr int kSlotPx = 256;           // pixels per slot = the MMA's largest N
+constexpr int kFilterTile = 128;       // filters per tile = the MMA's M
 constexpr int kAStages = 2;
 constexpr int kMaxBStages = 8;
-constexpr uint32_t kWaitIters = 1u << 24;   // bounded spin: try_wait itself suspends for a while per call
-constexpr int kCtrlBarrierBytes = 16 * kAStages + 16 * kMaxBStages + 8 + 8 * kMaxChunks;   // all mbarriers
+constexpr uint32_t kWaitIters = 1u << 22;   // bounded wait: polls back off with nanosleep, so this is seconds
+constexpr int kCtrlBarrierBytes = 16 * kAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
 
 struct TcPlan {
     int OH, OW, Wq, Hq;
-    int nn;              // images per strip (1: row tiles of one image)
-    int chunks;          // accumulator chunks per tile (<= kMaxChunks)
-    int total_chunks;    // row-tile mode: chunks per image
-    int tiles_img;       // row-tile mode: tiles per image
+    int nn;              // images per strip (1: runs of pixels of one image)
+    int px_tile;         // pixels per tile (multiple of 16, at most kSlots * kSlotPx)
+    int px_img;          // nn == 1: pixels of one image in the flattened padded numbering (OH * Wq)
+    int tiles_img;       // nn == 1: tiles per image
     int m_tiles;         // pixel tiles in the grid
     int Rs;              // box rows (per image)
     int strip_px, tail_px, stage_px;
-    int BN, n_tiles;     // filters per N tile, N tiles
-    int tmem_cols;
+    int n_tiles;         // filter tiles
+    int w_rows;          // rows of the filter box (min(128, padded filters))
     int b_stages;
-    uint32_t a_stage_bytes, b_stage_bytes, smem_bytes;
+    uint32_t a_stage_bytes, smem_bytes;
     bool ok;
 };
 
 struct TcArgs {
     const float *bias; float *out; int *status;
     int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
-    int nn, chunks, total_chunks, tiles_img, m_tiles, n_tiles, BN, Rs, strip_px, tail_px;
-    int tmem_cols, b_stages;
-    uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
+    int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
+    int b_stages;
+    uint32_t a_stage_bytes, a_box_bytes;
     int relu, accumulate;
 };
 
@@ -75,6 +84,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -84,15 +96,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or another role already gave up (abort flag set).
+// Bounded wait.  Returns false when the limit ran out or another role already gave up (abort flag set).  After a few
+// immediate retries the poll backs off with nanosleep so that waiting roles leave shared-memory bandwidth to the
+// tensor core, which reads its operands from the same shared memory.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
     for (uint32_t it = 0; it < kWaitIters; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (it >= 4) __nanosleep(it < 64 ? 40 : 400);
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(status, (int)SMALL_ERR_TIMEOUT);
     return false;
+}
+// One lane waits for the whole warp (all 32 lanes must call this together).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3, int c4) {
@@ -117,12 +138,16 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, FP32 accumulate, M = 128, N from the instruction descriptor, K = 8.
-__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// The two 64-bit shared-memory descriptors arrive as (low word, shared high word): only the low word changes between
+// MMAs, which keeps the single issuing thread's instruction count per MMA small.
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 // The mbarrier receives one arrival when every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -130,21 +155,16 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 }
 
 // Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows 128 bytes apart, groups of 8 rows 1024
-// bytes apart.  `addr` is the 128-byte-aligned row start plus the 32-byte K step.  The tensor core, like TMA, takes
-// the swizzle phase from the absolute shared-memory address (bits 7-9 select the XOR applied to the 16-byte chunk
-// index), so a start that is not on a 1024-byte boundary - every shifted tap - reads the strip exactly as TMA wrote
-// it and the descriptor's base-offset field stays 0 (checked on the device: a non-zero value permutes the chunks).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);            // start address
-    d |= (uint64_t)1 << 16;                              // leading byte offset (unused with this swizzle)
-    d |= (uint64_t)(1024u >> 4) << 32;                   // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                              // 128-byte swizzle
-    return d;
-}
+// bytes apart.  Low word: start address >> 4 (bits 0-13) and the leading byte offset (bits 16-29, unused with this
+// swizzle).  High word: stride byte offset 1024 >> 4 (bits 32-45), descriptor version 1 (bit 46), swizzle mode 2 =
+// 128 bytes (bits 61-63).  The tensor core, like TMA, takes the swizzle phase from the absolute shared-memory address
+// (bits 7-9 select the XOR applied to the 16-byte chunk index), so a start that is not on a 1024-byte boundary - every
+// shifted tap - reads the strip exactly as TMA wrote it and the base-offset field (bits 49-51) stays 0 (checked on
+// the device: a non-zero value permutes the chunks).  Advancing by n bytes adds n >> 4 to the low word.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
 
-// Instruction descriptor: FP32 accumulator, TF32 A and B, both K-major, M = 128, N = n.
+// Instruction descriptor: FP32 accumulator, TF32 A and B, both K-major, M = 128, N = n (a multiple of 16, <= 256).
 __device__ __forceinline__ uint32_t instr_desc(int n) {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
 }
@@ -166,7 +186,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 }
 
 // ---------------------------------------------------------------------------------------------- kernel
-struct Tile { int n_tile, n0, q0, row0, a0, chunks; };
+// One tile: `px` pixels starting at flattened index q0 of image n0 (nn == 1) or of the strip of images n0.. (nn > 1),
+// split over `slots` accumulator slots of `n_slot` pixels each (a multiple of 16), and filter tile n_tile.
+struct Tile { int n_tile, n0, q0, row0, a0, px, slots, n_slot; };
 
 __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
     Tile r;
@@ -175,29 +197,18 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
     if (a.nn == 1) {
         r.n0 = m_tile / a.tiles_img;
         const int ti = m_tile - r.n0 * a.tiles_img;
-        const int c0 = ti * a.chunks;
-        r.chunks = min(a.chunks, a.total_chunks - c0);
-        r.q0 = c0 * 128;
+        r.q0 = ti * a.px_tile;
+        r.px = min(a.px_tile, a.px_img - r.q0);
         r.row0 = r.q0 / a.Wq;
         r.a0 = r.q0 - r.row0 * a.Wq;
     } else {
         r.n0 = m_tile * a.nn;
         r.q0 = 0; r.row0 = 0; r.a0 = 0;
-        r.chunks = a.chunks;
+        r.px = a.px_tile;
     }
+    r.slots = r.px > kSlotPx ? 2 : 1;
+    r.n_slot = ((r.px + r.slots - 1) / r.slots + 15) & ~15;
     return r;
-}
-
-__device__ __forceinline__ void st_global_v8(float *p, const float *v) {
-    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
-}
-__device__ __forceinline__ void ld_global_v8(const float *p, float *v) {
-    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -207,13 +218,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t a_base = base;
     const uint32_t b_base = a_base + kAStages * a.a_stage_bytes;
-    const uint32_t ctrl = b_base + a.b_stages * a.b_stage_bytes;
+    constexpr uint32_t kBStageBytes = kFilterTile * 128;
+    const uint32_t ctrl = b_base + a.b_stages * kBStageBytes;
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
     // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias for all filters
     const uint32_t bar_a_full = ctrl, bar_a_empty = ctrl + 8 * kAStages;
     const uint32_t bar_b_full = ctrl + 16 * kAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
-    const uint32_t bar_acc = bar_b_empty + 8 * kMaxBStages;
-    const uint32_t bar_chunk_free = bar_acc + 8;                 // kMaxChunks barriers
+    const uint32_t bar_slot_full = bar_b_empty + 8 * kMaxBStages, bar_slot_free = bar_slot_full + 8 * kSlots;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
     float *bias_s = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16);
@@ -225,8 +236,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, 1); }
         for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, 1); }
-        mbar_init(bar_acc, 1);
-        for (int c = 0; c < kMaxChunks; ++c) mbar_init(bar_chunk_free + 8 * c, 4);   // one arrival per epilogue warp
+        for (int s = 0; s < kSlots; ++s) { mbar_init(bar_slot_full + 8 * s, 1); mbar_init(bar_slot_free + 8 * s, 4); }   // 4 epilogue warps
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -235,9 +245,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         float4 *tail = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + (size_t)a.strip_px * 128);
         for (int i = threadIdx.x; i < a.tail_px * 8; i += kThreads) tail[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    // filter rows the TMA box does not cover (fewer than 128 filters in the layer) stay zero for the whole kernel
+    if (a.w_rows < kFilterTile)
+        for (int s = 0; s < a.b_stages; ++s) {
+            float4 *rest = reinterpret_cast<float4 *>(base_ptr + (b_base - base) + (size_t)s * kBStageBytes + (size_t)a.w_rows * 128);
+            for (int i = threadIdx.x; i < (kFilterTile - a.w_rows) * 8; i += kThreads) rest[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
     for (int i = threadIdx.x; i < a.KB * 32; i += kThreads) bias_s[i] = (a.bias && i < a.K) ? a.bias[i] : 0.0f;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy zeros visible to the tensor core
-    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), (uint32_t)a.tmem_cols);
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), (uint32_t)(kSlots * kSlotPx));
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -263,13 +279,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         if (!alive)   // let copies that are still in flight land before the CTA exits
             for (int s = 0; s < kAStages; ++s)
-                if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_a_full + 8 * s, last_parity[s]); ++it) {}
+                if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_a_full + 8 * s, last_parity[s]); ++it) __nanosleep(200);
     } else if (warp == 2 && lane == 0) {
-        // ---- filter tiles: BN rows x 128 bytes per (tile, channel block, tap)
+        // ---- filter tiles: up to 128 rows x 128 bytes per (tile, channel block, tap)
         uint32_t armed_mask = 0, last_parity[kMaxBStages] = {};
         bool alive = true;
         uint32_t ib = 0;
         const int per_tile = a.CB * T;
+        const uint32_t box_bytes = (uint32_t)a.w_rows * 128u;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const int n_tile = t % a.n_tiles;
             for (int i = 0; i < per_tile && alive; ++i, ++ib) {
@@ -277,138 +294,127 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t use = ib / a.b_stages;
                 if (use > 0) alive = mbar_wait(bar_b_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
                 if (!alive) break;
-                mbar_expect_tx(bar_b_full + 8 * s, a.b_stage_bytes);
-                tma_load_4d(b_base + s * a.b_stage_bytes, &map_b, bar_b_full + 8 * s, 0, n_tile * a.BN, i % T, i / T);
+                mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
+                tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, n_tile * kFilterTile, i % T, i / T);
                 armed_mask |= 1u << s;
                 last_parity[s] = use & 1;
             }
         }
         if (!alive)
             for (int s = 0; s < a.b_stages; ++s)
-                if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_b_full + 8 * s, last_parity[s]); ++it) {}
+                if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_b_full + 8 * s, last_parity[s]); ++it) __nanosleep(200);
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issue
-        const uint32_t idesc = instr_desc(a.BN);
         bool alive = true;
-        uint32_t ia = 0, ib = 0, it = 0;
-        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x, ++it) {
+        uint32_t ia = 0, ib = 0, slot_uses = 0;   // slot_uses: slots taken so far; slot j of a tile is (slot_uses + j) % 2
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
+            const uint32_t idesc = instr_desc(tl.n_slot);
             for (int cb = 0; cb < a.CB && alive; ++cb, ++ia) {
                 const int sa = ia % kAStages;
                 alive = mbar_wait(bar_a_full + 8 * sa, (ia / kAStages) & 1, abort_flag, a.status);
                 if (!alive) break;
-                const uint32_t a_stage = a_base + sa * a.a_stage_bytes;
+                const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes);
                 for (int tap = 0; tap < T && alive; ++tap, ++ib) {
                     const int sb = ib % a.b_stages;
                     alive = mbar_wait(bar_b_full + 8 * sb, (ib / a.b_stages) & 1, abort_flag, a.status);
                     if (!alive) break;
                     tc_fence_after();
                     const int x = tap / a.FW, y = tap - x * a.FW;
-                    const uint32_t a_tap = a_stage + (uint32_t)(tl.a0 + x * a.Wq + y) * 128u;
-                    const uint32_t b_stage = b_base + sb * a.b_stage_bytes;
-                    for (int c = 0; c < tl.chunks && alive; ++c) {
-                        if (it > 0 && cb == 0 && tap == 0) {   // the previous tile's values of this chunk must have left tensor memory
-                            alive = mbar_wait(bar_chunk_free + 8 * c, (it - 1) & 1, abort_flag, a.status);
-                            if (!alive) break;
-                            tc_fence_after();
-                        }
+                    const uint32_t x_lo = x_stage + (uint32_t)(tl.a0 + x * a.Wq + y) * 8u;   // 128 bytes per pixel, >> 4
+                    const uint32_t w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
+                    const uint32_t first = (cb | tap) == 0 ? 0u : 1u;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            mma_tf32(tmem + (uint32_t)(c * a.BN), smem_desc(a_tap + (uint32_t)c * (128u * 128u) + k * 32u),
-                                     smem_desc(b_stage + k * 32u), idesc, (cb | tap | k) != 0);
+                    for (int j = 0; j < kSlots; ++j) {
+                        if (j < tl.slots && alive) {
+                            const uint32_t u = slot_uses + j;        // this slot's turn number
+                            const uint32_t s = u % kSlots;
+                            if (first == 0 && u >= kSlots) {         // its previous content must have left tensor memory
+                                alive = mbar_wait(bar_slot_free + 8 * s, (u / kSlots - 1) & 1, abort_flag, a.status);
+                                tc_fence_after();
+                            }
+                            if (alive) {
+                                const uint32_t d = tmem + s * kSlotPx;
+                                const uint32_t xs = x_lo + (uint32_t)(j * tl.n_slot) * 8u;
+                                mma_tf32(d, w_lo, xs, kDescHi, idesc, first);
+                                mma_tf32(d, w_lo + 2u, xs + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
+                                mma_tf32(d, w_lo + 4u, xs + 4u, kDescHi, idesc, 1u);
+                                mma_tf32(d, w_lo + 6u, xs + 6u, kDescHi, idesc, 1u);
+                            }
                         }
                     }
                     if (alive) mma_commit(bar_b_empty + 8 * sb);     // filter stage reusable once these MMAs have read it
                 }
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
             }
-            if (alive) mma_commit(bar_acc);
+            if (alive)
+                for (int j = 0; j < tl.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
+            slot_uses += tl.slots;
         }
     } else if (warp >= 4) {
-        // ---- epilogue: each warp owns the 32 tensor-memory lanes of its quarter; thread = one pixel of a chunk
+        // ---- epilogue: warp q owns tensor-memory lanes 32q.. = filters 32q.. of the tile; lane = filter, column = pixel
         const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
         bool alive = true;
-        uint32_t it = 0;
-        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x, ++it) {
+        uint32_t slot_uses = 0;
+        const int pv = a.Hq * a.Wq;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
-            alive = mbar_wait(bar_acc, it & 1, abort_flag, a.status);
-            if (!alive) break;
-            tc_fence_after();
-            const int kb0 = tl.n_tile * (a.BN / 32);
-            // every chunk slot is handed back each tile (also the ones this tile did not use), so that the MMA issuer's
-            // wait on a slot always refers to the previous tile
-            for (int c = 0; c < kMaxChunks; ++c) {
-                if (c >= tl.chunks) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_chunk_free + 8 * c);
-                    continue;
-                }
-                const int q = c * 128 + row;
-                bool valid;
-                int n, oh, ow;
-                if (a.nn == 1) {
-                    const int qq = tl.q0 + q;
-                    oh = qq / a.Wq; ow = qq - oh * a.Wq; n = tl.n0;
-                    valid = oh < a.OH && ow < a.OW;
-                } else {
-                    const int pv = a.Hq * a.Wq;
-                    const int img = q / pv, rem = q - img * pv;
-                    oh = rem / a.Wq; ow = rem - oh * a.Wq; n = tl.n0 + img;
-                    valid = img < a.nn && n < a.N && oh < a.OH && ow < a.OW;
-                }
-                const int nj = a.BN / 32;
-                for (int j = 0; j < nj; ++j) {
-                    float v[32];
-                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * a.BN + j * 32), v);
-                    if (j == nj - 1) {   // the chunk's values are in registers: give the slot back before storing
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_chunk_free + 8 * c);
-                    }
-                    const int kb = kb0 + j;
-                    if (!valid || kb >= a.KB) continue;
-                    float *dst = a.out + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow) * 32;
-                    const float *bs = bias_s + kb * 32;
+            const int kb = tl.n_tile * (kFilterTile / 32) + quarter;
+            const int k = kb * 32 + lane;
+            const float bv = kb < a.KB ? bias_s[k] : 0.0f;
+            const bool lane_real = k < a.K;
+            for (int j = 0; j < tl.slots && alive; ++j) {
+                const uint32_t u = slot_uses + j, s = u % kSlots;
+                alive = mbar_wait_warp(bar_slot_full + 8 * s, (u / kSlots) & 1, abort_flag, a.status);
+                if (!alive) break;
+                tc_fence_after();
+                const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
+                if (kb < a.KB) {
+                    for (int g = 0; g < px_here; g += 32) {
+                        float v[32];
+                        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + g), v);
+                        // pixel coordinates of column g (the same for all lanes), then walked incrementally
+                        int q = tl.q0 + j * tl.n_slot + g;
+                        int img = 0;
+                        if (a.nn > 1) { img = q / pv; q -= img * pv; }
+                        int oh = q / a.Wq, ow = q - oh * a.Wq;
+                        const int cnt = min(32, px_here - g);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float r[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) r[e] = v[8 * i + e] + bs[8 * i + e];
-                        if (a.accumulate) {
-                            float p[8];
-                            ld_global_v8(dst + 8 * i, p);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) r[e] += p[e];
+                        for (int e = 0; e < 32; ++e) {
+                            if (e < cnt) {
+                                const int n = tl.n0 + img;
+                                if (oh < a.OH && ow < a.OW && n < a.N && img < a.nn) {
+                                    float *dst = a.out + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow) * 32 + lane;
+                                    float r = v[e] + bv;
+                                    if (a.accumulate) r += *dst;
+                                    if (a.relu) r = fmaxf(r, 0.f);
+                                    *dst = lane_real ? r : 0.0f;     // pad lanes of the last filter block stay +0
+                                }
+                                if (++ow == a.Wq) { ow = 0; if (++oh == a.Hq && a.nn > 1) { oh = 0; ++img; } }
+                            }
                         }
-                        if (a.relu) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) r[e] = fmaxf(r[e], 0.f);
-                        }
-                        const int k = kb * 32 + 8 * i;   // pad lanes of the last filter block stay +0
-                        if (k + 7 >= a.K) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) if (k + e >= a.K) r[e] = 0.f;
-                        }
-                        st_global_v8(dst + 8 * i, r);
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_slot_free + 8 * s);
             }
+            slot_uses += tl.slots;
         }
         tc_fence_before();
     }
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+        tmem_dealloc(tmem, (uint32_t)(kSlots * kSlotPx));
     }
 }
 
 // ---------------------------------------------------------------------------------------------- host side
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4; }
 
-// Plan for at most `max_chunks` accumulator chunks per tile and filter tiles of `BN`; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_chunks, int BN) {
+// Plan with at most `max_px` pixels per tile; ok = false when it does not fit.
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;
@@ -419,84 +425,85 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_chunks, int BN) {
     p.Hq = g.H + padh;
     if (p.Wq > 256 || g.FH * g.FW > 64) return p;
     const int Kp = g.KB * 32;
-    p.BN = BN < Kp ? BN : Kp;
-    p.n_tiles = ceil_div(Kp, p.BN);
+    p.n_tiles = ceil_div(Kp, kFilterTile);
+    p.w_rows = Kp < kFilterTile ? Kp : kFilterTile;
     const long long pv = (long long)p.Hq * p.Wq;
-    int a0max;
-    if (pv <= max_chunks * 128 && p.Hq <= 256) {
-        // whole images per strip: as many as fill the chunks (at least one)
-        p.nn = (int)((max_chunks * 128) / pv);
+    int a0max, slot_reach;
+    if (pv <= max_px && p.Hq <= 256) {
+        // whole images per strip: as many as fill the tile (at least one)
+        p.nn = (int)(max_px / pv);
         if (p.nn > 256) p.nn = 256;
         if (p.nn > g.N) p.nn = g.N;
-        p.chunks = ceil_div((int)(p.nn * pv), 128);
-        p.total_chunks = p.chunks; p.tiles_img = 1;
+        p.px_tile = (int)(p.nn * pv);
+        p.px_img = p.px_tile; p.tiles_img = 1;
         p.Rs = p.Hq;
         p.m_tiles = ceil_div(g.N, p.nn);
         p.tail_px = minh * p.Wq + minw;
         p.strip_px = p.nn * p.Rs * p.Wq;
-        a0max = 0;   // with one image per strip the kernel's row-tile formulas describe the same geometry (q0 = 0)
+        a0max = 0;   // with one image per strip the kernel's run-of-pixels formulas describe the same geometry (q0 = 0)
     } else {
-        // row tiles of one image: runs of chunks * 128 pixels of the flattened padded plane
+        // runs of pixels of one image in the flattened padded numbering, balanced over the tiles
         p.nn = 1;
-        p.total_chunks = ceil_div(g.OH * p.Wq, 128);
-        const int tiles = ceil_div(p.total_chunks, max_chunks);
-        p.chunks = ceil_div(p.total_chunks, tiles);              // balanced: 7 chunks -> 4 + 3, not 4 + 4 slots
-        p.tiles_img = ceil_div(p.total_chunks, p.chunks);
-        p.Rs = (p.Wq - 1 + p.chunks * 128 - 1) / p.Wq + 1 + g.FH - 1;
+        p.px_img = g.OH * p.Wq;
+        const int tiles = ceil_div(p.px_img, max_px);
+        p.px_tile = ((ceil_div(p.px_img, tiles) + 31) / 32) * 32;    // two slots of a multiple of 16
+        if (p.px_tile > max_px) p.px_tile = max_px;
+        p.tiles_img = ceil_div(p.px_img, p.px_tile);
+        p.Rs = (p.Wq - 1 + p.px_tile - 1) / p.Wq + 1 + g.FH - 1;
         if (p.Rs > 256) return p;
         p.m_tiles = g.N * p.tiles_img;
         p.tail_px = minw;
         p.strip_px = p.Rs * p.Wq;
         a0max = p.Wq - 1;
     }
-    // every pixel an MMA can touch lies inside the stage: strip + zero tail, and the furthest shifted chunk
-    const int reach = a0max + p.chunks * 128 + (g.FH - 1) * p.Wq + g.FW - 1;
+    // every pixel an MMA can touch lies inside the stage: strip + zero tail, and the furthest shifted slot
+    {
+        const int slots = p.px_tile > kSlotPx ? 2 : 1;
+        const int n_slot = ((p.px_tile + slots - 1) / slots + 15) & ~15;
+        slot_reach = slots * n_slot;
+    }
+    const int reach = a0max + slot_reach + (g.FH - 1) * p.Wq + g.FW - 1;
     p.stage_px = p.strip_px + p.tail_px > reach ? p.strip_px + p.tail_px : reach;
     p.a_stage_bytes = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
-    p.b_stage_bytes = (uint32_t)p.BN * 128u;
-    int cols = p.chunks * p.BN;
-    p.tmem_cols = 32;
-    while (p.tmem_cols < cols) p.tmem_cols <<= 1;
-    if (p.tmem_cols > 512) return p;
+    const size_t b_stage = (size_t)kFilterTile * 128;
     const size_t fixed = 1024 + (size_t)kAStages * p.a_stage_bytes + ctrl_bytes(g.KB);
-    if (fixed + 2 * (size_t)p.b_stage_bytes > max_smem) return p;
-    size_t room = (max_smem - fixed) / p.b_stage_bytes;
+    if (fixed + 2 * b_stage > max_smem) return p;
+    size_t room = (max_smem - fixed) / b_stage;
     p.b_stages = (int)(room < (size_t)kMaxBStages ? room : kMaxBStages);
-    p.smem_bytes = (uint32_t)(fixed + (size_t)p.b_stages * p.b_stage_bytes);
+    p.smem_bytes = (uint32_t)(fixed + (size_t)p.b_stages * b_stage);
     if ((long long)p.m_tiles * p.n_tiles > 0x7fffffffLL) return p;
     p.ok = true;
     return p;
 }
 
-// Estimated cycles of the whole layer under a plan: the slower of MMA issue and L2 -> shared-memory traffic per tile,
-// plus a fixed hand-over cost, times the tiles the busiest SM gets.
+// Estimated cycles of the whole layer under a plan: MMA issue at the measured rates (128 cycles per 128x256x8 MMA,
+// about 119 for any narrower one) against L2 -> shared-memory traffic per tile, plus a fixed hand-over cost, times the
+// tiles the busiest SM gets.
 double plan_cost(const TcPlan &p, const Geom &g, int sms) {
     const double steps = (double)g.CB * g.FH * g.FW;
-    const double avg_chunks = p.nn == 1 ? (double)p.total_chunks / p.tiles_img : (double)p.chunks;
-    const double mma = avg_chunks * steps * 4.0 * (p.BN / 2.0 < 16.0 ? 16.0 : p.BN / 2.0);
-    const double bytes = (double)g.CB * p.strip_px * 128.0 + steps * p.b_stage_bytes + avg_chunks * 128.0 * p.BN * 4.0;
-    const double mem = bytes / 24.0;                 // bytes per clock one SM can expect from L2 when all SMs pull
-    const double starve = p.b_stages < 4 ? 1.15 : 1.0;   // few filter stages in flight: the MMA issuer waits on L2 latency
-    const double tile = (mma > mem ? mma : mem) * starve + 2500.0;
+    const double avg_px = p.nn == 1 ? (double)p.px_img / p.tiles_img : (double)p.px_tile;
+    const int slots = p.px_tile > kSlotPx ? 2 : 1;
+    const double n_slot = avg_px / slots;
+    const double mma = steps * 4.0 * slots * (n_slot / 2.0 > 119.0 ? n_slot / 2.0 : 119.0);
+    const double bytes = (double)g.CB * p.strip_px * 128.0 + steps * p.w_rows * 128.0 + avg_px * 128.0 * 4.0;
+    const double mem = bytes / 40.0;                 // bytes per clock one SM can expect from L2 when all SMs pull
+    const double tile = (mma > mem ? mma : mem) + 2500.0;
     const double tiles = (double)p.m_tiles * p.n_tiles;
     const double per_sm = tiles <= sms ? 1.0 : tiles / sms;
     const double waves = per_sm < 4.0 ? (double)(long long)(per_sm + 0.999) : per_sm;   // few tiles per SM: whole waves
     return waves * tile;
 }
 
-// The cheapest plan over the tile shapes that fit (wide rows or tall windows leave room for fewer chunks).
+// The cheapest plan over the tile sizes that fit (wide rows or tall windows leave room for fewer pixels per tile).
 TcPlan make_plan(const Geom &g, size_t max_smem, int sms) {
     TcPlan best{};
     double best_cost = 0.0;
-    const int bns[3] = {128, 64, 32};
-    for (int chunks = kMaxChunks; chunks >= 1; --chunks)
-        for (int b = 0; b < 3; ++b) {
-            if (b > 0 && bns[b] >= g.KB * 32) continue;      // same as the previous candidate
-            TcPlan p = make_plan_with(g, max_smem, chunks, bns[b]);
-            if (!p.ok) continue;
-            const double c = plan_cost(p, g, sms);
-            if (!best.ok || c < best_cost) { best = p; best_cost = c; }
-        }
+    for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
+        TcPlan p = make_plan_with(g, max_smem, px);
+        if (!p.ok) continue;
+        const double c = plan_cost(p, g, sms);
+        if (!best.ok || c < best_cost) { best = p; best_cost = c; }
+    }
     return best;
 }
 
@@ -527,11 +534,11 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
     }
-    {   // filters: [CB][FH*FW][KB*32][32 floats]; box = 32 x BN rows
+    {   // filters: [CB][FH*FW][KB*32][32 floats]; box = 32 x min(128, KB*32) rows
         const int T = g.FH * g.FW, Kp = g.KB * 32;
         cuuint64_t dims[4] = {32, (cuuint64_t)Kp, (cuuint64_t)T, (cuuint64_t)g.CB};
         cuuint64_t strides[3] = {128, (cuuint64_t)Kp * 128, (cuuint64_t)T * Kp * 128};
-        cuuint32_t box[4] = {32, (cuuint32_t)p.BN, 1, 1};
+        cuuint32_t box[4] = {32, (cuuint32_t)p.w_rows, 1, 1};
         cuuint32_t estr[4] = {1, 1, 1, 1};
         CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float *>(w_hi), dims, strides, box, estr,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -542,9 +549,9 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.bias = bias; a.out = out; a.status = ctx->dev_status;
     a.N = g.N; a.K = g.K; a.KB = g.KB; a.CB = g.CB; a.OH = g.OH; a.OW = g.OW; a.Wq = p.Wq; a.Hq = p.Hq;
     a.FH = g.FH; a.FW = g.FW; a.pt = g.pt; a.pl = g.pl;
-    a.nn = p.nn; a.chunks = p.chunks; a.total_chunks = p.total_chunks; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
-    a.BN = p.BN; a.Rs = p.Rs; a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.tmem_cols = p.tmem_cols; a.b_stages = p.b_stages;
-    a.a_stage_bytes = p.a_stage_bytes; a.b_stage_bytes = p.b_stage_bytes;
+    a.nn = p.nn; a.px_tile = p.px_tile; a.px_img = p.px_img; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
+    a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
+    a.a_stage_bytes = p.a_stage_bytes;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.relu = relu; a.accumulate = accumulate;
     cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
