@@ -370,27 +370,37 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_after();
                 const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
                 if (kb < a.KB) {
+                    // pixel coordinates of the slot's first column (the same for all lanes), then walked one pixel at a
+                    // time; valid pixels of one image are consecutive 128-byte lines of the output, so the store
+                    // pointer just advances by one line per valid pixel
+                    int q = tl.q0 + j * tl.n_slot;
+                    int img = 0;
+                    if (a.nn > 1) { img = q / pv; q -= img * pv; }
+                    int oh = q / a.Wq, ow = q - oh * a.Wq;
+                    const size_t plane = (size_t)a.OH * a.OW * 32;
+                    const size_t image = plane * a.KB;
+                    // line of (n, kb, oh, ow) if that pixel exists; rows past OH only occur at the end of an image
+                    float *dst = a.out + (size_t)(tl.n0 + img) * image + kb * plane +
+                                 ((size_t)min(oh, a.OH) * a.OW + (oh < a.OH ? min(ow, a.OW) : 0)) * 32 + lane;
+                    int imgs_left = min(a.nn, a.N - tl.n0) - img;      // images of this strip that exist, from img on
                     for (int g = 0; g < px_here; g += 32) {
                         float v[32];
                         tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + g), v);
-                        // pixel coordinates of column g (the same for all lanes), then walked incrementally
-                        int q = tl.q0 + j * tl.n_slot + g;
-                        int img = 0;
-                        if (a.nn > 1) { img = q / pv; q -= img * pv; }
-                        int oh = q / a.Wq, ow = q - oh * a.Wq;
                         const int cnt = min(32, px_here - g);
 #pragma unroll
                         for (int e = 0; e < 32; ++e) {
                             if (e < cnt) {
-                                const int n = tl.n0 + img;
-                                if (oh < a.OH && ow < a.OW && n < a.N && img < a.nn) {
-                                    float *dst = a.out + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow) * 32 + lane;
+                                if (ow < a.OW && oh < a.OH && imgs_left > 0) {
                                     float r = v[e] + bv;
                                     if (a.accumulate) r += *dst;
                                     if (a.relu) r = fmaxf(r, 0.f);
                                     *dst = lane_real ? r : 0.0f;     // pad lanes of the last filter block stay +0
+                                    dst += 32;
                                 }
-                                if (++ow == a.Wq) { ow = 0; if (++oh == a.Hq && a.nn > 1) { oh = 0; ++img; } }
+                                if (++ow == a.Wq) {
+                                    ow = 0;
+                                    if (++oh == a.Hq && a.nn > 1) { oh = 0; --imgs_left; dst += image - plane; }
+                                }
                             }
                         }
                     }
