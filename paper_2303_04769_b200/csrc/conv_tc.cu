@@ -185,6 +185,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Predicated global accesses as single instructions, so that the epilogue's unrolled loops stay free of branches.
+__device__ __forceinline__ void st_global_if(float *p, float v, uint32_t flag) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v), "r"(flag) : "memory");
+}
+__device__ __forceinline__ float ld_global_if(const float *p, uint32_t flag) {
+    float v = 0.0f;
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p ld.global.f32 %0, [%1];\n\t}" : "+f"(v) : "l"(p), "r"(flag) : "memory");
+    return v;
+}
+
 // ---------------------------------------------------------------------------------------------- kernel
 // One tile: `px` pixels starting at flattened index q0 of image n0 (nn == 1) or of the strip of images n0.. (nn > 1),
 // split over `slots` accumulator slots of `n_slot` pixels each (a multiple of 16), and filter tile n_tile.
@@ -370,38 +380,37 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_after();
                 const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
                 if (kb < a.KB) {
-                    // pixel coordinates of the slot's first column (the same for all lanes), then walked one pixel at a
-                    // time; valid pixels of one image are consecutive 128-byte lines of the output, so the store
-                    // pointer just advances by one line per valid pixel
-                    int q = tl.q0 + j * tl.n_slot;
-                    int img = 0;
-                    if (a.nn > 1) { img = q / pv; q -= img * pv; }
-                    int oh = q / a.Wq, ow = q - oh * a.Wq;
+                    // All lanes hold the same 32 pixels (columns) of different filters.  The pixel -> output line
+                    // mapping is therefore computed once per group with one pixel per lane (divisions in parallel)
+                    // and handed round by shuffle; the stores themselves are straight-line predicated code.
                     const size_t plane = (size_t)a.OH * a.OW * 32;
-                    const size_t image = plane * a.KB;
-                    // line of (n, kb, oh, ow) if that pixel exists; rows past OH only occur at the end of an image
-                    float *dst = a.out + (size_t)(tl.n0 + img) * image + kb * plane +
-                                 ((size_t)min(oh, a.OH) * a.OW + (oh < a.OH ? min(ow, a.OW) : 0)) * 32 + lane;
-                    int imgs_left = min(a.nn, a.N - tl.n0) - img;      // images of this strip that exist, from img on
+                    const uint32_t image = (uint32_t)(plane * a.KB);
+                    float *base_out = a.out + (size_t)tl.n0 * image + kb * plane + lane;
+                    const int q_slot = tl.q0 + j * tl.n_slot;
+                    const int imgs_here = min(a.nn, a.N - tl.n0);
                     for (int g = 0; g < px_here; g += 32) {
                         float v[32];
                         tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + g), v);
-                        const int cnt = min(32, px_here - g);
+                        int q = q_slot + g + lane, img = 0;
+                        if (a.nn > 1) { img = q / pv; q -= img * pv; }
+                        const int oh = q / a.Wq, ow = q - oh * a.Wq;
+                        const bool ok = g + lane < px_here && ow < a.OW && oh < a.OH && img < imgs_here;
+                        const uint32_t my_off = (uint32_t)img * image + (uint32_t)(oh * a.OW + ow) * 32u;   // floats from base_out
+                        const uint32_t mask = __ballot_sync(0xffffffffu, ok);
+                        // straight-line code: 32 independent shuffles, then 32 predicated stores (no branches, so the
+                        // single warp per scheduler can keep them all in flight)
+                        uint32_t off[32];
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) off[e] = __shfl_sync(0xffffffffu, my_off, e);
+                        if (a.accumulate) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) v[e] += ld_global_if(base_out + off[e], mask >> e & 1u);
+                        }
 #pragma unroll
                         for (int e = 0; e < 32; ++e) {
-                            if (e < cnt) {
-                                if (ow < a.OW && oh < a.OH && imgs_left > 0) {
-                                    float r = v[e] + bv;
-                                    if (a.accumulate) r += *dst;
-                                    if (a.relu) r = fmaxf(r, 0.f);
-                                    *dst = lane_real ? r : 0.0f;     // pad lanes of the last filter block stay +0
-                                    dst += 32;
-                                }
-                                if (++ow == a.Wq) {
-                                    ow = 0;
-                                    if (++oh == a.Hq && a.nn > 1) { oh = 0; --imgs_left; dst += image - plane; }
-                                }
-                            }
+                            float r = v[e] + bv;
+                            if (a.relu) r = fmaxf(r, 0.f);
+                            st_global_if(base_out + off[e], lane_real ? r : 0.0f, mask >> e & 1u);   // pad lanes stay +0
                         }
                     }
                 }
