@@ -250,7 +250,17 @@ def gpu_main(args):
         return sum(a.elapsed_time(b) for a, b in evs) / steps
 
     sampler = ClockSampler(local) if rank == 0 else None
-    ms_dev = timed(lambda i: gnet.run(in_blk[i % R]), args.steps, args.warmup)
+    ms_eager = timed(lambda i: gnet.run(in_blk[i % R]), args.steps, args.warmup)
+    # the same call captured once per input set and replayed: the step the headline number times
+    step_graphs = []
+    for r in range(R):
+        gnet.run(in_blk[r])
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            gnet.run(in_blk[r])
+        step_graphs.append(g)
+    ms_dev = timed(lambda i: step_graphs[i % R].replay(), args.steps, args.warmup)
     ms_e2e = timed(lambda i: gnet.run_host(host_in[i % R], host_out), args.steps, args.warmup)
     clocks = sampler.stop() if sampler else None
     value, ms = whole_job_throughput(N, ms_dev, world, dev)
@@ -264,16 +274,27 @@ def gpu_main(args):
         return
 
     # ---- per-kernel timing of the same network, one launch at a time on the same stream
+    def capture(fn, inner=1):
+        """CUDA graph of `inner` back-to-back calls of fn (the library only enqueues kernels, so its calls capture)."""
+        fn()                                   # once outside the capture: first-use set-up of the kernels
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(inner):
+                fn()
+        return g
+
     def time_launch(fn, reps=20, warm=3, inner=1):
-        """Device time of one launch: `inner` back-to-back launches between two events, minimum and median over `reps`."""
+        """Device time of one launch: a graph of `inner` back-to-back launches replayed between two events (so that
+        host launch overhead does not hide kernels of a few microseconds); minimum and median over `reps`."""
+        g = capture(fn, inner)
         for _ in range(warm):
-            fn()
+            g.replay()
         ts = []
         for _ in range(reps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for _ in range(inner):
-                fn()
+            g.replay()
             e1.record()
             e1.synchronize()
             ts.append(e0.elapsed_time(e1) / inner)
@@ -322,7 +343,8 @@ def gpu_main(args):
             "data": "synthetic",
             "config": {"workload": f"{WORKLOAD}: 8-layer residual CNN, 3x32x32 input, batch {N} per GPU (configs[1])",
                        "math": args.math, "tolerance_rel_l2": TOL[args.math], "l2": "flushed between steps (256 MB write)",
-                       "inputs": f"{R} rotating seeded input sets", "parallelism": f"batch shards x{world}, no collective"},
+                       "inputs": f"{R} rotating seeded input sets", "parallelism": f"batch shards x{world}, no collective",
+                       "launch": "small_run_net captured in a CUDA graph per input set and replayed", "eager_ms_per_step": ms_eager},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * N * c * h * w, "d2h_bytes_per_step": 4 * N * oc * oh * ow,
                     "ms_per_step": ms_e2e},
             "gpu_launches": len(gnet.layer_rows) * args.steps,

@@ -43,23 +43,31 @@ __global__ void __launch_bounds__(256) add_kernel(const float4 *__restrict__ a, 
     }
 }
 
-static int stream_grid(small_ctx *ctx, size_t n4, int unroll) {
+// Launch shape from a sweep on B200: tensors well beyond L2 stream best with few loads per thread and 4 CTAs per SM;
+// smaller ones (where ramp-up and tail are a large part of the run) want 8 CTAs per SM and 8 loads in flight each.
+static int stream_grid(small_ctx *ctx, size_t n4, int unroll, int ctas_per_sm) {
     size_t want = (n4 + 256ull * unroll - 1) / (256ull * unroll);
-    size_t cap = (size_t)ctx->sm_count * 8;      // 8 resident CTAs of 256 threads per SM
+    size_t cap = (size_t)ctx->sm_count * ctas_per_sm;
     if (want < 1) want = 1;
     return (int)(want < cap ? want : cap);
 }
+static bool is_large(size_t n4) { return n4 * 16 >= (size_t)64 << 20; }
 
 int launch_relu(small_ctx *ctx, const float *in, float *out, size_t n, cudaStream_t st) {
     size_t n4 = n / 4;   // a blocked tensor is a whole number of 32-float lines
-    relu_kernel<4><<<stream_grid(ctx, n4, 4), 256, 0, st>>>(reinterpret_cast<const float4 *>(in), reinterpret_cast<float4 *>(out), n4);
+    const float4 *i4 = reinterpret_cast<const float4 *>(in);
+    float4 *o4 = reinterpret_cast<float4 *>(out);
+    if (is_large(n4)) relu_kernel<2><<<stream_grid(ctx, n4, 2, 4), 256, 0, st>>>(i4, o4, n4);
+    else relu_kernel<8><<<stream_grid(ctx, n4, 8, 8), 256, 0, st>>>(i4, o4, n4);
     return check_launch(ctx);
 }
 
 int launch_add(small_ctx *ctx, const float *a, const float *b, float *out, size_t n, bool relu, cudaStream_t st) {
     size_t n4 = n / 4;
-    add_kernel<4><<<stream_grid(ctx, n4, 4), 256, 0, st>>>(reinterpret_cast<const float4 *>(a), reinterpret_cast<const float4 *>(b),
-                                                         reinterpret_cast<float4 *>(out), n4, relu);
+    const float4 *a4 = reinterpret_cast<const float4 *>(a), *b4 = reinterpret_cast<const float4 *>(b);
+    float4 *o4 = reinterpret_cast<float4 *>(out);
+    if (is_large(n4)) add_kernel<2><<<stream_grid(ctx, n4, 2, 4), 256, 0, st>>>(a4, b4, o4, n4, relu);
+    else add_kernel<4><<<stream_grid(ctx, n4, 4, 8), 256, 0, st>>>(a4, b4, o4, n4, relu);
     return check_launch(ctx);
 }
 

@@ -40,6 +40,7 @@ class Net:
         self.in_shape = tuple(net["input"])
         self.math = B.MATH[math]
         self.keep = []            # device tensors the descriptors point into
+        self._offsets = None
         slot_of, _ = assign_slots(net["layers"])
         self.slot_of = slot_of
         dims = {"in": self.in_shape}
@@ -117,7 +118,9 @@ class Net:
             return in_blk.data_ptr()
         if slot == B.SLOT_OUTPUT:
             return out_blk.data_ptr()
-        return self.workspace.data_ptr() + self.slot_offsets()[slot]
+        if self._offsets is None:
+            self._offsets = self.slot_offsets()
+        return self.workspace.data_ptr() + self._offsets[slot]
 
     def run_layer(self, i, in_blk, out_blk=None, stream=None):
         """Launches layer i alone through its own entry point, on the same buffers small_run_net would use."""
