@@ -185,16 +185,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// Bulk asynchronous copy shared -> global (the epilogue's store path): `bytes` is a multiple of 16, both addresses
-// 16-byte aligned.  Copies are grouped per commit; wait_read returns when all but `pending` groups have been read out
-// of shared memory (the staging buffer may be rewritten), wait_all when every copy has completed.
-__device__ __forceinline__ void bulk_store(float *gdst, uint32_t ssrc, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
 // Predicated global accesses as single instructions, so that the epilogue's unrolled loops stay free of branches.
 __device__ __forceinline__ void st_global_if(float *p, float v, uint32_t flag) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v), "r"(flag) : "memory");
@@ -248,8 +238,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
     float *bias_s = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16);
-    // per epilogue warp: two staging buffers of 32 pixels x 128 bytes for the bulk stores
-    const uint32_t stage_off = ((uint32_t)(kCtrlBarrierBytes + 16 + a.KB * 32 * 4) + 127u) & ~127u;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = a.FH * a.FW;
@@ -377,7 +365,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ---- epilogue: warp q owns tensor-memory lanes 32q.. = filters 32q.. of the tile; lane = filter, column = pixel
         const int quarter = warp & 3;
         bool alive = true;
-        uint32_t slot_uses = 0, groups_done = 0;
+        uint32_t slot_uses = 0;
         const int pv = a.Hq * a.Wq;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
@@ -392,54 +380,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_after();
                 const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
                 if (kb < a.KB) {
+                    // All lanes hold the same 32 pixels (columns) of different filters.  The pixel -> output line
+                    // mapping is therefore computed once per group with one pixel per lane (divisions in parallel)
+                    // and handed round by shuffle; the stores themselves are straight-line predicated code.
                     const size_t plane = (size_t)a.OH * a.OW * 32;
                     const uint32_t image = (uint32_t)(plane * a.KB);
+                    float *base_out = a.out + (size_t)tl.n0 * image + kb * plane + lane;
                     const int q_slot = tl.q0 + j * tl.n_slot;
                     const int imgs_here = min(a.nn, a.N - tl.n0);
-                    if (!a.accumulate) {
-                        // All lanes hold the same 32 pixels (columns) of different filters: written to shared memory
-                        // as 32 lines of 128 bytes, exactly the blocked output's bytes.  Runs of valid pixels of one
-                        // output row are contiguous in global memory and leave by bulk asynchronous copies, so the
-                        // warp spends three instructions per pixel and no address arithmetic.
-                        float *stage = reinterpret_cast<float *>(ctrl_ptr + stage_off) + quarter * 2048;
-                        const uint32_t stage_addr = ctrl + stage_off + quarter * 8192u;
-                        float *out_kb = a.out + (size_t)tl.n0 * image + kb * plane;
-                        for (int g = 0; g < px_here; g += 32, ++groups_done) {
-                            float v[32];
-                            tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + g), v);
-                            const uint32_t buf = groups_done & 1u;
-                            if (lane == 0) bulk_wait_read_1();          // the copy that last read this buffer is done with it
-                            __syncwarp();
-                            float *sb = stage + buf * 1024 + lane;
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) {
-                                float r = v[e] + bv;
-                                if (a.relu) r = fmaxf(r, 0.f);
-                                sb[e * 32] = lane_real ? r : 0.0f;       // pad lanes of the last filter block stay +0
-                            }
-                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                            __syncwarp();
-                            // row segments of this group (the same on all lanes; lane 0 issues the copies)
-                            const int cnt = min(32, px_here - g);
-                            int q = q_slot + g, img = 0;
-                            if (a.nn > 1) { img = q / pv; q -= img * pv; }
-                            int oh = q / a.Wq, ow = q - oh * a.Wq;
-                            for (int e = 0; e < cnt;) {
-                                const int seg = min(cnt - e, a.Wq - ow);
-                                const int nvalid = min(ow + seg, a.OW) - ow;
-                                if (nvalid > 0 && oh < a.OH && img < imgs_here && lane == 0)
-                                    bulk_store(out_kb + (size_t)img * image + ((size_t)oh * a.OW + ow) * 32,
-                                               stage_addr + buf * 4096u + (uint32_t)e * 128u, (uint32_t)nvalid * 128u);
-                                e += seg; ow = 0;
-                                if (++oh == a.Hq && a.nn > 1) { oh = 0; ++img; }
-                            }
-                            if (lane == 0) bulk_commit();
-                        }
-                    } else {
-                    // Accumulate (residual join): the previous output has to be read, so this path uses plain
-                    // predicated loads and stores.  The pixel -> output line mapping is computed once per group with
-                    // one pixel per lane (divisions in parallel) and handed round by shuffle.
-                    float *base_out = a.out + (size_t)tl.n0 * image + kb * plane + lane;
                     for (int g = 0; g < px_here; g += 32) {
                         float v[32];
                         tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + g), v);
@@ -449,18 +397,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const bool ok = g + lane < px_here && ow < a.OW && oh < a.OH && img < imgs_here;
                         const uint32_t my_off = (uint32_t)img * image + (uint32_t)(oh * a.OW + ow) * 32u;   // floats from base_out
                         const uint32_t mask = __ballot_sync(0xffffffffu, ok);
+                        // straight-line code: 32 independent shuffles, then 32 predicated stores (no branches, so the
+                        // single warp per scheduler can keep them all in flight)
                         uint32_t off[32];
 #pragma unroll
                         for (int e = 0; e < 32; ++e) off[e] = __shfl_sync(0xffffffffu, my_off, e);
+                        if (a.accumulate) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) v[e] += ld_global_if(base_out + off[e], mask >> e & 1u);
+                            for (int e = 0; e < 32; ++e) v[e] += ld_global_if(base_out + off[e], mask >> e & 1u);
+                        }
 #pragma unroll
                         for (int e = 0; e < 32; ++e) {
                             float r = v[e] + bv;
                             if (a.relu) r = fmaxf(r, 0.f);
                             st_global_if(base_out + off[e], lane_real ? r : 0.0f, mask >> e & 1u);   // pad lanes stay +0
                         }
-                    }
                     }
                 }
                 tc_fence_before();
@@ -469,7 +420,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             slot_uses += tl.slots;
         }
-        if (lane == 0) bulk_wait_all();               // the staging buffers must outlive their copies
         tc_fence_before();
     }
     __syncthreads();
@@ -480,8 +430,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 // ---------------------------------------------------------------------------------------------- host side
-// control block + bias, then the epilogue's staging buffers (4 warps x 2 x 4 KB)
-size_t ctrl_bytes(int KB) { return ((kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + 127) & ~(size_t)127) + 4 * 8192; }
+size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4; }
 
 // Plan with at most `max_px` pixels per tile; ok = false when it does not fit.
 TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
