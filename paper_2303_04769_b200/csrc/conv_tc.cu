@@ -62,7 +62,10 @@ struct TcPlan {
     int n_tiles;         // filter tiles
     int w_rows;          // rows of the filter box (min(128, padded filters))
     int b_stages;
-    uint32_t a_stage_bytes, smem_bytes;
+    int pixel_m;         // 1: pixels are the MMA's M rows (128 per chunk) and filters its N; 0: the other way round
+    int w_tile;          // filters per tile: 128 (filters on M) or up to 256 (filters on N)
+    int cps;             // pixel_m: 128-pixel chunks per accumulator slot (2 when the tile has <= 128 filters, else 1)
+    uint32_t a_stage_bytes, b_stage_bytes, smem_bytes;
     bool ok;
 };
 
@@ -70,8 +73,8 @@ struct TcArgs {
     const float *bias; float *out; int *status;
     int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
     int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
-    int b_stages;
-    uint32_t a_stage_bytes, a_box_bytes;
+    int b_stages, pixel_m, w_tile, cps;
+    uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     int relu, accumulate;
 };
 
@@ -185,6 +188,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 256-bit global accesses (32-byte aligned addresses).
+__device__ __forceinline__ void st_global_v8(float *p, const float *v) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+__device__ __forceinline__ void ld_global_v8(const float *p, float *v) {
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p) : "memory");
+}
+
 // Predicated global accesses as single instructions, so that the epilogue's unrolled loops stay free of branches.
 __device__ __forceinline__ void st_global_if(float *p, float v, uint32_t flag) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v), "r"(flag) : "memory");
@@ -216,8 +229,13 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
         r.q0 = 0; r.row0 = 0; r.a0 = 0;
         r.px = a.px_tile;
     }
-    r.slots = r.px > kSlotPx ? 2 : 1;
-    r.n_slot = ((r.px + r.slots - 1) / r.slots + 15) & ~15;
+    if (a.pixel_m) {                       // slots hold cps chunks of 128 pixels
+        r.n_slot = a.cps * 128;
+        r.slots = r.px > r.n_slot ? 2 : 1;
+    } else {
+        r.slots = r.px > kSlotPx ? 2 : 1;
+        r.n_slot = ((r.px + r.slots - 1) / r.slots + 15) & ~15;
+    }
     return r;
 }
 
@@ -228,7 +246,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t a_base = base;
     const uint32_t b_base = a_base + kAStages * a.a_stage_bytes;
-    constexpr uint32_t kBStageBytes = kFilterTile * 128;
+    const uint32_t kBStageBytes = a.b_stage_bytes;
     const uint32_t ctrl = b_base + a.b_stages * kBStageBytes;
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
     // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias for all filters
@@ -256,7 +274,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int i = threadIdx.x; i < a.tail_px * 8; i += kThreads) tail[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     // filter rows the TMA box does not cover (fewer than 128 filters in the layer) stay zero for the whole kernel
-    if (a.w_rows < kFilterTile)
+    if (!a.pixel_m && a.w_rows < kFilterTile)
         for (int s = 0; s < a.b_stages; ++s) {
             float4 *rest = reinterpret_cast<float4 *>(base_ptr + (b_base - base) + (size_t)s * kBStageBytes + (size_t)a.w_rows * 128);
             for (int i = threadIdx.x; i < (kFilterTile - a.w_rows) * 8; i += kThreads) rest[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -305,7 +323,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (use > 0) alive = mbar_wait(bar_b_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
                 if (!alive) break;
                 mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
-                tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, n_tile * kFilterTile, i % T, i / T);
+                tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, n_tile * a.w_tile, i % T, i / T);
                 armed_mask |= 1u << s;
                 last_parity[s] = use & 1;
             }
@@ -319,7 +337,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t ia = 0, ib = 0, slot_uses = 0;   // slot_uses: slots taken so far; slot j of a tile is (slot_uses + j) % 2
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
-            const uint32_t idesc = instr_desc(tl.n_slot);
+            // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
+            const uint32_t idesc = instr_desc(a.pixel_m ? a.w_rows : tl.n_slot);
+            const uint32_t sw = a.cps == 2 ? 128u : 256u;      // pixel_m: tensor-memory columns per 128-pixel chunk
             for (int cb = 0; cb < a.CB && alive; ++cb, ++ia) {
                 const int sa = ia % kAStages;
                 alive = mbar_wait(bar_a_full + 8 * sa, (ia / kAStages) & 1, abort_flag, a.status);
@@ -343,13 +363,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 alive = mbar_wait(bar_slot_free + 8 * s, (u / kSlots - 1) & 1, abort_flag, a.status);
                                 tc_fence_after();
                             }
-                            if (alive) {
+                            if (alive && !a.pixel_m) {
                                 const uint32_t d = tmem + s * kSlotPx;
                                 const uint32_t xs = x_lo + (uint32_t)(j * tl.n_slot) * 8u;
                                 mma_tf32(d, w_lo, xs, kDescHi, idesc, first);
                                 mma_tf32(d, w_lo + 2u, xs + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
                                 mma_tf32(d, w_lo + 4u, xs + 4u, kDescHi, idesc, 1u);
                                 mma_tf32(d, w_lo + 6u, xs + 6u, kDescHi, idesc, 1u);
+                            } else if (alive) {
+                                // pixels on M: one MMA chain per 128-pixel chunk of the slot, D = [pixel][filter]
+                                const int px_slot = min(tl.n_slot, tl.px - j * tl.n_slot);
+                                for (int c = 0; c * 128 < px_slot; ++c) {
+                                    const uint32_t d = tmem + s * kSlotPx + (uint32_t)c * sw;
+                                    const uint32_t xs = x_lo + (uint32_t)(j * tl.n_slot + c * 128) * 8u;
+                                    mma_tf32(d, xs, w_lo, kDescHi, idesc, first);
+                                    mma_tf32(d, xs + 2u, w_lo + 2u, kDescHi, idesc, 1u);
+                                    mma_tf32(d, xs + 4u, w_lo + 4u, kDescHi, idesc, 1u);
+                                    mma_tf32(d, xs + 6u, w_lo + 6u, kDescHi, idesc, 1u);
+                                }
                             }
                         }
                     }
@@ -379,7 +410,50 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!alive) break;
                 tc_fence_after();
                 const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
-                if (kb < a.KB) {
+                if (a.pixel_m) {
+                    // pixels on M: this thread owns one pixel of each 128-pixel chunk (tensor-memory lane = pixel) and
+                    // reads 32 filters at a time = one whole 128-byte output line, stored as four 32-byte vectors
+                    const uint32_t sw = a.cps == 2 ? 128u : 256u;
+                    const int kb_tile = tl.n_tile * (a.w_tile / 32);
+                    for (int c = 0; c * 128 < px_here; ++c) {
+                        const int p = c * 128 + quarter * 32 + lane;            // pixel within the slot
+                        int q = tl.q0 + j * tl.n_slot + p, img = 0;
+                        if (a.nn > 1) { img = q / pv; q -= img * pv; }
+                        const int oh = q / a.Wq, ow = q - oh * a.Wq;
+                        const int n = tl.n0 + img;
+                        const bool ok = p < px_here && ow < a.OW && oh < a.OH && img < a.nn && n < a.N;
+                        for (int jj = 0; jj * 32 < a.w_rows; ++jj) {
+                            float v[32];
+                            tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx) + (uint32_t)c * sw + jj * 32u, v);
+                            const int kbj = kb_tile + jj;
+                            if (!ok || kbj >= a.KB) continue;
+                            float *dst = a.out + ((((size_t)n * a.KB + kbj) * a.OH + oh) * a.OW + ow) * 32;
+                            const float *bs = bias_s + kbj * 32;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                float r[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) r[e] = v[8 * i + e] + bs[8 * i + e];
+                                if (a.accumulate) {
+                                    float o[8];
+                                    ld_global_v8(dst + 8 * i, o);
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) r[e] += o[e];
+                                }
+                                if (a.relu) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) r[e] = fmaxf(r[e], 0.f);
+                                }
+                                const int k0 = kbj * 32 + 8 * i;               // pad lanes of the last filter block stay +0
+                                if (k0 + 7 >= a.K) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) if (k0 + e >= a.K) r[e] = 0.f;
+                                }
+                                st_global_v8(dst + 8 * i, r);
+                            }
+                        }
+                    }
+                } else if (kb < a.KB) {
                     // All lanes hold the same 32 pixels (columns) of different filters.  The pixel -> output line
                     // mapping is therefore computed once per group with one pixel per lane (divisions in parallel)
                     // and handed round by shuffle; the stores themselves are straight-line predicated code.
@@ -432,8 +506,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------- host side
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4; }
 
-// Plan with at most `max_px` pixels per tile; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
+// Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;
@@ -444,8 +518,12 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
     p.Hq = g.H + padh;
     if (p.Wq > 256 || g.FH * g.FW > 64) return p;
     const int Kp = g.KB * 32;
-    p.n_tiles = ceil_div(Kp, kFilterTile);
-    p.w_rows = Kp < kFilterTile ? Kp : kFilterTile;
+    p.pixel_m = pixel_m;
+    p.w_tile = pixel_m ? 256 : kFilterTile;
+    p.n_tiles = ceil_div(Kp, p.w_tile);
+    p.w_rows = Kp < p.w_tile ? Kp : p.w_tile;
+    p.cps = (pixel_m && p.w_rows <= 128) ? 2 : 1;
+    if (pixel_m && max_px > kSlots * p.cps * 128) return p;       // more pixels than the accumulator slots hold
     const long long pv = (long long)p.Hq * p.Wq;
     int a0max, slot_reach;
     if (pv <= max_px && p.Hq <= 256) {
@@ -466,6 +544,7 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
         p.px_img = g.OH * p.Wq;
         const int tiles = ceil_div(p.px_img, max_px);
         p.px_tile = ((ceil_div(p.px_img, tiles) + 31) / 32) * 32;    // two slots of a multiple of 16
+        if (pixel_m) p.px_tile = ((p.px_tile + 127) / 128) * 128;    // whole 128-pixel chunks
         if (p.px_tile > max_px) p.px_tile = max_px;
         p.tiles_img = ceil_div(p.px_img, p.px_tile);
         p.Rs = (p.Wq - 1 + p.px_tile - 1) / p.Wq + 1 + g.FH - 1;
@@ -476,7 +555,9 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
         a0max = p.Wq - 1;
     }
     // every pixel an MMA can touch lies inside the stage: strip + zero tail, and the furthest shifted slot
-    {
+    if (pixel_m) {
+        slot_reach = ceil_div(p.px_tile, 128) * 128;
+    } else {
         const int slots = p.px_tile > kSlotPx ? 2 : 1;
         const int n_slot = ((p.px_tile + slots - 1) / slots + 15) & ~15;
         slot_reach = slots * n_slot;
@@ -484,7 +565,8 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
     const int reach = a0max + slot_reach + (g.FH - 1) * p.Wq + g.FW - 1;
     p.stage_px = p.strip_px + p.tail_px > reach ? p.strip_px + p.tail_px : reach;
     p.a_stage_bytes = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
-    const size_t b_stage = (size_t)kFilterTile * 128;
+    const size_t b_stage = ((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023;
+    p.b_stage_bytes = (uint32_t)b_stage;
     const size_t fixed = 1024 + (size_t)kAStages * p.a_stage_bytes + ctrl_bytes(g.KB);
     if (fixed + 2 * b_stage > max_smem) return p;
     size_t room = (max_smem - fixed) / b_stage;
@@ -495,34 +577,48 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px) {
     return p;
 }
 
-// Estimated cycles of the whole layer under a plan: MMA issue at the measured rates (128 cycles per 128x256x8 MMA,
-// about 119 for any narrower one) against L2 -> shared-memory traffic per tile, plus a fixed hand-over cost, times the
-// tiles the busiest SM gets.
+// Estimated cycles of the whole layer under a plan, from measured rates: a 128 x N x 8 MMA takes about 119 cycles for
+// N <= 224 and 128 for N = 256; with filters on M the epilogue spends about 34 cycles per pixel (one 4-byte store per
+// pixel and warp), with pixels on M about 1.2 cycles per pixel and 32 filters (32-byte vector stores).  Per tile the
+// slower of MMA issue, epilogue and L2 -> shared-memory traffic counts, plus a fixed hand-over cost, times the tiles
+// the busiest SM gets.
 double plan_cost(const TcPlan &p, const Geom &g, int sms) {
     const double steps = (double)g.CB * g.FH * g.FW;
     const double avg_px = p.nn == 1 ? (double)p.px_img / p.tiles_img : (double)p.px_tile;
-    const int slots = p.px_tile > kSlotPx ? 2 : 1;
-    const double n_slot = avg_px / slots;
-    const double mma = steps * 4.0 * slots * (n_slot / 2.0 > 119.0 ? n_slot / 2.0 : 119.0);
-    const double bytes = (double)g.CB * p.strip_px * 128.0 + steps * p.w_rows * 128.0 + avg_px * 128.0 * 4.0;
+    double mma, epi;
+    if (p.pixel_m) {
+        const double chunks = (avg_px + 127.0) / 128.0;
+        mma = steps * 4.0 * (double)(long long)chunks * (p.w_rows / 2.0 > 119.0 ? p.w_rows / 2.0 : 119.0);
+        epi = avg_px * 1.2 * (p.w_rows / 32.0) / 4.0 + 300.0 * chunks;
+    } else {
+        const int slots = p.px_tile > kSlotPx ? 2 : 1;
+        const double n_slot = avg_px / slots;
+        mma = steps * 4.0 * slots * (n_slot / 2.0 > 119.0 ? n_slot / 2.0 : 119.0);
+        epi = avg_px * 34.0;
+    }
+    const double bytes = (double)g.CB * p.strip_px * 128.0 + steps * p.w_rows * 128.0 + avg_px * 128.0 * (p.w_rows / 32.0);
     const double mem = bytes / 40.0;                 // bytes per clock one SM can expect from L2 when all SMs pull
-    const double tile = (mma > mem ? mma : mem) + 2500.0;
+    double tile = mma > mem ? mma : mem;
+    if (epi > tile) tile = epi;
+    tile += 2500.0;
     const double tiles = (double)p.m_tiles * p.n_tiles;
     const double per_sm = tiles <= sms ? 1.0 : tiles / sms;
     const double waves = per_sm < 4.0 ? (double)(long long)(per_sm + 0.999) : per_sm;   // few tiles per SM: whole waves
     return waves * tile;
 }
 
-// The cheapest plan over the tile sizes that fit (wide rows or tall windows leave room for fewer pixels per tile).
-TcPlan make_plan(const Geom &g, size_t max_smem, int sms) {
+// The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
+// fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32) {
     TcPlan best{};
     double best_cost = 0.0;
-    for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-        TcPlan p = make_plan_with(g, max_smem, px);
-        if (!p.ok) continue;
-        const double c = plan_cost(p, g, sms);
-        if (!best.ok || c < best_cost) { best = p; best_cost = c; }
-    }
+    for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
+        for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m);
+            if (!p.ok) continue;
+            const double c = plan_cost(p, g, sms);
+            if (!best.ok || c < best_cost) { best = p; best_cost = c; }
+        }
     return best;
 }
 
@@ -533,13 +629,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 }  // namespace
 
 bool conv_tc_supported(const Geom &g) {
-    return make_plan(g, 227 * 1024, 148).ok;
+    return make_plan(g, 227 * 1024, 148, false).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &g, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
     (void)w_lo; (void)mode;
-    TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count);
+    TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
+                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_a, map_b;
@@ -570,6 +667,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.FH = g.FH; a.FW = g.FW; a.pt = g.pt; a.pl = g.pl;
     a.nn = p.nn; a.px_tile = p.px_tile; a.px_img = p.px_img; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
     a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
+    a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
     a.a_stage_bytes = p.a_stage_bytes;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.relu = relu; a.accumulate = accumulate;
