@@ -45,10 +45,10 @@ constexpr int kThreads = 256;
 constexpr int kSlots = 2;              // accumulator slots of 256 tensor-memory columns
 constexpr int kSlotPx = 256;           // pixels per slot = the MMA's largest N
 constexpr int kFilterTile = 128;       // filters per tile = the MMA's M
-constexpr int kAStages = 2;
+constexpr int kMaxAStages = 6;         // input strips in flight (at least 2; as many as shared memory allows)
 constexpr int kMaxBStages = 8;
 constexpr uint32_t kWaitIters = 1u << 22;   // bounded wait: polls back off with nanosleep, so this is seconds
-constexpr int kCtrlBarrierBytes = 16 * kAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
+constexpr int kCtrlBarrierBytes = 16 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
 
 struct TcPlan {
     int OH, OW, Wq, Hq;
@@ -61,7 +61,7 @@ struct TcPlan {
     int strip_px, tail_px, stage_px;
     int n_tiles;         // filter tiles
     int w_rows;          // rows of the filter box (min(128, padded filters))
-    int b_stages;
+    int a_stages, b_stages;
     int pixel_m;         // 1: pixels are the MMA's M rows (128 per chunk) and filters its N; 0: the other way round
     int w_tile;          // filters per tile: 128 (filters on M) or up to 256 (filters on N)
     int cps;             // pixel_m: 128-pixel chunks per accumulator slot (2 when the tile has <= 128 filters, else 1)
@@ -73,7 +73,7 @@ struct TcArgs {
     const float *bias; float *out; int *status;
     int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
     int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
-    int b_stages, pixel_m, w_tile, cps;
+    int a_stages, b_stages, pixel_m, w_tile, cps;
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     int relu, accumulate;
 };
@@ -245,13 +245,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t a_base = base;
+    const int kAStages = a.a_stages;
     const uint32_t b_base = a_base + kAStages * a.a_stage_bytes;
     const uint32_t kBStageBytes = a.b_stage_bytes;
     const uint32_t ctrl = b_base + a.b_stages * kBStageBytes;
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
     // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias for all filters
-    const uint32_t bar_a_full = ctrl, bar_a_empty = ctrl + 8 * kAStages;
-    const uint32_t bar_b_full = ctrl + 16 * kAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
+    const uint32_t bar_a_full = ctrl, bar_a_empty = ctrl + 8 * kMaxAStages;
+    const uint32_t bar_b_full = ctrl + 16 * kMaxAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
     const uint32_t bar_slot_full = bar_b_empty + 8 * kMaxBStages, bar_slot_free = bar_slot_full + 8 * kSlots;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
@@ -289,7 +290,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0 && lane == 0) {
         // ---- input strips: one box per (tile, channel block)
-        uint32_t armed_mask = 0, last_parity[kAStages] = {0, 0};
+        uint32_t armed_mask = 0, last_parity[kMaxAStages] = {};
         bool alive = true;
         uint32_t ia = 0;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
@@ -546,13 +547,16 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
         p.px_tile = ((ceil_div(p.px_img, tiles) + 31) / 32) * 32;    // two slots of a multiple of 16
         if (pixel_m) p.px_tile = ((p.px_tile + 127) / 128) * 128;    // whole 128-pixel chunks
         if (p.px_tile > max_px) p.px_tile = max_px;
+        // whole rows per tile when at least two fit: the strip then needs no partial rows at either end
+        if (p.Wq <= p.px_tile && (g.FH == 1 || 2 * p.Wq <= p.px_tile)) p.px_tile = (p.px_tile / p.Wq) * p.Wq;
         p.tiles_img = ceil_div(p.px_img, p.px_tile);
-        p.Rs = (p.Wq - 1 + p.px_tile - 1) / p.Wq + 1 + g.FH - 1;
+        const bool row_aligned = p.px_tile % p.Wq == 0;             // every tile starts at a row start
+        p.Rs = row_aligned ? p.px_tile / p.Wq + g.FH - 1 : (p.Wq - 1 + p.px_tile - 1) / p.Wq + 1 + g.FH - 1;
         if (p.Rs > 256) return p;
         p.m_tiles = g.N * p.tiles_img;
         p.tail_px = minw;
         p.strip_px = p.Rs * p.Wq;
-        a0max = p.Wq - 1;
+        a0max = row_aligned ? 0 : p.Wq - 1;
     }
     // every pixel an MMA can touch lies inside the stage: strip + zero tail, and the furthest shifted slot
     if (pixel_m) {
@@ -567,40 +571,51 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
     p.a_stage_bytes = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
     const size_t b_stage = ((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023;
     p.b_stage_bytes = (uint32_t)b_stage;
-    const size_t fixed = 1024 + (size_t)kAStages * p.a_stage_bytes + ctrl_bytes(g.KB);
-    if (fixed + 2 * b_stage > max_smem) return p;
-    size_t room = (max_smem - fixed) / b_stage;
-    p.b_stages = (int)(room < (size_t)kMaxBStages ? room : kMaxBStages);
-    p.smem_bytes = (uint32_t)(fixed + (size_t)p.b_stages * b_stage);
+    // shared memory: at least two strips and two filter tiles; then filter tiles up to one per tap plus two, then
+    // further strips (deeper prefetch across tiles, which is what the bandwidth-bound layers need), then the rest
+    const size_t fixed = 1024 + ctrl_bytes(g.KB);
+    if (fixed + 2 * (size_t)p.a_stage_bytes + 2 * b_stage > max_smem) return p;
+    size_t room = max_smem - fixed - 2 * (size_t)p.a_stage_bytes - 2 * b_stage;
+    p.a_stages = 2; p.b_stages = 2;
+    const int b_want = g.FH * g.FW + 2 < kMaxBStages ? g.FH * g.FW + 2 : kMaxBStages;
+    while (p.b_stages < b_want && room >= b_stage) { ++p.b_stages; room -= b_stage; }
+    while (p.a_stages < kMaxAStages && room >= p.a_stage_bytes) { ++p.a_stages; room -= p.a_stage_bytes; }
+    while (p.b_stages < kMaxBStages && room >= b_stage) { ++p.b_stages; room -= b_stage; }
+    p.smem_bytes = (uint32_t)(fixed + (size_t)p.a_stages * p.a_stage_bytes + (size_t)p.b_stages * b_stage);
     if ((long long)p.m_tiles * p.n_tiles > 0x7fffffffLL) return p;
     p.ok = true;
     return p;
 }
 
 // Estimated cycles of the whole layer under a plan, from measured rates: a 128 x N x 8 MMA takes about 119 cycles for
-// N <= 224 and 128 for N = 256; with filters on M the epilogue spends about 34 cycles per pixel (one 4-byte store per
-// pixel and warp), with pixels on M about 1.2 cycles per pixel and 32 filters (32-byte vector stores).  Per tile the
-// slower of MMA issue, epilogue and L2 -> shared-memory traffic counts, plus a fixed hand-over cost, times the tiles
-// the busiest SM gets.
+// N <= 224 and 128 for N = 256.  The epilogue's stores run at memory speed in either orientation; what differs is how
+// many of the four epilogue warps have filters to store (filters on M: one warp per 32 filters of the tile) and the
+// instructions per pixel (about 20 cycles per pixel and warp with 4-byte stores, about 1.2 per pixel and 32 filters
+// with 32-byte vector stores).  Per tile the slowest of MMA issue, epilogue and L2 -> shared-memory traffic counts,
+// plus a hand-over cost and, when the strips of two tiles do not fit in the stages, the exposed load of one tile;
+// times the tiles the busiest SM gets.
 double plan_cost(const TcPlan &p, const Geom &g, int sms) {
     const double steps = (double)g.CB * g.FH * g.FW;
     const double avg_px = p.nn == 1 ? (double)p.px_img / p.tiles_img : (double)p.px_tile;
     double mma, epi;
     if (p.pixel_m) {
-        const double chunks = (avg_px + 127.0) / 128.0;
-        mma = steps * 4.0 * (double)(long long)chunks * (p.w_rows / 2.0 > 119.0 ? p.w_rows / 2.0 : 119.0);
-        epi = avg_px * 1.2 * (p.w_rows / 32.0) / 4.0 + 300.0 * chunks;
+        const double chunks = (double)(long long)((avg_px + 127.0) / 128.0);
+        mma = steps * 4.0 * chunks * (p.w_rows / 2.0 > 119.0 ? p.w_rows / 2.0 : 119.0);
+        epi = avg_px * 1.2 * (p.w_rows / 32.0) + 300.0 * chunks;
     } else {
         const int slots = p.px_tile > kSlotPx ? 2 : 1;
         const double n_slot = avg_px / slots;
         mma = steps * 4.0 * slots * (n_slot / 2.0 > 119.0 ? n_slot / 2.0 : 119.0);
-        epi = avg_px * 34.0;
+        const double warps = p.w_rows >= 128 ? 4.0 : p.w_rows / 32.0;
+        epi = avg_px * 20.0 * 4.0 / warps;
     }
-    const double bytes = (double)g.CB * p.strip_px * 128.0 + steps * p.w_rows * 128.0 + avg_px * 128.0 * (p.w_rows / 32.0);
-    const double mem = bytes / 40.0;                 // bytes per clock one SM can expect from L2 when all SMs pull
+    const double strip_bytes = (double)g.CB * p.strip_px * 128.0;
+    const double bytes = strip_bytes + steps * p.w_rows * 128.0 + avg_px * 128.0 * (p.w_rows / 32.0);
+    const double mem = bytes / 30.0;                 // bytes per clock one SM can expect when all SMs pull
     double tile = mma > mem ? mma : mem;
     if (epi > tile) tile = epi;
     tile += 2500.0;
+    if (p.a_stages < 2 * g.CB) tile += strip_bytes / 30.0 * 0.5;     // the next tile's strips cannot all be in flight
     const double tiles = (double)p.m_tiles * p.n_tiles;
     const double per_sm = tiles <= sms ? 1.0 : tiles / sms;
     const double waves = per_sm < 4.0 ? (double)(long long)(per_sm + 0.999) : per_sm;   // few tiles per SM: whole waves
@@ -628,13 +643,30 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 }  // namespace
 
+// A 1x1 window without padding never looks at a neighbour, so the plane may be viewed with any row length that
+// divides H*W: the longest one that still fits a TMA box makes every tile a run of whole rows and every strip exactly
+// the pixels the tile needs.
+static Geom flatten_pointwise(const Geom &g) {
+    if (g.FH != 1 || g.FW != 1 || g.S != 1 || (g.pt | g.pb | g.pl | g.pr)) return g;
+    const long long hw = (long long)g.H * g.W;
+    int best = 0;
+    for (int w = 256; w >= 1; --w)
+        if (hw % w == 0) { best = w; break; }
+    if (best <= g.W) return g;
+    Geom f = g;
+    f.W = f.OW = best;
+    f.H = f.OH = (int)(hw / best);
+    return f;
+}
+
 bool conv_tc_supported(const Geom &g) {
-    return make_plan(g, 227 * 1024, 148, false).ok;
+    return make_plan(flatten_pointwise(g), 227 * 1024, 148, false).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
-                   const Geom &g, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
+                   const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
     (void)w_lo; (void)mode;
+    const Geom g = flatten_pointwise(g_in);
     TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
                          (reinterpret_cast<uintptr_t>(out) & 31u) == 0);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
@@ -667,7 +699,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.FH = g.FH; a.FW = g.FW; a.pt = g.pt; a.pl = g.pl;
     a.nn = p.nn; a.px_tile = p.px_tile; a.px_img = p.px_img; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
     a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
-    a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
+    a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
     a.a_stage_bytes = p.a_stage_bytes;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.relu = relu; a.accumulate = accumulate;
