@@ -64,7 +64,9 @@ struct TcPlan {
     int a_stages, b_stages;
     int pixel_m;         // 1: pixels are the MMA's M rows (128 per chunk) and filters its N; 0: the other way round
     int w_tile;          // filters per tile: 128 (filters on M) or up to 256 (filters on N)
-    int cps;             // pixel_m: 128-pixel chunks per accumulator slot (2 when the tile has <= 128 filters, else 1)
+    int cps;             // pixel_m: 128-pixel chunks per accumulator slot (4, 2 or 1 for up to 64, 128 or 256 filters)
+    int b_resident;      // all filter tiles of the layer stay in shared memory for the whole kernel
+    int ks_last;         // K steps (8 channels each) of the last channel block that hold real channels
     uint32_t a_stage_bytes, b_stage_bytes, smem_bytes;
     bool ok;
 };
@@ -73,7 +75,7 @@ struct TcArgs {
     const float *bias; float *out; int *status;
     int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
     int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
-    int a_stages, b_stages, pixel_m, w_tile, cps;
+    int a_stages, b_stages, pixel_m, w_tile, cps, b_resident, ks_last;
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     int relu, accumulate;
 };
@@ -288,106 +290,138 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // Stages a producer has armed and the parity of each stage's latest fill, kept past the role loops: if any role
+    // gave up, the producers wait (bounded) for their copies in flight before the CTA may exit.
+    uint32_t armed_mask = 0, armed_parity = 0;
+    uint32_t drain_bar = 0;
+
+    // The three single-thread roles below keep their loops free of divisions: stage indices, phase bits and tap
+    // offsets advance incrementally, because every scalar instruction of the one issuing thread is a few cycles that
+    // the tensor pipe may have to wait for.
     if (warp == 0 && lane == 0) {
         // ---- input strips: one box per (tile, channel block)
-        uint32_t armed_mask = 0, last_parity[kMaxAStages] = {};
-        bool alive = true;
-        uint32_t ia = 0;
+        drain_bar = bar_a_full;
+        bool alive = true, wrapped = false;
+        uint32_t s = 0, phase = 0;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
-            for (int cb = 0; cb < a.CB && alive; ++cb, ++ia) {
-                const int s = ia % kAStages;
-                const uint32_t use = ia / kAStages;
-                if (use > 0) alive = mbar_wait(bar_a_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
+            for (int cb = 0; cb < a.CB; ++cb) {
+                if (wrapped) alive = mbar_wait(bar_a_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
                 if (!alive) break;
                 mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
                 tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, -a.pl, tl.row0 - a.pt, cb, tl.n0);
                 armed_mask |= 1u << s;
-                last_parity[s] = use & 1;
+                armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
+                if (++s == (uint32_t)kAStages) { s = 0; phase ^= 1u; wrapped = true; }
             }
         }
-        if (!alive)   // let copies that are still in flight land before the CTA exits
-            for (int s = 0; s < kAStages; ++s)
-                if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_a_full + 8 * s, last_parity[s]); ++it) __nanosleep(200);
     } else if (warp == 2 && lane == 0) {
-        // ---- filter tiles: up to 128 rows x 128 bytes per (tile, channel block, tap)
-        uint32_t armed_mask = 0, last_parity[kMaxBStages] = {};
-        bool alive = true;
-        uint32_t ib = 0;
-        const int per_tile = a.CB * T;
+        // ---- filter tiles: w_rows x 128 bytes per (channel block, tap).  Resident: all of them once, on one barrier.
+        drain_bar = bar_b_full;
         const uint32_t box_bytes = (uint32_t)a.w_rows * 128u;
-        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
-            const int n_tile = t % a.n_tiles;
-            for (int i = 0; i < per_tile && alive; ++i, ++ib) {
-                const int s = ib % a.b_stages;
-                const uint32_t use = ib / a.b_stages;
-                if (use > 0) alive = mbar_wait(bar_b_empty + 8 * s, (use - 1) & 1, abort_flag, a.status);
-                if (!alive) break;
-                mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
-                tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, n_tile * a.w_tile, i % T, i / T);
-                armed_mask |= 1u << s;
-                last_parity[s] = use & 1;
+        if (a.b_resident) {
+            mbar_expect_tx(bar_b_full, box_bytes * (uint32_t)(a.CB * T));
+            uint32_t dst = b_base;
+            for (int cb = 0; cb < a.CB; ++cb)
+                for (int tap = 0; tap < T; ++tap, dst += kBStageBytes) tma_load_4d(dst, &map_b, bar_b_full, 0, 0, tap, cb);
+            armed_mask = 1u;
+        } else {
+            bool alive = true, wrapped = false;
+            uint32_t s = 0, phase = 0;
+            for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+                const int row = (t % a.n_tiles) * a.w_tile;
+                for (int cb = 0; cb < a.CB && alive; ++cb)
+                    for (int tap = 0; tap < T; ++tap) {
+                        if (wrapped) alive = mbar_wait(bar_b_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                        if (!alive) break;
+                        mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
+                        tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, row, tap, cb);
+                        armed_mask |= 1u << s;
+                        armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
+                        if (++s == (uint32_t)a.b_stages) { s = 0; phase ^= 1u; wrapped = true; }
+                    }
             }
         }
-        if (!alive)
-            for (int s = 0; s < a.b_stages; ++s)
-                if (armed_mask >> s & 1) for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(bar_b_full + 8 * s, last_parity[s]); ++it) __nanosleep(200);
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issue
         bool alive = true;
-        uint32_t ia = 0, ib = 0, slot_uses = 0;   // slot_uses: slots taken so far; slot j of a tile is (slot_uses + j) % 2
+        uint32_t sa = 0, pa = 0, sb = 0, pb = 0;
+        uint32_t slot_uses = 0;                   // slots taken so far; slot j of a tile is (slot_uses + j) % 2
+        const uint32_t b_step = kBStageBytes >> 4;
+        const uint32_t row_wrap = (uint32_t)(a.Wq - a.FW + 1) * 8u;     // tap offset step from the end of a window row
+        const uint32_t sw = 256u / (uint32_t)a.cps;                     // pixel_m: tensor-memory columns per chunk
+        const int cps_log2 = a.cps == 4 ? 2 : a.cps == 2 ? 1 : 0;
+        if (a.b_resident) alive = mbar_wait(bar_b_full, 0, abort_flag, a.status);
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
             // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
             const uint32_t idesc = instr_desc(a.pixel_m ? a.w_rows : tl.n_slot);
-            const uint32_t sw = a.cps == 2 ? 128u : 256u;      // pixel_m: tensor-memory columns per 128-pixel chunk
-            for (int cb = 0; cb < a.CB && alive; ++cb, ++ia) {
-                const int sa = ia % kAStages;
-                alive = mbar_wait(bar_a_full + 8 * sa, (ia / kAStages) & 1, abort_flag, a.status);
+            // the previous content of the slots this tile takes must have left tensor memory
+            for (int j = 0; j < tl.slots && alive; ++j) {
+                const uint32_t u = slot_uses + j;
+                if (u >= kSlots) alive = mbar_wait(bar_slot_free + 8 * (u % kSlots), (u / kSlots - 1) & 1, abort_flag, a.status);
+            }
+            if (!alive) break;
+            tc_fence_after();
+            // accumulator address and strip offset (in 16-byte units) of each MMA chain of the tile: one per slot
+            // (filters on M) or one per 128-pixel chunk (pixels on M)
+            uint32_t acc[4], xo[4];
+            int chains;
+            if (a.pixel_m) {
+                chains = (tl.px + 127) >> 7;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int j = c >> cps_log2;
+                    acc[c] = tmem + ((slot_uses + j) % kSlots) * kSlotPx + (uint32_t)(c - j * a.cps) * sw;
+                    xo[c] = (uint32_t)c * 128u * 8u;
+                }
+            } else {
+                chains = tl.slots;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    acc[c] = tmem + ((slot_uses + c) % kSlots) * kSlotPx;
+                    xo[c] = (uint32_t)(c * tl.n_slot) * 8u;
+                }
+            }
+            uint32_t w_res = smem_desc_lo(b_base);
+            for (int cb = 0; cb < a.CB && alive; ++cb) {
+                alive = mbar_wait(bar_a_full + 8 * sa, pa, abort_flag, a.status);
                 if (!alive) break;
-                const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes);
-                for (int tap = 0; tap < T && alive; ++tap, ++ib) {
-                    const int sb = ib % a.b_stages;
-                    alive = mbar_wait(bar_b_full + 8 * sb, (ib / a.b_stages) & 1, abort_flag, a.status);
-                    if (!alive) break;
+                const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
+                const int ks = cb == a.CB - 1 ? a.ks_last : 4;           // K steps of 8 channels that hold real channels
+                uint32_t off = 0;
+                int y = 0;
+                for (int tap = 0; tap < T; ++tap) {
+                    uint32_t w_lo;
+                    if (a.b_resident) {
+                        w_lo = w_res; w_res += b_step;
+                    } else {
+                        alive = mbar_wait(bar_b_full + 8 * sb, pb, abort_flag, a.status);
+                        if (!alive) break;
+                        w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
+                    }
                     tc_fence_after();
-                    const int x = tap / a.FW, y = tap - x * a.FW;
-                    const uint32_t x_lo = x_stage + (uint32_t)(tl.a0 + x * a.Wq + y) * 8u;   // 128 bytes per pixel, >> 4
-                    const uint32_t w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
+                    const uint32_t x_lo = x_stage + off;
                     const uint32_t first = (cb | tap) == 0 ? 0u : 1u;
 #pragma unroll
-                    for (int j = 0; j < kSlots; ++j) {
-                        if (j < tl.slots && alive) {
-                            const uint32_t u = slot_uses + j;        // this slot's turn number
-                            const uint32_t s = u % kSlots;
-                            if (first == 0 && u >= kSlots) {         // its previous content must have left tensor memory
-                                alive = mbar_wait(bar_slot_free + 8 * s, (u / kSlots - 1) & 1, abort_flag, a.status);
-                                tc_fence_after();
-                            }
-                            if (alive && !a.pixel_m) {
-                                const uint32_t d = tmem + s * kSlotPx;
-                                const uint32_t xs = x_lo + (uint32_t)(j * tl.n_slot) * 8u;
-                                mma_tf32(d, w_lo, xs, kDescHi, idesc, first);
-                                mma_tf32(d, w_lo + 2u, xs + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
-                                mma_tf32(d, w_lo + 4u, xs + 4u, kDescHi, idesc, 1u);
-                                mma_tf32(d, w_lo + 6u, xs + 6u, kDescHi, idesc, 1u);
-                            } else if (alive) {
-                                // pixels on M: one MMA chain per 128-pixel chunk of the slot, D = [pixel][filter]
-                                const int px_slot = min(tl.n_slot, tl.px - j * tl.n_slot);
-                                for (int c = 0; c * 128 < px_slot; ++c) {
-                                    const uint32_t d = tmem + s * kSlotPx + (uint32_t)c * sw;
-                                    const uint32_t xs = x_lo + (uint32_t)(j * tl.n_slot + c * 128) * 8u;
-                                    mma_tf32(d, xs, w_lo, kDescHi, idesc, first);
-                                    mma_tf32(d, xs + 2u, w_lo + 2u, kDescHi, idesc, 1u);
-                                    mma_tf32(d, xs + 4u, w_lo + 4u, kDescHi, idesc, 1u);
-                                    mma_tf32(d, xs + 6u, w_lo + 6u, kDescHi, idesc, 1u);
-                                }
-                            }
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < chains) {
+                            const uint32_t xs = x_lo + xo[c];
+                            const uint32_t da = a.pixel_m ? xs : w_lo, db = a.pixel_m ? w_lo : xs;
+                            mma_tf32(acc[c], da, db, kDescHi, idesc, first);
+                            if (ks > 1) mma_tf32(acc[c], da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
+                            if (ks > 2) mma_tf32(acc[c], da + 4u, db + 4u, kDescHi, idesc, 1u);
+                            if (ks > 3) mma_tf32(acc[c], da + 6u, db + 6u, kDescHi, idesc, 1u);
                         }
                     }
-                    if (alive) mma_commit(bar_b_empty + 8 * sb);     // filter stage reusable once these MMAs have read it
+                    if (!a.b_resident) {
+                        mma_commit(bar_b_empty + 8 * sb);                // filter stage reusable once these MMAs have read it
+                        if (++sb == (uint32_t)a.b_stages) { sb = 0; pb ^= 1u; }
+                    }
+                    if (++y == a.FW) { y = 0; off += row_wrap; } else off += 8u;
                 }
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
+                if (++sa == (uint32_t)kAStages) { sa = 0; pa ^= 1u; }
             }
             if (alive)
                 for (int j = 0; j < tl.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
@@ -414,7 +448,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (a.pixel_m) {
                     // pixels on M: this thread owns one pixel of each 128-pixel chunk (tensor-memory lane = pixel) and
                     // reads 32 filters at a time = one whole 128-byte output line, stored as four 32-byte vectors
-                    const uint32_t sw = a.cps == 2 ? 128u : 256u;
+                    const uint32_t sw = 256u / (uint32_t)a.cps;
                     const int kb_tile = tl.n_tile * (a.w_tile / 32);
                     for (int c = 0; c * 128 < px_here; ++c) {
                         const int p = c * 128 + quarter * 32 + lane;            // pixel within the slot
@@ -498,6 +532,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tc_fence_before();
     }
     __syncthreads();
+    if (*abort_flag && armed_mask) {   // a role gave up: let the copies that are still in flight land before the CTA exits
+        for (int st = 0; st < 32; ++st)
+            if (armed_mask >> st & 1u)
+                for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(drain_bar + 8 * st, armed_parity >> st & 1u); ++it) __nanosleep(200);
+    }
+    __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem, (uint32_t)(kSlots * kSlotPx));
@@ -523,7 +563,8 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
     p.w_tile = pixel_m ? 256 : kFilterTile;
     p.n_tiles = ceil_div(Kp, p.w_tile);
     p.w_rows = Kp < p.w_tile ? Kp : p.w_tile;
-    p.cps = (pixel_m && p.w_rows <= 128) ? 2 : 1;
+    p.cps = !pixel_m ? 1 : p.w_rows <= 64 ? 4 : p.w_rows <= 128 ? 2 : 1;
+    p.ks_last = (g.C - (g.CB - 1) * 32 + 7) / 8;
     if (pixel_m && max_px > kSlots * p.cps * 128) return p;       // more pixels than the accumulator slots hold
     const long long pv = (long long)p.Hq * p.Wq;
     int a0max, slot_reach;
@@ -571,55 +612,74 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
     p.a_stage_bytes = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
     const size_t b_stage = ((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023;
     p.b_stage_bytes = (uint32_t)b_stage;
-    // shared memory: at least two strips and two filter tiles; then filter tiles up to one per tap plus two, then
-    // further strips (deeper prefetch across tiles, which is what the bandwidth-bound layers need), then the rest
+    // shared memory.  When one filter tile covers the layer and all its (channel block, tap) boxes fit beside enough
+    // strips, the filters are loaded once and stay; otherwise at least two strips and two filter boxes, then filter
+    // boxes up to one per tap plus two, then further strips (deeper prefetch across tiles, which is what the
+    // bandwidth-bound layers need), then the rest as filter boxes.
     const size_t fixed = 1024 + ctrl_bytes(g.KB);
-    if (fixed + 2 * (size_t)p.a_stage_bytes + 2 * b_stage > max_smem) return p;
-    size_t room = max_smem - fixed - 2 * (size_t)p.a_stage_bytes - 2 * b_stage;
-    p.a_stages = 2; p.b_stages = 2;
-    const int b_want = g.FH * g.FW + 2 < kMaxBStages ? g.FH * g.FW + 2 : kMaxBStages;
-    while (p.b_stages < b_want && room >= b_stage) { ++p.b_stages; room -= b_stage; }
-    while (p.a_stages < kMaxAStages && room >= p.a_stage_bytes) { ++p.a_stages; room -= p.a_stage_bytes; }
-    while (p.b_stages < kMaxBStages && room >= b_stage) { ++p.b_stages; room -= b_stage; }
+    const size_t all_b = (size_t)g.CB * g.FH * g.FW * b_stage;
+    p.b_resident = 0;
+    if (p.n_tiles == 1 && fixed + all_b + 2 * (size_t)p.a_stage_bytes <= max_smem) {
+        size_t fit = (max_smem - fixed - all_b) / p.a_stage_bytes;
+        if (fit > (size_t)kMaxAStages) fit = kMaxAStages;
+        const size_t want = g.CB + 1 < 4 ? g.CB + 1 : 4;
+        if (fit >= want) { p.b_resident = 1; p.a_stages = (int)fit; p.b_stages = g.CB * g.FH * g.FW; }
+    }
+    if (!p.b_resident) {
+        if (fixed + 2 * (size_t)p.a_stage_bytes + 2 * b_stage > max_smem) return p;
+        size_t room = max_smem - fixed - 2 * (size_t)p.a_stage_bytes - 2 * b_stage;
+        p.a_stages = 2; p.b_stages = 2;
+        const int b_want = g.FH * g.FW + 2 < kMaxBStages ? g.FH * g.FW + 2 : kMaxBStages;
+        while (p.b_stages < b_want && room >= b_stage) { ++p.b_stages; room -= b_stage; }
+        while (p.a_stages < kMaxAStages && room >= p.a_stage_bytes) { ++p.a_stages; room -= p.a_stage_bytes; }
+        while (p.b_stages < kMaxBStages && room >= b_stage) { ++p.b_stages; room -= b_stage; }
+    }
     p.smem_bytes = (uint32_t)(fixed + (size_t)p.a_stages * p.a_stage_bytes + (size_t)p.b_stages * b_stage);
     if ((long long)p.m_tiles * p.n_tiles > 0x7fffffffLL) return p;
     p.ok = true;
     return p;
 }
 
-// Estimated cycles of the whole layer under a plan, from measured rates: a 128 x N x 8 MMA takes about 119 cycles for
-// N <= 224 and 128 for N = 256.  The epilogue's stores run at memory speed in either orientation; what differs is how
-// many of the four epilogue warps have filters to store (filters on M: one warp per 32 filters of the tile) and the
-// instructions per pixel (about 20 cycles per pixel and warp with 4-byte stores, about 1.2 per pixel and 32 filters
-// with 32-byte vector stores).  Per tile the slowest of MMA issue, epilogue and L2 -> shared-memory traffic counts,
-// plus a hand-over cost and, when the strips of two tiles do not fit in the stages, the exposed load of one tile;
-// times the tiles the busiest SM gets.
+// Estimated cycles of the whole layer under a plan, from measured rates.  A 128 x N x 8 TF32 MMA occupies the pipe
+// for N / 2 cycles, with a floor of about 48; each tap costs the issuing thread some tens of cycles more (waiting for
+// and releasing a filter stage when the filters stream).  The epilogue's stores run at memory speed in either
+// orientation; what differs is how many of the four epilogue warps have filters to store (filters on M: one warp per
+// 32 filters of the tile) and the instructions per pixel (about 20 cycles per pixel and warp with 4-byte stores, about
+// 1.2 per pixel and 32 filters with 32-byte vector stores).  A tile that takes one accumulator slot overlaps its
+// epilogue with the next tile's MMAs (the slots alternate); a tile that takes both cannot.  Per tile the slowest of
+// MMA issue, epilogue and L2 -> shared-memory traffic counts, plus a hand-over cost and, when the strips of two tiles
+// do not fit in the stages, the exposed load of one tile; times the tiles the busiest SM gets.
 double plan_cost(const TcPlan &p, const Geom &g, int sms) {
-    const double steps = (double)g.CB * g.FH * g.FW;
+    const double taps = (double)g.FH * g.FW;
+    const double ksteps = (g.CB - 1) * 4.0 + p.ks_last;
     const double avg_px = p.nn == 1 ? (double)p.px_img / p.tiles_img : (double)p.px_tile;
     double mma, epi;
+    int slots;
     if (p.pixel_m) {
         const double chunks = (double)(long long)((avg_px + 127.0) / 128.0);
-        mma = steps * 4.0 * chunks * (p.w_rows / 2.0 > 119.0 ? p.w_rows / 2.0 : 119.0);
+        slots = p.px_tile > p.cps * 128 ? 2 : 1;
+        mma = taps * ksteps * chunks * (p.w_rows / 2.0 > 48.0 ? p.w_rows / 2.0 : 48.0);
         epi = avg_px * 1.2 * (p.w_rows / 32.0) + 300.0 * chunks;
     } else {
-        const int slots = p.px_tile > kSlotPx ? 2 : 1;
+        slots = p.px_tile > kSlotPx ? 2 : 1;
         const double n_slot = avg_px / slots;
-        mma = steps * 4.0 * slots * (n_slot / 2.0 > 119.0 ? n_slot / 2.0 : 119.0);
+        mma = taps * ksteps * slots * (n_slot / 2.0 > 48.0 ? n_slot / 2.0 : 48.0);
         const double warps = p.w_rows >= 128 ? 4.0 : p.w_rows / 32.0;
         epi = avg_px * 20.0 * 4.0 / warps;
     }
+    mma += taps * g.CB * (p.b_resident ? 40.0 : 120.0);
     const double strip_bytes = (double)g.CB * p.strip_px * 128.0;
-    const double bytes = strip_bytes + steps * p.w_rows * 128.0 + avg_px * 128.0 * (p.w_rows / 32.0);
+    const double bytes = strip_bytes + (p.b_resident ? 0.0 : taps * g.CB * p.w_rows * 128.0) + avg_px * 128.0 * (p.w_rows / 32.0);
     const double mem = bytes / 30.0;                 // bytes per clock one SM can expect when all SMs pull
     double tile = mma > mem ? mma : mem;
-    if (epi > tile) tile = epi;
-    tile += 2500.0;
+    if (slots == 2) tile += epi;
+    else if (epi > tile) tile = epi;
+    tile += 1500.0;
     if (p.a_stages < 2 * g.CB) tile += strip_bytes / 30.0 * 0.5;     // the next tile's strips cannot all be in flight
     const double tiles = (double)p.m_tiles * p.n_tiles;
     const double per_sm = tiles <= sms ? 1.0 : tiles / sms;
     const double waves = per_sm < 4.0 ? (double)(long long)(per_sm + 0.999) : per_sm;   // few tiles per SM: whole waves
-    return waves * tile;
+    return waves * tile + (p.b_resident ? g.CB * taps * p.w_rows * 128.0 / 30.0 : 0.0);
 }
 
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
@@ -702,6 +762,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
     a.a_stage_bytes = p.a_stage_bytes;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
+    a.b_resident = p.b_resident; a.ks_last = p.ks_last;
     a.relu = relu; a.accumulate = accumulate;
     cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
