@@ -35,6 +35,8 @@
 // tensor memory and returns.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace small {
@@ -76,6 +78,8 @@ struct TcArgs {
     int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
     int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
     int a_stages, b_stages, pixel_m, w_tile, cps, b_resident, ks_last;
+    int rows_tile;       // whole rows per tile when every tile starts at a row start, else 0
+    int slots, n_slot;   // accumulator slots per tile and pixels per slot: the same for every tile of the layer
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     int relu, accumulate;
 };
@@ -217,30 +221,33 @@ struct Tile { int n_tile, n0, q0, row0, a0, px, slots, n_slot; };
 
 __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
     Tile r;
-    r.n_tile = t % a.n_tiles;
-    const int m_tile = t / a.n_tiles;
+    // the common shapes (one filter tile, one tile per image, row-aligned tiles) need no division at all
+    int m_tile = t;
+    r.n_tile = 0;
+    if (a.n_tiles > 1) { m_tile = (int)((unsigned)t / (unsigned)a.n_tiles); r.n_tile = t - m_tile * a.n_tiles; }
     if (a.nn == 1) {
-        r.n0 = m_tile / a.tiles_img;
+        r.n0 = a.tiles_img > 1 ? (int)((unsigned)m_tile / (unsigned)a.tiles_img) : m_tile;
         const int ti = m_tile - r.n0 * a.tiles_img;
         r.q0 = ti * a.px_tile;
         r.px = min(a.px_tile, a.px_img - r.q0);
-        r.row0 = r.q0 / a.Wq;
-        r.a0 = r.q0 - r.row0 * a.Wq;
+        if (a.rows_tile > 0) { r.row0 = ti * a.rows_tile; r.a0 = 0; }
+        else { r.row0 = (int)((unsigned)r.q0 / (unsigned)a.Wq); r.a0 = r.q0 - r.row0 * a.Wq; }
     } else {
         r.n0 = m_tile * a.nn;
         r.q0 = 0; r.row0 = 0; r.a0 = 0;
         r.px = a.px_tile;
     }
-    if (a.pixel_m) {                       // slots hold cps chunks of 128 pixels
-        r.n_slot = a.cps * 128;
-        r.slots = r.px > r.n_slot ? 2 : 1;
-    } else {
-        r.slots = r.px > kSlotPx ? 2 : 1;
-        r.n_slot = ((r.px + r.slots - 1) / r.slots + 15) & ~15;
-    }
+    // every tile takes the slots of a full tile; a ragged last tile leaves the tail of them unused
+    r.slots = a.slots;
+    r.n_slot = a.n_slot;
     return r;
 }
 
+// CH: MMA chains per tile (accumulator slots with filters on M, 128-pixel chunks with pixels on M); KS_LAST: K steps
+// of the last channel block that hold real channels (1, 2 or 4); PM: pixels on the MMA's M axis.  They are template
+// parameters so that the single issuing thread runs straight-line code: with run-time chain and K-step counts every
+// MMA costs it about 100 cycles of branches and selects, more than a small MMA occupies the pipe (measured).
+template <int CH, int KS_LAST, bool PM>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -277,7 +284,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int i = threadIdx.x; i < a.tail_px * 8; i += kThreads) tail[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     // filter rows the TMA box does not cover (fewer than 128 filters in the layer) stay zero for the whole kernel
-    if (!a.pixel_m && a.w_rows < kFilterTile)
+    if (!PM && a.w_rows < kFilterTile)
         for (int s = 0; s < a.b_stages; ++s) {
             float4 *rest = reinterpret_cast<float4 *>(base_ptr + (b_base - base) + (size_t)s * kBStageBytes + (size_t)a.w_rows * 128);
             for (int i = threadIdx.x; i < (kFilterTile - a.w_rows) * 8; i += kThreads) rest[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -349,38 +356,64 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t slot_uses = 0;                   // slots taken so far; slot j of a tile is (slot_uses + j) % 2
         const uint32_t b_step = kBStageBytes >> 4;
         const uint32_t row_wrap = (uint32_t)(a.Wq - a.FW + 1) * 8u;     // tap offset step from the end of a window row
-        const uint32_t sw = 256u / (uint32_t)a.cps;                     // pixel_m: tensor-memory columns per chunk
-        const int cps_log2 = a.cps == 4 ? 2 : a.cps == 2 ? 1 : 0;
+        // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
+        const uint32_t idesc = instr_desc(PM ? a.w_rows : a.n_slot);
+        // strip offset (in 16-byte units) of each MMA chain of a tile: one per slot or one per 128-pixel chunk
+        uint32_t xo[CH];
+#pragma unroll
+        for (int c = 0; c < CH; ++c) xo[c] = (uint32_t)(c * (PM ? 128 : a.n_slot)) * 8u;
         if (a.b_resident) alive = mbar_wait(bar_b_full, 0, abort_flag, a.status);
+
+        // all taps of one channel block with KS K-steps each; straight-line MMA issue
+        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const bool first_block, uint32_t &w_res) {
+            constexpr int KS = decltype(ks_tag)::value;
+            uint32_t off = 0;
+            int y = 0;
+            for (int tap = 0; tap < T; ++tap) {
+                uint32_t w_lo;
+                if (a.b_resident) {
+                    w_lo = w_res; w_res += b_step;
+                } else {
+                    alive = mbar_wait(bar_b_full + 8 * sb, pb, abort_flag, a.status);
+                    if (!alive) return;
+                    w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
+                }
+                const uint32_t x_lo = x_stage + off;
+                const uint32_t first = (first_block && tap == 0) ? 0u : 1u;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const uint32_t xs = x_lo + xo[c];
+                    const uint32_t da = PM ? xs : w_lo, db = PM ? w_lo : xs;
+                    mma_tf32(acc[c], da, db, kDescHi, idesc, first);
+                    if (KS > 1) mma_tf32(acc[c], da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
+                    if (KS > 2) mma_tf32(acc[c], da + 4u, db + 4u, kDescHi, idesc, 1u);
+                    if (KS > 3) mma_tf32(acc[c], da + 6u, db + 6u, kDescHi, idesc, 1u);
+                }
+                if (!a.b_resident) {
+                    mma_commit(bar_b_empty + 8 * sb);                // filter stage reusable once these MMAs have read it
+                    if (++sb == (uint32_t)a.b_stages) { sb = 0; pb ^= 1u; }
+                }
+                if (++y == a.FW) { y = 0; off += row_wrap; } else off += 8u;
+            }
+        };
+
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
-            // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
-            const uint32_t idesc = instr_desc(a.pixel_m ? a.w_rows : tl.n_slot);
             // the previous content of the slots this tile takes must have left tensor memory
-            for (int j = 0; j < tl.slots && alive; ++j) {
+            for (int j = 0; j < a.slots && alive; ++j) {
                 const uint32_t u = slot_uses + j;
                 if (u >= kSlots) alive = mbar_wait(bar_slot_free + 8 * (u % kSlots), (u / kSlots - 1) & 1, abort_flag, a.status);
             }
             if (!alive) break;
             tc_fence_after();
-            // accumulator address and strip offset (in 16-byte units) of each MMA chain of the tile: one per slot
-            // (filters on M) or one per 128-pixel chunk (pixels on M)
-            uint32_t acc[4], xo[4];
-            int chains;
-            if (a.pixel_m) {
-                chains = (tl.px + 127) >> 7;
+            uint32_t acc[CH];                     // accumulator address of each chain
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int j = c >> cps_log2;
-                    acc[c] = tmem + ((slot_uses + j) % kSlots) * kSlotPx + (uint32_t)(c - j * a.cps) * sw;
-                    xo[c] = (uint32_t)c * 128u * 8u;
-                }
-            } else {
-                chains = tl.slots;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < CH; ++c) {
+                if (PM) {
+                    const int j = c / a.cps;
+                    acc[c] = tmem + ((slot_uses + j) % kSlots) * kSlotPx + (uint32_t)(c - j * a.cps) * (256u / (uint32_t)a.cps);
+                } else {
                     acc[c] = tmem + ((slot_uses + c) % kSlots) * kSlotPx;
-                    xo[c] = (uint32_t)(c * tl.n_slot) * 8u;
                 }
             }
             uint32_t w_res = smem_desc_lo(b_base);
@@ -388,44 +421,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 alive = mbar_wait(bar_a_full + 8 * sa, pa, abort_flag, a.status);
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
-                const int ks = cb == a.CB - 1 ? a.ks_last : 4;           // K steps of 8 channels that hold real channels
-                uint32_t off = 0;
-                int y = 0;
-                for (int tap = 0; tap < T; ++tap) {
-                    uint32_t w_lo;
-                    if (a.b_resident) {
-                        w_lo = w_res; w_res += b_step;
-                    } else {
-                        alive = mbar_wait(bar_b_full + 8 * sb, pb, abort_flag, a.status);
-                        if (!alive) break;
-                        w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
-                    }
-                    tc_fence_after();
-                    const uint32_t x_lo = x_stage + off;
-                    const uint32_t first = (cb | tap) == 0 ? 0u : 1u;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < chains) {
-                            const uint32_t xs = x_lo + xo[c];
-                            const uint32_t da = a.pixel_m ? xs : w_lo, db = a.pixel_m ? w_lo : xs;
-                            mma_tf32(acc[c], da, db, kDescHi, idesc, first);
-                            if (ks > 1) mma_tf32(acc[c], da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
-                            if (ks > 2) mma_tf32(acc[c], da + 4u, db + 4u, kDescHi, idesc, 1u);
-                            if (ks > 3) mma_tf32(acc[c], da + 6u, db + 6u, kDescHi, idesc, 1u);
-                        }
-                    }
-                    if (!a.b_resident) {
-                        mma_commit(bar_b_empty + 8 * sb);                // filter stage reusable once these MMAs have read it
-                        if (++sb == (uint32_t)a.b_stages) { sb = 0; pb ^= 1u; }
-                    }
-                    if (++y == a.FW) { y = 0; off += row_wrap; } else off += 8u;
-                }
+                if (cb == a.CB - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, cb == 0, w_res);
+                else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, cb == 0, w_res);
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
                 if (++sa == (uint32_t)kAStages) { sa = 0; pa ^= 1u; }
             }
             if (alive)
-                for (int j = 0; j < tl.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
-            slot_uses += tl.slots;
+                for (int j = 0; j < a.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
+            slot_uses += a.slots;
         }
     } else if (warp >= 4) {
         // ---- epilogue: warp q owns tensor-memory lanes 32q.. = filters 32q.. of the tile; lane = filter, column = pixel
@@ -445,7 +448,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!alive) break;
                 tc_fence_after();
                 const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
-                if (a.pixel_m) {
+                if (PM) {
                     // pixels on M: this thread owns one pixel of each 128-pixel chunk (tensor-memory lane = pixel) and
                     // reads 32 filters at a time = one whole 128-byte output line, stored as four 32-byte vectors
                     const uint32_t sw = 256u / (uint32_t)a.cps;
@@ -697,6 +700,29 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32) {
     return best;
 }
 
+typedef void (*TcKernel)(const CUtensorMap, const CUtensorMap, const TcArgs);
+
+template <int CH, bool PM>
+TcKernel pick_ks(int ks) {
+    switch (ks) {
+        case 1: return conv_tc_kernel<CH, 1, PM>;
+        case 2: return conv_tc_kernel<CH, 2, PM>;
+        case 4: return conv_tc_kernel<CH, 4, PM>;
+        default: return nullptr;
+    }
+}
+// Filters on M: one chain per accumulator slot (1 or 2); pixels on M: one per 128-pixel chunk (1 to 4).
+TcKernel pick_kernel(int chains, int ks, bool pixel_m) {
+    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks) : chains == 2 ? pick_ks<2, false>(ks) : nullptr;
+    switch (chains) {
+        case 1: return pick_ks<1, true>(ks);
+        case 2: return pick_ks<2, true>(ks);
+        case 3: return pick_ks<3, true>(ks);
+        case 4: return pick_ks<4, true>(ks);
+        default: return nullptr;
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -763,12 +789,26 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.a_stage_bytes = p.a_stage_bytes;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
+    a.rows_tile = (p.nn == 1 && p.px_tile % p.Wq == 0) ? p.px_tile / p.Wq : 0;
+    int chains;
+    if (p.pixel_m) {
+        a.n_slot = p.cps * 128;
+        a.slots = p.px_tile > a.n_slot ? 2 : 1;
+        chains = ceil_div(p.px_tile, 128);
+    } else {
+        a.slots = p.px_tile > kSlotPx ? 2 : 1;
+        a.n_slot = ((p.px_tile + a.slots - 1) / a.slots + 15) & ~15;
+        chains = a.slots;
+    }
+    const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
     a.relu = relu; a.accumulate = accumulate;
-    cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0);
+    if (!kern) return SMALL_ERR_UNSUPPORTED;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
-    conv_tc_kernel<<<grid, kThreads, p.smem_bytes, st>>>(map_a, map_b, a);
+    kern<<<grid, kThreads, p.smem_bytes, st>>>(map_a, map_b, a);
     return check_launch(ctx);
 }
 
