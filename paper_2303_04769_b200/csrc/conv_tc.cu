@@ -51,6 +51,7 @@ constexpr int kMaxAStages = 6;         // input strips in flight (at least 2; as
 constexpr int kMaxBStages = 8;
 constexpr uint32_t kWaitIters = 1u << 22;   // bounded wait: polls back off with nanosleep, so this is seconds
 constexpr int kCtrlBarrierBytes = 16 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
+constexpr int kTapTabEntries = 4 * 64;   // original tap of every (phase plane, view tap), -1 where the view tap has none
 
 struct TcPlan {
     int OH, OW, Wq, Hq;
@@ -68,6 +69,7 @@ struct TcPlan {
     int w_tile;          // filters per tile: 128 (filters on M) or up to 256 (filters on N)
     int cps;             // pixel_m: 128-pixel chunks per accumulator slot (4, 2 or 1 for up to 64, 128 or 256 filters)
     int b_resident;      // all filter tiles of the layer stay in shared memory for the whole kernel
+    double taps_eff;     // taps per block that exist (a stride-2 view has empty ones)
     int ks_last;         // K steps (8 channels each) of the last channel block that hold real channels
     uint32_t a_stage_bytes, b_stage_bytes, smem_bytes;
     bool ok;
@@ -75,7 +77,8 @@ struct TcPlan {
 
 struct TcArgs {
     const float *bias; float *out; int *status;
-    int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;
+    int N, K, KB, CB, OH, OW, Wq, Hq, FH, FW, pt, pl;   // CB, FH, FW, pt, pl: the stride-1 view (see Virt)
+    int S, n_phase, CBr, phase_bits, FHo, FWo, pto, plo;  // stride, phase planes, real channel blocks, original window
     int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
     int a_stages, b_stages, pixel_m, w_tile, cps, b_resident, ks_last;
     int rows_tile;       // whole rows per tile when every tile starts at a row start, else 0
@@ -266,6 +269,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
     float *bias_s = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16);
+    volatile short *tap_tab = reinterpret_cast<volatile short *>(ctrl_ptr + kCtrlBarrierBytes + 16 + (size_t)a.KB * 32 * 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = a.FH * a.FW;
@@ -290,6 +294,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int i = threadIdx.x; i < (kFilterTile - a.w_rows) * 8; i += kThreads) rest[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
     for (int i = threadIdx.x; i < a.KB * 32; i += kThreads) bias_s[i] = (a.bias && i < a.K) ? a.bias[i] : 0.0f;
+    // view tap (x', y') of phase plane (ph, pw) is the original tap x = S (x' - pt') + ph + pt, y likewise, if it exists
+    for (int i = threadIdx.x; i < a.n_phase * T; i += kThreads) {
+        const int p = i / T, tv = i - p * T, xv = tv / a.FW, yv = tv - xv * a.FW;
+        const int x = a.S * (xv - a.pt) + ((a.phase_bits >> (2 * p)) & 1) + a.pto;
+        const int y = a.S * (yv - a.pl) + ((a.phase_bits >> (2 * p + 1)) & 1) + a.plo;
+        tap_tab[i] = (short)((x >= 0 && x < a.FHo && y >= 0 && y < a.FWo) ? x * a.FWo + y : -1);
+    }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy zeros visible to the tensor core
     if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), (uint32_t)(kSlots * kSlotPx));
     tc_fence_before();
@@ -312,14 +323,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t s = 0, phase = 0;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
-            for (int cb = 0; cb < a.CB; ++cb) {
-                if (wrapped) alive = mbar_wait(bar_a_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
-                if (!alive) break;
-                mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
-                tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, -a.pl, tl.row0 - a.pt, cb, tl.n0);
-                armed_mask |= 1u << s;
-                armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
-                if (++s == (uint32_t)kAStages) { s = 0; phase ^= 1u; wrapped = true; }
+            // one box per (phase plane, real channel block); with stride 2 the map's element strides pick every
+            // other row and column, starting at the plane's parity
+            const int c1 = a.S * (-a.pl), c2 = a.S * (tl.row0 - a.pt);
+            for (int p = 0; p < a.n_phase && alive; ++p) {
+                const int ph = (a.phase_bits >> (2 * p)) & 1, pw = (a.phase_bits >> (2 * p + 1)) & 1;
+                for (int cb = 0; cb < a.CBr; ++cb) {
+                    if (wrapped) alive = mbar_wait(bar_a_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                    if (!alive) break;
+                    mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
+                    tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, c1 + pw, c2 + ph, cb, tl.n0);
+                    armed_mask |= 1u << s;
+                    armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
+                    if (++s == (uint32_t)kAStages) { s = 0; phase ^= 1u; wrapped = true; }
+                }
             }
         }
     } else if (warp == 2 && lane == 0) {
@@ -327,26 +344,35 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         drain_bar = bar_b_full;
         const uint32_t box_bytes = (uint32_t)a.w_rows * 128u;
         if (a.b_resident) {
-            mbar_expect_tx(bar_b_full, box_bytes * (uint32_t)(a.CB * T));
+            int boxes = 0;
+            for (int i = 0; i < a.n_phase * T; ++i) boxes += tap_tab[i] >= 0 ? 1 : 0;
+            mbar_expect_tx(bar_b_full, box_bytes * (uint32_t)(boxes * a.CBr));
             uint32_t dst = b_base;
-            for (int cb = 0; cb < a.CB; ++cb)
-                for (int tap = 0; tap < T; ++tap, dst += kBStageBytes) tma_load_4d(dst, &map_b, bar_b_full, 0, 0, tap, cb);
+            for (int p = 0; p < a.n_phase; ++p)
+                for (int cb = 0; cb < a.CBr; ++cb)
+                    for (int tap = 0; tap < T; ++tap, dst += kBStageBytes) {
+                        const int orig = tap_tab[p * T + tap];
+                        if (orig >= 0) tma_load_4d(dst, &map_b, bar_b_full, 0, 0, orig, cb);
+                    }
             armed_mask = 1u;
         } else {
             bool alive = true, wrapped = false;
             uint32_t s = 0, phase = 0;
             for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
                 const int row = (t % a.n_tiles) * a.w_tile;
-                for (int cb = 0; cb < a.CB && alive; ++cb)
-                    for (int tap = 0; tap < T; ++tap) {
-                        if (wrapped) alive = mbar_wait(bar_b_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
-                        if (!alive) break;
-                        mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
-                        tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, row, tap, cb);
-                        armed_mask |= 1u << s;
-                        armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
-                        if (++s == (uint32_t)a.b_stages) { s = 0; phase ^= 1u; wrapped = true; }
-                    }
+                for (int p = 0; p < a.n_phase && alive; ++p)
+                    for (int cb = 0; cb < a.CBr && alive; ++cb)
+                        for (int tap = 0; tap < T; ++tap) {
+                            const int orig = tap_tab[p * T + tap];
+                            if (orig < 0) continue;
+                            if (wrapped) alive = mbar_wait(bar_b_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                            if (!alive) break;
+                            mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
+                            tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, row, orig, cb);
+                            armed_mask |= 1u << s;
+                            armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
+                            if (++s == (uint32_t)a.b_stages) { s = 0; phase ^= 1u; wrapped = true; }
+                        }
             }
         }
     } else if (warp == 1 && lane == 0) {
@@ -365,12 +391,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (a.b_resident) alive = mbar_wait(bar_b_full, 0, abort_flag, a.status);
 
         // all taps of one channel block with KS K-steps each; straight-line MMA issue
-        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const bool first_block, uint32_t &w_res) {
+        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const volatile short *taps, uint32_t &started, uint32_t &w_res) {
             constexpr int KS = decltype(ks_tag)::value;
             uint32_t off = 0;
             int y = 0;
             for (int tap = 0; tap < T; ++tap) {
                 uint32_t w_lo;
+                if (taps[tap] < 0) {             // the view has no such tap in this phase plane
+                    if (a.b_resident) w_res += b_step;
+                    if (++y == a.FW) { y = 0; off += row_wrap; } else off += 8u;
+                    continue;
+                }
                 if (a.b_resident) {
                     w_lo = w_res; w_res += b_step;
                 } else {
@@ -379,7 +410,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
                 }
                 const uint32_t x_lo = x_stage + off;
-                const uint32_t first = (first_block && tap == 0) ? 0u : 1u;
+                const uint32_t first = started;   // 0 for the first MMAs of the tile: they overwrite the accumulator
+                started = 1u;
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
                     const uint32_t xs = x_lo + xo[c];
@@ -416,15 +448,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     acc[c] = tmem + ((slot_uses + c) % kSlots) * kSlotPx;
                 }
             }
-            uint32_t w_res = smem_desc_lo(b_base);
-            for (int cb = 0; cb < a.CB && alive; ++cb) {
+            uint32_t w_res = smem_desc_lo(b_base), started = 0;
+            int cb = 0;
+            const volatile short *taps = tap_tab;
+            for (int blk = 0; blk < a.CB && alive; ++blk) {       // blocks = phase planes x real channel blocks
                 alive = mbar_wait(bar_a_full + 8 * sa, pa, abort_flag, a.status);
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
-                if (cb == a.CB - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, cb == 0, w_res);
-                else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, cb == 0, w_res);
+                if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, started, w_res);
+                else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, taps, started, w_res);
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
                 if (++sa == (uint32_t)kAStages) { sa = 0; pa ^= 1u; }
+                if (++cb == a.CBr) { cb = 0; taps += T; }
             }
             if (alive)
                 for (int j = 0; j < a.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
@@ -548,19 +583,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 // ---------------------------------------------------------------------------------------------- host side
-size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4; }
+size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + kTapTabEntries * sizeof(short); }
 
 // Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff) {
     TcPlan p{};
     p.ok = false;
-    if (g.S != 1) return p;
+    if (g.S != 1) return p;                      // g is the stride-1 view; S scales the TMA box of the real tensor
+    p.taps_eff = taps_eff;
     p.OH = g.OH; p.OW = g.OW;
     const int padw = g.pl > g.pr ? g.pl : g.pr, padh = g.pt > g.pb ? g.pt : g.pb;
     const int minw = g.pl < g.pr ? g.pl : g.pr, minh = g.pt < g.pb ? g.pt : g.pb;
     p.Wq = g.W + padw;
     p.Hq = g.H + padh;
-    if (p.Wq > 256 || g.FH * g.FW > 64) return p;
+    if (p.Wq * S > 256 || g.FH * g.FW > 64) return p;
     const int Kp = g.KB * 32;
     p.pixel_m = pixel_m;
     p.w_tile = pixel_m ? 256 : kFilterTile;
@@ -571,7 +607,7 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
     if (pixel_m && max_px > kSlots * p.cps * 128) return p;       // more pixels than the accumulator slots hold
     const long long pv = (long long)p.Hq * p.Wq;
     int a0max, slot_reach;
-    if (pv <= max_px && p.Hq <= 256) {
+    if (pv <= max_px && p.Hq * S <= 256) {
         // whole images per strip: as many as fill the tile (at least one)
         p.nn = (int)(max_px / pv);
         if (p.nn > 256) p.nn = 256;
@@ -596,7 +632,7 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
         p.tiles_img = ceil_div(p.px_img, p.px_tile);
         const bool row_aligned = p.px_tile % p.Wq == 0;             // every tile starts at a row start
         p.Rs = row_aligned ? p.px_tile / p.Wq + g.FH - 1 : (p.Wq - 1 + p.px_tile - 1) / p.Wq + 1 + g.FH - 1;
-        if (p.Rs > 256) return p;
+        if (p.Rs * S > 256) return p;
         p.m_tiles = g.N * p.tiles_img;
         p.tail_px = minw;
         p.strip_px = p.Rs * p.Wq;
@@ -653,7 +689,7 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m) {
 // MMA issue, epilogue and L2 -> shared-memory traffic counts, plus a hand-over cost and, when the strips of two tiles
 // do not fit in the stages, the exposed load of one tile; times the tiles the busiest SM gets.
 double plan_cost(const TcPlan &p, const Geom &g, int sms) {
-    const double taps = (double)g.FH * g.FW;
+    const double taps = p.taps_eff;
     const double ksteps = (g.CB - 1) * 4.0 + p.ks_last;
     const double avg_px = p.nn == 1 ? (double)p.px_img / p.tiles_img : (double)p.px_tile;
     double mma, epi;
@@ -687,12 +723,12 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
 
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
 // fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
-TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32) {
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff) {
     TcPlan best{};
     double best_cost = 0.0;
     for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
         for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-            TcPlan p = make_plan_with(g, max_smem, px, pixel_m);
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff);
             if (!p.ok) continue;
             const double c = plan_cost(p, g, sms);
             if (!best.ok || c < best_cost) { best = p; best_cost = c; }
@@ -745,32 +781,79 @@ static Geom flatten_pointwise(const Geom &g) {
     return f;
 }
 
+// The stride-1 view of a layer.  A stride-2 window over X is a stride-1 window over X's four phase planes
+// P(ph,pw)[i][j] = X[2i+ph][2j+pw]: tap x of the original window reads row 2 oh + x - pt = 2 (oh + dh) + ph with
+// ph = (x - pt) mod 2 and dh = floor((x - pt) / 2), i.e. row oh + dh of plane ph.  So the layer becomes a stride-1
+// convolution with window (dh_max - dh_min + 1), top pad -dh_min, and n_phase x CB "channel blocks", one per (phase
+// plane, real block); view taps that no original tap maps to are skipped.  TMA reads a phase plane straight from the
+// blocked tensor with element strides 2, so nothing is reformatted.  (Stride 1: the view is the layer itself.)
+struct Virt { Geom g; int S, n_phase, CBr, phase_bits, FHo, FWo, pto, plo; double taps_eff; };
+
+static int floor_half(int v) { return v >= 0 ? v / 2 : -((1 - v) / 2); }
+
+static bool make_virt(const Geom &g_in, Virt &v) {
+    v.S = g_in.S; v.FHo = g_in.FH; v.FWo = g_in.FW; v.pto = g_in.pt; v.plo = g_in.pl; v.CBr = g_in.CB;
+    if (g_in.S == 1) {
+        v.g = flatten_pointwise(g_in);
+        v.n_phase = 1; v.phase_bits = 0; v.taps_eff = (double)g_in.FH * g_in.FW;
+        return true;
+    }
+    if (g_in.S != 2) return false;
+    const int dh0 = floor_half(-g_in.pt), dh1 = floor_half(g_in.FH - 1 - g_in.pt);
+    const int dw0 = floor_half(-g_in.pl), dw1 = floor_half(g_in.FW - 1 - g_in.pl);
+    bool has_h[2] = {false, false}, has_w[2] = {false, false};
+    for (int x = 0; x < g_in.FH; ++x) has_h[(x - g_in.pt) & 1] = true;
+    for (int y = 0; y < g_in.FW; ++y) has_w[(y - g_in.pl) & 1] = true;
+    v.n_phase = 0; v.phase_bits = 0;
+    for (int ph = 0; ph < 2; ++ph)
+        for (int pw = 0; pw < 2; ++pw)
+            if (has_h[ph] && has_w[pw]) { v.phase_bits |= (ph | (pw << 1)) << (2 * v.n_phase); ++v.n_phase; }
+    Geom g = g_in;
+    g.S = 1;
+    g.FH = dh1 - dh0 + 1; g.FW = dw1 - dw0 + 1;
+    g.pt = -dh0; g.pl = -dw0; g.pb = 0; g.pr = 0;
+    g.H = g_in.OH + g.FH - 1 - g.pt; g.W = g_in.OW + g.FW - 1 - g.pl;     // rows and columns of a plane that outputs reach
+    if (g.H < 1 || g.W < 1 || g.pt < 0 || g.pl < 0) return false;
+    g.CB = v.n_phase * g_in.CB;
+    g.C = (g.CB - 1) * 32 + (g_in.C - (g_in.CB - 1) * 32);                  // keeps the K steps of the last real block
+    v.g = g;
+    v.taps_eff = (double)g_in.FH * g_in.FW / v.n_phase;
+    return g.FH * g.FW <= 64;
+}
+
 bool conv_tc_supported(const Geom &g) {
-    return make_plan(flatten_pointwise(g), 227 * 1024, 148, false).ok;
+    Virt v;
+    return make_virt(g, v) && make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
     (void)w_lo; (void)mode;
-    const Geom g = flatten_pointwise(g_in);
+    Virt v;
+    if (!make_virt(g_in, v)) return SMALL_ERR_UNSUPPORTED;
+    const Geom &g = v.g;
     TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
-                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0);
+                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_a, map_b;
     {   // activations: [N][CB][H][W][32 floats]; box = 32 x Wq x Rs x 1 x nn, out-of-range elements read as zero
-        cuuint64_t dims[5] = {32, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.CB, (cuuint64_t)g.N};
-        cuuint64_t strides[4] = {128, (cuuint64_t)g.W * 128, (cuuint64_t)g.H * g.W * 128, (cuuint64_t)g.CB * g.H * g.W * 128};
-        cuuint32_t box[5] = {32, (cuuint32_t)p.Wq, (cuuint32_t)p.Rs, 1, (cuuint32_t)p.nn};
-        cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        // the real tensor (for stride 1 possibly with a 1x1 layer's rows re-cut); with stride 2 the box spans 2 Wq x 2 Rs
+        // elements and the element strides keep every other one, so shared memory receives Wq x Rs pixels either way
+        const int Hr = v.S == 1 ? g.H : g_in.H, Wr = v.S == 1 ? g.W : g_in.W;
+        const cuuint32_t es = (cuuint32_t)v.S;
+        cuuint64_t dims[5] = {32, (cuuint64_t)Wr, (cuuint64_t)Hr, (cuuint64_t)v.CBr, (cuuint64_t)g.N};
+        cuuint64_t strides[4] = {128, (cuuint64_t)Wr * 128, (cuuint64_t)Hr * Wr * 128, (cuuint64_t)v.CBr * Hr * Wr * 128};
+        cuuint32_t box[5] = {32, (cuuint32_t)p.Wq * es, (cuuint32_t)p.Rs * es, 1, (cuuint32_t)p.nn};
+        cuuint32_t estr[5] = {1, es, es, 1, 1};
         CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float *>(in), dims, strides, box, estr,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
     }
     {   // filters: [CB][FH*FW][KB*32][32 floats]; box = 32 x min(128, KB*32) rows
-        const int T = g.FH * g.FW, Kp = g.KB * 32;
-        cuuint64_t dims[4] = {32, (cuuint64_t)Kp, (cuuint64_t)T, (cuuint64_t)g.CB};
+        const int T = v.FHo * v.FWo, Kp = g.KB * 32;
+        cuuint64_t dims[4] = {32, (cuuint64_t)Kp, (cuuint64_t)T, (cuuint64_t)v.CBr};
         cuuint64_t strides[3] = {128, (cuuint64_t)Kp * 128, (cuuint64_t)T * Kp * 128};
         cuuint32_t box[4] = {32, (cuuint32_t)p.w_rows, 1, 1};
         cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -783,6 +866,8 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.bias = bias; a.out = out; a.status = ctx->dev_status;
     a.N = g.N; a.K = g.K; a.KB = g.KB; a.CB = g.CB; a.OH = g.OH; a.OW = g.OW; a.Wq = p.Wq; a.Hq = p.Hq;
     a.FH = g.FH; a.FW = g.FW; a.pt = g.pt; a.pl = g.pl;
+    a.S = v.S; a.n_phase = v.n_phase; a.CBr = v.CBr; a.phase_bits = v.phase_bits;
+    a.FHo = v.FHo; a.FWo = v.FWo; a.pto = v.S == 1 ? g.pt : v.pto; a.plo = v.S == 1 ? g.pl : v.plo;
     a.nn = p.nn; a.px_tile = p.px_tile; a.px_img = p.px_img; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
     a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
     a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;

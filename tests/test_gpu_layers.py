@@ -252,3 +252,43 @@ def test_conv_tf32_tensor_cores(case):
     out2 = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out2, N, C, K, H, W, FH, FW, 1, pad, B.RELU | B.MATH_TF32)
     assert torch.equal(out.view(torch.int32), out2.view(torch.int32))
+
+
+CONV_TC_STRIDE2_CASES = [  # N, C, K, H, W, FH, FW, pad  (stride 2: read as a stride-1 window over the input's four phase planes)
+    (3, 16, 32, 32, 32, 3, 3, (1, 1, 1, 1)),       # the residual network's downsampling convolutions
+    (3, 16, 32, 32, 32, 1, 1, (0, 0, 0, 0)),       # and its 1x1 shortcut: a single phase plane
+    (2, 32, 64, 16, 16, 3, 3, (1, 1, 1, 1)),
+    (2, 3, 8, 96, 96, 3, 3, (1, 1, 1, 1)),         # depthwise-separable stem
+    (5, 1, 64, 49, 10, 10, 4, (4, 5, 1, 1)),       # keyword-spotting stem: tall window, odd height, asymmetric pads
+    (2, 70, 45, 17, 19, 3, 3, (0, 1, 1, 0)),       # odd planes, ragged channels, pads on one side only
+    (2, 40, 40, 15, 15, 2, 2, (0, 0, 0, 0)),       # window = stride: every phase plane has one tap
+    (3, 64, 64, 9, 9, 5, 5, (2, 2, 2, 2)),
+    (2, 32, 32, 31, 33, 1, 1, (0, 0, 0, 0)),
+    (2, 32, 300, 12, 12, 3, 3, (1, 0, 0, 1)),      # two filter tiles
+]
+
+
+@pytest.mark.parametrize("case", CONV_TC_STRIDE2_CASES)
+def test_conv_tf32_tensor_cores_stride2(case):
+    N, C, K, H, W, FH, FW, pad = case
+    x, w, b = rnd((N, C, H, W), 26), rnd((K, C, FH, FW), 27), rnd((K,), 28)
+    wb = torch.empty(B.small_conv_weight_elems(C, K, FH, FW, B.MATH_TF32), device="cuda")
+    B.small_pack_conv_weights(ctx(), dev(w), wb, C, K, FH, FW, B.MATH_TF32)
+    bx = to_blk(x)
+    ref = oracle.conv2d(x, w, b, 2, pad, relu=True)
+    OH, OW = ref.shape[2:]
+    assert B.small_conv2d_uses_tensor_cores(N, C, K, H, W, FH, FW, 2, pad)
+    out = new_blk(N, K, OH, OW)
+    B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, 2, pad, B.RELU | B.MATH_TF32)
+    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    assert B.small_device_status(ctx()) == 0
+    assert 1e-7 < err <= 2e-3, err
+    assert pad_lanes_are_zero(out, N, K, OH, OW)
+    prev = rnd((N, K, OH, OW), 29)
+    acc = to_blk(prev)
+    B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, 2, pad, B.ACCUMULATE | B.MATH_TF32)
+    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, 2, pad, accumulate_into=prev)) <= 2e-3
+    # the FP32 mode of the same layer stays within its own bound
+    out32 = new_blk(N, K, OH, OW)
+    B.small_conv2d(ctx(), bx, wb, dev(b), out32, N, C, K, H, W, FH, FW, 2, pad, B.RELU | B.MATH_FP32)
+    assert rel_l2(from_blk(out32, N, K, OH, OW), ref) <= 1e-5
