@@ -247,10 +247,11 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
 }
 
 // CH: MMA chains per tile (accumulator slots with filters on M, 128-pixel chunks with pixels on M); KS_LAST: K steps
-// of the last channel block that hold real channels (1, 2 or 4); PM: pixels on the MMA's M axis.  They are template
+// of the last channel block that hold real channels (1, 2 or 4); PM: pixels on the MMA's M axis;
+// MASKED: some view taps do not exist (stride-2 layers).  They are template
 // parameters so that the single issuing thread runs straight-line code: with run-time chain and K-step counts every
 // MMA costs it about 100 cycles of branches and selects, more than a small MMA occupies the pipe (measured).
-template <int CH, int KS_LAST, bool PM>
+template <int CH, int KS_LAST, bool PM, bool MASKED>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -391,13 +392,22 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (a.b_resident) alive = mbar_wait(bar_b_full, 0, abort_flag, a.status);
 
         // all taps of one channel block with KS K-steps each; straight-line MMA issue
-        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const volatile short *taps, uint32_t &started, uint32_t &w_res) {
+        // bit t set: view tap t of the phase plane exists (all of them for stride 1); kept in a register so that the
+        // tap loop reads no memory
+        auto load_mask = [&](int p) {
+            unsigned long long m = 0;
+            for (int tv = 0; tv < T; ++tv) m |= (unsigned long long)(tap_tab[p * T + tv] >= 0 ? 1 : 0) << tv;
+            return m;
+        };
+        const unsigned long long mask0 = MASKED ? load_mask(0) : ~0ull;
+
+        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const unsigned long long taps, uint32_t &started, uint32_t &w_res) {
             constexpr int KS = decltype(ks_tag)::value;
             uint32_t off = 0;
             int y = 0;
             for (int tap = 0; tap < T; ++tap) {
                 uint32_t w_lo;
-                if (taps[tap] < 0) {             // the view has no such tap in this phase plane
+                if (MASKED && !((taps >> tap) & 1ull)) {   // the view has no such tap in this phase plane
                     if (a.b_resident) w_res += b_step;
                     if (++y == a.FW) { y = 0; off += row_wrap; } else off += 8u;
                     continue;
@@ -449,8 +459,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
             uint32_t w_res = smem_desc_lo(b_base), started = 0;
-            int cb = 0;
-            const volatile short *taps = tap_tab;
+            int cb = 0, plane = 0;
+            unsigned long long taps = mask0;
             for (int blk = 0; blk < a.CB && alive; ++blk) {       // blocks = phase planes x real channel blocks
                 alive = mbar_wait(bar_a_full + 8 * sa, pa, abort_flag, a.status);
                 if (!alive) break;
@@ -459,7 +469,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, taps, started, w_res);
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
                 if (++sa == (uint32_t)kAStages) { sa = 0; pa ^= 1u; }
-                if (++cb == a.CBr) { cb = 0; taps += T; }
+                if (++cb == a.CBr) { cb = 0; if (MASKED && ++plane < a.n_phase) taps = load_mask(plane); }
             }
             if (alive)
                 for (int j = 0; j < a.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
@@ -739,22 +749,22 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, in
 typedef void (*TcKernel)(const CUtensorMap, const CUtensorMap, const TcArgs);
 
 template <int CH, bool PM>
-TcKernel pick_ks(int ks) {
+TcKernel pick_ks(int ks, bool masked) {
     switch (ks) {
-        case 1: return conv_tc_kernel<CH, 1, PM>;
-        case 2: return conv_tc_kernel<CH, 2, PM>;
-        case 4: return conv_tc_kernel<CH, 4, PM>;
+        case 1: return masked ? conv_tc_kernel<CH, 1, PM, true> : conv_tc_kernel<CH, 1, PM, false>;
+        case 2: return masked ? conv_tc_kernel<CH, 2, PM, true> : conv_tc_kernel<CH, 2, PM, false>;
+        case 4: return masked ? conv_tc_kernel<CH, 4, PM, true> : conv_tc_kernel<CH, 4, PM, false>;
         default: return nullptr;
     }
 }
 // Filters on M: one chain per accumulator slot (1 or 2); pixels on M: one per 128-pixel chunk (1 to 4).
-TcKernel pick_kernel(int chains, int ks, bool pixel_m) {
-    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks) : chains == 2 ? pick_ks<2, false>(ks) : nullptr;
+TcKernel pick_kernel(int chains, int ks, bool pixel_m, bool masked) {
+    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks, masked) : chains == 2 ? pick_ks<2, false>(ks, masked) : nullptr;
     switch (chains) {
-        case 1: return pick_ks<1, true>(ks);
-        case 2: return pick_ks<2, true>(ks);
-        case 3: return pick_ks<3, true>(ks);
-        case 4: return pick_ks<4, true>(ks);
+        case 1: return pick_ks<1, true>(ks, masked);
+        case 2: return pick_ks<2, true>(ks, masked);
+        case 3: return pick_ks<3, true>(ks, masked);
+        case 4: return pick_ks<4, true>(ks, masked);
         default: return nullptr;
     }
 }
@@ -887,7 +897,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     }
     const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
     a.relu = relu; a.accumulate = accumulate;
-    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0);
+    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1);
     if (!kern) return SMALL_ERR_UNSUPPORTED;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
