@@ -273,13 +273,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile short *tap_tab = reinterpret_cast<volatile short *>(ctrl_ptr + kCtrlBarrierBytes + 16 + (size_t)a.KB * 32 * 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Tiles with two or more MMA chains split them over two issuing threads (warps 1 and 3, on different schedulers):
+    // issuing a small MMA costs a thread more cycles than the pipe needs to run it.
+    constexpr int kIssuers = CH >= 2 ? 2 : 1;
+    constexpr int kSplit = (CH + 1) / 2;       // chains [0, kSplit) belong to warp 1, the rest to warp 3
     const int T = a.FH * a.FW;
     const int total_tiles = a.m_tiles * a.n_tiles;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, 1); }
-        for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, 1); }
-        for (int s = 0; s < kSlots; ++s) { mbar_init(bar_slot_full + 8 * s, 1); mbar_init(bar_slot_free + 8 * s, 4); }   // 4 epilogue warps
+        // every MMA issuer commits to the stage-empty and slot-full barriers; 4 epilogue warps free a slot
+        for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, kIssuers); }
+        for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, kIssuers); }
+        for (int s = 0; s < kSlots; ++s) { mbar_init(bar_slot_full + 8 * s, kIssuers); mbar_init(bar_slot_free + 8 * s, 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -376,8 +381,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
             }
         }
-    } else if (warp == 1 && lane == 0) {
-        // ---- MMA issue
+    } else if ((warp == 1 || (kIssuers == 2 && warp == 3)) && lane == 0) {
+        // ---- MMA issue: this thread's chains are [C0, C1)
+        auto mma_role = [&](auto c0_tag, auto c1_tag) {
+        constexpr int C0 = decltype(c0_tag)::value, C1 = decltype(c1_tag)::value;
         bool alive = true;
         uint32_t sa = 0, pa = 0, sb = 0, pb = 0;
         uint32_t slot_uses = 0;                   // slots taken so far; slot j of a tile is (slot_uses + j) % 2
@@ -423,7 +430,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t first = started;   // 0 for the first MMAs of the tile: they overwrite the accumulator
                 started = 1u;
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
+                for (int c = C0; c < C1; ++c) {
                     const uint32_t xs = x_lo + xo[c];
                     const uint32_t da = PM ? xs : w_lo, db = PM ? w_lo : xs;
                     mma_tf32(acc[c], da, db, kDescHi, idesc, first);
@@ -475,6 +482,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int j = 0; j < a.slots; ++j) mma_commit(bar_slot_full + 8 * ((slot_uses + j) % kSlots));
             slot_uses += a.slots;
         }
+        };
+        if (kIssuers == 1 || warp == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, kIssuers == 1 ? CH : kSplit>{});
+        else mma_role(std::integral_constant<int, kSplit>{}, std::integral_constant<int, CH>{});
     } else if (warp >= 4) {
         // ---- epilogue: warp q owns tensor-memory lanes 32q.. = filters 32q.. of the tile; lane = filter, column = pixel
         const int quarter = warp & 3;
