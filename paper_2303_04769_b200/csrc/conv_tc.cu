@@ -672,9 +672,8 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     const size_t b_stage = ((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023;
     p.b_stage_bytes = (uint32_t)b_stage;
     // shared memory.  When one filter tile covers the layer and all its (channel block, tap) boxes fit beside enough
-    // strips, the filters are loaded once and stay; otherwise at least two strips and two filter boxes, then filter
-    // boxes up to one per tap plus two, then further strips (deeper prefetch across tiles, which is what the
-    // bandwidth-bound layers need), then the rest as filter boxes.
+    // strips, the filters are loaded once and stay; otherwise at least two strips and two filter boxes, and the rest
+    // shared out as described below.
     const size_t fixed = 1024 + ctrl_bytes(g.KB);
     const size_t all_b = (size_t)g.CB * g.FH * g.FW * b_stage;
     p.b_resident = 0;
@@ -688,10 +687,18 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
         if (fixed + 2 * (size_t)p.a_stage_bytes + 2 * b_stage > max_smem) return p;
         size_t room = max_smem - fixed - 2 * (size_t)p.a_stage_bytes - 2 * b_stage;
         p.a_stages = 2; p.b_stages = 2;
-        const int b_want = g.FH * g.FW + 2 < kMaxBStages ? g.FH * g.FW + 2 : kMaxBStages;
-        while (p.b_stages < b_want && room >= b_stage) { ++p.b_stages; room -= b_stage; }
-        while (p.a_stages < kMaxAStages && room >= p.a_stage_bytes) { ++p.a_stages; room -= p.a_stage_bytes; }
-        while (p.b_stages < kMaxBStages && room >= b_stage) { ++p.b_stages; room -= b_stage; }
+        // Both streams are latency bound (a stage is refilled only after its MMAs have finished), so what counts is
+        // how many channel-block steps of MMA work the stages in flight cover: a strip covers one, a filter box 1/taps.
+        // Grow whichever side covers less until nothing more fits.
+        const int taps = g.FH * g.FW;
+        for (;;) {
+            const bool can_a = p.a_stages < kMaxAStages && room >= p.a_stage_bytes;
+            const bool can_b = p.b_stages < kMaxBStages && room >= b_stage;
+            if (!can_a && !can_b) break;
+            const bool b_behind = (double)p.b_stages / taps <= (double)p.a_stages;
+            if (can_b && (b_behind || !can_a)) { ++p.b_stages; room -= b_stage; }
+            else { ++p.a_stages; room -= p.a_stage_bytes; }
+        }
     }
     p.smem_bytes = (uint32_t)(fixed + (size_t)p.a_stages * p.a_stage_bytes + (size_t)p.b_stages * b_stage);
     if ((long long)p.m_tiles * p.n_tiles > 0x7fffffffLL) return p;
