@@ -213,7 +213,7 @@ SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     bool relu = flags & SMALL_RELU, acc = flags & SMALL_ACCUMULATE;
     // the tensor-core epilogue may store 32 bytes per thread: an output that is only 16-byte aligned takes the FP32 kernel
-    if (math == SMALL_MATH_TF32 && conv_tc_supported(g) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0) {   // 3XTF32 runs the FP32 kernel until its split path lands
+    if (math != SMALL_MATH_FP32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
         const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);
         const float *w_lo = w_hi + conv_w_tc_elems(C, K, FH, FW);
         return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, relu, acc, math, st);

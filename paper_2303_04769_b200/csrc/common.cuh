@@ -67,7 +67,7 @@ int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, f
 int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
                      bool relu, bool accumulate, cudaStream_t);
 // tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32
-bool conv_tc_supported(const Geom &);
+bool conv_tc_supported(const Geom &, bool x3 = false);   // x3: with the doubled stages of 3xTF32
 int launch_conv_tc(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t);
 

@@ -43,14 +43,15 @@ namespace small {
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;            // roles of the TF32 kernel; the 3xTF32 kernel adds four splitting warps
+constexpr int kThreadsX3 = 384;
 constexpr int kSlots = 2;              // accumulator slots of 256 tensor-memory columns
 constexpr int kSlotPx = 256;           // pixels per slot = the MMA's largest N
 constexpr int kFilterTile = 128;       // filters per tile = the MMA's M
 constexpr int kMaxAStages = 6;         // input strips in flight (at least 2; as many as shared memory allows)
 constexpr int kMaxBStages = 8;
 constexpr uint32_t kWaitIters = 1u << 22;   // bounded wait: polls back off with nanosleep, so this is seconds
-constexpr int kCtrlBarrierBytes = 16 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
+constexpr int kCtrlBarrierBytes = 24 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
 constexpr int kTapTabEntries = 4 * 64;   // original tap of every (phase plane, view tap), -1 where the view tap has none
 
 struct TcPlan {
@@ -69,9 +70,11 @@ struct TcPlan {
     int w_tile;          // filters per tile: 128 (filters on M) or up to 256 (filters on N)
     int cps;             // pixel_m: 128-pixel chunks per accumulator slot (4, 2 or 1 for up to 64, 128 or 256 filters)
     int b_resident;      // all filter tiles of the layer stay in shared memory for the whole kernel
+    int x3;              // 3xTF32: stages hold both halves, three MMAs per K step
     double taps_eff;     // taps per block that exist (a stride-2 view has empty ones)
     int ks_last;         // K steps (8 channels each) of the last channel block that hold real channels
     uint32_t a_stage_bytes, b_stage_bytes, smem_bytes;
+    uint32_t a_half, b_half;   // 3xTF32: each stage holds the TF32 part and, a_half / b_half bytes on, the residual
     bool ok;
 };
 
@@ -84,6 +87,7 @@ struct TcArgs {
     int rows_tile;       // whole rows per tile when every tile starts at a row start, else 0
     int slots, n_slot;   // accumulator slots per tile and pixels per slot: the same for every tile of the layer
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
+    uint32_t a_half, b_half;   // 3xTF32: byte offset of the residual half of a strip stage / filter stage
     int relu, accumulate;
 };
 
@@ -251,9 +255,15 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
 // MASKED: some view taps do not exist (stride-2 layers).  They are template
 // parameters so that the single issuing thread runs straight-line code: with run-time chain and K-step counts every
 // MMA costs it about 100 cycles of branches and selects, more than a small MMA occupies the pipe (measured).
-template <int CH, int KS_LAST, bool PM, bool MASKED>
-__global__ void __launch_bounds__(kThreads, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
+// X3: 3xTF32.  Every FP32 operand is split into its TF32 part and the residual (x = x_hi + x_lo, w = w_hi + w_lo) and
+// each K step issues x_lo*w_hi, x_hi*w_lo and x_hi*w_hi into the same FP32 accumulator (x_lo*w_lo is below FP32
+// resolution).  Filters arrive split (packed so); the activations are split in shared memory by four extra warps as
+// each strip lands: hi = the top 19 bits, in place; lo = x - hi, exact, in the second half of the stage.
+template <int CH, int KS_LAST, bool PM, bool MASKED, bool X3>
+__global__ void __launch_bounds__(X3 ? kThreadsX3 : kThreads, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_b_lo, const TcArgs a) {
+    constexpr int kNT = X3 ? kThreadsX3 : kThreads;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -265,7 +275,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
     // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias for all filters
     const uint32_t bar_a_full = ctrl, bar_a_empty = ctrl + 8 * kMaxAStages;
-    const uint32_t bar_b_full = ctrl + 16 * kMaxAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
+    const uint32_t bar_a_split = ctrl + 16 * kMaxAStages;      // 3xTF32: strip split into hi and lo
+    const uint32_t bar_b_full = ctrl + 24 * kMaxAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
     const uint32_t bar_slot_full = bar_b_empty + 8 * kMaxBStages, bar_slot_free = bar_slot_full + 8 * kSlots;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
@@ -282,7 +293,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         // every MMA issuer commits to the stage-empty and slot-full barriers; 4 epilogue warps free a slot
-        for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, kIssuers); }
+        for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, kIssuers); mbar_init(bar_a_split + 8 * s, 128); }
         for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, kIssuers); }
         for (int s = 0; s < kSlots; ++s) { mbar_init(bar_slot_full + 8 * s, kIssuers); mbar_init(bar_slot_free + 8 * s, 4); }
         *abort_flag = 0;
@@ -291,17 +302,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // zero tail behind each strip: the padding pixels a row (or image) wrap runs into after the last strip row
     for (int s = 0; s < kAStages; ++s) {
         float4 *tail = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + (size_t)a.strip_px * 128);
-        for (int i = threadIdx.x; i < a.tail_px * 8; i += kThreads) tail[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = threadIdx.x; i < a.tail_px * 8; i += kNT) tail[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     // filter rows the TMA box does not cover (fewer than 128 filters in the layer) stay zero for the whole kernel
     if (!PM && a.w_rows < kFilterTile)
         for (int s = 0; s < a.b_stages; ++s) {
             float4 *rest = reinterpret_cast<float4 *>(base_ptr + (b_base - base) + (size_t)s * kBStageBytes + (size_t)a.w_rows * 128);
-            for (int i = threadIdx.x; i < (kFilterTile - a.w_rows) * 8; i += kThreads) rest[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = threadIdx.x; i < (kFilterTile - a.w_rows) * 8; i += kNT) {
+                rest[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (X3) rest[i + a.b_half / 16] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
-    for (int i = threadIdx.x; i < a.KB * 32; i += kThreads) bias_s[i] = (a.bias && i < a.K) ? a.bias[i] : 0.0f;
+    for (int i = threadIdx.x; i < a.KB * 32; i += kNT) bias_s[i] = (a.bias && i < a.K) ? a.bias[i] : 0.0f;
     // view tap (x', y') of phase plane (ph, pw) is the original tap x = S (x' - pt') + ph + pt, y likewise, if it exists
-    for (int i = threadIdx.x; i < a.n_phase * T; i += kThreads) {
+    for (int i = threadIdx.x; i < a.n_phase * T; i += kNT) {
         const int p = i / T, tv = i - p * T, xv = tv / a.FW, yv = tv - xv * a.FW;
         const int x = a.S * (xv - a.pt) + ((a.phase_bits >> (2 * p)) & 1) + a.pto;
         const int y = a.S * (yv - a.pl) + ((a.phase_bits >> (2 * p + 1)) & 1) + a.plo;
@@ -352,13 +366,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (a.b_resident) {
             int boxes = 0;
             for (int i = 0; i < a.n_phase * T; ++i) boxes += tap_tab[i] >= 0 ? 1 : 0;
-            mbar_expect_tx(bar_b_full, box_bytes * (uint32_t)(boxes * a.CBr));
+            mbar_expect_tx(bar_b_full, box_bytes * (uint32_t)(boxes * a.CBr) * (X3 ? 2u : 1u));
             uint32_t dst = b_base;
             for (int p = 0; p < a.n_phase; ++p)
                 for (int cb = 0; cb < a.CBr; ++cb)
                     for (int tap = 0; tap < T; ++tap, dst += kBStageBytes) {
                         const int orig = tap_tab[p * T + tap];
-                        if (orig >= 0) tma_load_4d(dst, &map_b, bar_b_full, 0, 0, orig, cb);
+                        if (orig >= 0) {
+                            tma_load_4d(dst, &map_b, bar_b_full, 0, 0, orig, cb);
+                            if (X3) tma_load_4d(dst + a.b_half, &map_b_lo, bar_b_full, 0, 0, orig, cb);
+                        }
                     }
             armed_mask = 1u;
         } else {
@@ -373,8 +390,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             if (orig < 0) continue;
                             if (wrapped) alive = mbar_wait(bar_b_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
                             if (!alive) break;
-                            mbar_expect_tx(bar_b_full + 8 * s, box_bytes);
+                            mbar_expect_tx(bar_b_full + 8 * s, X3 ? 2u * box_bytes : box_bytes);
                             tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, row, orig, cb);
+                            if (X3) tma_load_4d(b_base + s * kBStageBytes + a.b_half, &map_b_lo, bar_b_full + 8 * s, 0, row, orig, cb);
                             armed_mask |= 1u << s;
                             armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
                             if (++s == (uint32_t)a.b_stages) { s = 0; phase ^= 1u; wrapped = true; }
@@ -389,6 +407,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t sa = 0, pa = 0, sb = 0, pb = 0;
         uint32_t slot_uses = 0;                   // slots taken so far; slot j of a tile is (slot_uses + j) % 2
         const uint32_t b_step = kBStageBytes >> 4;
+        const uint32_t x_half = a.a_half >> 4, w_half = a.b_half >> 4;
         const uint32_t row_wrap = (uint32_t)(a.Wq - a.FW + 1) * 8u;     // tap offset step from the end of a window row
         // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
         const uint32_t idesc = instr_desc(PM ? a.w_rows : a.n_slot);
@@ -433,10 +452,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int c = C0; c < C1; ++c) {
                     const uint32_t xs = x_lo + xo[c];
                     const uint32_t da = PM ? xs : w_lo, db = PM ? w_lo : xs;
-                    mma_tf32(acc[c], da, db, kDescHi, idesc, first);
-                    if (KS > 1) mma_tf32(acc[c], da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
-                    if (KS > 2) mma_tf32(acc[c], da + 4u, db + 4u, kDescHi, idesc, 1u);
-                    if (KS > 3) mma_tf32(acc[c], da + 6u, db + 6u, kDescHi, idesc, 1u);
+                    if (!X3) {
+                        mma_tf32(acc[c], da, db, kDescHi, idesc, first);
+                        if (KS > 1) mma_tf32(acc[c], da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
+                        if (KS > 2) mma_tf32(acc[c], da + 4u, db + 4u, kDescHi, idesc, 1u);
+                        if (KS > 3) mma_tf32(acc[c], da + 6u, db + 6u, kDescHi, idesc, 1u);
+                    } else {
+                        // the residual halves sit x_half / w_half (16-byte units) behind the TF32 halves
+                        const uint32_t da_lo = da + (PM ? x_half : w_half), db_lo = db + (PM ? w_half : x_half);
+#pragma unroll
+                        for (int k = 0; k < KS; ++k) {
+                            mma_tf32(acc[c], da_lo + 2u * k, db + 2u * k, kDescHi, idesc, k == 0 ? first : 1u);   // small terms first
+                            mma_tf32(acc[c], da + 2u * k, db_lo + 2u * k, kDescHi, idesc, 1u);
+                            mma_tf32(acc[c], da + 2u * k, db + 2u * k, kDescHi, idesc, 1u);
+                        }
+                    }
                 }
                 if (!a.b_resident) {
                     mma_commit(bar_b_empty + 8 * sb);                // filter stage reusable once these MMAs have read it
@@ -469,7 +499,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int cb = 0, plane = 0;
             unsigned long long taps = mask0;
             for (int blk = 0; blk < a.CB && alive; ++blk) {       // blocks = phase planes x real channel blocks
-                alive = mbar_wait(bar_a_full + 8 * sa, pa, abort_flag, a.status);
+                alive = mbar_wait((X3 ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status);   // 3xTF32: once split
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
                 if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, started, w_res);
@@ -485,7 +515,30 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         };
         if (kIssuers == 1 || warp == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, kIssuers == 1 ? CH : kSplit>{});
         else mma_role(std::integral_constant<int, kSplit>{}, std::integral_constant<int, CH>{});
-    } else if (warp >= 4) {
+    } else if (X3 && warp >= 8) {
+        // ---- 3xTF32: split each strip as it lands.  Elementwise at equal offsets, so the swizzled layout carries over.
+        const int tid = threadIdx.x - 256;
+        bool alive = true;
+        uint32_t s = 0, phase = 0;
+        const int n4 = (a.strip_px + a.tail_px) * 8;          // 16-byte vectors of the strip and its zero tail
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x)
+            for (int blk = 0; blk < a.CB; ++blk) {
+                alive = mbar_wait_warp(bar_a_full + 8 * s, phase, abort_flag, a.status);
+                if (!alive) break;
+                uint4 *hi = reinterpret_cast<uint4 *>(base_ptr + (size_t)s * a.a_stage_bytes);
+                float4 *lo = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + a.a_half);
+                for (int i = tid; i < n4; i += 128) {
+                    const uint4 v = hi[i];
+                    const uint4 h = make_uint4(v.x & 0xffffe000u, v.y & 0xffffe000u, v.z & 0xffffe000u, v.w & 0xffffe000u);
+                    lo[i] = make_float4(__uint_as_float(v.x) - __uint_as_float(h.x), __uint_as_float(v.y) - __uint_as_float(h.y),
+                                        __uint_as_float(v.z) - __uint_as_float(h.z), __uint_as_float(v.w) - __uint_as_float(h.w));
+                    hi[i] = h;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these writes are read by the tensor core
+                mbar_arrive(bar_a_split + 8 * s);
+                if (++s == (uint32_t)kAStages) { s = 0; phase ^= 1u; }
+            }
+    } else if (warp >= 4 && warp < 8) {
         // ---- epilogue: warp q owns tensor-memory lanes 32q.. = filters 32q.. of the tile; lane = filter, column = pixel
         const int quarter = warp & 3;
         bool alive = true;
@@ -606,7 +659,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + kTapTabEntries * sizeof(short); }
 
 // Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff) {
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;                      // g is the stride-1 view; S scales the TMA box of the real tensor
@@ -668,8 +721,11 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     }
     const int reach = a0max + slot_reach + (g.FH - 1) * p.Wq + g.FW - 1;
     p.stage_px = p.strip_px + p.tail_px > reach ? p.strip_px + p.tail_px : reach;
-    p.a_stage_bytes = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
-    const size_t b_stage = ((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023;
+    p.a_half = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
+    p.b_half = (uint32_t)(((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023);
+    p.x3 = x3 ? 1 : 0;
+    p.a_stage_bytes = p.a_half * (x3 ? 2u : 1u);         // 3xTF32: TF32 part and residual side by side
+    const size_t b_stage = (size_t)p.b_half * (x3 ? 2 : 1);
     p.b_stage_bytes = (uint32_t)b_stage;
     // shared memory.  When one filter tile covers the layer and all its (channel block, tap) boxes fit beside enough
     // strips, the filters are loaded once and stay; otherwise at least two strips and two filter boxes, and the rest
@@ -733,9 +789,10 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
         const double warps = p.w_rows >= 128 ? 4.0 : p.w_rows / 32.0;
         epi = avg_px * 20.0 * 4.0 / warps;
     }
+    if (p.x3) mma *= 3.0;
     mma += taps * g.CB * (p.b_resident ? 40.0 : 120.0);
     const double strip_bytes = (double)g.CB * p.strip_px * 128.0;
-    const double bytes = strip_bytes + (p.b_resident ? 0.0 : taps * g.CB * p.w_rows * 128.0) + avg_px * 128.0 * (p.w_rows / 32.0);
+    const double bytes = strip_bytes + (p.b_resident ? 0.0 : taps * g.CB * p.w_rows * 128.0 * (p.x3 ? 2.0 : 1.0)) + avg_px * 128.0 * (p.w_rows / 32.0);
     const double mem = bytes / 30.0;                 // bytes per clock one SM can expect when all SMs pull
     double tile = mma > mem ? mma : mem;
     if (slots == 2) tile += epi;
@@ -750,12 +807,12 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
 
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
 // fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
-TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff) {
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3) {
     TcPlan best{};
     double best_cost = 0.0;
     for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
         for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff);
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3);
             if (!p.ok) continue;
             const double c = plan_cost(p, g, sms);
             if (!best.ok || c < best_cost) { best = p; best_cost = c; }
@@ -763,25 +820,30 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, in
     return best;
 }
 
-typedef void (*TcKernel)(const CUtensorMap, const CUtensorMap, const TcArgs);
+typedef void (*TcKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
 
+template <int CH, int KS, bool PM>
+TcKernel pick_flags(bool masked, bool x3) {
+    if (x3) return masked ? conv_tc_kernel<CH, KS, PM, true, true> : conv_tc_kernel<CH, KS, PM, false, true>;
+    return masked ? conv_tc_kernel<CH, KS, PM, true, false> : conv_tc_kernel<CH, KS, PM, false, false>;
+}
 template <int CH, bool PM>
-TcKernel pick_ks(int ks, bool masked) {
+TcKernel pick_ks(int ks, bool masked, bool x3) {
     switch (ks) {
-        case 1: return masked ? conv_tc_kernel<CH, 1, PM, true> : conv_tc_kernel<CH, 1, PM, false>;
-        case 2: return masked ? conv_tc_kernel<CH, 2, PM, true> : conv_tc_kernel<CH, 2, PM, false>;
-        case 4: return masked ? conv_tc_kernel<CH, 4, PM, true> : conv_tc_kernel<CH, 4, PM, false>;
+        case 1: return pick_flags<CH, 1, PM>(masked, x3);
+        case 2: return pick_flags<CH, 2, PM>(masked, x3);
+        case 4: return pick_flags<CH, 4, PM>(masked, x3);
         default: return nullptr;
     }
 }
 // Filters on M: one chain per accumulator slot (1 or 2); pixels on M: one per 128-pixel chunk (1 to 4).
-TcKernel pick_kernel(int chains, int ks, bool pixel_m, bool masked) {
-    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks, masked) : chains == 2 ? pick_ks<2, false>(ks, masked) : nullptr;
+TcKernel pick_kernel(int chains, int ks, bool pixel_m, bool masked, bool x3) {
+    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks, masked, x3) : chains == 2 ? pick_ks<2, false>(ks, masked, x3) : nullptr;
     switch (chains) {
-        case 1: return pick_ks<1, true>(ks, masked);
-        case 2: return pick_ks<2, true>(ks, masked);
-        case 3: return pick_ks<3, true>(ks, masked);
-        case 4: return pick_ks<4, true>(ks, masked);
+        case 1: return pick_ks<1, true>(ks, masked, x3);
+        case 2: return pick_ks<2, true>(ks, masked, x3);
+        case 3: return pick_ks<3, true>(ks, masked, x3);
+        case 4: return pick_ks<4, true>(ks, masked, x3);
         default: return nullptr;
     }
 }
@@ -848,22 +910,30 @@ static bool make_virt(const Geom &g_in, Virt &v) {
     return g.FH * g.FW <= 64;
 }
 
-bool conv_tc_supported(const Geom &g) {
+// The tensor core adds each K step's products to its FP32 accumulator with truncation, an error that grows with the
+// number of accumulation steps (measured: about 5e-8 relative per K step of 8 channels).  TF32's own tolerance absorbs
+// it; 3xTF32 promises 1e-5, which holds up to about 180 steps, so longer reductions are left to the FP32 kernel.
+constexpr int kMaxKStepsX3 = 160;
+
+bool conv_tc_supported(const Geom &g, bool x3) {
     Virt v;
-    return make_virt(g, v) && make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff).ok;
+    if (!make_virt(g, v)) return false;
+    if (x3 && g.CB * 4 * g.FH * g.FW > kMaxKStepsX3) return false;
+    return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
-    (void)w_lo; (void)mode;
+    const bool x3 = mode == SMALL_MATH_3XTF32;
+    if (x3 && !w_lo) return SMALL_ERR_INVALID_ARG;
     Virt v;
     if (!make_virt(g_in, v)) return SMALL_ERR_UNSUPPORTED;
     const Geom &g = v.g;
     TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
-                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff);
+                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
-    CUtensorMap map_a, map_b;
+    CUtensorMap map_a, map_b, map_b_lo;
     {   // activations: [N][CB][H][W][32 floats]; box = 32 x Wq x Rs x 1 x nn, out-of-range elements read as zero
         // the real tensor (for stride 1 possibly with a 1x1 layer's rows re-cut); with stride 2 the box spans 2 Wq x 2 Rs
         // elements and the element strides keep every other one, so shared memory receives Wq x Rs pixels either way
@@ -878,17 +948,18 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
     }
-    {   // filters: [CB][FH*FW][KB*32][32 floats]; box = 32 x min(128, KB*32) rows
+    for (int half = 0; half < (x3 ? 2 : 1); ++half) {   // filters: [CB][FH*FW][KB*32][32 floats], TF32 part and (3xTF32) residual
         const int T = v.FHo * v.FWo, Kp = g.KB * 32;
         cuuint64_t dims[4] = {32, (cuuint64_t)Kp, (cuuint64_t)T, (cuuint64_t)v.CBr};
         cuuint64_t strides[3] = {128, (cuuint64_t)Kp * 128, (cuuint64_t)T * Kp * 128};
         cuuint32_t box[4] = {32, (cuuint32_t)p.w_rows, 1, 1};
         cuuint32_t estr[4] = {1, 1, 1, 1};
-        CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float *>(w_hi), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CUresult r = encode(half ? &map_b_lo : &map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float *>(half ? w_lo : w_hi), dims, strides,
+                            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
     }
+    if (!x3) map_b_lo = map_b;
     TcArgs a{};
     a.bias = bias; a.out = out; a.status = ctx->dev_status;
     a.N = g.N; a.K = g.K; a.KB = g.KB; a.CB = g.CB; a.OH = g.OH; a.OW = g.OW; a.Wq = p.Wq; a.Hq = p.Hq;
@@ -898,7 +969,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.nn = p.nn; a.px_tile = p.px_tile; a.px_img = p.px_img; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
     a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
     a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
-    a.a_stage_bytes = p.a_stage_bytes;
+    a.a_stage_bytes = p.a_stage_bytes; a.a_half = p.a_half; a.b_half = p.b_half;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
     a.rows_tile = (p.nn == 1 && p.px_tile % p.Wq == 0) ? p.px_tile / p.Wq : 0;
@@ -914,13 +985,13 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     }
     const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
     a.relu = relu; a.accumulate = accumulate;
-    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1);
+    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3);
     if (!kern) return SMALL_ERR_UNSUPPORTED;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
-    kern<<<grid, kThreads, p.smem_bytes, st>>>(map_a, map_b, a);
+    kern<<<grid, x3 ? kThreadsX3 : kThreads, p.smem_bytes, st>>>(map_a, map_b, map_b_lo, a);
     return check_launch(ctx);
 }
 

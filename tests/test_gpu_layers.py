@@ -292,3 +292,46 @@ def test_conv_tf32_tensor_cores_stride2(case):
     out32 = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out32, N, C, K, H, W, FH, FW, 2, pad, B.RELU | B.MATH_FP32)
     assert rel_l2(from_blk(out32, N, K, OH, OW), ref) <= 1e-5
+
+
+CONV_3XTF32_CASES = [  # N, C, K, H, W, FH, FW, stride, pad
+    (1, 16, 16, 32, 32, 3, 3, 1, (1, 1, 1, 1)),
+    (2, 64, 64, 56, 56, 3, 3, 1, (1, 1, 1, 1)),
+    (3, 128, 128, 28, 28, 3, 3, 1, (1, 1, 1, 1)),
+    (5, 256, 256, 14, 14, 3, 3, 1, (1, 1, 1, 1)),
+    (19, 512, 512, 7, 7, 1, 1, 1, (0, 0, 0, 0)),
+    (2, 64, 64, 56, 56, 1, 1, 1, (0, 0, 0, 0)),
+    (2, 3, 16, 32, 32, 3, 3, 1, (1, 1, 1, 1)),
+    (2, 70, 45, 9, 11, 3, 3, 1, (1, 1, 1, 1)),
+    (2, 33, 200, 17, 19, 5, 3, 1, (2, 1, 0, 2)),
+    (3, 16, 32, 32, 32, 3, 3, 2, (1, 1, 1, 1)),
+    (3, 16, 32, 32, 32, 1, 1, 2, (0, 0, 0, 0)),
+    (5, 1, 64, 49, 10, 10, 4, 2, (4, 5, 1, 1)),
+]
+
+
+@pytest.mark.parametrize("case", CONV_3XTF32_CASES)
+def test_conv_3xtf32_tensor_cores(case):
+    """3xTF32: TF32 part and residual of both operands, three MMAs per K step, FP32-level accuracy."""
+    N, C, K, H, W, FH, FW, S, pad = case
+    x, w, b = rnd((N, C, H, W), 36), rnd((K, C, FH, FW), 37), rnd((K,), 38)
+    wb = torch.empty(B.small_conv_weight_elems(C, K, FH, FW, B.MATH_3XTF32), device="cuda")
+    B.small_pack_conv_weights(ctx(), dev(w), wb, C, K, FH, FW, B.MATH_3XTF32)
+    bx = to_blk(x)
+    ref = oracle.conv2d(x, w, b, S, pad, relu=True)
+    OH, OW = ref.shape[2:]
+    out = new_blk(N, K, OH, OW)
+    B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH_3XTF32)
+    assert B.small_device_status(ctx()) == 0
+    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    assert err <= 1e-5, err
+    assert pad_lanes_are_zero(out, N, K, OH, OW)
+    # not the CUDA-core kernel under another name: the same layer in FP32 mode sums in another order
+    out32 = new_blk(N, K, OH, OW)
+    B.small_conv2d(ctx(), bx, wb, dev(b), out32, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH_FP32)
+    if ((C + 31) // 32) * 4 * FH * FW <= 160:      # longer reductions stay on the FP32 kernel (accumulator truncation)
+        assert not torch.equal(out.view(torch.int32), out32.view(torch.int32))
+    prev = rnd((N, K, OH, OW), 39)
+    acc = to_blk(prev)
+    B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, S, pad, B.ACCUMULATE | B.MATH_3XTF32)
+    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad, accumulate_into=prev)) <= 1e-5
