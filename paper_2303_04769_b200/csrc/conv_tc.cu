@@ -70,6 +70,7 @@ struct TcPlan {
     int w_tile;          // filters per tile: 128 (filters on M) or up to 256 (filters on N)
     int cps;             // pixel_m: 128-pixel chunks per accumulator slot (4, 2 or 1 for up to 64, 128 or 256 filters)
     int b_resident;      // all filter tiles of the layer stay in shared memory for the whole kernel
+    int racc;            // accumulators per slot, 256 / racc tensor-memory columns apart (bounds the accumulation chains)
     int x3;              // 3xTF32: stages hold both halves, three MMAs per K step
     double taps_eff;     // taps per block that exist (a stride-2 view has empty ones)
     int ks_last;         // K steps (8 channels each) of the last channel block that hold real channels
@@ -88,6 +89,7 @@ struct TcArgs {
     int slots, n_slot;   // accumulator slots per tile and pixels per slot: the same for every tile of the layer
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     uint32_t a_half, b_half;   // 3xTF32: byte offset of the residual half of a strip stage / filter stage
+    int racc;                  // accumulators per slot that the channel blocks rotate over (filters on M only)
     int relu, accumulate;
 };
 
@@ -427,7 +429,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         };
         const unsigned long long mask0 = MASKED ? load_mask(0) : ~0ull;
 
-        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const unsigned long long taps, uint32_t &started, uint32_t &w_res) {
+        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const unsigned long long taps, const uint32_t r_sel, uint32_t &started, uint32_t &w_res) {
+            const uint32_t r_col = r_sel * (uint32_t)(kSlotPx / a.racc);   // this block's accumulator within each slot
             constexpr int KS = decltype(ks_tag)::value;
             uint32_t off = 0;
             int y = 0;
@@ -446,25 +449,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
                 }
                 const uint32_t x_lo = x_stage + off;
-                const uint32_t first = started;   // 0 for the first MMAs of the tile: they overwrite the accumulator
-                started = 1u;
+                const uint32_t first = (started >> r_sel) & 1u;   // 0 for an accumulator's first MMAs of the tile: they overwrite
+                started |= 1u << r_sel;
 #pragma unroll
                 for (int c = C0; c < C1; ++c) {
                     const uint32_t xs = x_lo + xo[c];
                     const uint32_t da = PM ? xs : w_lo, db = PM ? w_lo : xs;
                     if (!X3) {
-                        mma_tf32(acc[c], da, db, kDescHi, idesc, first);
-                        if (KS > 1) mma_tf32(acc[c], da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
-                        if (KS > 2) mma_tf32(acc[c], da + 4u, db + 4u, kDescHi, idesc, 1u);
-                        if (KS > 3) mma_tf32(acc[c], da + 6u, db + 6u, kDescHi, idesc, 1u);
+                        mma_tf32(acc[c] + r_col, da, db, kDescHi, idesc, first);
+                        if (KS > 1) mma_tf32(acc[c] + r_col, da + 2u, db + 2u, kDescHi, idesc, 1u);        // K steps of 32 bytes
+                        if (KS > 2) mma_tf32(acc[c] + r_col, da + 4u, db + 4u, kDescHi, idesc, 1u);
+                        if (KS > 3) mma_tf32(acc[c] + r_col, da + 6u, db + 6u, kDescHi, idesc, 1u);
                     } else {
                         // the residual halves sit x_half / w_half (16-byte units) behind the TF32 halves
                         const uint32_t da_lo = da + (PM ? x_half : w_half), db_lo = db + (PM ? w_half : x_half);
 #pragma unroll
                         for (int k = 0; k < KS; ++k) {
-                            mma_tf32(acc[c], da_lo + 2u * k, db + 2u * k, kDescHi, idesc, k == 0 ? first : 1u);   // small terms first
-                            mma_tf32(acc[c], da + 2u * k, db_lo + 2u * k, kDescHi, idesc, 1u);
-                            mma_tf32(acc[c], da + 2u * k, db + 2u * k, kDescHi, idesc, 1u);
+                            mma_tf32(acc[c] + r_col, da_lo + 2u * k, db + 2u * k, kDescHi, idesc, k == 0 ? first : 1u);   // small terms first
+                            mma_tf32(acc[c] + r_col, da + 2u * k, db_lo + 2u * k, kDescHi, idesc, 1u);
+                            mma_tf32(acc[c] + r_col, da + 2u * k, db + 2u * k, kDescHi, idesc, 1u);
                         }
                     }
                 }
@@ -495,15 +498,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     acc[c] = tmem + ((slot_uses + c) % kSlots) * kSlotPx;
                 }
             }
-            uint32_t w_res = smem_desc_lo(b_base), started = 0;
+            uint32_t w_res = smem_desc_lo(b_base), started = 0, r_sel = 0;
             int cb = 0, plane = 0;
             unsigned long long taps = mask0;
             for (int blk = 0; blk < a.CB && alive; ++blk) {       // blocks = phase planes x real channel blocks
                 alive = mbar_wait((X3 ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status);   // 3xTF32: once split
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
-                if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, started, w_res);
-                else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, taps, started, w_res);
+                if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, r_sel, started, w_res);
+                else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, taps, r_sel, started, w_res);
+                if (++r_sel == (uint32_t)a.racc) r_sel = 0;
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
                 if (++sa == (uint32_t)kAStages) { sa = 0; pa ^= 1u; }
                 if (++cb == a.CBr) { cb = 0; if (MASKED && ++plane < a.n_phase) taps = load_mask(plane); }
@@ -611,6 +615,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     for (int g = 0; g < px_here; g += 32) {
                         float v[32];
                         tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + g), v);
+                        for (int r = 1; r < a.racc; ++r) {       // channel blocks rotated over several accumulators: add them up
+                            float v2[32];
+                            tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx + r * (kSlotPx / a.racc) + g), v2);
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) v[e] += v2[e];
+                        }
                         int q = q_slot + g + lane, img = 0;
                         if (a.nn > 1) { img = q / pv; q -= img * pv; }
                         const int oh = q / a.Wq, ow = q - oh * a.Wq;
@@ -659,7 +669,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + kTapTabEntries * sizeof(short); }
 
 // Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3) {
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;                      // g is the stride-1 view; S scales the TMA box of the real tensor
@@ -678,6 +688,8 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     p.cps = !pixel_m ? 1 : p.w_rows <= 64 ? 4 : p.w_rows <= 128 ? 2 : 1;
     p.ks_last = (g.C - (g.CB - 1) * 32 + 7) / 8;
     if (pixel_m && max_px > kSlots * p.cps * 128) return p;       // more pixels than the accumulator slots hold
+    p.racc = racc;
+    if (racc > 1 && (pixel_m || max_px > kSlots * (kSlotPx / racc))) return p;   // each slot holds racc accumulators
     const long long pv = (long long)p.Hq * p.Wq;
     int a0max, slot_reach;
     if (pv <= max_px && p.Hq * S <= 256) {
@@ -715,7 +727,7 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     if (pixel_m) {
         slot_reach = ceil_div(p.px_tile, 128) * 128;
     } else {
-        const int slots = p.px_tile > kSlotPx ? 2 : 1;
+        const int slots = p.px_tile > kSlotPx / racc ? 2 : 1;
         const int n_slot = ((p.px_tile + slots - 1) / slots + 15) & ~15;
         slot_reach = slots * n_slot;
     }
@@ -762,6 +774,11 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     return p;
 }
 
+// The tensor core adds each K step's products to its FP32 accumulator with truncation, an error that grows with the
+// number of accumulation steps (measured: about 5e-8 relative per K step of 8 channels).  TF32's own tolerance absorbs
+// it; 3xTF32 promises 1e-5, which holds up to about 180 steps per accumulator.
+constexpr int kMaxKStepsX3 = 160;
+
 // Estimated cycles of the whole layer under a plan, from measured rates.  A 128 x N x 8 TF32 MMA occupies the pipe
 // for N / 2 cycles, with a floor of about 48; each tap costs the issuing thread some tens of cycles more (waiting for
 // and releasing a filter stage when the filters stream).  The epilogue's stores run at memory speed in either
@@ -783,7 +800,7 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
         mma = taps * ksteps * chunks * (p.w_rows / 2.0 > 48.0 ? p.w_rows / 2.0 : 48.0);
         epi = avg_px * 1.2 * (p.w_rows / 32.0) + 300.0 * chunks;
     } else {
-        slots = p.px_tile > kSlotPx ? 2 : 1;
+        slots = p.px_tile > kSlotPx / p.racc ? 2 : 1;
         const double n_slot = avg_px / slots;
         mma = taps * ksteps * slots * (n_slot / 2.0 > 48.0 ? n_slot / 2.0 : 48.0);
         const double warps = p.w_rows >= 128 ? 4.0 : p.w_rows / 32.0;
@@ -808,11 +825,19 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
 // fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
 TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3) {
+    // 3xTF32 keeps every accumulation chain within kMaxKStepsX3 K steps by rotating the channel blocks over 2 or 4
+    // accumulators (added up in the epilogue); TF32's tolerance needs none of that
+    int racc = 1;
+    if (x3) {
+        const int ksteps = g.CB * 4 * g.FH * g.FW;
+        racc = ksteps <= kMaxKStepsX3 ? 1 : ksteps <= 2 * kMaxKStepsX3 ? 2 : 4;
+        if (ksteps > 4 * kMaxKStepsX3) return TcPlan{};
+    }
     TcPlan best{};
     double best_cost = 0.0;
     for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
         for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3);
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc);
             if (!p.ok) continue;
             const double c = plan_cost(p, g, sms);
             if (!best.ok || c < best_cost) { best = p; best_cost = c; }
@@ -910,15 +935,9 @@ static bool make_virt(const Geom &g_in, Virt &v) {
     return g.FH * g.FW <= 64;
 }
 
-// The tensor core adds each K step's products to its FP32 accumulator with truncation, an error that grows with the
-// number of accumulation steps (measured: about 5e-8 relative per K step of 8 channels).  TF32's own tolerance absorbs
-// it; 3xTF32 promises 1e-5, which holds up to about 180 steps, so longer reductions are left to the FP32 kernel.
-constexpr int kMaxKStepsX3 = 160;
-
 bool conv_tc_supported(const Geom &g, bool x3) {
     Virt v;
     if (!make_virt(g, v)) return false;
-    if (x3 && g.CB * 4 * g.FH * g.FW > kMaxKStepsX3) return false;
     return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3).ok;
 }
 
@@ -969,7 +988,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.nn = p.nn; a.px_tile = p.px_tile; a.px_img = p.px_img; a.tiles_img = p.tiles_img; a.m_tiles = p.m_tiles; a.n_tiles = p.n_tiles;
     a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
     a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
-    a.a_stage_bytes = p.a_stage_bytes; a.a_half = p.a_half; a.b_half = p.b_half;
+    a.a_stage_bytes = p.a_stage_bytes; a.a_half = p.a_half; a.b_half = p.b_half; a.racc = p.racc;
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
     a.rows_tile = (p.nn == 1 && p.px_tile % p.Wq == 0) ? p.px_tile / p.Wq : 0;
@@ -979,7 +998,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
         a.slots = p.px_tile > a.n_slot ? 2 : 1;
         chains = ceil_div(p.px_tile, 128);
     } else {
-        a.slots = p.px_tile > kSlotPx ? 2 : 1;
+        a.slots = p.px_tile > kSlotPx / p.racc ? 2 : 1;
         a.n_slot = ((p.px_tile + a.slots - 1) / a.slots + 15) & ~15;
         chains = a.slots;
     }
