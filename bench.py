@@ -374,6 +374,14 @@ def gpu_main(args):
             other_modes[m] = {"value": N / (oms * 1e-3), "unit": UNIT, "ms_per_step": oms, "tolerance_rel_l2": TOL[m]}
             del og, onet
 
+    # the library's own issue-rate probe: what the TF32 pipe sustains with operands resident in shared memory
+    probe = None
+    if world == 1:
+        probe = {}
+        for n in (256, 128, 64, 32):
+            tf, cpm = B.small_measure_tf32_peak(ctx, n, 4096)
+            probe[f"n{n}"] = {"tflops": round(tf, 1), "cycles_per_mma": round(cpm, 1)}
+
     sweep = None if (args.no_sweep or world > 1) else run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch)
 
     cpu = None
@@ -384,7 +392,8 @@ def gpu_main(args):
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": {"fp32": "f32", "tf32": "tf32 products, f32 accumulate", "3xtf32": "3xtf32 products, f32 accumulate"}[args.math],
+            "dtype": {"fp32": "f32", "tf32": "tf32 products, f32 accumulate",
+                      "3xtf32": "f32 via 3xTF32 (TF32 part + residual of both operands, f32 accumulate)"}[args.math],
             "data": "synthetic",
             "config": {"workload": f"{WORKLOAD}: 8-layer residual CNN, 3x32x32 input, batch {N} per GPU (configs[1])",
                        "math": args.math, "tolerance_rel_l2": TOL[args.math], "l2": "flushed between steps (256 MB write)",
@@ -393,7 +402,7 @@ def gpu_main(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * N * c * h * w, "d2h_bytes_per_step": 4 * N * oc * oh * ow,
                     "ms_per_step": ms_e2e},
             "gpu_launches": len(gnet.layer_rows) * args.steps,
-            "clocks": clocks, "roofline": roofline, "other_math_modes": other_modes, "cpu_baseline": cpu, "device_status": status,
+            "clocks": clocks, "roofline": roofline, "other_math_modes": other_modes, "tf32_issue_probe": probe, "cpu_baseline": cpu, "device_status": status,
             "kernels": {k: {"launches_per_step": v["launches"], "ms": round(v["ms"], 4),
                             "share": round(v["ms"] / sum(x["ms"] for x in by_kernel.values()), 3)} for k, v in by_kernel.items()},
             "layers": layer_table, "sweep": sweep}
@@ -544,7 +553,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--math", default="tf32", choices=["fp32", "tf32", "3xtf32"])
+    ap.add_argument("--math", default="3xtf32", choices=["fp32", "tf32", "3xtf32"],
+                    help="arithmetic of the convolutions; the default keeps FP32-level accuracy (1e-5) on the tensor cores")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--layer", default=None, help="KIND:C:HW[:BATCH] - run one sweep layer only (for profiler captures)")

@@ -99,7 +99,8 @@ int small_last_cuda_error(small_ctx *ctx);
 int small_device_status(small_ctx *ctx, int *status, void *stream);
 
 /* Measures the dense TF32 tensor-core rate of this device: every SM issues `iters` x 4 back-to-back
- * tcgen05.mma kind::tf32 of shape 128 x n x 8 (n = 64, 128 or 256) on operands resident in shared memory.
+ * tcgen05.mma kind::tf32 of shape 128 x n x 8 (n = 32, 64, 128 or 256; iters a multiple of 8) on operands resident in
+ * shared memory.
  * cycles_dev: device buffer of one 64-bit word per SM (receives each SM's cycle count).  *tflops: whole-device rate
  * from CUDA events; *cycles_per_mma: SM 0's cycles per MMA instruction.  Synchronises `stream`.  This is the
  * measured denominator of the tensor-bound rooflines (the paper has no counterpart: its kernels are CPU SIMD). */

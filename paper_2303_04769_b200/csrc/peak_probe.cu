@@ -36,19 +36,28 @@ __global__ void __launch_bounds__(128, 1) tf32_peak_kernel(int n, int iters, lon
         const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
         const uint32_t a_lo = ((a_addr & 0x3FFFFu) >> 4) | (1u << 16), b_lo = ((b_addr & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
-        const int slots = 512 / n;                      // independent accumulators, used round robin
-        const long long t0 = clock64();
-        for (int i = 0; i < iters; ++i) {
-            const uint32_t d = tmem + (uint32_t)((i % slots) * n);
+        // Eight MMA chains per loop trip, round robin over the independent accumulators that fit in tensor memory,
+        // issued as straight-line code: with index arithmetic or branches between the MMAs the issuing thread, not
+        // the pipe, sets the pace for small n.
+        const int slots = 512 / n > 8 ? 8 : 512 / n;
+        uint32_t dd[8];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                asm volatile(
-                    "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-                    "setp.ne.b32 p, %5, 0;\n\t"
-                    "mov.b64 da, {%1, %3};\n\t"
-                    "mov.b64 db, {%2, %3};\n\t"
-                    "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %4, p;\n\t}"
-                    ::"r"(d), "r"(a_lo + 2u * k), "r"(b_lo + 2u * k), "r"(desc_hi), "r"(idesc), "r"((uint32_t)(i >= slots || k > 0)) : "memory");
+        for (int j = 0; j < 8; ++j) dd[j] = tmem + (uint32_t)((j % slots) * n);
+        const long long t0 = clock64();
+        for (int i = 0; i < iters; i += 8) {
+            const uint32_t acc = i > 0 ? 1u : 0u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+                        "setp.ne.b32 p, %5, 0;\n\t"
+                        "mov.b64 da, {%1, %3};\n\t"
+                        "mov.b64 db, {%2, %3};\n\t"
+                        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %4, p;\n\t}"
+                        ::"r"(dd[j]), "r"(a_lo + 2u * k), "r"(b_lo + 2u * k), "r"(desc_hi), "r"(idesc), "r"(k > 0 ? 1u : acc) : "memory");
+                }
             }
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr) : "memory");
@@ -79,7 +88,7 @@ SMALL_API int small_measure_tf32_peak(small_ctx *ctx, int n, int iters, long lon
                                       double *cycles_per_mma, void *stream) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     if (!cycles_dev || !tflops || !cycles_per_mma) return SMALL_ERR_INVALID_ARG;
-    if ((n != 64 && n != 128 && n != 256) || iters < 1 || iters > (1 << 20)) return SMALL_ERR_INVALID_ARG;
+    if ((n != 32 && n != 64 && n != 128 && n != 256) || iters < 8 || iters > (1 << 20) || iters % 8) return SMALL_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = 1024 + (size_t)(128 + n) * 128;
     cudaError_t e = cudaFuncSetAttribute(tf32_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

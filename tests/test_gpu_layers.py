@@ -335,3 +335,15 @@ def test_conv_3xtf32_tensor_cores(case):
     acc = to_blk(prev)
     B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, S, pad, B.ACCUMULATE | B.MATH_3XTF32)
     assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad, accumulate_into=prev)) <= 1e-5
+
+
+def test_tf32_issue_probe():
+    """The probe's straight-line MMA chains run at the pipe's rate: N / 2 cycles per 128 x N x 8 MMA for N >= 128."""
+    tf256, c256 = B.small_measure_tf32_peak(ctx(), 256, 2048)
+    tf128, c128 = B.small_measure_tf32_peak(ctx(), 128, 2048)
+    tf32, c32 = B.small_measure_tf32_peak(ctx(), 32, 2048)
+    assert B.small_device_status(ctx()) == 0
+    assert 120.0 <= c256 <= 140.0 and 60.0 <= c128 <= 75.0 and 20.0 <= c32 <= 75.0, (c256, c128, c32)
+    assert tf256 > 600.0 and abs(tf128 / tf256 - 1.0) < 0.15
+    with pytest.raises(B.SmallError):
+        B.small_measure_tf32_peak(ctx(), 48, 2048)
