@@ -167,7 +167,8 @@ def whole_job_throughput(units_local, ms_local, world, device=None):
 
 # ------------------------------------------------------------------------------------------- CPU oracle legs
 def time_oracle_net(batch_cap, target_s=12.0):
-    """The oracle as it stands on the host cores: a bounded sample of the workload's batch."""
+    """The oracle as it stands on the host cores: a bounded sample of the workload (at most the full batch per pass,
+    whole passes repeated until about target_s seconds of CPU work are done)."""
     import oracle
     from oracle import nets
     net = configs.NETWORKS[WORKLOAD]()
@@ -179,10 +180,13 @@ def time_oracle_net(batch_cap, target_s=12.0):
     dt = time.perf_counter() - t0
     n = int(max(probe, min(batch_cap, probe * target_s / max(dt, 1e-6))))
     x = configs.make_input(net, n)
-    t0 = time.perf_counter()
-    nets.run_net(net, params, x)
-    dt = time.perf_counter() - t0
-    return n / dt, n, dt, oracle.num_threads()
+    passes, total = 0, 0.0
+    while passes == 0 or (total < target_s and passes < 64):
+        t0 = time.perf_counter()
+        nets.run_net(net, params, x)
+        total += time.perf_counter() - t0
+        passes += 1
+    return n * passes / total, n, total, oracle.num_threads(), passes
 
 
 def reference_arm(args):
@@ -190,14 +194,17 @@ def reference_arm(args):
     if rank != 0:
         return
     net = configs.NETWORKS[WORKLOAD]()
-    times, n_used, cores = [], 0, 0
+    # every step is a bounded sample of the workload, sized so that the whole run stays within a few minutes
+    per_step_s = max(0.05, min(6.0, 150.0 / (args.steps + args.warmup)))
+    rates, n_used, cores, passes = [], 0, 0, 0
     for i in range(args.warmup + args.steps):
-        ips, n_used, dt, cores = time_oracle_net(net["batch"], target_s=6.0)
+        ips, n_used, dt, cores, passes = time_oracle_net(net["batch"], target_s=per_step_s)
         if i >= args.warmup:
-            times.append(n_used / ips)
-    ms = 1e3 * sum(times) / len(times)
-    value = n_used / (ms * 1e-3)
-    sample = f"{n_used} of {net['batch']} images per step, double accumulation, OpenMP"
+            rates.append(ips)
+    value = sum(rates) / len(rates)
+    ms = 1e3 * net["batch"] / value                     # one full batch at the sampled rate
+    sample = (f"{n_used} of {net['batch']} images per pass, {passes} passes per step (about {per_step_s:.2f} s), "
+              "double accumulation, OpenMP; ms_per_step is scaled to the full batch")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64 accumulate over f32 data", "data": "synthetic",
@@ -386,9 +393,9 @@ def gpu_main(args):
 
     cpu = None
     if world == 1 and not args.no_cpu:
-        ips, n_used, dt, cores = time_oracle_net(N)
+        ips, n_used, dt, cores, passes = time_oracle_net(N)
         cpu = {"value": ips, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"{n_used} of {N} images, one pass, {dt:.1f} s, double accumulation, OpenMP"}
+               "sample": f"{n_used} of {N} images per pass, {passes} passes, {dt:.1f} s of CPU work, double accumulation, OpenMP"}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -137,14 +137,16 @@ int small_pack_fc_weights(small_ctx *ctx, const float *w_kj, float *w_blk, int J
  *   out[n,k,oh,ow] = [out[n,k,oh,ow] +] bias[k] + sum_{c,x,y} in[n,c,oh*s+x-pad_t,ow*s+y-pad_l] * w[k,c,x,y]
  * in: blocked [N][C][H][W]; out: blocked [N][K][OH][OW]; bias: K floats or NULL.
  * flags: SMALL_RELU | SMALL_ACCUMULATE | one SMALL_MATH_*.  The tensor-core modes apply to the shapes
- * small_conv2d_uses_tensor_cores accepts (stride 1, padded row within the kernel's tile); any other shape
- * runs the FP32 kernel (tighter accuracy, no error).
+ * small_conv2d_uses_tensor_cores accepts (stride 1 or 2, padded row within the kernel's tile, at most 64
+ * taps in the stride-1 view of the window); any other shape runs the FP32 kernel (tighter accuracy, no
+ * error).  3XTF32 needs roughly twice the shared memory per tile and falls back the same way where even
+ * its smallest tile does not fit.  `out` must be 32-byte aligned for the tensor-core kernel (16 otherwise).
  * Errors: NOT_INIT, INVALID_ARG, SHAPE (dims < 1, empty output, pad >= window), ALIGN, OVERLAP,
  * UNSUPPORTED (window so large that one input tile exceeds shared memory). */
 int small_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
                  int N, int C, int K, int H, int W, int FH, int FW, int stride,
                  int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
-/* 1 if small_conv2d would run this shape on the tensor cores under a tensor-core math mode, else 0. */
+/* 1 if small_conv2d would run this shape on the tensor cores under SMALL_MATH_TF32, else 0. */
 int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
                                    int pad_t, int pad_b, int pad_l, int pad_r);
 
