@@ -71,6 +71,7 @@ struct TcPlan {
     int cps;             // pixel_m: 128-pixel chunks per accumulator slot (4, 2 or 1 for up to 64, 128 or 256 filters)
     int b_resident;      // all filter tiles of the layer stay in shared memory for the whole kernel
     int racc;            // accumulators per slot, 256 / racc tensor-memory columns apart (bounds the accumulation chains)
+    int x_packed;        // 3xTF32 with one channel block of <= 16 channels: hi in lanes [0, h), lo in [h, 2h) of each row
     int x3;              // 3xTF32: stages hold both halves, three MMAs per K step
     double taps_eff;     // taps per block that exist (a stride-2 view has empty ones)
     int ks_last;         // K steps (8 channels each) of the last channel block that hold real channels
@@ -90,6 +91,8 @@ struct TcArgs {
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     uint32_t a_half, b_half;   // 3xTF32: byte offset of the residual half of a strip stage / filter stage
     int racc;                  // accumulators per slot that the channel blocks rotate over (filters on M only)
+    int x_packed;              // 3xTF32, at most 16 channels: the residual sits in the unused lanes of the same row
+    uint32_t x_lo_off;         // 3xTF32: 16-byte units from a strip's TF32 part to its residual
     int relu, accumulate;
 };
 
@@ -409,7 +412,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t sa = 0, pa = 0, sb = 0, pb = 0;
         uint32_t slot_uses = 0;                   // slots taken so far; slot j of a tile is (slot_uses + j) % 2
         const uint32_t b_step = kBStageBytes >> 4;
-        const uint32_t x_half = a.a_half >> 4, w_half = a.b_half >> 4;
+        const uint32_t x_half = a.x_lo_off, w_half = a.b_half >> 4;
         const uint32_t row_wrap = (uint32_t)(a.Wq - a.FW + 1) * 8u;     // tap offset step from the end of a window row
         // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
         const uint32_t idesc = instr_desc(PM ? a.w_rows : a.n_slot);
@@ -531,6 +534,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!alive) break;
                 uint4 *hi = reinterpret_cast<uint4 *>(base_ptr + (size_t)s * a.a_stage_bytes);
                 float4 *lo = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + a.a_half);
+                if (a.x_packed) {
+                    // at most 16 channels: lanes [h, 2h) of every row are pad lanes (zero), and the residual goes
+                    // there instead of into a second half-stage.  A row's 16-byte chunk j sits at chunk j ^ (row & 7)
+                    // (128-byte swizzle; stages start on 1024-byte boundaries).
+                    const int hc = (int)a.x_lo_off >> 0;              // chunks per half: 2 (h = 8) or 4 (h = 16)
+                    const int rows = a.strip_px + a.tail_px;
+                    for (int i = tid; i < rows * hc; i += 128) {
+                        const int r = i / hc, j = i - r * hc;
+                        const int sw7 = r & 7;
+                        uint4 *src = hi + r * 8 + (j ^ sw7);
+                        const uint4 v = *src;
+                        const uint4 h = make_uint4(v.x & 0xffffe000u, v.y & 0xffffe000u, v.z & 0xffffe000u, v.w & 0xffffe000u);
+                        reinterpret_cast<float4 *>(hi)[r * 8 + ((j + hc) ^ sw7)] =
+                            make_float4(__uint_as_float(v.x) - __uint_as_float(h.x), __uint_as_float(v.y) - __uint_as_float(h.y),
+                                        __uint_as_float(v.z) - __uint_as_float(h.z), __uint_as_float(v.w) - __uint_as_float(h.w));
+                        *src = h;
+                    }
+                } else
                 for (int i = tid; i < n4; i += 128) {
                     const uint4 v = hi[i];
                     const uint4 h = make_uint4(v.x & 0xffffe000u, v.y & 0xffffe000u, v.z & 0xffffe000u, v.w & 0xffffe000u);
@@ -669,7 +690,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + kTapTabEntries * sizeof(short); }
 
 // Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc) {
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc, bool pack_ok) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;                      // g is the stride-1 view; S scales the TMA box of the real tensor
@@ -736,7 +757,8 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     p.a_half = (uint32_t)(((size_t)p.stage_px * 128 + 1023) & ~(size_t)1023);
     p.b_half = (uint32_t)(((size_t)(pixel_m ? p.w_rows : kFilterTile) * 128 + 1023) & ~(size_t)1023);
     p.x3 = x3 ? 1 : 0;
-    p.a_stage_bytes = p.a_half * (x3 ? 2u : 1u);         // 3xTF32: TF32 part and residual side by side
+    p.x_packed = (x3 && pack_ok) ? 1 : 0;
+    p.a_stage_bytes = p.a_half * ((x3 && !p.x_packed) ? 2u : 1u);   // 3xTF32: TF32 part and residual side by side
     const size_t b_stage = (size_t)p.b_half * (x3 ? 2 : 1);
     p.b_stage_bytes = (uint32_t)b_stage;
     // shared memory.  When one filter tile covers the layer and all its (channel block, tap) boxes fit beside enough
@@ -824,7 +846,7 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
 
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
 // fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
-TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3) {
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3, bool pack_ok) {
     // 3xTF32 keeps every accumulation chain within kMaxKStepsX3 K steps by rotating the channel blocks over 2 or 4
     // accumulators (added up in the epilogue); TF32's tolerance needs none of that
     int racc = 1;
@@ -837,7 +859,7 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, in
     double best_cost = 0.0;
     for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
         for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc);
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc, pack_ok);
             if (!p.ok) continue;
             const double c = plan_cost(p, g, sms);
             if (!best.ok || c < best_cost) { best = p; best_cost = c; }
@@ -938,7 +960,7 @@ static bool make_virt(const Geom &g_in, Virt &v) {
 bool conv_tc_supported(const Geom &g, bool x3) {
     Virt v;
     if (!make_virt(g, v)) return false;
-    return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3).ok;
+    return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, v.CBr == 1 && g.C <= 16).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
@@ -949,7 +971,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     if (!make_virt(g_in, v)) return SMALL_ERR_UNSUPPORTED;
     const Geom &g = v.g;
     TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
-                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3);
+                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3, v.CBr == 1 && g_in.C <= 16);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_a, map_b, map_b_lo;
@@ -989,6 +1011,8 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.strip_px = p.strip_px; a.tail_px = p.tail_px; a.w_rows = p.w_rows; a.b_stages = p.b_stages;
     a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
     a.a_stage_bytes = p.a_stage_bytes; a.a_half = p.a_half; a.b_half = p.b_half; a.racc = p.racc;
+    a.x_packed = p.x_packed;
+    a.x_lo_off = p.x_packed ? 2u * (uint32_t)p.ks_last : (p.a_half >> 4);   // packed: the residual starts h = 8 ks_last lanes on
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
     a.rows_tile = (p.nn == 1 && p.px_tile % p.Wq == 0) ? p.px_tile / p.Wq : 0;
