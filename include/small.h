@@ -123,6 +123,13 @@ size_t small_conv_weight_elems(int C, int K, int FH, int FW, unsigned math);
 /* w_kcrs: device float[K][C][FH][FW].  w_blk: device, small_conv_weight_elems floats. */
 int small_pack_conv_weights(small_ctx *ctx, const float *w_kcrs, float *w_blk, int C, int K, int FH, int FW,
                             unsigned math, void *stream);
+/* Group convolution filters (Section 3.1.3: the filter tensor is F_H x F_W x F_C x K x G).
+ * w_gkcrs: device float[G][K][F_C][FH][FW], G = small_group_count(C, F_C, S_C) (0 if the channel window does
+ * not tile the channels: (C - F_C) must be a multiple of S_C). */
+int small_group_count(int C, int F_C, int S_C);
+size_t small_group_conv_weight_elems(int C, int F_C, int S_C, int K, int FH, int FW);
+int small_pack_group_conv_weights(small_ctx *ctx, const float *w_gkcrs, float *w_blk, int C, int F_C, int S_C, int K,
+                                  int FH, int FW, void *stream);
 size_t small_dw_weight_elems(int C, int FH, int FW);
 /* w_crs: device float[C][FH][FW] (one filter per channel: Table 1, single channel reduction). */
 int small_pack_dw_weights(small_ctx *ctx, const float *w_crs, float *w_blk, int C, int FH, int FW, void *stream);
@@ -146,6 +153,14 @@ int small_pack_fc_weights(small_ctx *ctx, const float *w_kj, float *w_blk, int J
 int small_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
                  int N, int C, int K, int H, int W, int FH, int FW, int stride,
                  int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
+/* Partial channel reduction (Section 3.1.2, Figure 1; Table 1 "group convolution"): the window also slides over
+ * the channels.  Group g = 0..G-1 reduces input channels g*S_C .. g*S_C + F_C - 1 with its own K filters and
+ * writes output channels g*K .. g*K + K - 1 (O_C = K*G); S_C = F_C is the usual grouped convolution, S_C < F_C
+ * gives overlapping groups, F_C = S_C = 1 with K = 1 is a depthwise convolution.  Same epilogue, flags, padding
+ * and errors as small_conv2d; bias has K*G entries.  Runs on the FP32 kernel in every math mode. */
+int small_group_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
+                       int N, int C, int F_C, int S_C, int K, int H, int W, int FH, int FW, int stride,
+                       int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
 /* 1 if small_conv2d would run this shape on the tensor cores under SMALL_MATH_TF32, else 0. */
 int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
                                    int pad_t, int pad_b, int pad_l, int pad_r);

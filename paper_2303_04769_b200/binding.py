@@ -26,7 +26,8 @@ MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
     "small_last_cuda_error", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
-    "small_pack_conv_weights", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
+    "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
+    "small_group_conv2d", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
     "small_relu", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
@@ -75,6 +76,11 @@ def lib():
     L.small_conv_weight_elems.argtypes = [I, I, I, I, U]
     L.small_conv_weight_elems.restype = Z
     L.small_pack_conv_weights.argtypes = [P, P, P, I, I, I, I, U, P]
+    L.small_group_count.argtypes = [I, I, I]
+    L.small_group_conv_weight_elems.argtypes = [I] * 6
+    L.small_group_conv_weight_elems.restype = Z
+    L.small_pack_group_conv_weights.argtypes = [P, P, P] + [I] * 6 + [P]
+    L.small_group_conv2d.argtypes = [P, P, P, P, P] + [I] * 14 + [U, P]
     L.small_dw_weight_elems.argtypes = [I, I, I]
     L.small_dw_weight_elems.restype = Z
     L.small_pack_dw_weights.argtypes = [P, P, P, I, I, I, P]
@@ -189,6 +195,25 @@ def small_conv2d(ctx, inp, w_blk, bias, out, N, C, K, H, W, FH, FW, stride, pad,
     pt, pb, pl, pr = pad
     _check(lib().small_conv2d(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, C, K, H, W, FH, FW, stride,
                               pt, pb, pl, pr, flags, _stream(stream)), "small_conv2d")
+
+
+def small_group_count(C, F_C, S_C):
+    return int(lib().small_group_count(C, F_C, S_C))
+
+
+def small_group_conv_weight_elems(C, F_C, S_C, K, FH, FW):
+    return int(lib().small_group_conv_weight_elems(C, F_C, S_C, K, FH, FW))
+
+
+def small_pack_group_conv_weights(ctx, w_gkcrs, w_blk, C, F_C, S_C, K, FH, FW, stream=None):
+    _check(lib().small_pack_group_conv_weights(ctx, _ptr(w_gkcrs), _ptr(w_blk), C, F_C, S_C, K, FH, FW, _stream(stream)),
+           "small_pack_group_conv_weights")
+
+
+def small_group_conv2d(ctx, inp, w_blk, bias, out, N, C, F_C, S_C, K, H, W, FH, FW, stride, pad, flags=0, stream=None):
+    pt, pb, pl, pr = pad
+    _check(lib().small_group_conv2d(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, C, F_C, S_C, K, H, W, FH, FW, stride,
+                                    pt, pb, pl, pr, flags, _stream(stream)), "small_group_conv2d")
 
 
 def small_conv2d_uses_tensor_cores(N, C, K, H, W, FH, FW, stride, pad):

@@ -164,6 +164,53 @@ SMALL_API int small_pack_conv_weights(small_ctx *ctx, const float *w, float *wb,
     return launch_pack_conv_weights(ctx, w, wb, C, K, FH, FW, math, static_cast<cudaStream_t>(stream));
 }
 
+// ---- group convolution (partial channel reduction)
+static bool group_shape_ok(int C, int F_C, int S_C, int K) {
+    return C >= 1 && F_C >= 1 && F_C <= C && S_C >= 1 && K >= 1 && (C - F_C) % S_C == 0;
+}
+
+SMALL_API int small_group_count(int C, int F_C, int S_C) {
+    if (C < 1 || F_C < 1 || F_C > C || S_C < 1 || (C - F_C) % S_C != 0) return 0;
+    return (C - F_C) / S_C + 1;
+}
+
+SMALL_API size_t small_group_conv_weight_elems(int C, int F_C, int S_C, int K, int FH, int FW) {
+    if (!group_shape_ok(C, F_C, S_C, K) || FH < 1 || FW < 1) return 0;
+    const int G = (C - F_C) / S_C + 1;
+    return (size_t)blocks_of(K * G) * group_conv_span(C, F_C, S_C, K) * FH * FW * SMALL_CB * SMALL_CB;
+}
+
+SMALL_API int small_pack_group_conv_weights(small_ctx *ctx, const float *w, float *wb, int C, int F_C, int S_C, int K,
+                                            int FH, int FW, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({w, wb})) return s;
+    if (!group_shape_ok(C, F_C, S_C, K) || FH < 1 || FW < 1) return SMALL_ERR_SHAPE;
+    const int G = (C - F_C) / S_C + 1;
+    if (ranges_overlap(w, sizeof(float) * (size_t)G * K * F_C * FH * FW, wb,
+                       sizeof(float) * small_group_conv_weight_elems(C, F_C, S_C, K, FH, FW)))
+        return SMALL_ERR_OVERLAP;
+    return launch_pack_group_conv_weights(ctx, w, wb, C, F_C, S_C, K, FH, FW, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_group_conv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
+                                 int N, int C, int F_C, int S_C, int K, int H, int W, int FH, int FW, int stride,
+                                 int pt, int pb, int pl, int pr, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    if (!math_valid(math_of(flags))) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, w, out}, {bias})) return s;
+    if (!group_shape_ok(C, F_C, S_C, K)) return SMALL_ERR_SHAPE;
+    const int G = (C - F_C) / S_C + 1;
+    if ((long long)K * G > 0x7fffffLL) return SMALL_ERR_SHAPE;
+    Geom g;
+    if (int s = make_geom(g, N, C, K * G, H, W, FH, FW, stride, pt, pb, pl, pr)) return s;
+    if (ranges_overlap(in, sizeof(float) * packed_elems(N, C, H, W), out, sizeof(float) * packed_elems(N, K * G, g.OH, g.OW)))
+        return SMALL_ERR_OVERLAP;
+    // every math mode runs the FP32 kernel here (tighter than the tensor-core modes promise)
+    return launch_conv_fp32(ctx, in, w, bias, out, g, flags & SMALL_RELU, flags & SMALL_ACCUMULATE, static_cast<cudaStream_t>(stream),
+                            group_conv_span(C, F_C, S_C, K), K, S_C);
+}
+
 SMALL_API size_t small_dw_weight_elems(int C, int FH, int FW) {
     if (C < 1 || FH < 1 || FW < 1) return 0;
     return (size_t)blocks_of(C) * FH * FW * SMALL_CB;

@@ -64,8 +64,12 @@ int launch_add(small_ctx *, const float *a, const float *b, float *out, size_t n
 int launch_pool(small_ctx *, const float *in, float *out, int32_t *idx, const Geom &, int mode, cudaStream_t);
 int launch_dwconv(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
 int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, float *out, int N, int J, int K, bool relu, cudaStream_t);
+// span > 0: group convolution - filter block kb reads `span` channel blocks from that of its first group on
+// (Kg filters per group, groups S_C channels apart); span = 0: full reduction over all channel blocks
 int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
-                     bool relu, bool accumulate, cudaStream_t);
+                     bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
+int group_conv_span(int C, int F_C, int S_C, int Kg);      // channel blocks a filter block of a group convolution needs
+int launch_pack_group_conv_weights(small_ctx *, const float *w, float *wb, int C, int F_C, int S_C, int Kg, int FH, int FW, cudaStream_t);
 // tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32
 bool conv_tc_supported(const Geom &, bool x3 = false);   // x3: with the doubled stages of 3xTF32
 int launch_conv_tc(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,

@@ -17,6 +17,10 @@ struct ConvArgs {
     const float *in; const float *w; const float *bias; float *out;
     int C, K, H, W, FH, FW, S, pt, pl, OH, OW, CB, KB;
     int tiles_h, tiles_w, rows, cols;   // output tiles per plane; input tile extent in shared memory
+    // Partial channel reduction (group convolution, Section 3.1.2): the 32 filters of block kb only read the
+    // input channel blocks [cb0(kb), cb0(kb) + span); the packed filters hold zeros where a (channel, filter)
+    // pair lies in different groups.  A full reduction has span = CB and cb0 = 0.
+    int span, Kg, S_C;                  // blocks per filter block; filters per group; channel step between groups
     bool relu, accumulate;
 };
 
@@ -42,7 +46,10 @@ __global__ void __launch_bounds__(256) conv_fp32_kernel(ConvArgs a) {
     float4 *in_tile = reinterpret_cast<float4 *>(smem);
     float *w_tile = smem + (size_t)a.rows * a.cols * max_ci4 * 4;
 
-    for (int cb = 0; cb < a.CB; ++cb) {
+    const int cb0 = a.Kg > 0 ? ((kb * 32) / a.Kg * a.S_C) / 32 : 0;       // first channel block of this filter block's groups
+    for (int cbj = 0; cbj < a.span; ++cbj) {
+        const int cb = cb0 + cbj;
+        if (cb >= a.CB) break;
         const int ci_n = min(32, a.C - cb * 32);
         const int ci4 = (ci_n + 3) >> 2;
         __syncthreads();   // the previous block's tile is no longer read
@@ -61,7 +68,7 @@ __global__ void __launch_bounds__(256) conv_fp32_kernel(ConvArgs a) {
         for (int x = 0; x < a.FH; ++x) {
             __syncthreads();   // input tile visible (first x); previous filter row no longer read
             // filter row x of (kb, cb): [FW][ci][32 ko], only the channels that exist
-            const float *wsrc = a.w + ((((size_t)kb * a.CB + cb) * a.FH + x) * a.FW) * 32 * 32;
+            const float *wsrc = a.w + ((((size_t)kb * a.span + cbj) * a.FH + x) * a.FW) * 32 * 32;
             const int w_elems = a.FW * ci4 * 4 * 32;
             for (int e = threadIdx.x; e < w_elems; e += 256) {
                 int ko = e & 31;
@@ -118,10 +125,10 @@ static int launch_variant(small_ctx *ctx, ConvArgs &a, long long blocks, size_t 
 }
 
 int launch_conv_fp32(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, const Geom &g,
-                     bool relu, bool accumulate, cudaStream_t st) {
+                     bool relu, bool accumulate, cudaStream_t st, int span, int Kg, int S_C) {
     const int PIX = g.OW <= 8 ? 8 : 16;
     ConvArgs a{in, w, bias, out, g.C, g.K, g.H, g.W, g.FH, g.FW, g.S, g.pt, g.pl, g.OH, g.OW, g.CB, g.KB,
-               ceil_div(g.OH, 8), ceil_div(g.OW, PIX), 0, 0, relu, accumulate};
+               ceil_div(g.OH, 8), ceil_div(g.OW, PIX), 0, 0, span > 0 ? span : g.CB, span > 0 ? Kg : 0, S_C, relu, accumulate};
     // the shared input tile covers the whole 8 x PIX thread tile, so threads whose outputs fall outside the plane
     // still read inside the allocation (their results are not stored)
     a.rows = 7 * g.S + g.FH;

@@ -98,6 +98,34 @@ __global__ void pack_conv_w_fp32_kernel(const float *__restrict__ w, float *__re
     }
 }
 
+// Group convolution (Section 3.1.2-3.1.3: G groups of K filters, group g reduces channels g*S_C .. g*S_C + F_C - 1;
+// filters given as [G][K][F_C][FH][FW]).  Packed for the FP32 kernel as [KB][span][FH][FW][32 ci][32 ko]: block j of
+// filter block kb is channel block cb0(kb) + j, cb0 = channel block of kb's first group; a (channel, filter) pair of
+// different groups is stored as zero, so the kernel needs no group logic in its inner loops.
+__global__ void pack_group_conv_w_kernel(const float *__restrict__ w, float *__restrict__ wb, int C, int F_C, int S_C, int Kg, int G,
+                                         int span, int FH, int FW, size_t total) {
+    const int OC = Kg * G;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        size_t r = i;
+        int ko = (int)(r % 32); r /= 32;
+        int ci = (int)(r % 32); r /= 32;
+        int y = (int)(r % FW); r /= FW;
+        int x = (int)(r % FH); r /= FH;
+        int j = (int)(r % span); r /= span;
+        int kb = (int)r;
+        const int oc = kb * 32 + ko;
+        float v = 0.0f;
+        if (oc < OC) {
+            const int g = oc / Kg;
+            const int cb0 = ((kb * 32) / Kg * S_C) / 32;
+            const int c = (cb0 + j) * 32 + ci;
+            const int rel = c - g * S_C;
+            if (c < C && rel >= 0 && rel < F_C) v = w[(((size_t)oc * F_C + rel) * FH + x) * FW + y];
+        }
+        wb[i] = v;
+    }
+}
+
 // Tensor-core sections: [CB][FH*FW][KB*32 k][32 ci], ci fastest (the K-major B operand: one 128-byte row per
 // output channel and input block).  hi = round-to-nearest TF32 of w; lo = TF32 of the exact residual w - hi.
 __global__ void pack_conv_w_tc_kernel(const float *__restrict__ w, float *__restrict__ hi, float *__restrict__ lo,
@@ -155,6 +183,26 @@ int launch_pack_conv_weights(small_ctx *ctx, const float *w, float *wb, int C, i
         if (int s = check_launch(ctx)) return s;
     }
     return SMALL_OK;
+}
+
+int group_conv_span(int C, int F_C, int S_C, int Kg) {
+    const int G = (C - F_C) / S_C + 1, OC = Kg * G, KB = blocks_of(OC);
+    int span = 1;
+    for (int kb = 0; kb < KB; ++kb) {
+        const int g0 = (kb * 32) / Kg;
+        int g1 = (kb * 32 + 31) / Kg;
+        if (g1 > G - 1) g1 = G - 1;
+        const int need = (g1 * S_C + F_C - 1) / 32 - (g0 * S_C) / 32 + 1;
+        if (need > span) span = need;
+    }
+    return span;
+}
+
+int launch_pack_group_conv_weights(small_ctx *ctx, const float *w, float *wb, int C, int F_C, int S_C, int Kg, int FH, int FW, cudaStream_t st) {
+    const int G = (C - F_C) / S_C + 1, span = group_conv_span(C, F_C, S_C, Kg);
+    const size_t total = (size_t)blocks_of(Kg * G) * span * FH * FW * 32 * 32;
+    pack_group_conv_w_kernel<<<flat_grid(ctx, total), 256, 0, st>>>(w, wb, C, F_C, S_C, Kg, G, span, FH, FW, total);
+    return check_launch(ctx);
 }
 
 int launch_pack_dw_weights(small_ctx *ctx, const float *w, float *wb, int C, int FH, int FW, cudaStream_t st) {
