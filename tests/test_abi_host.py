@@ -58,6 +58,20 @@ def test_weight_sizes(lib):
     assert B.small_fc_weight_elems(0, 10) == 0
 
 
+def test_group_convolution_sizes(lib):
+    # the group count is Section 3.1.2's sliding-window formula applied to the channels
+    for C, F_C, S_C in [(8, 4, 2), (64, 16, 16), (40, 1, 1), (96, 48, 48), (64, 64, 1), (36, 8, 4)]:
+        assert B.small_group_count(C, F_C, S_C) == oracle.groups(C, F_C, S_C)
+    assert B.small_group_count(10, 4, 4) == 0 and B.small_group_count(8, 9, 1) == 0 and B.small_group_count(8, 4, 0) == 0
+    # packed size = filter blocks x channel blocks one filter block can touch x window x 32 x 32
+    assert B.small_group_conv_weight_elems(64, 16, 16, 16, 3, 3) == 2 * 1 * 9 * 1024      # 2 groups per filter block, one channel block
+    assert B.small_group_conv_weight_elems(128, 32, 32, 32, 3, 3) == 4 * 1 * 9 * 1024     # block-diagonal
+    assert B.small_group_conv_weight_elems(64, 64, 1, 8, 1, 1) == 1 * 2 * 1024            # one group: the dense size
+    assert B.small_group_conv_weight_elems(40, 1, 1, 1, 3, 3) == 2 * 1 * 9 * 1024         # depthwise as a group convolution
+    assert B.small_group_conv_weight_elems(96, 48, 48, 20, 1, 1) == 2 * 3 * 1024          # filter block 0 spans both groups
+    assert B.small_group_conv_weight_elems(10, 4, 4, 2, 3, 3) == 0
+
+
 def test_status_strings_and_null_context(lib):
     for s in range(0, 10):
         assert len(lib.small_strerror(s)) > 0
