@@ -383,6 +383,31 @@ def gpu_main(args):
             other_modes[m] = {"value": N / (oms * 1e-3), "unit": UNIT, "ms_per_step": oms, "tolerance_rel_l2": TOL[m]}
             del og, onet
 
+    # second workload, for context: the fully-connected autoencoder (batch 4096), each math mode, graph-replayed.  In the
+    # tensor-core modes its layers run as 1x1 convolutions over a 1x1 plane on the convolution kernel.
+    other_workloads = {}
+    if world == 1:
+        anet = configs.NETWORKS["autoencoder_fc"]()
+        aN = anet["batch"]
+        aparams = configs.make_params(anet)
+        ax = torch.from_numpy(configs.make_input(anet, aN)).to(dev)
+        ablk = torch.empty(B.small_packed_elems(aN, *anet["input"]), device=dev)
+        B.small_pack(ctx, ax, ablk, aN, *anet["input"])
+        flops = sum(2.0 * aN * L["C"] * L["K"] for L in anet["layers"])
+        res = {}
+        for m in ("3xtf32", "tf32", "fp32"):
+            an = Net(ctx, anet, aparams, math=m, device=dev)
+            an.run(ablk)
+            torch.cuda.synchronize()
+            ag = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(ag):
+                an.run(ablk)
+            ams = timed(lambda i: ag.replay(), min(args.steps, 100), 5)
+            res[m] = {"value": aN / (ams * 1e-3), "unit": UNIT, "ms_per_step": ams, "gflops": flops / ams / 1e6}
+            del ag, an
+        other_workloads["autoencoder_fc"] = {"batch": aN, "layers": len(anet["layers"]), "modes": res}
+        del ax, ablk
+
     # the library's own issue-rate probe: what the TF32 pipe sustains with operands resident in shared memory
     probe = None
     if world == 1:
@@ -411,7 +436,7 @@ def gpu_main(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * N * c * h * w, "d2h_bytes_per_step": 4 * N * oc * oh * ow,
                     "ms_per_step": ms_e2e},
             "gpu_launches": len(gnet.layer_rows) * args.steps,
-            "clocks": clocks, "roofline": roofline, "other_math_modes": other_modes, "tf32_issue_probe": probe, "cpu_baseline": cpu, "device_status": status,
+            "clocks": clocks, "roofline": roofline, "other_math_modes": other_modes, "tf32_issue_probe": probe, "other_workloads": other_workloads, "cpu_baseline": cpu, "device_status": status,
             "kernels": {k: {"launches_per_step": v["launches"], "ms": round(v["ms"], 4),
                             "share": round(v["ms"] / sum(x["ms"] for x in by_kernel.values()), 3)} for k, v in by_kernel.items()},
             "layers": layer_table, "sweep": sweep}

@@ -73,6 +73,15 @@ class Net:
                 d.op = B.OP_POOL
                 d.pool_mode = B.POOL_MAX if L["pool"] == "max" else B.POOL_AVG
                 wb = None
+            elif L["op"] == "fc" and self.math != B.MATH["fp32"] and h == 1 and wd == 1:
+                # a full reduction over a 1x1 plane is a 1x1 convolution whose pixels are the images: in the
+                # tensor-core modes it runs on the convolution kernel (same arithmetic, same blocked buffers)
+                d.op = B.OP_CONV
+                d.FH = d.FW = 1
+                flags |= self.math
+                wb = torch.empty(B.small_conv_weight_elems(L["C"], L["K"], 1, 1, self.math), device=device)
+                B.small_pack_conv_weights(ctx, wt.reshape(L["K"], L["C"], 1, 1).contiguous(), wb, L["C"], L["K"], 1, 1, self.math)
+                oh = ow = 1
             elif L["op"] == "fc":
                 d.op = B.OP_FC
                 wb = torch.empty(B.small_fc_weight_elems(L["C"], L["K"]), device=device)

@@ -41,9 +41,9 @@ def _gap(name, src, dst, C):
                 relu=False, accumulate=False, pool="avg")
 
 
-def _fc(name, src, dst, J, K):
+def _fc(name, src, dst, J, K, relu=False):
     return dict(op="fc", name=name, src=src, dst=dst, C=J, K=K, FH=1, FW=1, stride=1, pad=P0,
-                relu=False, accumulate=False)
+                relu=relu, accumulate=False)
 
 
 def single_conv_pool():
@@ -107,8 +107,23 @@ def kws_cnn(batch=1024):
                 weight_dist="he_normal", layers=L)
 
 
+def autoencoder_fc(batch=4096):
+    """Fully-connected autoencoder on 640 features (the Deep-Autoencoder-shaped model, Section 5.1.1): an encoder of
+    four 128-wide layers, an 8-wide bottleneck, a mirrored decoder; ReLU after every layer but the last (normalisation
+    folded into the biases).  Every layer is a full reduction (Table 1) over a 1x1 plane."""
+    widths = [640, 128, 128, 128, 128, 8, 128, 128, 128, 128, 640]
+    L, cur = [], "in"
+    for i in range(1, len(widths)):
+        last = i == len(widths) - 1
+        dst = "out" if last else f"h{i}"
+        L.append(_fc(f"fc{i}", cur, dst, widths[i - 1], widths[i], relu=not last))
+        cur = dst
+    return dict(name="autoencoder_fc", batch=batch, input=(640, 1, 1), input_dist=("normal", 0.0, 1.0),
+                weight_dist="he_normal", layers=L)
+
+
 NETWORKS = {"single_conv_pool": single_conv_pool, "residual_cnn": residual_cnn,
-            "dwsep_cnn": dwsep_cnn, "kws_cnn": kws_cnn}
+            "dwsep_cnn": dwsep_cnn, "kws_cnn": kws_cnn, "autoencoder_fc": autoencoder_fc}
 
 # GPU-scale layer sweep: batch 128, C = K, square planes, stride 1 (conv3x3 / depthwise pad 1, conv1x1 pad 0)
 SWEEP_BATCH = 128

@@ -13,7 +13,8 @@ from gpu_util import ctx, to_blk, from_blk, rel_l2
 pytestmark = pytest.mark.gpu
 TOL = {"fp32": 1e-5, "3xtf32": 1e-5, "tf32": 2e-3}
 
-CASES = [("single_conv_pool", 1), ("residual_cnn", 4), ("dwsep_cnn", 2), ("kws_cnn", 8)]
+CASES = [("single_conv_pool", 1), ("residual_cnn", 4), ("dwsep_cnn", 2), ("kws_cnn", 8),
+         ("autoencoder_fc", 64), ("autoencoder_fc", 300)]      # 300 images: a full strip of 256 and a ragged one
 
 
 @pytest.mark.parametrize("name,batch", CASES)
