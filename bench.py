@@ -495,17 +495,19 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
                 tmin, tmed = time_launch(call, reps=5 if slow else 20, warm=2, inner=1 if slow else 10)
                 record(kind, mode, fl, by, tmin, tmed, mode)
             del w, wb
-        # group convolution, groups of 32 channels with 32 filters each (G = C / 32): FP32 kernel, block-diagonal filters
+        # group convolution, groups of 32 channels with 32 filters each (G = C / 32): block-diagonal filters on the FP32 kernel,
+        # one filter tile per group on the tensor-core kernel
         G = C // 32
         wg = torch.from_numpy(synth.uniform((G, 32, 32, 3, 3), -1.0, 1.0, 900 + C)).to(dev)
         wgb = torch.empty(B.small_group_conv_weight_elems(C, 32, 32, 32, 3, 3), device=dev)
         B.small_pack_group_conv_weights(ctx, wg, wgb, C, 32, 32, 32, 3, 3)
 
-        def gc():
-            a, o = rot()
-            B.small_group_conv2d(ctx, a, wgb, bias, o, N, C, 32, 32, 32, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU)
-        tmin, tmed = time_launch(gc, reps=10, warm=2, inner=4)
-        record(f"groupconv3x3_g{G}", "fp32", 2.0 * N * HW * HW * C * 32 * 9, 4.0 * (2 * N * C * HW * HW + C * 32 * 9 + C), tmin, tmed, "fp32")
+        for mode in ("fp32", "tf32", "3xtf32"):
+            def gc(mode=mode):
+                a, o = rot()
+                B.small_group_conv2d(ctx, a, wgb, bias, o, N, C, 32, 32, 32, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU | B.MATH[mode])
+            tmin, tmed = time_launch(gc, reps=10, warm=2, inner=4 if mode == "fp32" else 10)
+            record(f"groupconv3x3_g{G}", mode, 2.0 * N * HW * HW * C * 32 * 9, 4.0 * (2 * N * C * HW * HW + C * 32 * 9 + C), tmin, tmed, mode)
         del wg, wgb
         wdw = torch.from_numpy(synth.uniform((C, 3, 3), -1.0, 1.0, 800 + C)).to(dev)
         wdb = torch.empty(B.small_dw_weight_elems(C, 3, 3), device=dev)

@@ -157,7 +157,9 @@ int small_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const floa
  * the channels.  Group g = 0..G-1 reduces input channels g*S_C .. g*S_C + F_C - 1 with its own K filters and
  * writes output channels g*K .. g*K + K - 1 (O_C = K*G); S_C = F_C is the usual grouped convolution, S_C < F_C
  * gives overlapping groups, F_C = S_C = 1 with K = 1 is a depthwise convolution.  Same epilogue, flags, padding
- * and errors as small_conv2d; bias has K*G entries.  Runs on the FP32 kernel in every math mode. */
+ * and errors as small_conv2d; bias has K*G entries.  Under SMALL_MATH_TF32 / 3XTF32, groups that are whole channel
+ * blocks (F_C = S_C a multiple of 32) with K a multiple of 32 (at most 256) run on the tensor-core kernel, one filter
+ * tile per group; every other shape, and SMALL_MATH_FP32, runs the FP32 kernel. */
 int small_group_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
                        int N, int C, int F_C, int S_C, int K, int H, int W, int FH, int FW, int stride,
                        int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);

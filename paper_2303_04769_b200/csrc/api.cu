@@ -174,10 +174,19 @@ SMALL_API int small_group_count(int C, int F_C, int S_C) {
     return (C - F_C) / S_C + 1;
 }
 
+// groups that are whole channel blocks with a multiple of 32 filters each can run on the tensor-core kernel
+static bool group_tc_layout(int F_C, int S_C, int K) { return F_C == S_C && F_C % 32 == 0 && K % 32 == 0 && K <= 256; }
+static size_t group_fp32_elems(int C, int F_C, int S_C, int K, int FH, int FW) {
+    const int G = (C - F_C) / S_C + 1;
+    return (size_t)blocks_of(K * G) * group_conv_span(C, F_C, S_C, K) * FH * FW * SMALL_CB * SMALL_CB;
+}
+
 SMALL_API size_t small_group_conv_weight_elems(int C, int F_C, int S_C, int K, int FH, int FW) {
     if (!group_shape_ok(C, F_C, S_C, K) || FH < 1 || FW < 1) return 0;
     const int G = (C - F_C) / S_C + 1;
-    return (size_t)blocks_of(K * G) * group_conv_span(C, F_C, S_C, K) * FH * FW * SMALL_CB * SMALL_CB;
+    size_t n = group_fp32_elems(C, F_C, S_C, K, FH, FW);
+    if (group_tc_layout(F_C, S_C, K)) n += 2 * group_conv_w_tc_elems(F_C, K, G, FH, FW);    // TF32 part and residual
+    return n;
 }
 
 SMALL_API int small_pack_group_conv_weights(small_ctx *ctx, const float *w, float *wb, int C, int F_C, int S_C, int K,
@@ -189,7 +198,13 @@ SMALL_API int small_pack_group_conv_weights(small_ctx *ctx, const float *w, floa
     if (ranges_overlap(w, sizeof(float) * (size_t)G * K * F_C * FH * FW, wb,
                        sizeof(float) * small_group_conv_weight_elems(C, F_C, S_C, K, FH, FW)))
         return SMALL_ERR_OVERLAP;
-    return launch_pack_group_conv_weights(ctx, w, wb, C, F_C, S_C, K, FH, FW, static_cast<cudaStream_t>(stream));
+    if (int s = launch_pack_group_conv_weights(ctx, w, wb, C, F_C, S_C, K, FH, FW, static_cast<cudaStream_t>(stream))) return s;
+    if (group_tc_layout(F_C, S_C, K)) {
+        float *hi = wb + group_fp32_elems(C, F_C, S_C, K, FH, FW);
+        return launch_pack_group_conv_weights_tc(ctx, w, hi, hi + group_conv_w_tc_elems(F_C, K, G, FH, FW), F_C, K, G, FH, FW,
+                                                 static_cast<cudaStream_t>(stream));
+    }
+    return SMALL_OK;
 }
 
 SMALL_API int small_group_conv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
@@ -206,7 +221,19 @@ SMALL_API int small_group_conv2d(small_ctx *ctx, const float *in, const float *w
     if (int s = make_geom(g, N, C, K * G, H, W, FH, FW, stride, pt, pb, pl, pr)) return s;
     if (ranges_overlap(in, sizeof(float) * packed_elems(N, C, H, W), out, sizeof(float) * packed_elems(N, K * G, g.OH, g.OW)))
         return SMALL_ERR_OVERLAP;
-    // every math mode runs the FP32 kernel here (tighter than the tensor-core modes promise)
+    // tensor-core modes: groups of whole channel blocks run on the tensor-core kernel, one filter tile per group
+    const unsigned math = math_of(flags);
+    if (math != SMALL_MATH_FP32 && G > 1 && group_tc_layout(F_C, S_C, K) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
+        Geom gg;
+        if (make_geom(gg, N, F_C, K * G, H, W, FH, FW, stride, pt, pb, pl, pr) == SMALL_OK &&
+            conv_tc_supported(gg, math == SMALL_MATH_3XTF32, G)) {
+            const float *w_hi = w + group_fp32_elems(C, F_C, S_C, K, FH, FW);
+            const float *w_lo = w_hi + group_conv_w_tc_elems(F_C, K, G, FH, FW);
+            return launch_conv_tc(ctx, in, w_hi, w_lo, bias, out, gg, flags & SMALL_RELU, flags & SMALL_ACCUMULATE, math,
+                                  static_cast<cudaStream_t>(stream), G);
+        }
+    }
+    // everything else runs the FP32 kernel (tighter than the tensor-core modes promise)
     return launch_conv_fp32(ctx, in, w, bias, out, g, flags & SMALL_RELU, flags & SMALL_ACCUMULATE, static_cast<cudaStream_t>(stream),
                             group_conv_span(C, F_C, S_C, K), K, S_C);
 }

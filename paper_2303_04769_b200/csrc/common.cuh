@@ -71,9 +71,14 @@ int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *
 int group_conv_span(int C, int F_C, int S_C, int Kg);      // channel blocks a filter block of a group convolution needs
 int launch_pack_group_conv_weights(small_ctx *, const float *w, float *wb, int C, int F_C, int S_C, int Kg, int FH, int FW, cudaStream_t);
 // tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32
-bool conv_tc_supported(const Geom &, bool x3 = false);   // x3: with the doubled stages of 3xTF32
+// x3: with the doubled stages of 3xTF32.  groups > 1: a group convolution whose groups are whole channel blocks; the
+// Geom then holds one group's channels (C = F_C) and all filters (K = groups x filters per group).
+bool conv_tc_supported(const Geom &, bool x3 = false, int groups = 1);
 int launch_conv_tc(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
-                   const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t);
+                   const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t, int groups = 1);
+// tensor-core filter sections of a group convolution: [F_C/32][FH*FW][G*K][32 ci], TF32 part and residual
+size_t group_conv_w_tc_elems(int F_C, int K, int G, int FH, int FW);
+int launch_pack_group_conv_weights_tc(small_ctx *, const float *w, float *hi, float *lo, int F_C, int K, int G, int FH, int FW, cudaStream_t);
 
 // Sizes (in floats) of the sections of a packed convolution filter buffer.
 size_t conv_w_fp32_elems(int C, int K, int FH, int FW);   // [KB][CB][FH][FW][32 ci][32 ko]

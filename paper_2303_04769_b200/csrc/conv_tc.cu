@@ -87,6 +87,7 @@ struct TcArgs {
     int nn, px_tile, px_img, tiles_img, m_tiles, n_tiles, strip_px, tail_px, w_rows;
     int a_stages, b_stages, pixel_m, w_tile, cps, b_resident, ks_last;
     int rows_tile;       // whole rows per tile when every tile starts at a row start, else 0
+    int cb_group;        // group convolution: channel blocks per group (filter tile g reads blocks g * cb_group ..), else 0
     int slots, n_slot;   // accumulator slots per tile and pixels per slot: the same for every tile of the layer
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     uint32_t a_half, b_half;   // 3xTF32: byte offset of the residual half of a strip stage / filter stage
@@ -357,7 +358,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (wrapped) alive = mbar_wait(bar_a_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
                     if (!alive) break;
                     mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
-                    tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, c1 + pw, c2 + ph, cb, tl.n0);
+                    tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, c1 + pw, c2 + ph, cb + tl.n_tile * a.cb_group, tl.n0);
                     armed_mask |= 1u << s;
                     armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
                     if (++s == (uint32_t)kAStages) { s = 0; phase ^= 1u; wrapped = true; }
@@ -571,7 +572,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int pv = a.Hq * a.Wq;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
-            const int kb = tl.n_tile * (kFilterTile / 32) + quarter;
+            const int kb = tl.n_tile * (a.w_tile / 32) + quarter;        // quarters past the tile's filters have nothing to store
             const int k = kb * 32 + lane;
             const float bv = kb < a.KB ? bias_s[k] : 0.0f;
             const bool lane_real = k < a.K;
@@ -624,7 +625,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             }
                         }
                     }
-                } else if (kb < a.KB) {
+                } else if (kb < a.KB && quarter * 32 < a.w_rows) {
                     // All lanes hold the same 32 pixels (columns) of different filters.  The pixel -> output line
                     // mapping is therefore computed once per group with one pixel per lane (divisions in parallel)
                     // and handed round by shuffle; the stores themselves are straight-line predicated code.
@@ -690,7 +691,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + kTapTabEntries * sizeof(short); }
 
 // Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc, bool pack_ok) {
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc, bool pack_ok, int group_k) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;                      // g is the stride-1 view; S scales the TMA box of the real tensor
@@ -706,6 +707,10 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     p.w_tile = pixel_m ? 256 : kFilterTile;
     p.n_tiles = ceil_div(Kp, p.w_tile);
     p.w_rows = Kp < p.w_tile ? Kp : p.w_tile;
+    if (group_k > 0) {                           // group convolution: one filter tile per group
+        if (group_k > p.w_tile) return p;
+        p.w_tile = group_k; p.w_rows = group_k; p.n_tiles = Kp / group_k;
+    }
     p.cps = !pixel_m ? 1 : p.w_rows <= 64 ? 4 : p.w_rows <= 128 ? 2 : 1;
     p.ks_last = (g.C - (g.CB - 1) * 32 + 7) / 8;
     if (pixel_m && max_px > kSlots * p.cps * 128) return p;       // more pixels than the accumulator slots hold
@@ -846,7 +851,7 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
 
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
 // fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
-TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3, bool pack_ok) {
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3, bool pack_ok, int group_k = 0) {
     // 3xTF32 keeps every accumulation chain within kMaxKStepsX3 K steps by rotating the channel blocks over 2 or 4
     // accumulators (added up in the epilogue); TF32's tolerance needs none of that
     int racc = 1;
@@ -859,7 +864,7 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, in
     double best_cost = 0.0;
     for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
         for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc, pack_ok);
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc, pack_ok, group_k);
             if (!p.ok) continue;
             const double c = plan_cost(p, g, sms);
             if (!best.ok || c < best_cost) { best = p; best_cost = c; }
@@ -957,21 +962,25 @@ static bool make_virt(const Geom &g_in, Virt &v) {
     return g.FH * g.FW <= 64;
 }
 
-bool conv_tc_supported(const Geom &g, bool x3) {
+// groups > 1: g describes one group's channels (C = F_C) and all the filters (K = groups * filters per group)
+bool conv_tc_supported(const Geom &g, bool x3, int groups) {
     Virt v;
     if (!make_virt(g, v)) return false;
+    if (groups > 1) return (g.C % 32 == 0) && (g.K % (32 * groups) == 0) &&
+                           make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, false, g.K / groups).ok;
     return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, v.CBr == 1 && g.C <= 16).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
-                   const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
+                   const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st, int groups) {
     const bool x3 = mode == SMALL_MATH_3XTF32;
     if (x3 && !w_lo) return SMALL_ERR_INVALID_ARG;
     Virt v;
     if (!make_virt(g_in, v)) return SMALL_ERR_UNSUPPORTED;
     const Geom &g = v.g;
     TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
-                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3, v.CBr == 1 && g_in.C <= 16);
+                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3, groups == 1 && v.CBr == 1 && g_in.C <= 16,
+                         groups > 1 ? g_in.K / groups : 0);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_a, map_b, map_b_lo;
@@ -980,8 +989,9 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
         // elements and the element strides keep every other one, so shared memory receives Wq x Rs pixels either way
         const int Hr = v.S == 1 ? g.H : g_in.H, Wr = v.S == 1 ? g.W : g_in.W;
         const cuuint32_t es = (cuuint32_t)v.S;
-        cuuint64_t dims[5] = {32, (cuuint64_t)Wr, (cuuint64_t)Hr, (cuuint64_t)v.CBr, (cuuint64_t)g.N};
-        cuuint64_t strides[4] = {128, (cuuint64_t)Wr * 128, (cuuint64_t)Hr * Wr * 128, (cuuint64_t)v.CBr * Hr * Wr * 128};
+        const cuuint64_t cb_all = (cuuint64_t)v.CBr * groups;      // a group's tiles address their blocks inside the whole tensor
+        cuuint64_t dims[5] = {32, (cuuint64_t)Wr, (cuuint64_t)Hr, cb_all, (cuuint64_t)g.N};
+        cuuint64_t strides[4] = {128, (cuuint64_t)Wr * 128, (cuuint64_t)Hr * Wr * 128, cb_all * Hr * Wr * 128};
         cuuint32_t box[5] = {32, (cuuint32_t)p.Wq * es, (cuuint32_t)p.Rs * es, 1, (cuuint32_t)p.nn};
         cuuint32_t estr[5] = {1, es, es, 1, 1};
         CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float *>(in), dims, strides, box, estr,
@@ -1016,6 +1026,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
     a.rows_tile = (p.nn == 1 && p.px_tile % p.Wq == 0) ? p.px_tile / p.Wq : 0;
+    a.cb_group = groups > 1 ? v.CBr : 0;
     int chains;
     if (p.pixel_m) {
         a.n_slot = p.cps * 128;

@@ -185,6 +185,33 @@ int launch_pack_conv_weights(small_ctx *ctx, const float *w, float *wb, int C, i
     return SMALL_OK;
 }
 
+// Tensor-core sections of a group convolution whose groups are whole channel blocks (F_C = S_C, multiples of 32, K a
+// multiple of 32): [F_C/32][FH*FW][G*K rows][32 ci] - row g*K + k holds filter k of group g, so one box of K rows is one
+// group's filter tile.  hi = TF32 rounding, lo = TF32 of the residual.
+__global__ void pack_group_conv_w_tc_kernel(const float *__restrict__ w, float *__restrict__ hi, float *__restrict__ lo,
+                                            int F_C, int K, int G, int FH, int FW, size_t total) {
+    const int T = FH * FW, rows = G * K;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        size_t r = i;
+        int ci = (int)(r % 32); r /= 32;
+        int row = (int)(r % rows); r /= rows;
+        int tap = (int)(r % T); r /= T;
+        int cb = (int)r;
+        const float v = w[((size_t)row * F_C + cb * 32 + ci) * T + tap];
+        const float h = round_tf32(v);
+        hi[i] = h;
+        lo[i] = round_tf32(v - h);
+    }
+}
+
+size_t group_conv_w_tc_elems(int F_C, int K, int G, int FH, int FW) { return (size_t)(F_C / 32) * FH * FW * G * K * 32; }
+
+int launch_pack_group_conv_weights_tc(small_ctx *ctx, const float *w, float *hi, float *lo, int F_C, int K, int G, int FH, int FW, cudaStream_t st) {
+    const size_t total = group_conv_w_tc_elems(F_C, K, G, FH, FW);
+    pack_group_conv_w_tc_kernel<<<flat_grid(ctx, total), 256, 0, st>>>(w, hi, lo, F_C, K, G, FH, FW, total);
+    return check_launch(ctx);
+}
+
 int group_conv_span(int C, int F_C, int S_C, int Kg) {
     const int G = (C - F_C) / S_C + 1, OC = Kg * G, KB = blocks_of(OC);
     int span = 1;

@@ -65,7 +65,9 @@ def test_group_convolution_sizes(lib):
     assert B.small_group_count(10, 4, 4) == 0 and B.small_group_count(8, 9, 1) == 0 and B.small_group_count(8, 4, 0) == 0
     # packed size = filter blocks x channel blocks one filter block can touch x window x 32 x 32
     assert B.small_group_conv_weight_elems(64, 16, 16, 16, 3, 3) == 2 * 1 * 9 * 1024      # 2 groups per filter block, one channel block
-    assert B.small_group_conv_weight_elems(128, 32, 32, 32, 3, 3) == 4 * 1 * 9 * 1024     # block-diagonal
+    # groups of whole channel blocks with a multiple of 32 filters also carry the tensor-core sections (TF32 part and
+    # residual): [F_C/32][taps][G*K][32]
+    assert B.small_group_conv_weight_elems(128, 32, 32, 32, 3, 3) == 4 * 1 * 9 * 1024 + 2 * (1 * 9 * 128 * 32)
     assert B.small_group_conv_weight_elems(64, 64, 1, 8, 1, 1) == 1 * 2 * 1024            # one group: the dense size
     assert B.small_group_conv_weight_elems(40, 1, 1, 1, 3, 3) == 2 * 1 * 9 * 1024         # depthwise as a group convolution
     assert B.small_group_conv_weight_elems(96, 48, 48, 20, 1, 1) == 2 * 3 * 1024          # filter block 0 spans both groups

@@ -91,3 +91,43 @@ def test_group_conv_rejects_bad_channel_windows():
     with pytest.raises(B.SmallError) as e:
         B.small_group_conv2d(ctx(), x, w, None, out, 1, 10, 4, 4, 2, 4, 4, 1, 1, 1, (0, 0, 0, 0), 0)
     assert "shape" in str(e.value).lower() or e.value.status != 0
+
+
+TC_CASES = [  # groups of whole channel blocks: N, C, F_C, K, H, W, FH, FW, stride, pad
+    (2, 128, 32, 32, 9, 11, 3, 3, 1, (1, 1, 1, 1)),
+    (3, 256, 64, 64, 14, 14, 3, 3, 1, (1, 1, 1, 1)),       # two channel blocks per group
+    (2, 128, 32, 32, 16, 16, 3, 3, 2, (1, 1, 1, 1)),       # stride 2: phase planes per group
+    (2, 64, 32, 128, 9, 9, 1, 1, 1, (0, 0, 0, 0)),         # more filters than channels per group
+    (5, 512, 32, 32, 7, 7, 3, 3, 1, (1, 1, 1, 1)),         # 16 groups, several images per strip
+    (2, 96, 32, 96, 12, 10, 3, 1, 1, (1, 1, 0, 0)),        # three groups, rectangular window
+]
+
+
+@pytest.mark.parametrize("case", TC_CASES)
+def test_group_conv_on_tensor_cores(case):
+    N, C, F_C, K, H, W, FH, FW, S, pad = case
+    G = C // F_C
+    OC = K * G
+    x, w, b = rnd((N, C, H, W), 56), rnd((G, K, F_C, FH, FW), 57), rnd((OC,), 58)
+    wb = torch.full((B.small_group_conv_weight_elems(C, F_C, F_C, K, FH, FW),), float("nan"), device="cuda")
+    B.small_pack_group_conv_weights(ctx(), dev(w), wb, C, F_C, F_C, K, FH, FW)
+    ref = oracle_group_conv(x, w, b, F_C, F_C, K, S, pad, relu=True)
+    OH, OW = ref.shape[2:]
+    bx = to_blk(x)
+    outs = {}
+    for math, tol in (("fp32", 1e-5), ("tf32", 2e-3), ("3xtf32", 1e-5)):
+        out = new_blk(N, OC, OH, OW)
+        B.small_group_conv2d(ctx(), bx, wb, dev(b), out, N, C, F_C, F_C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH[math])
+        assert B.small_device_status(ctx()) == 0
+        got = from_blk(out, N, OC, OH, OW)
+        err = rel_l2(got, ref)
+        assert err <= tol, (math, err)
+        assert pad_lanes_are_zero(out, N, OC, OH, OW)
+        outs[math] = (out, err)
+    assert outs["tf32"][1] > 1e-6                                    # TF32 products: the tensor-core kernel ran
+    assert not torch.equal(outs["3xtf32"][0].view(torch.int32), outs["fp32"][0].view(torch.int32))
+    prev = rnd((N, OC, OH, OW), 59)
+    acc = to_blk(prev)
+    B.small_group_conv2d(ctx(), bx, wb, None, acc, N, C, F_C, F_C, K, H, W, FH, FW, S, pad, B.ACCUMULATE | B.MATH_3XTF32)
+    ref_acc = oracle_group_conv(x, w, np.zeros(OC, np.float32), F_C, F_C, K, S, pad, relu=False).astype(np.float64) + prev
+    assert rel_l2(from_blk(acc, N, OC, OH, OW), ref_acc.astype(np.float32)) <= 1e-5
