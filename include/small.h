@@ -70,6 +70,7 @@ enum {
     SMALL_MATH_FP32 = 0u << 4,   /* FP32 FMA on CUDA cores, FP32 accumulate */
     SMALL_MATH_TF32 = 1u << 4,   /* TF32 tensor-core products, FP32 accumulate */
     SMALL_MATH_3XTF32 = 2u << 4, /* three TF32 products per term (hi*hi + hi*lo + lo*hi), FP32 accumulate */
+    SMALL_RELU_MID = 4u,   /* small_dwpw_conv2d only: max(x, 0) on the depthwise result, before the 1x1 convolution */
     SMALL_MATH_MASK = 3u << 4
 };
 
@@ -163,6 +164,21 @@ int small_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const floa
 int small_group_conv2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
                        int N, int C, int F_C, int S_C, int K, int H, int W, int FH, int FW, int stride,
                        int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
+/* Abstract fused layer (Section 6, future directions): depthwise 3x3 (+ dw_bias, + ReLU with SMALL_RELU_MID) followed
+ * by a 1x1 convolution to K channels (+ pw_bias, + ReLU with SMALL_RELU), as one layer:
+ *   out = act( pw( act_mid( dw(in) + dw_bias ) ) + pw_bias )
+ * in: blocked [N][C][H][W]; out: blocked [N][K][OH][OW], OH/OW from the depthwise window (3x3, `stride`, the pads).
+ * dw_w_blk from small_pack_dw_weights(C, 3, 3); pw_w_blk from small_pack_conv_weights(C, K, 1, 1, math).
+ * Under SMALL_MATH_TF32 / 3XTF32, shapes small_dwpw_fused accepts run as ONE kernel: the depthwise result is computed
+ * in shared memory and feeds the tensor cores without going to global memory.  Otherwise the two layers run one after
+ * the other through `scratch` (device, small_packed_elems(N, C, OH, OW) floats; may be NULL when the fused kernel
+ * runs - SMALL_ERR_WORKSPACE if it is needed and NULL).  Errors as small_conv2d. */
+int small_dwpw_conv2d(small_ctx *ctx, const float *in, const float *dw_w_blk, const float *dw_bias,
+                      const float *pw_w_blk, const float *pw_bias, float *out, float *scratch,
+                      int N, int C, int K, int H, int W, int stride,
+                      int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
+/* 1 if small_dwpw_conv2d runs this shape as one fused kernel under the given tensor-core math mode, else 0. */
+int small_dwpw_fused(int N, int C, int K, int H, int W, int stride, int pad_t, int pad_b, int pad_l, int pad_r, unsigned math);
 /* 1 if small_conv2d would run this shape on the tensor cores under SMALL_MATH_TF32, else 0. */
 int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
                                    int pad_t, int pad_b, int pad_l, int pad_r);

@@ -309,6 +309,56 @@ SMALL_API int small_dwconv2d(small_ctx *ctx, const float *in, const float *w, co
     return launch_dwconv(ctx, in, w, bias, out, g, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
 }
 
+// ---- fused depthwise 3x3 -> 1x1 convolution
+static bool dwpw_geoms(Geom &gd, Geom &gp, int N, int C, int K, int H, int W, int stride, int pt, int pb, int pl, int pr) {
+    if (make_geom(gd, N, C, C, H, W, 3, 3, stride, pt, pb, pl, pr) != SMALL_OK) return false;
+    return make_geom(gp, N, C, K, gd.OH, gd.OW, 1, 1, 1, 0, 0, 0, 0) == SMALL_OK;
+}
+
+SMALL_API int small_dwpw_fused(int N, int C, int K, int H, int W, int stride, int pt, int pb, int pl, int pr, unsigned math) {
+    if (math != SMALL_MATH_TF32 && math != SMALL_MATH_3XTF32) return 0;
+    if (stride != 1 && stride != 2) return 0;
+    Geom gd, gp;
+    if (!dwpw_geoms(gd, gp, N, C, K, H, W, stride, pt, pb, pl, pr)) return 0;
+    DwFuse f{nullptr, nullptr, C, H, W, stride, pt, pl, 0};
+    return conv_tc_supported(gp, math == SMALL_MATH_3XTF32, 1, &f) ? 1 : 0;
+}
+
+SMALL_API int small_dwpw_conv2d(small_ctx *ctx, const float *in, const float *dw_w, const float *dw_bias,
+                                const float *pw_w, const float *pw_bias, float *out, float *scratch,
+                                int N, int C, int K, int H, int W, int stride,
+                                int pt, int pb, int pl, int pr, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_RELU_MID | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    const unsigned math = math_of(flags);
+    if (!math_valid(math)) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, dw_w, pw_w, out}, {dw_bias, pw_bias, scratch})) return s;
+    Geom gd, gp;
+    if (int s = make_geom(gd, N, C, C, H, W, 3, 3, stride, pt, pb, pl, pr)) return s;
+    if (int s = make_geom(gp, N, C, K, gd.OH, gd.OW, 1, 1, 1, 0, 0, 0, 0)) return s;
+    if (ranges_overlap(in, sizeof(float) * packed_elems(N, C, H, W), out, sizeof(float) * packed_elems(N, K, gd.OH, gd.OW)))
+        return SMALL_ERR_OVERLAP;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool relu = flags & SMALL_RELU, relu_mid = flags & SMALL_RELU_MID;
+    if (math != SMALL_MATH_FP32 && (stride == 1 || stride == 2) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
+        DwFuse f{dw_w, dw_bias, C, H, W, stride, pt, pl, relu_mid ? 1 : 0};
+        if (conv_tc_supported(gp, math == SMALL_MATH_3XTF32, 1, &f)) {
+            const float *w_hi = pw_w + conv_w_fp32_elems(C, K, 1, 1);
+            const float *w_lo = w_hi + conv_w_tc_elems(C, K, 1, 1);
+            return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, pw_bias, out, gp, relu, false, math, st, 1, &f);
+        }
+    }
+    // the two layers one after the other, through the caller's scratch tensor
+    if (!scratch) return SMALL_ERR_WORKSPACE;
+    const size_t mid = sizeof(float) * packed_elems(N, C, gd.OH, gd.OW);
+    if (ranges_overlap(scratch, mid, in, sizeof(float) * packed_elems(N, C, H, W)) ||
+        ranges_overlap(scratch, mid, out, sizeof(float) * packed_elems(N, K, gd.OH, gd.OW)))
+        return SMALL_ERR_OVERLAP;
+    if (int s = launch_dwconv(ctx, in, dw_w, dw_bias, scratch, gd, relu_mid, st)) return s;
+    return small_conv2d(ctx, scratch, pw_w, pw_bias, out, N, C, K, gd.OH, gd.OW, 1, 1, 1, 0, 0, 0, 0,
+                        (relu ? SMALL_RELU : 0u) | math, stream);
+}
+
 SMALL_API int small_pool2d(small_ctx *ctx, const float *in, float *out, int32_t *idx,
                            int N, int C, int H, int W, int FH, int FW, int stride,
                            int pt, int pb, int pl, int pr, int mode, void *stream) {

@@ -73,9 +73,12 @@ int launch_pack_group_conv_weights(small_ctx *, const float *w, float *wb, int C
 // tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32
 // x3: with the doubled stages of 3xTF32.  groups > 1: a group convolution whose groups are whole channel blocks; the
 // Geom then holds one group's channels (C = F_C) and all filters (K = groups x filters per group).
-bool conv_tc_supported(const Geom &, bool x3 = false, int groups = 1);
+// A depthwise 3x3 fused in front of a 1x1 convolution: the Geom given to the two functions below is the 1x1 layer over
+// the depthwise output (H = W = that output's size); this describes the depthwise layer and its input.
+struct DwFuse { const float *w; const float *bias; int C, H, W, s, pt, pl, relu; };
+bool conv_tc_supported(const Geom &, bool x3 = false, int groups = 1, const DwFuse *dw = nullptr);
 int launch_conv_tc(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
-                   const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t, int groups = 1);
+                   const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t, int groups = 1, const DwFuse *dw = nullptr);
 // tensor-core filter sections of a group convolution: [F_C/32][FH*FW][G*K][32 ci], TF32 part and residual
 size_t group_conv_w_tc_elems(int F_C, int K, int G, int FH, int FW);
 int launch_pack_group_conv_weights_tc(small_ctx *, const float *w, float *hi, float *lo, int F_C, int K, int G, int FH, int FW, cudaStream_t);

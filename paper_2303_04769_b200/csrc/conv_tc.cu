@@ -51,7 +51,8 @@ constexpr int kFilterTile = 128;       // filters per tile = the MMA's M
 constexpr int kMaxAStages = 6;         // input strips in flight (at least 2; as many as shared memory allows)
 constexpr int kMaxBStages = 8;
 constexpr uint32_t kWaitIters = 1u << 22;   // bounded wait: polls back off with nanosleep, so this is seconds
-constexpr int kCtrlBarrierBytes = 24 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots;   // all mbarriers
+constexpr int kRawStages = 2;           // fused depthwise: halo tiles in flight
+constexpr int kCtrlBarrierBytes = 24 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots + 16 * kRawStages;   // all mbarriers
 constexpr int kTapTabEntries = 4 * 64;   // original tap of every (phase plane, view tap), -1 where the view tap has none
 
 struct TcPlan {
@@ -71,6 +72,7 @@ struct TcPlan {
     int cps;             // pixel_m: 128-pixel chunks per accumulator slot (4, 2 or 1 for up to 64, 128 or 256 filters)
     int b_resident;      // all filter tiles of the layer stay in shared memory for the whole kernel
     int racc;            // accumulators per slot, 256 / racc tensor-memory columns apart (bounds the accumulation chains)
+    uint32_t raw_stage_bytes; int dw_Hb, dw_Wb, dw_rows;   // fused depthwise: halo tile per (tile, channel block)
     int x_packed;        // 3xTF32 with one channel block of <= 16 channels: hi in lanes [0, h), lo in [h, 2h) of each row
     int x3;              // 3xTF32: stages hold both halves, three MMAs per K step
     double taps_eff;     // taps per block that exist (a stride-2 view has empty ones)
@@ -92,6 +94,10 @@ struct TcArgs {
     uint32_t a_stage_bytes, b_stage_bytes, a_box_bytes;
     uint32_t a_half, b_half;   // 3xTF32: byte offset of the residual half of a strip stage / filter stage
     int racc;                  // accumulators per slot that the channel blocks rotate over (filters on M only)
+    // fused depthwise 3x3 in front of a 1x1 convolution: the strips are computed in shared memory from halo tiles
+    const float *dw_w; const float *dw_bias;   // depthwise filters [CB][9][32] and bias (C floats or null)
+    int dw_s, dw_Wb, dw_Hb, dw_pt, dw_pl, dw_relu, dw_rows, dw_C;   // stride, halo box, pads, ReLU, strip rows per image
+    uint32_t raw_stage_bytes, raw_box_bytes;
     int x_packed;              // 3xTF32, at most 16 channels: the residual sits in the unused lanes of the same row
     uint32_t x_lo_off;         // 3xTF32: 16-byte units from a strip's TF32 part to its residual
     int relu, accumulate;
@@ -265,11 +271,14 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
 // each K step issues x_lo*w_hi, x_hi*w_lo and x_hi*w_hi into the same FP32 accumulator (x_lo*w_lo is below FP32
 // resolution).  Filters arrive split (packed so); the activations are split in shared memory by four extra warps as
 // each strip lands: hi = the top 19 bits, in place; lo = x - hi, exact, in the second half of the stage.
-template <int CH, int KS_LAST, bool PM, bool MASKED, bool X3>
-__global__ void __launch_bounds__(X3 ? kThreadsX3 : kThreads, 1)
+// DW: a depthwise 3x3 (+ bias, ReLU) is computed in front of this 1x1 convolution: TMA loads halo tiles of the layer's
+// input, warps 8-11 compute the depthwise result straight into the strip the MMAs read (and split it for 3xTF32),
+// so the depthwise output never goes to global memory.
+template <int CH, int KS_LAST, bool PM, bool MASKED, bool X3, bool DW>
+__global__ void __launch_bounds__((X3 || DW) ? kThreadsX3 : kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_b_lo, const TcArgs a) {
-    constexpr int kNT = X3 ? kThreadsX3 : kThreads;
+    constexpr int kNT = (X3 || DW) ? kThreadsX3 : kThreads;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -277,17 +286,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int kAStages = a.a_stages;
     const uint32_t b_base = a_base + kAStages * a.a_stage_bytes;
     const uint32_t kBStageBytes = a.b_stage_bytes;
-    const uint32_t ctrl = b_base + a.b_stages * kBStageBytes;
+    const uint32_t raw_base = b_base + a.b_stages * kBStageBytes;          // fused depthwise: halo tiles (no swizzle)
+    const uint32_t ctrl = raw_base + (DW ? kRawStages * a.raw_stage_bytes : 0u);
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
     // control block: barriers (8 bytes each), tensor-memory address, abort flag, bias for all filters
     const uint32_t bar_a_full = ctrl, bar_a_empty = ctrl + 8 * kMaxAStages;
     const uint32_t bar_a_split = ctrl + 16 * kMaxAStages;      // 3xTF32: strip split into hi and lo
     const uint32_t bar_b_full = ctrl + 24 * kMaxAStages, bar_b_empty = bar_b_full + 8 * kMaxBStages;
     const uint32_t bar_slot_full = bar_b_empty + 8 * kMaxBStages, bar_slot_free = bar_slot_full + 8 * kSlots;
+    const uint32_t bar_raw_full = bar_slot_free + 8 * kSlots, bar_raw_empty = bar_raw_full + 8 * kRawStages;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_ptr + kCtrlBarrierBytes);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_ptr + kCtrlBarrierBytes + 4);
     float *bias_s = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16);
     volatile short *tap_tab = reinterpret_cast<volatile short *>(ctrl_ptr + kCtrlBarrierBytes + 16 + (size_t)a.KB * 32 * 4);
+    float *dw_s_w = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16 + (size_t)a.KB * 32 * 4 + kTapTabEntries * sizeof(short));   // [CB][10][32]: 9 taps + bias
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Tiles with two or more MMA chains split them over two issuing threads (warps 1 and 3, on different schedulers):
@@ -302,6 +314,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, kIssuers); mbar_init(bar_a_split + 8 * s, 128); }
         for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, kIssuers); }
         for (int s = 0; s < kSlots; ++s) { mbar_init(bar_slot_full + 8 * s, kIssuers); mbar_init(bar_slot_free + 8 * s, 4); }
+        for (int s = 0; s < kRawStages; ++s) { mbar_init(bar_raw_full + 8 * s, 1); mbar_init(bar_raw_empty + 8 * s, 128); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -320,6 +333,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     for (int i = threadIdx.x; i < a.KB * 32; i += kNT) bias_s[i] = (a.bias && i < a.K) ? a.bias[i] : 0.0f;
+    if (DW)
+        for (int i = threadIdx.x; i < a.CBr * 10 * 32; i += kNT) {
+            const int cb = i / 320, rest = i - cb * 320, tap = rest >> 5, c = rest & 31;
+            dw_s_w[i] = tap < 9 ? a.dw_w[(cb * 9 + tap) * 32 + c] : (a.dw_bias && cb * 32 + c < a.dw_C ? a.dw_bias[cb * 32 + c] : 0.0f);
+        }
     // view tap (x', y') of phase plane (ph, pw) is the original tap x = S (x' - pt') + ph + pt, y likewise, if it exists
     for (int i = threadIdx.x; i < a.n_phase * T; i += kNT) {
         const int p = i / T, tv = i - p * T, xv = tv / a.FW, yv = tv - xv * a.FW;
@@ -344,9 +362,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // the tensor pipe may have to wait for.
     if (warp == 0 && lane == 0) {
         // ---- input strips: one box per (tile, channel block)
-        drain_bar = bar_a_full;
+        drain_bar = DW ? bar_raw_full : bar_a_full;
         bool alive = true, wrapped = false;
         uint32_t s = 0, phase = 0;
+        if (DW) {
+            // fused depthwise: one halo box of the layer's input per (tile, channel block), into the raw-tile ring
+            for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+                const Tile tl = decode_tile(a, t);
+                for (int cb = 0; cb < a.CBr; ++cb) {
+                    if (wrapped) alive = mbar_wait(bar_raw_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                    if (!alive) break;
+                    mbar_expect_tx(bar_raw_full + 8 * s, a.raw_box_bytes);
+                    tma_load_5d(raw_base + s * a.raw_stage_bytes, &map_a, bar_raw_full + 8 * s, 0, -a.dw_pl, tl.row0 * a.dw_s - a.dw_pt, cb, tl.n0);
+                    armed_mask |= 1u << s;
+                    armed_parity = (armed_parity & ~(1u << s)) | (phase << s);
+                    if (++s == (uint32_t)kRawStages) { s = 0; phase ^= 1u; wrapped = true; }
+                }
+            }
+        } else
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const Tile tl = decode_tile(a, t);
             // one box per (phase plane, real channel block); with stride 2 the map's element strides pick every
@@ -506,7 +539,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int cb = 0, plane = 0;
             unsigned long long taps = mask0;
             for (int blk = 0; blk < a.CB && alive; ++blk) {       // blocks = phase planes x real channel blocks
-                alive = mbar_wait((X3 ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status);   // 3xTF32: once split
+                alive = mbar_wait(((X3 || DW) ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status);   // once split / computed
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
                 if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, r_sel, started, w_res);
@@ -523,6 +556,55 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         };
         if (kIssuers == 1 || warp == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, kIssuers == 1 ? CH : kSplit>{});
         else mma_role(std::integral_constant<int, kSplit>{}, std::integral_constant<int, CH>{});
+    } else if (DW && warp >= 8) {
+        // ---- fused depthwise 3x3: halo tile -> strip.  One item = 4 channels of one output pixel: nine 16-byte loads
+        // from the halo tile, FMAs, bias, ReLU, one 16-byte store at the swizzled place of the K-major strip.
+        const int tid = threadIdx.x - 256;
+        bool alive = true, wrapped = false;
+        uint32_t r = 0, pr = 0, s = 0, ps = 0;
+        const int px_img = a.dw_rows * a.OW;                     // strip pixels per image (row pitch = OW: a 1x1 view)
+        const int items = a.nn * px_img * 8;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x)
+            for (int cb = 0; cb < a.CBr; ++cb) {
+                alive = mbar_wait_warp(bar_raw_full + 8 * r, pr, abort_flag, a.status);
+                if (alive && wrapped) alive = mbar_wait_warp(bar_a_empty + 8 * s, ps ^ 1u, abort_flag, a.status);
+                if (!alive) break;
+                const float4 *raw = reinterpret_cast<const float4 *>(base_ptr + (raw_base - base) + (size_t)r * a.raw_stage_bytes);
+                float4 *hi = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes);
+                float4 *lo = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + a.a_half);
+                const float4 *w4 = reinterpret_cast<const float4 *>(dw_s_w + cb * 320);
+                for (int i = tid; i < items; i += 128) {
+                    const int j = i & 7, q = i >> 3;
+                    const int img = q / px_img, rem = q - img * px_img;
+                    const int rr = rem / a.OW, ow = rem - rr * a.OW;
+                    const float4 *src = raw + ((size_t)(img * a.dw_Hb + rr * a.dw_s) * a.dw_Wb + ow * a.dw_s) * 8 + j;
+                    float4 acc = w4[9 * 8 + j];                                   // bias
+#pragma unroll
+                    for (int x = 0; x < 3; ++x)
+#pragma unroll
+                        for (int y = 0; y < 3; ++y) {
+                            const float4 v = src[(x * a.dw_Wb + y) * 8];
+                            const float4 w = w4[(x * 3 + y) * 8 + j];
+                            acc.x = fmaf(v.x, w.x, acc.x); acc.y = fmaf(v.y, w.y, acc.y);
+                            acc.z = fmaf(v.z, w.z, acc.z); acc.w = fmaf(v.w, w.w, acc.w);
+                        }
+                    if (a.dw_relu) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+                    const int at = q * 8 + (j ^ (q & 7));                          // 128-byte swizzle of the K-major strip
+                    if (X3) {
+                        const float4 h = make_float4(__uint_as_float(__float_as_uint(acc.x) & 0xffffe000u), __uint_as_float(__float_as_uint(acc.y) & 0xffffe000u),
+                                                     __uint_as_float(__float_as_uint(acc.z) & 0xffffe000u), __uint_as_float(__float_as_uint(acc.w) & 0xffffe000u));
+                        hi[at] = h;
+                        lo[at] = make_float4(acc.x - h.x, acc.y - h.y, acc.z - h.z, acc.w - h.w);
+                    } else {
+                        hi[at] = acc;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these writes are read by the tensor core
+                mbar_arrive(bar_a_split + 8 * s);
+                mbar_arrive(bar_raw_empty + 8 * r);
+                if (++r == (uint32_t)kRawStages) { r = 0; pr ^= 1u; }
+                if (++s == (uint32_t)kAStages) { s = 0; ps ^= 1u; wrapped = true; }
+            }
     } else if (X3 && warp >= 8) {
         // ---- 3xTF32: split each strip as it lands.  Elementwise at equal offsets, so the swizzled layout carries over.
         const int tid = threadIdx.x - 256;
@@ -691,7 +773,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 size_t ctrl_bytes(int KB) { return kCtrlBarrierBytes + 16 + (size_t)KB * 32 * 4 + kTapTabEntries * sizeof(short); }
 
 // Plan with at most `max_px` pixels per tile in the given orientation; ok = false when it does not fit.
-TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc, bool pack_ok, int group_k) {
+TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, int S, double taps_eff, bool x3, int racc, bool pack_ok, int group_k, const DwFuse *dw) {
     TcPlan p{};
     p.ok = false;
     if (g.S != 1) return p;                      // g is the stride-1 view; S scales the TMA box of the real tensor
@@ -769,7 +851,18 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
     // shared memory.  When one filter tile covers the layer and all its (channel block, tap) boxes fit beside enough
     // strips, the filters are loaded once and stay; otherwise at least two strips and two filter boxes, and the rest
     // shared out as described below.
-    const size_t fixed = 1024 + ctrl_bytes(g.KB);
+    size_t dw_extra = 0;
+    if (dw) {
+        // the depthwise result of whole output rows (or whole images) is computed from one halo box of the input
+        if (p.nn == 1 && p.px_tile % p.Wq != 0) return p;
+        p.dw_rows = p.nn == 1 ? p.px_tile / p.Wq : p.Hq;
+        p.dw_Hb = (p.dw_rows - 1) * dw->s + 3;
+        p.dw_Wb = (g.OW - 1) * dw->s + 3;
+        if (p.dw_Hb > 256 || p.dw_Wb > 256) return p;
+        p.raw_stage_bytes = (uint32_t)(((size_t)p.nn * p.dw_Hb * p.dw_Wb * 128 + 1023) & ~(size_t)1023);
+        dw_extra = (size_t)kRawStages * p.raw_stage_bytes + (size_t)g.CB * 320 * sizeof(float);
+    }
+    const size_t fixed = 1024 + ctrl_bytes(g.KB) + dw_extra;
     const size_t all_b = (size_t)g.CB * g.FH * g.FW * b_stage;
     p.b_resident = 0;
     if (p.n_tiles == 1 && fixed + all_b + 2 * (size_t)p.a_stage_bytes <= max_smem) {
@@ -851,7 +944,7 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
 
 // The cheapest plan over both orientations and the tile sizes that fit (wide rows or tall windows leave room for
 // fewer pixels per tile).  The pixels-on-M orientation stores 32-byte vectors and needs `out` aligned to 32 bytes.
-TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3, bool pack_ok, int group_k = 0) {
+TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, int S, double taps_eff, bool x3, bool pack_ok, int group_k = 0, const DwFuse *dw = nullptr) {
     // 3xTF32 keeps every accumulation chain within kMaxKStepsX3 K steps by rotating the channel blocks over 2 or 4
     // accumulators (added up in the epilogue); TF32's tolerance needs none of that
     int racc = 1;
@@ -864,7 +957,7 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, in
     double best_cost = 0.0;
     for (int pixel_m = 0; pixel_m <= (out_aligned32 ? 1 : 0); ++pixel_m)
         for (int px = kSlots * kSlotPx; px >= 64; px -= 64) {
-            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc, pack_ok, group_k);
+            TcPlan p = make_plan_with(g, max_smem, px, pixel_m, S, taps_eff, x3, racc, pack_ok, group_k, dw);
             if (!p.ok) continue;
             const double c = plan_cost(p, g, sms);
             if (!best.ok || c < best_cost) { best = p; best_cost = c; }
@@ -875,27 +968,28 @@ TcPlan make_plan(const Geom &g, size_t max_smem, int sms, bool out_aligned32, in
 typedef void (*TcKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
 
 template <int CH, int KS, bool PM>
-TcKernel pick_flags(bool masked, bool x3) {
-    if (x3) return masked ? conv_tc_kernel<CH, KS, PM, true, true> : conv_tc_kernel<CH, KS, PM, false, true>;
-    return masked ? conv_tc_kernel<CH, KS, PM, true, false> : conv_tc_kernel<CH, KS, PM, false, false>;
+TcKernel pick_flags(bool masked, bool x3, bool dw) {
+    if (dw) return masked ? nullptr : x3 ? conv_tc_kernel<CH, KS, PM, false, true, true> : conv_tc_kernel<CH, KS, PM, false, false, true>;
+    if (x3) return masked ? conv_tc_kernel<CH, KS, PM, true, true, false> : conv_tc_kernel<CH, KS, PM, false, true, false>;
+    return masked ? conv_tc_kernel<CH, KS, PM, true, false, false> : conv_tc_kernel<CH, KS, PM, false, false, false>;
 }
 template <int CH, bool PM>
-TcKernel pick_ks(int ks, bool masked, bool x3) {
+TcKernel pick_ks(int ks, bool masked, bool x3, bool dw) {
     switch (ks) {
-        case 1: return pick_flags<CH, 1, PM>(masked, x3);
-        case 2: return pick_flags<CH, 2, PM>(masked, x3);
-        case 4: return pick_flags<CH, 4, PM>(masked, x3);
+        case 1: return pick_flags<CH, 1, PM>(masked, x3, dw);
+        case 2: return pick_flags<CH, 2, PM>(masked, x3, dw);
+        case 4: return pick_flags<CH, 4, PM>(masked, x3, dw);
         default: return nullptr;
     }
 }
 // Filters on M: one chain per accumulator slot (1 or 2); pixels on M: one per 128-pixel chunk (1 to 4).
-TcKernel pick_kernel(int chains, int ks, bool pixel_m, bool masked, bool x3) {
-    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks, masked, x3) : chains == 2 ? pick_ks<2, false>(ks, masked, x3) : nullptr;
+TcKernel pick_kernel(int chains, int ks, bool pixel_m, bool masked, bool x3, bool dw) {
+    if (!pixel_m) return chains == 1 ? pick_ks<1, false>(ks, masked, x3, dw) : chains == 2 ? pick_ks<2, false>(ks, masked, x3, dw) : nullptr;
     switch (chains) {
-        case 1: return pick_ks<1, true>(ks, masked, x3);
-        case 2: return pick_ks<2, true>(ks, masked, x3);
-        case 3: return pick_ks<3, true>(ks, masked, x3);
-        case 4: return pick_ks<4, true>(ks, masked, x3);
+        case 1: return pick_ks<1, true>(ks, masked, x3, dw);
+        case 2: return pick_ks<2, true>(ks, masked, x3, dw);
+        case 3: return pick_ks<3, true>(ks, masked, x3, dw);
+        case 4: return pick_ks<4, true>(ks, masked, x3, dw);
         default: return nullptr;
     }
 }
@@ -932,10 +1026,10 @@ struct Virt { Geom g; int S, n_phase, CBr, phase_bits, FHo, FWo, pto, plo; doubl
 
 static int floor_half(int v) { return v >= 0 ? v / 2 : -((1 - v) / 2); }
 
-static bool make_virt(const Geom &g_in, Virt &v) {
+static bool make_virt(const Geom &g_in, Virt &v, bool keep_rows = false) {
     v.S = g_in.S; v.FHo = g_in.FH; v.FWo = g_in.FW; v.pto = g_in.pt; v.plo = g_in.pl; v.CBr = g_in.CB;
     if (g_in.S == 1) {
-        v.g = flatten_pointwise(g_in);
+        v.g = keep_rows ? g_in : flatten_pointwise(g_in);
         v.n_phase = 1; v.phase_bits = 0; v.taps_eff = (double)g_in.FH * g_in.FW;
         return true;
     }
@@ -963,28 +1057,38 @@ static bool make_virt(const Geom &g_in, Virt &v) {
 }
 
 // groups > 1: g describes one group's channels (C = F_C) and all the filters (K = groups * filters per group)
-bool conv_tc_supported(const Geom &g, bool x3, int groups) {
+bool conv_tc_supported(const Geom &g, bool x3, int groups, const DwFuse *dw) {
     Virt v;
-    if (!make_virt(g, v)) return false;
+    if (!make_virt(g, v, dw != nullptr)) return false;
+    if (dw) return groups == 1 && make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, false, 0, dw).ok;
     if (groups > 1) return (g.C % 32 == 0) && (g.K % (32 * groups) == 0) &&
                            make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, false, g.K / groups).ok;
     return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, v.CBr == 1 && g.C <= 16).ok;
 }
 
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
-                   const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st, int groups) {
+                   const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st, int groups, const DwFuse *dw) {
     const bool x3 = mode == SMALL_MATH_3XTF32;
     if (x3 && !w_lo) return SMALL_ERR_INVALID_ARG;
     Virt v;
-    if (!make_virt(g_in, v)) return SMALL_ERR_UNSUPPORTED;
+    if (!make_virt(g_in, v, dw != nullptr)) return SMALL_ERR_UNSUPPORTED;
     const Geom &g = v.g;
     TcPlan p = make_plan(g, ctx->max_smem_optin < 227 * 1024 ? ctx->max_smem_optin : 227 * 1024, ctx->sm_count,
-                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3, groups == 1 && v.CBr == 1 && g_in.C <= 16,
-                         groups > 1 ? g_in.K / groups : 0);
+                         (reinterpret_cast<uintptr_t>(out) & 31u) == 0, v.S, v.taps_eff, x3, groups == 1 && !dw && v.CBr == 1 && g_in.C <= 16,
+                         groups > 1 ? g_in.K / groups : 0, dw);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_a, map_b, map_b_lo;
-    {   // activations: [N][CB][H][W][32 floats]; box = 32 x Wq x Rs x 1 x nn, out-of-range elements read as zero
+    if (dw) {   // fused depthwise: halo boxes of the depthwise layer's input, read by CUDA threads (no swizzle)
+        cuuint64_t dims[5] = {32, (cuuint64_t)dw->W, (cuuint64_t)dw->H, (cuuint64_t)v.CBr, (cuuint64_t)g.N};
+        cuuint64_t strides[4] = {128, (cuuint64_t)dw->W * 128, (cuuint64_t)dw->H * dw->W * 128, (cuuint64_t)v.CBr * dw->H * dw->W * 128};
+        cuuint32_t box[5] = {32, (cuuint32_t)p.dw_Wb, (cuuint32_t)p.dw_Hb, 1, (cuuint32_t)p.nn};
+        cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float *>(in), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
+    } else {   // activations: [N][CB][H][W][32 floats]; box = 32 x Wq x Rs x 1 x nn, out-of-range elements read as zero
         // the real tensor (for stride 1 possibly with a 1x1 layer's rows re-cut); with stride 2 the box spans 2 Wq x 2 Rs
         // elements and the element strides keep every other one, so shared memory receives Wq x Rs pixels either way
         const int Hr = v.S == 1 ? g.H : g_in.H, Wr = v.S == 1 ? g.W : g_in.W;
@@ -1027,6 +1131,11 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
     a.rows_tile = (p.nn == 1 && p.px_tile % p.Wq == 0) ? p.px_tile / p.Wq : 0;
     a.cb_group = groups > 1 ? v.CBr : 0;
+    if (dw) {
+        a.dw_w = dw->w; a.dw_bias = dw->bias; a.dw_C = dw->C; a.dw_s = dw->s; a.dw_pt = dw->pt; a.dw_pl = dw->pl; a.dw_relu = dw->relu;
+        a.dw_Wb = p.dw_Wb; a.dw_Hb = p.dw_Hb; a.dw_rows = p.dw_rows; a.raw_stage_bytes = p.raw_stage_bytes;
+        a.raw_box_bytes = (uint32_t)((size_t)p.nn * p.dw_Hb * p.dw_Wb * 128);
+    }
     int chains;
     if (p.pixel_m) {
         a.n_slot = p.cps * 128;
@@ -1039,13 +1148,13 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     }
     const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
     a.relu = relu; a.accumulate = accumulate;
-    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3);
+    const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3, dw != nullptr);
     if (!kern) return SMALL_ERR_UNSUPPORTED;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
-    kern<<<grid, x3 ? kThreadsX3 : kThreads, p.smem_bytes, st>>>(map_a, map_b, map_b_lo, a);
+    kern<<<grid, (x3 || dw) ? kThreadsX3 : kThreads, p.smem_bytes, st>>>(map_a, map_b, map_b_lo, a);
     return check_launch(ctx);
 }
 
