@@ -512,6 +512,19 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
         wdw = torch.from_numpy(synth.uniform((C, 3, 3), -1.0, 1.0, 800 + C)).to(dev)
         wdb = torch.empty(B.small_dw_weight_elems(C, 3, 3), device=dev)
         B.small_pack_dw_weights(ctx, wdw, wdb, C, 3, 3)
+        # depthwise 3x3 -> 1x1 as one fused layer (C -> C): no intermediate tensor in the algorithmic bytes
+        wpw = torch.from_numpy(synth.uniform((C, C, 1, 1), -1.0, 1.0, 850 + C)).to(dev)
+        wpb = torch.empty(B.small_conv_weight_elems(C, C, 1, 1, B.MATH_3XTF32), device=dev)
+        B.small_pack_conv_weights(ctx, wpw, wpb, C, C, 1, 1, B.MATH_3XTF32)
+        for mode in ("tf32", "3xtf32"):
+            if not B.small_dwpw_fused(N, C, C, HW, HW, 1, (1, 1, 1, 1), B.MATH[mode]):
+                continue
+            def fz(mode=mode):
+                a, o = rot()
+                B.small_dwpw_conv2d(ctx, a, wdb, bias, wpb, bias, o, None, N, C, C, HW, HW, 1, (1, 1, 1, 1), B.RELU | B.RELU_MID | B.MATH[mode])
+            tmin, tmed = time_launch(fz, inner=10)
+            record("dw3x3+conv1x1_fused", mode, 2.0 * N * HW * HW * C * (9 + C), 4.0 * (2 * N * C * HW * HW + C * C + 12 * C), tmin, tmed, mode)
+        del wpw, wpb
 
         def dw():
             a, o = rot()

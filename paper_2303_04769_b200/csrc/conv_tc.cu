@@ -45,6 +45,7 @@ namespace {
 
 constexpr int kThreads = 256;            // roles of the TF32 kernel; the 3xTF32 kernel adds four splitting warps
 constexpr int kThreadsX3 = 384;
+constexpr int kThreadsDW = 512;          // fused depthwise: eight warps compute the strips
 constexpr int kSlots = 2;              // accumulator slots of 256 tensor-memory columns
 constexpr int kSlotPx = 256;           // pixels per slot = the MMA's largest N
 constexpr int kFilterTile = 128;       // filters per tile = the MMA's M
@@ -275,10 +276,11 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs &a, int t) {
 // input, warps 8-11 compute the depthwise result straight into the strip the MMAs read (and split it for 3xTF32),
 // so the depthwise output never goes to global memory.
 template <int CH, int KS_LAST, bool PM, bool MASKED, bool X3, bool DW>
-__global__ void __launch_bounds__((X3 || DW) ? kThreadsX3 : kThreads, 1)
+__global__ void __launch_bounds__(DW ? kThreadsDW : X3 ? kThreadsX3 : kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_b_lo, const TcArgs a) {
-    constexpr int kNT = (X3 || DW) ? kThreadsX3 : kThreads;
+    constexpr int kNT = DW ? kThreadsDW : X3 ? kThreadsX3 : kThreads;
+    constexpr int kXform = DW ? 256 : 128;     // threads that split (3xTF32) or compute (fused depthwise) the strips
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -311,10 +313,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         // every MMA issuer commits to the stage-empty and slot-full barriers; 4 epilogue warps free a slot
-        for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, kIssuers); mbar_init(bar_a_split + 8 * s, 128); }
+        for (int s = 0; s < kAStages; ++s) { mbar_init(bar_a_full + 8 * s, 1); mbar_init(bar_a_empty + 8 * s, kIssuers); mbar_init(bar_a_split + 8 * s, kXform); }
         for (int s = 0; s < a.b_stages; ++s) { mbar_init(bar_b_full + 8 * s, 1); mbar_init(bar_b_empty + 8 * s, kIssuers); }
         for (int s = 0; s < kSlots; ++s) { mbar_init(bar_slot_full + 8 * s, kIssuers); mbar_init(bar_slot_free + 8 * s, 4); }
-        for (int s = 0; s < kRawStages; ++s) { mbar_init(bar_raw_full + 8 * s, 1); mbar_init(bar_raw_empty + 8 * s, 128); }
+        for (int s = 0; s < kRawStages; ++s) { mbar_init(bar_raw_full + 8 * s, 1); mbar_init(bar_raw_empty + 8 * s, kXform); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -557,13 +559,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (kIssuers == 1 || warp == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, kIssuers == 1 ? CH : kSplit>{});
         else mma_role(std::integral_constant<int, kSplit>{}, std::integral_constant<int, CH>{});
     } else if (DW && warp >= 8) {
-        // ---- fused depthwise 3x3: halo tile -> strip.  One item = 4 channels of one output pixel: nine 16-byte loads
-        // from the halo tile, FMAs, bias, ReLU, one 16-byte store at the swizzled place of the K-major strip.
+        // ---- fused depthwise 3x3: halo tile -> strip (FMAs, bias, ReLU, 16-byte stores at the swizzled places of the
+        // K-major strip the MMAs read).
         const int tid = threadIdx.x - 256;
         bool alive = true, wrapped = false;
         uint32_t r = 0, pr = 0, s = 0, ps = 0;
         const int px_img = a.dw_rows * a.OW;                     // strip pixels per image (row pitch = OW: a 1x1 view)
-        const int items = a.nn * px_img * 8;
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x)
             for (int cb = 0; cb < a.CBr; ++cb) {
                 alive = mbar_wait_warp(bar_raw_full + 8 * r, pr, abort_flag, a.status);
@@ -573,30 +574,58 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 float4 *hi = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes);
                 float4 *lo = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + a.a_half);
                 const float4 *w4 = reinterpret_cast<const float4 *>(dw_s_w + cb * 320);
-                for (int i = tid; i < items; i += 128) {
-                    const int j = i & 7, q = i >> 3;
-                    const int img = q / px_img, rem = q - img * px_img;
-                    const int rr = rem / a.OW, ow = rem - rr * a.OW;
-                    const float4 *src = raw + ((size_t)(img * a.dw_Hb + rr * a.dw_s) * a.dw_Wb + ow * a.dw_s) * 8 + j;
-                    float4 acc = w4[9 * 8 + j];                                   // bias
+                // One unit = 4 channels (chunk j) of one output column of one image; the thread walks down the column
+                // with the 3x3 window in registers, so each output costs three (stride 2: six) 16-byte loads.  j is
+                // the same for all units of a thread (128 threads, 8 chunks), so its nine filter vectors load once.
+                const int j = tid & 7;                                  // (256 threads: 32 column groups in flight)
+                float4 wv[9];
 #pragma unroll
-                    for (int x = 0; x < 3; ++x)
+                for (int k = 0; k < 9; ++k) wv[k] = w4[k * 8 + j];
+                const float4 bias4 = w4[9 * 8 + j];
+                const int units = a.nn * a.OW;                       // (image, column) pairs; this thread takes every 16th
+                for (int u = tid >> 3; u < units; u += kXform / 8) {
+                    const int img = u / a.OW, ow = u - img * a.OW;
+                    const float4 *col = raw + ((size_t)img * a.dw_Hb * a.dw_Wb + ow * a.dw_s) * 8 + j;
+                    const int q0 = img * px_img + ow;
+                    float4 win[3][3];
+                    // rows 0 .. (3 - stride) - 1 of the first window; the loop loads the remaining `stride` rows per output
+                    if (a.dw_s == 1) {
 #pragma unroll
-                        for (int y = 0; y < 3; ++y) {
-                            const float4 v = src[(x * a.dw_Wb + y) * 8];
-                            const float4 w = w4[(x * 3 + y) * 8 + j];
-                            acc.x = fmaf(v.x, w.x, acc.x); acc.y = fmaf(v.y, w.y, acc.y);
-                            acc.z = fmaf(v.z, w.z, acc.z); acc.w = fmaf(v.w, w.w, acc.w);
-                        }
-                    if (a.dw_relu) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
-                    const int at = q * 8 + (j ^ (q & 7));                          // 128-byte swizzle of the K-major strip
-                    if (X3) {
-                        const float4 h = make_float4(__uint_as_float(__float_as_uint(acc.x) & 0xffffe000u), __uint_as_float(__float_as_uint(acc.y) & 0xffffe000u),
-                                                     __uint_as_float(__float_as_uint(acc.z) & 0xffffe000u), __uint_as_float(__float_as_uint(acc.w) & 0xffffe000u));
-                        hi[at] = h;
-                        lo[at] = make_float4(acc.x - h.x, acc.y - h.y, acc.z - h.z, acc.w - h.w);
+                        for (int y = 0; y < 3; ++y) { win[1][y] = col[y * 8]; win[2][y] = col[(a.dw_Wb + y) * 8]; }
                     } else {
-                        hi[at] = acc;
+#pragma unroll
+                        for (int y = 0; y < 3; ++y) win[2][y] = col[y * 8];
+                    }
+                    for (int rr = 0; rr < a.dw_rows; ++rr) {
+                        if (a.dw_s == 1) {
+                            const float4 *row = col + (size_t)(rr + 2) * a.dw_Wb * 8;
+#pragma unroll
+                            for (int y = 0; y < 3; ++y) { win[0][y] = win[1][y]; win[1][y] = win[2][y]; win[2][y] = row[y * 8]; }
+                        } else {
+                            const float4 *row = col + (size_t)(2 * rr + 1) * a.dw_Wb * 8;
+#pragma unroll
+                            for (int y = 0; y < 3; ++y) { win[0][y] = win[2][y]; win[1][y] = row[y * 8]; win[2][y] = row[(a.dw_Wb + y) * 8]; }
+                        }
+                        float4 acc = bias4;
+#pragma unroll
+                        for (int x = 0; x < 3; ++x)
+#pragma unroll
+                            for (int y = 0; y < 3; ++y) {
+                                const float4 v = win[x][y], w = wv[x * 3 + y];
+                                acc.x = fmaf(v.x, w.x, acc.x); acc.y = fmaf(v.y, w.y, acc.y);
+                                acc.z = fmaf(v.z, w.z, acc.z); acc.w = fmaf(v.w, w.w, acc.w);
+                            }
+                        if (a.dw_relu) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+                        const int q = q0 + rr * a.OW;
+                        const int at = q * 8 + (j ^ (q & 7));                      // 128-byte swizzle of the K-major strip
+                        if (X3) {
+                            const float4 h = make_float4(__uint_as_float(__float_as_uint(acc.x) & 0xffffe000u), __uint_as_float(__float_as_uint(acc.y) & 0xffffe000u),
+                                                         __uint_as_float(__float_as_uint(acc.z) & 0xffffe000u), __uint_as_float(__float_as_uint(acc.w) & 0xffffe000u));
+                            hi[at] = h;
+                            lo[at] = make_float4(acc.x - h.x, acc.y - h.y, acc.z - h.z, acc.w - h.w);
+                        } else {
+                            hi[at] = acc;
+                        }
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these writes are read by the tensor core
@@ -1154,7 +1183,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
-    kern<<<grid, (x3 || dw) ? kThreadsX3 : kThreads, p.smem_bytes, st>>>(map_a, map_b, map_b_lo, a);
+    kern<<<grid, dw ? kThreadsDW : x3 ? kThreadsX3 : kThreads, p.smem_bytes, st>>>(map_a, map_b, map_b_lo, a);
     return check_launch(ctx);
 }
 
