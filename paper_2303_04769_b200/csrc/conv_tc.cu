@@ -1,21 +1,22 @@
-// Full channel reduction on the tensor cores (paper Section 3.2 item 4; Algorithms 1 and 2) for stride-1 windows:
-// an implicit GEMM straight from the blocked layout, with no im2col buffer and no reformatting (Section 4.4).
+// Full channel reduction on the tensor cores (paper Section 3.2 item 4; Algorithms 1 and 2), strides 1 and 2: an
+// implicit GEMM straight from the blocked layout, with no im2col buffer and no reformatting (Section 4.4).
 //
 //   D[k, pixel] = sum over (channel block cb, tap (x,y), 32 channels ci)  W[k, ci] * X[pixel + shift(x,y), ci]
 //
 // How the paper's loop nest maps onto the SM:
-//   k block loop (parallel)        -> filter tiles of 128 (the MMA's M rows), one tile = (pixel tile, filter tile)
+//   k block loop (parallel)        -> filter tiles, one tile = (pixel tile, filter tile); groups = filter tiles too
 //   i loop over F_C in F_Cb steps  -> cb loop over 32-channel blocks: one TMA box of the input per block
 //   x, y kernel loops              -> taps: the SAME shared-memory strip is re-read with a shifted start address
-//   ii loop                        -> four K=8 TF32 MMAs per 32-channel block (tcgen05.mma kind::tf32)
-//   O_wb x K_b register tile       -> 128 filters x up to 256 pixels per accumulator slot in tensor memory, 2 slots
+//   ii loop                        -> up to four K=8 TF32 MMAs per 32-channel block (tcgen05.mma kind::tf32)
+//   O_wb x K_b register tile       -> accumulator slots in tensor memory (2 slots x 256 columns x 128 lanes)
 //   LOAD / STORE phases            -> epilogue: tensor memory -> registers, + bias, (+ previous output), ReLU, store
 //
-// Filters are the MMA's M operand and pixels its N operand because the pipe only runs at full rate for N = 256
-// (measured with this library's issue probe: 128 cycles per 128x256x8 MMA, but about 119 cycles for any N <= 224),
-// and a layer always has hundreds of pixels while it may have only 64 or 128 filters.  As a bonus the accumulator
-// comes out as [filter][pixel]: a warp holds 32 consecutive filters of one pixel = one 128-byte line of the blocked
-// output, so every store is fully coalesced.
+// Two orientations, chosen per layer by the host's cost model.  Filters on the MMA's M axis: 128 filters x up to 256
+// pixels per slot; the accumulator comes out as [filter][pixel], a warp holds 32 consecutive filters of one pixel =
+// one 128-byte line of the blocked output, so its 4-byte stores are fully coalesced.  Pixels on M: 128-pixel chunks x
+// up to 256 filters; a thread holds 32 filters of its pixel and stores the line as four 32-byte vectors - the choice for
+// layers with few filters, where M = 128 filters would be mostly padding.  The pipe needs N / 2 cycles per 128 x N x 8
+// MMA for N >= 128 and 40 to 52 cycles below that, whatever M is (measured with this library's issue probe).
 //
 // The strip.  A blocked input plane is [H][W][32 floats]: one pixel and channel block = one 128-byte row, the K-major
 // operand row of a TF32 MMA with the 128-byte swizzle.  TMA copies a box of Rs rows x Wq pixels (starting at column
@@ -25,14 +26,16 @@
 // numbered with pitch Wq) needs strip pixel q + x*Wq + y for tap (x, y).  Any run of consecutive q is a valid MMA
 // operand: rows 128 bytes apart, start address (q + x*Wq + y) * 128.  Columns ow >= OW of each row are computed and
 // dropped.  Small planes put several whole images in one strip the same way (image pitch Hq = H + max(pad_t, pad_b)).
+// Stride 2 is a stride-1 window over the input's phase planes (see Virt); 3xTF32 and the fused depthwise layer put a
+// transform between the copy and the MMAs (see the X3 and DW template flags).
 //
 // Persistent CTAs (one per SM) walk the tile list with stride gridDim.x.  Roles: warp 0 = TMA producer for input
-// strips, warp 2 = TMA producer for filter tiles, warp 1 = MMA issuer (one elected thread each), warps 4-7 = epilogue
-// (warp q owns filters 32q..32q+31 of the tile).  The producers run ahead across tiles; accumulator slots are handed
-// back to the MMA issuer as soon as the epilogue has read them out of tensor memory, so the next tile's MMAs overlap
-// the current tile's stores (one-slot tiles alternate between the two slots).  Every mbarrier wait is bounded; on
-// expiry the kernel records SMALL_ERR_TIMEOUT in the context's status word, lets its in-flight copies land, frees
-// tensor memory and returns.
+// strips, warp 2 = TMA producer for filter tiles, warps 1 and 3 = MMA issuers (one thread each; a tile's chains are
+// split between them), warps 4-7 = epilogue, warps 8 and up = strip transform where there is one.  The producers run
+// ahead across tiles; accumulator slots are handed back to the issuers as soon as the epilogue has read them out of
+// tensor memory, so the next tile's MMAs overlap the current tile's stores (one-slot tiles alternate between the two
+// slots).  Every mbarrier wait is bounded; on expiry the kernel records SMALL_ERR_TIMEOUT in the context's status
+// word, lets its in-flight copies land, frees tensor memory and returns.
 #include <cuda.h>
 
 #include <type_traits>
