@@ -407,6 +407,27 @@ def gpu_main(args):
             del ag, an
         other_workloads["autoencoder_fc"] = {"batch": aN, "layers": len(anet["layers"]), "modes": res}
         del ax, ablk
+        # the other two network workloads of the configuration list, at their full batch, same protocol
+        for wname in ("dwsep_cnn", "kws_cnn"):
+            wnet = configs.NETWORKS[wname]()
+            wN = wnet["batch"]
+            wparams = configs.make_params(wnet)
+            wx = torch.from_numpy(configs.make_input(wnet, wN)).to(dev)
+            wblk = torch.empty(B.small_packed_elems(wN, *wnet["input"]), device=dev)
+            B.small_pack(ctx, wx, wblk, wN, *wnet["input"])
+            res = {}
+            for m in ("3xtf32", "tf32", "fp32"):
+                wn = Net(ctx, wnet, wparams, math=m, device=dev)
+                wn.run(wblk)
+                torch.cuda.synchronize()
+                wg = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(wg):
+                    wn.run(wblk)
+                wms = timed(lambda i: wg.replay(), min(args.steps, 100), 5)
+                res[m] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms}
+                del wg, wn
+            other_workloads[wname] = {"batch": wN, "layers": len(wnet["layers"]), "modes": res}
+            del wx, wblk
 
     # the library's own issue-rate probe: what the TF32 pipe sustains with operands resident in shared memory
     probe = None
