@@ -424,8 +424,18 @@ def gpu_main(args):
                 with torch.cuda.graph(wg):
                     wn.run(wblk)
                 wms = timed(lambda i: wg.replay(), min(args.steps, 100), 5)
-                res[m] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms}
+                res[m] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms, "launches": len(wn.layer_rows)}
                 del wg, wn
+                if m != "fp32":     # the same network with every depthwise and 1x1 layer launched on its own
+                    wn = Net(ctx, wnet, wparams, math=m, device=dev, fuse_dwpw=False)
+                    wn.run(wblk)
+                    torch.cuda.synchronize()
+                    wg = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(wg):
+                        wn.run(wblk)
+                    wms = timed(lambda i: wg.replay(), min(args.steps, 100), 5)
+                    res[m + "_unfused"] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms, "launches": len(wn.layer_rows)}
+                    del wg, wn
             other_workloads[wname] = {"batch": wN, "layers": len(wnet["layers"]), "modes": res}
             del wx, wblk
 

@@ -216,7 +216,8 @@ int small_fc(small_ctx *ctx, const float *in, const float *w_blk, const float *b
 
 /* ---- networks (Section 5.3: layers share intermediate buffers; Section 5.4: end-to-end inference) -- */
 
-enum { SMALL_OP_CONV = 0, SMALL_OP_DWCONV = 1, SMALL_OP_POOL = 2, SMALL_OP_RELU = 3, SMALL_OP_ADD = 4, SMALL_OP_FC = 5 };
+enum { SMALL_OP_CONV = 0, SMALL_OP_DWCONV = 1, SMALL_OP_POOL = 2, SMALL_OP_RELU = 3, SMALL_OP_ADD = 4, SMALL_OP_FC = 5,
+       SMALL_OP_DWPW = 6 };  /* depthwise 3x3 then 1x1 convolution as one fused layer (small_dwpw_conv2d) */
 enum { SMALL_SLOT_INPUT = -1, SMALL_SLOT_OUTPUT = -2 }; /* the caller's in_blk / out_blk */
 
 typedef struct small_layer {
@@ -225,12 +226,15 @@ typedef struct small_layer {
     int H, W;               /* input plane (1 x 1 for FC) */
     int FH, FW, stride;     /* window and stride (CONV, DWCONV, POOL) */
     int pad_t, pad_b, pad_l, pad_r;
-    unsigned flags;         /* SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_* as the op allows */
+    unsigned flags;         /* SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_* as the op allows; DWPW: RELU, RELU_MID and a
+                             * tensor-core math mode - the shape must be one small_dwpw_fused accepts */
     int pool_mode;          /* SMALL_POOL_* */
     const float *w_blk;     /* packed filters (device) or NULL */
     const float *bias;      /* device or NULL */
     int src, dst;           /* slot ids >= 0, or SMALL_SLOT_INPUT / SMALL_SLOT_OUTPUT */
     int src2;               /* second operand of ADD; ignored otherwise */
+    const float *w_blk2;    /* DWPW: packed 1x1 filters (w_blk, bias are the depthwise layer's); else ignored */
+    const float *bias2;     /* DWPW: bias of the 1x1 convolution or NULL */
 } small_layer;
 
 /* Bytes of workspace for `layers` at batch N: slot s is as large as the largest tensor any layer reads

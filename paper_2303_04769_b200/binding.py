@@ -19,7 +19,7 @@ OK = 0
 RELU, ACCUMULATE, RELU_MID = 1, 2, 4
 MATH_FP32, MATH_TF32, MATH_3XTF32 = 0 << 4, 1 << 4, 2 << 4
 POOL_MAX, POOL_AVG = 0, 1
-OP_CONV, OP_DWCONV, OP_POOL, OP_RELU, OP_ADD, OP_FC = range(6)
+OP_CONV, OP_DWCONV, OP_POOL, OP_RELU, OP_ADD, OP_FC, OP_DWPW = range(7)
 SLOT_INPUT, SLOT_OUTPUT = -1, -2
 MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
@@ -46,7 +46,8 @@ class small_layer(ctypes.Structure):
                 ("pad_t", ctypes.c_int), ("pad_b", ctypes.c_int), ("pad_l", ctypes.c_int), ("pad_r", ctypes.c_int),
                 ("flags", ctypes.c_uint), ("pool_mode", ctypes.c_int),
                 ("w_blk", ctypes.c_void_p), ("bias", ctypes.c_void_p),
-                ("src", ctypes.c_int), ("dst", ctypes.c_int), ("src2", ctypes.c_int)]
+                ("src", ctypes.c_int), ("dst", ctypes.c_int), ("src2", ctypes.c_int),
+                ("w_blk2", ctypes.c_void_p), ("bias2", ctypes.c_void_p)]
 
 
 _lib = None

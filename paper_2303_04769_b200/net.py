@@ -31,22 +31,60 @@ def assign_slots(layers):
     return slot_of, n_slots
 
 
+# Fusing a depthwise 3x3 with the 1x1 convolution behind it pays where the two separate launches are short (measured:
+# a few percent on the depthwise-separable network at batch 64, a loss on large intermediate tensors, where the fused
+# kernel's eight depthwise warps per SM cannot keep up with two full-size kernels); above this size of the
+# intermediate tensor the pair runs as two layers.  fuse_dwpw="all" fuses every pair the kernel takes, False none.
+FUSE_DWPW_MAX_BYTES = 24 << 20
+
+
 class Net:
     """A network resident on the device: packed filters, descriptors and workspace."""
 
-    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda"):
+    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda", fuse_dwpw=True):
         self.ctx = ctx
         self.N = net["batch"] if batch is None else batch
         self.in_shape = tuple(net["input"])
         self.math = B.MATH[math]
         self.keep = []            # device tensors the descriptors point into
         self._offsets = None
-        slot_of, _ = assign_slots(net["layers"])
+        # which depthwise 3x3 -> 1x1 pairs run as one fused layer (tensor-core modes, shapes the fused kernel takes, the
+        # depthwise result used by nothing else); slots are then assigned over the layers as they will run
+        layers_in = net["layers"]
+        uses = {}
+        for L in layers_in:
+            uses[L["src"]] = uses.get(L["src"], 0) + 1
+        shape = {"in": self.in_shape}
+        fused_at = set()
+        for li, L in enumerate(layers_in):
+            c, h, wd = shape[L["src"]]
+            fh, fw = (h, wd) if (L["op"] == "pool" and L["FH"] == 0) else (L["FH"], L["FW"])
+            pt, pb, pl, pr = L["pad"]
+            oh, ow = (1, 1) if L["op"] == "fc" else (B.small_out_size(h, fh, L["stride"], pt, pb), B.small_out_size(wd, fw, L["stride"], pl, pr))
+            shape[L["dst"]] = (L["K"], oh, ow)
+            nxt = layers_in[li + 1] if li + 1 < len(layers_in) else None
+            if (fuse_dwpw and self.math != B.MATH["fp32"] and (li - 1) not in fused_at and L["op"] == "dwconv" and fh == 3 and fw == 3
+                    and nxt is not None and nxt["op"] == "conv" and nxt["src"] == L["dst"] and uses.get(L["dst"], 0) == 1
+                    and nxt["FH"] == 1 and nxt["FW"] == 1 and nxt["stride"] == 1 and tuple(nxt["pad"]) == (0, 0, 0, 0)
+                    and not nxt.get("accumulate")
+                    and (fuse_dwpw == "all" or 4 * B.small_packed_elems(self.N, L["C"], oh, ow) <= FUSE_DWPW_MAX_BYTES)
+                    and B.small_dwpw_fused(self.N, L["C"], nxt["K"], h, wd, L["stride"], L["pad"], self.math)):
+                fused_at.add(li)
+        eff = []
+        for li, L in enumerate(layers_in):
+            if li - 1 in fused_at:
+                continue
+            eff.append(dict(L, dst=layers_in[li + 1]["dst"]) if li in fused_at else L)
+        slot_of, _ = assign_slots(eff)
         self.slot_of = slot_of
         dims = {"in": self.in_shape}
         descs = []
         self.layer_rows = []
-        for L, (w, b) in zip(net["layers"], params):
+        skip = False
+        for li, (L, (w, b)) in enumerate(zip(layers_in, params)):
+            if skip:            # the 1x1 convolution already folded into the previous (fused) descriptor
+                skip = False
+                continue
             c, h, wd = dims[L["src"]]
             fh, fw = L["FH"], L["FW"]
             if L["op"] == "pool" and fh == 0:
@@ -55,11 +93,39 @@ class Net:
             d = B.small_layer()
             d.C, d.K, d.H, d.W, d.FH, d.FW, d.stride = L["C"], L["K"], h, wd, fh, fw, L["stride"]
             d.pad_t, d.pad_b, d.pad_l, d.pad_r = pt, pb, pl, pr
-            d.src, d.dst, d.src2 = slot_of[L["src"]], slot_of[L["dst"]], 0
+            d.src, d.dst, d.src2 = slot_of[L["src"]], slot_of.get(L["dst"], 0), 0
             flags = (B.RELU if L["relu"] else 0) | (B.ACCUMULATE if L.get("accumulate") else 0)
             wt = None if w is None else torch.from_numpy(w).to(device)
             bt = None if b is None else torch.from_numpy(b).to(device)
             oh, ow = B.small_out_size(h, fh, L["stride"], pt, pb), B.small_out_size(wd, fw, L["stride"], pl, pr)
+            nxt = layers_in[li + 1] if li + 1 < len(layers_in) else None
+            if li in fused_at:
+                # depthwise 3x3 -> 1x1 as one fused layer: the depthwise result stays in shared memory
+                w2, b2 = params[li + 1]
+                d.op = B.OP_DWPW
+                d.K = nxt["K"]
+                d.dst = slot_of[nxt["dst"]]
+                flags = (B.RELU_MID if L["relu"] else 0) | (B.RELU if nxt["relu"] else 0) | self.math
+                wb = torch.empty(B.small_dw_weight_elems(L["C"], 3, 3), device=device)
+                B.small_pack_dw_weights(ctx, wt, wb, L["C"], 3, 3)
+                wt2 = torch.from_numpy(w2).to(device)
+                bt2 = None if b2 is None else torch.from_numpy(b2).to(device)
+                wb2 = torch.empty(B.small_conv_weight_elems(L["C"], nxt["K"], 1, 1, self.math), device=device)
+                B.small_pack_conv_weights(ctx, wt2, wb2, L["C"], nxt["K"], 1, 1, self.math)
+                d.w_blk2 = wb2.data_ptr()
+                d.bias2 = None if bt2 is None else bt2.data_ptr()
+                self.keep += [wt2, bt2, wb2]
+                d.flags = flags
+                d.w_blk = wb.data_ptr()
+                d.bias = None if bt is None else bt.data_ptr()
+                self.keep += [wb, bt, wt]
+                dims[L["dst"]] = (L["C"], oh, ow)
+                dims[nxt["dst"]] = (nxt["K"], oh, ow)
+                self.layer_rows.append(dict(name=L["name"] + "+" + nxt["name"], op="dwpw", C=L["C"], K=nxt["K"], H=h, W=wd, FH=3, FW=3,
+                                            stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=nxt["dst"], upto=li + 2))
+                descs.append(d)
+                skip = True
+                continue
             if L["op"] == "conv":
                 d.op = B.OP_CONV
                 flags |= self.math
@@ -95,7 +161,7 @@ class Net:
             self.keep += [wb, bt, wt]
             dims[L["dst"]] = (L["K"], oh, ow)
             self.layer_rows.append(dict(name=L["name"], op=L["op"], C=L["C"], K=L["K"], H=h, W=wd, FH=fh, FW=fw,
-                                        stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=L["dst"]))
+                                        stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=L["dst"], upto=li + 1))
             descs.append(d)
         torch.cuda.synchronize()
         self.dims = dims
@@ -145,6 +211,9 @@ class Net:
             B.small_pool2d(self.ctx, src, dst, None, N, L.C, L.H, L.W, L.FH, L.FW, L.stride, pad, L.pool_mode, stream)
         elif L.op == B.OP_FC:
             B.small_fc(self.ctx, src, L.w_blk, L.bias, dst, N, L.C, L.K, L.flags, stream)
+        elif L.op == B.OP_DWPW:
+            B.small_dwpw_conv2d(self.ctx, src, L.w_blk, L.bias, L.w_blk2, L.bias2, dst, None, N, L.C, L.K, L.H, L.W, L.stride, pad,
+                                L.flags, stream)
         else:
             raise ValueError(L.op)
 

@@ -24,7 +24,7 @@ def test_network_matches_oracle_layer_by_layer(name, batch, math):
     params = configs.make_params(net)
     x = configs.make_input(net, batch)
     ref = nets.run_net(net, params, x)
-    gnet = Net(ctx(), net, params, batch=batch, math=math)
+    gnet = Net(ctx(), net, params, batch=batch, math=math, fuse_dwpw="all")     # every pair the fused kernel takes
     in_blk = to_blk(x)
     tol = TOL[math]
     # prefixes of the layer list: the tensor each layer has just written is checked before a later layer reuses its slot
@@ -32,8 +32,9 @@ def test_network_matches_oracle_layer_by_layer(name, batch, math):
         if row["dst"] == "out":
             continue
         # a prefix cannot end on an accumulate target that the oracle dict has since overwritten: recompute the oracle prefix
-        sub = dict(net, layers=net["layers"][:i + 1])
-        ref_i = nets.run_net(sub, params[:i + 1], x)[row["dst"]]
+        upto = row["upto"]          # configuration layers this descriptor completes (two for a fused depthwise + 1x1 pair)
+        sub = dict(net, layers=net["layers"][:upto])
+        ref_i = nets.run_net(sub, params[:upto], x)[row["dst"]]
         gnet.run(in_blk, n_layers=i + 1)
         got = from_blk(gnet.slot_tensor(row["dst"]), batch, row["K"], row["OH"], row["OW"])
         assert rel_l2(got, ref_i) <= tol * (1 + i), (row["name"], rel_l2(got, ref_i))
