@@ -960,13 +960,17 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
     }
     if (p.x3) mma *= 3.0;
     mma += taps * g.CB * (p.b_resident ? 40.0 : 120.0);
-    const double strip_bytes = (double)g.CB * p.strip_px * 128.0;
+    // fused depthwise: what is loaded is the halo tile, and eight warps compute the strip from it (about 6 cycles per
+    // pixel and channel block, measured)
+    const double strip_bytes = p.raw_stage_bytes ? (double)g.CB * p.nn * p.dw_Hb * p.dw_Wb * 128.0 : (double)g.CB * p.strip_px * 128.0;
     const double bytes = strip_bytes + (p.b_resident ? 0.0 : taps * g.CB * p.w_rows * 128.0 * (p.x3 ? 2.0 : 1.0)) + avg_px * 128.0 * (p.w_rows / 32.0);
     const double mem = bytes / 30.0;                 // bytes per clock one SM can expect when all SMs pull
     double tile = mma > mem ? mma : mem;
+    if (p.raw_stage_bytes && g.CB * avg_px * 6.0 > tile) tile = g.CB * avg_px * 6.0;
     if (slots == 2) tile += epi;
     else if (epi > tile) tile = epi;
-    tile += 1500.0;
+    if (p.raw_stage_bytes && !p.x3 && p.a_stages < 3) tile *= 1.25;   // measured: two strips starve the load -> compute -> MMA chain
+    tile += p.raw_stage_bytes ? 8000.0 : 1500.0;     // hand-over per tile; the fused depthwise adds a load -> compute -> MMA chain
     if (p.a_stages < 2 * g.CB) tile += strip_bytes / 30.0 * 0.5;     // the next tile's strips cannot all be in flight
     const double tiles = (double)p.m_tiles * p.n_tiles;
     const double per_sm = tiles <= sms ? 1.0 : tiles / sms;
