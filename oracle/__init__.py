@@ -60,6 +60,8 @@ def lib():
         L.so_pool2d.argtypes = [_f32p, _f32p, _i32p] + [I] * 12
         L.so_relu.argtypes = [_f32p, _f32p, ctypes.c_long]
         L.so_add.argtypes = [_f32p, _f32p, _f32p, ctypes.c_long, I]
+        L.so_scale_shift.argtypes = [_f32p, _f32p, _f32p, _f32p, I, I, I, I, I]
+        L.so_upsample_nearest.argtypes = [_f32p, _f32p, I, I, I, I, I]
         L.so_fc.argtypes = [_f32p, _f32p, _f32p, _f32p] + [I] * 4
         L.so_abstract_layer.argtypes = [_f32p, _f32p, _f32p] + [I] * 15 + [ctypes.c_double]
         L.so_abstract_layer.restype = I
@@ -182,6 +184,27 @@ def relu(x):
     x, xp = _f(x)
     out = np.empty_like(x)
     lib().so_relu(xp, out.ctypes.data_as(_f32p), x.size)
+    return out
+
+
+def scale_shift(x, scale, shift, relu=False):
+    """Inference batch normalisation as the paper classes it (Table 2): out = scale[c] * x + shift[c]."""
+    x, xp = _f(x)
+    s, sp = _f(scale)
+    t, tp = _f(shift)
+    N, C, H, W = x.shape
+    assert s.shape == (C,) and t.shape == (C,)
+    out = np.empty_like(x)
+    lib().so_scale_shift(xp, sp, tp, out.ctypes.data_as(_f32p), N, C, H, W, int(relu))
+    return out
+
+
+def upsample_nearest(x, f):
+    """Nearest-neighbour upsampling by an integer factor (Table 2)."""
+    x, xp = _f(x)
+    N, C, H, W = x.shape
+    out = np.empty((N, C, H * f, W * f), dtype=np.float32)
+    lib().so_upsample_nearest(xp, out.ctypes.data_as(_f32p), N, C, H, W, int(f))
     return out
 
 

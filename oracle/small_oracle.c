@@ -14,7 +14,7 @@
  * zero padding for the FMA layers and as "ignored positions" for pooling.
  *
  * Two independent statements of the arithmetic live here on purpose:
- *   - so_conv2d / so_dwconv2d / so_pool2d / so_relu / so_fc: the per-output
+ *   - so_conv2d / so_dwconv2d / so_pool2d / so_relu / so_scale_shift / so_upsample_nearest / so_fc: the per-output
  *     definitions of Section 3.2 (classes of layers);
  *   - so_abstract_layer: Algorithm 1 (the abstract layer loop nest) with its
  *     blocking parameters, taken in the paper's loop order, for any
@@ -232,6 +232,29 @@ SO_EXPORT void so_relu(const float *in, float *out, long n) {
 
 SO_EXPORT void so_add(const float *a, const float *b, float *out, long n, int relu) {
     for (long i = 0; i < n; ++i) out[i] = so_finish((double)a[i] + (double)b[i], relu);
+}
+
+/* Batch normalisation at inference (Table 2: single element, FMA): one multiply-add per element with the channel's
+ * scale and shift, out = scale[c] * in + shift[c].  NCHW. */
+SO_EXPORT void so_scale_shift(const float *in, const float *scale, const float *shift, float *out,
+                              int N, int C, int H, int W, int relu) {
+    long plane = (long)H * W;
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (long i = 0; i < plane; ++i) {
+                long at = ((long)n * C + c) * plane + i;
+                out[at] = so_finish((double)scale[c] * (double)in[at] + (double)shift[c], relu);
+            }
+}
+
+/* Upsample (Table 2: nearest neighbour interpolation): every input element is repeated f x f times,
+ * out[n][c][oh][ow] = in[n][c][oh / f][ow / f], out is [N][C][H*f][W*f]. */
+SO_EXPORT void so_upsample_nearest(const float *in, float *out, int N, int C, int H, int W, int f) {
+    long OH = (long)H * f, OW = (long)W * f;
+    for (long nc = 0; nc < (long)N * C; ++nc)
+        for (long oh = 0; oh < OH; ++oh)
+            for (long ow = 0; ow < OW; ++ow)
+                out[(nc * OH + oh) * OW + ow] = in[(nc * H + oh / f) * W + ow / f];
 }
 
 /* ---- Full reduction (Section 3.2 item 5): the flattened input [N][J] times a J x K filter bank,

@@ -424,3 +424,35 @@ def test_generator_is_counter_based_and_in_range():
     assert abs(z.mean()) < 0.03 and abs(z.std() - 1) < 0.03
     w = synth.he_normal((64, 64, 3, 3), 576, 8)
     assert abs(w.std() - np.sqrt(2 / 576)) < 2e-3
+
+
+# ---- the other single-element layers of Table 2: batch normalisation (FMA) and upsampling (nearest neighbour)
+def test_scale_shift_pins():
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((2, 5, 3, 4)).astype(np.float32)
+    s = rng.standard_normal(5).astype(np.float32)
+    t = rng.standard_normal(5).astype(np.float32)
+    got = oracle.scale_shift(x, s, t)
+    # brute force, one element at a time, exact rational arithmetic rounded once
+    from fractions import Fraction
+    for n, c, h, w in [(0, 0, 0, 0), (1, 4, 2, 3), (0, 2, 1, 1), (1, 1, 0, 2)]:
+        exact = Fraction(float(s[c])) * Fraction(float(x[n, c, h, w])) + Fraction(float(t[c]))
+        assert got[n, c, h, w] == np.float32(float(exact))
+    # special cases: identity, pure shift, a 1x1 depthwise convolution with bias is the same layer
+    assert np.array_equal(oracle.scale_shift(x, np.ones(5, np.float32), np.zeros(5, np.float32)), x)
+    assert np.array_equal(oracle.scale_shift(np.zeros_like(x), s, t), np.broadcast_to(t[None, :, None, None], x.shape))
+    assert np.array_equal(got, oracle.dwconv2d(x, s.reshape(5, 1, 1), t, 1, (0, 0, 0, 0)))
+    assert np.array_equal(oracle.scale_shift(x, s, t, relu=True), np.maximum(got, 0))
+
+
+def test_upsample_nearest_pins():
+    rng = np.random.default_rng(6)
+    x = rng.standard_normal((2, 3, 4, 5)).astype(np.float32)
+    for f in (1, 2, 3):
+        up = oracle.upsample_nearest(x, f)
+        assert up.shape == (2, 3, 4 * f, 5 * f)
+        assert np.array_equal(up, np.repeat(np.repeat(x, f, axis=2), f, axis=3))       # library statement of the same thing
+        assert np.array_equal(up[:, :, ::f, ::f], x)                                    # subsampling undoes it
+        assert np.array_equal(oracle.pool2d(up, f, f, f, mode="max"), x)                # so does pooling each f x f block
+    up = oracle.upsample_nearest(x, 2)
+    assert up[1, 2, 7, 9] == x[1, 2, 3, 4] and up[0, 1, 2, 1] == x[0, 1, 1, 0]
