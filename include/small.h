@@ -202,6 +202,15 @@ int small_pool2d(small_ctx *ctx, const float *in, float *out, int32_t *idx,
  * out may equal in (in place); any other overlap is an error. */
 int small_relu(small_ctx *ctx, const float *in, float *out, int N, int C, int H, int W, void *stream);
 
+/* Batch normalisation at inference (Table 2: a single element layer whose operation is FMA):
+ *   out[n,c,h,w] = scale[c] * in[n,c,h,w] + shift[c]   (then max(., 0) with SMALL_RELU)
+ * scale, shift: device, C floats each (gamma / sqrt(var + eps) and beta - mean * that, folded by the caller).
+ * in, out: blocked [N][C][H][W]; out may be the same buffer as in; pad lanes are written as +0. */
+int small_scale_shift(small_ctx *ctx, const float *in, const float *scale, const float *shift, float *out,
+                      int N, int C, int H, int W, unsigned flags, void *stream);
+/* Upsample (Table 2: nearest neighbour interpolation) by an integer factor in both plane dimensions:
+ *   out[n,c,oh,ow] = in[n,c,oh / factor,ow / factor];  out: blocked [N][C][H*factor][W*factor].  Bit-exact move. */
+int small_upsample_nearest(small_ctx *ctx, const float *in, float *out, int N, int C, int H, int W, int factor, void *stream);
 /* Single element reduction "addition" (Section 3.2 item 1): out = a + b, then ReLU if SMALL_RELU.
  * out may equal a or b. */
 int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N, int C, int H, int W,

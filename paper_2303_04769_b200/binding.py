@@ -29,7 +29,7 @@ EXPORTS = [
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
-    "small_relu", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
+    "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
 ]
 
@@ -96,6 +96,8 @@ def lib():
     L.small_pool2d.argtypes = [P, P, P, P] + [I] * 11 + [I, P]
     L.small_relu.argtypes = [P, P, P, I, I, I, I, P]
     L.small_add.argtypes = [P, P, P, P, I, I, I, I, U, P]
+    L.small_scale_shift.argtypes = [P, P, P, P, P, I, I, I, I, U, P]
+    L.small_upsample_nearest.argtypes = [P, P, P, I, I, I, I, I, P]
     L.small_fc.argtypes = [P, P, P, P, P, I, I, I, U, P]
     L.small_net_workspace_bytes.argtypes = [ctypes.POINTER(small_layer), I, I]
     L.small_net_workspace_bytes.restype = Z
@@ -249,6 +251,14 @@ def small_pool2d(ctx, inp, out, idx, N, C, H, W, FH, FW, stride, pad, mode=POOL_
 
 def small_relu(ctx, inp, out, N, C, H, W, stream=None):
     _check(lib().small_relu(ctx, _ptr(inp), _ptr(out), N, C, H, W, _stream(stream)), "small_relu")
+
+
+def small_scale_shift(ctx, inp, scale, shift, out, N, C, H, W, flags=0, stream=None):
+    _check(lib().small_scale_shift(ctx, _ptr(inp), _ptr(scale), _ptr(shift), _ptr(out), N, C, H, W, flags, _stream(stream)), "small_scale_shift")
+
+
+def small_upsample_nearest(ctx, inp, out, N, C, H, W, factor, stream=None):
+    _check(lib().small_upsample_nearest(ctx, _ptr(inp), _ptr(out), N, C, H, W, factor, _stream(stream)), "small_upsample_nearest")
 
 
 def small_add(ctx, a, b, out, N, C, H, W, flags=0, stream=None):

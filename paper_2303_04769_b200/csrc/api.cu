@@ -383,6 +383,28 @@ SMALL_API int small_relu(small_ctx *ctx, const float *in, float *out, int N, int
     return launch_relu(ctx, in, out, n, static_cast<cudaStream_t>(stream));
 }
 
+SMALL_API int small_scale_shift(small_ctx *ctx, const float *in, const float *scale, const float *shift, float *out,
+                                int N, int C, int H, int W, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~SMALL_RELU) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, out}, {})) return s;
+    if (!scale || !shift) return SMALL_ERR_INVALID_ARG;
+    size_t n = packed_elems(N, C, H, W);
+    if (n == 0) return SMALL_ERR_SHAPE;
+    if (in != out && ranges_overlap(in, n * sizeof(float), out, n * sizeof(float))) return SMALL_ERR_OVERLAP;
+    return launch_scale_shift(ctx, in, scale, shift, out, N, C, H, W, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
+}
+
+SMALL_API int small_upsample_nearest(small_ctx *ctx, const float *in, float *out, int N, int C, int H, int W, int factor, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (int s = check_ptrs({in, out})) return s;
+    if (factor < 1 || factor > 64) return SMALL_ERR_INVALID_ARG;
+    size_t n = packed_elems(N, C, H, W);
+    if (n == 0 || (long long)H * factor > 0x7fffffLL || (long long)W * factor > 0x7fffffLL) return SMALL_ERR_SHAPE;
+    if (ranges_overlap(in, n * sizeof(float), out, n * sizeof(float) * factor * factor)) return SMALL_ERR_OVERLAP;
+    return launch_upsample_nearest(ctx, in, out, N, C, H, W, factor, static_cast<cudaStream_t>(stream));
+}
+
 SMALL_API int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N, int C, int H, int W,
                         unsigned flags, void *stream) {
     if (!ctx) return SMALL_ERR_NOT_INIT;

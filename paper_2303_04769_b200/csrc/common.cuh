@@ -61,6 +61,9 @@ int launch_pack_dw_weights(small_ctx *, const float *w, float *wb, int C, int FH
 int launch_pack_fc_weights(small_ctx *, const float *w, float *wb, int J, int K, cudaStream_t);
 int launch_relu(small_ctx *, const float *in, float *out, size_t n, cudaStream_t);
 int launch_add(small_ctx *, const float *a, const float *b, float *out, size_t n, bool relu, cudaStream_t);
+int launch_scale_shift(small_ctx *, const float *in, const float *scale, const float *shift, float *out, int N, int C, int H, int W,
+                       bool relu, cudaStream_t);
+int launch_upsample_nearest(small_ctx *, const float *in, float *out, int N, int C, int H, int W, int f, cudaStream_t);
 int launch_pool(small_ctx *, const float *in, float *out, int32_t *idx, const Geom &, int mode, cudaStream_t);
 int launch_dwconv(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
 int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, float *out, int N, int J, int K, bool relu, cudaStream_t);

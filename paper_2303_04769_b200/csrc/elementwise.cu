@@ -53,6 +53,57 @@ static int stream_grid(small_ctx *ctx, size_t n4, int unroll, int ctas_per_sm) {
 }
 static bool is_large(size_t n4) { return n4 * 16 >= (size_t)64 << 20; }
 
+// Batch normalisation at inference (paper Table 2: single element, FMA): out = scale[c] * in + shift[c].  One thread =
+// four channels of one pixel; the channel's scale and shift come from the 128-byte line position (chunk of the block),
+// pad lanes (c >= C) are written as +0.
+__global__ void __launch_bounds__(256) scale_shift_kernel(const float4 *__restrict__ in, const float *__restrict__ scale,
+                                                          const float *__restrict__ shift, float4 *__restrict__ out,
+                                                          size_t n4, int C, int CB, size_t plane4, bool relu) {
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const int cb = (int)((i / plane4) % CB);            // plane4 = H * W * 8 vectors per (image, channel block)
+        const int c = cb * 32 + (int)(i & 7) * 4;
+        const float4 v = __ldcs(in + i);
+        float4 r;
+        r.x = c + 0 < C ? fmaf(scale[c + 0], v.x, shift[c + 0]) : 0.0f;
+        r.y = c + 1 < C ? fmaf(scale[c + 1], v.y, shift[c + 1]) : 0.0f;
+        r.z = c + 2 < C ? fmaf(scale[c + 2], v.z, shift[c + 2]) : 0.0f;
+        r.w = c + 3 < C ? fmaf(scale[c + 3], v.w, shift[c + 3]) : 0.0f;
+        __stcs(out + i, relu ? relu4(r) : r);
+    }
+}
+
+// Upsample (paper Table 2: nearest neighbour): out[n][cb][oh][ow] = in[n][cb][oh / f][ow / f]; one thread writes four
+// channels of one output pixel, so a warp writes four whole output lines.
+__global__ void __launch_bounds__(256) upsample_nearest_kernel(const float4 *__restrict__ in, float4 *__restrict__ out,
+                                                               size_t n4_out, int H, int W, int f) {
+    const int OW = W * f, OH = H * f;
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4_out; i += stride) {
+        const int j = (int)(i & 7);
+        size_t p = i >> 3;
+        const int ow = (int)(p % OW); p /= OW;
+        const int oh = (int)(p % OH); p /= OH;             // p = image * channel blocks + block
+        __stcs(out + i, __ldg(in + ((p * H + oh / f) * W + ow / f) * 8 + j));
+    }
+}
+
+int launch_scale_shift(small_ctx *ctx, const float *in, const float *scale, const float *shift, float *out,
+                       int N, int C, int H, int W, bool relu, cudaStream_t st) {
+    const int CB = blocks_of(C);
+    const size_t plane4 = (size_t)H * W * 8, n4 = (size_t)N * CB * plane4;
+    scale_shift_kernel<<<stream_grid(ctx, n4, 1, 8), 256, 0, st>>>(reinterpret_cast<const float4 *>(in), scale, shift,
+                                                                  reinterpret_cast<float4 *>(out), n4, C, CB, plane4, relu);
+    return check_launch(ctx);
+}
+
+int launch_upsample_nearest(small_ctx *ctx, const float *in, float *out, int N, int C, int H, int W, int f, cudaStream_t st) {
+    const size_t n4 = (size_t)N * blocks_of(C) * H * f * W * f * 8;
+    upsample_nearest_kernel<<<stream_grid(ctx, n4, 1, 8), 256, 0, st>>>(reinterpret_cast<const float4 *>(in),
+                                                                        reinterpret_cast<float4 *>(out), n4, H, W, f);
+    return check_launch(ctx);
+}
+
 int launch_relu(small_ctx *ctx, const float *in, float *out, size_t n, cudaStream_t st) {
     size_t n4 = n / 4;   // a blocked tensor is a whole number of 32-float lines
     const float4 *i4 = reinterpret_cast<const float4 *>(in);

@@ -347,3 +347,33 @@ def test_tf32_issue_probe():
     assert tf256 > 600.0 and abs(tf128 / tf256 - 1.0) < 0.15
     with pytest.raises(B.SmallError):
         B.small_measure_tf32_peak(ctx(), 48, 2048)
+
+
+@pytest.mark.parametrize("shape", [(2, 16, 9, 7), (3, 40, 5, 5), (1, 64, 56, 56), (2, 3, 4, 4), (1, 70, 3, 11)])
+def test_scale_shift(shape):
+    """Batch normalisation as a per-channel FMA: one fused multiply-add per element, so within one rounding of the oracle."""
+    N, C, H, W = shape
+    x, s, t = rnd(shape, 81), rnd((C,), 82), rnd((C,), 83)
+    for relu in (False, True):
+        ref = oracle.scale_shift(x, s, t, relu)
+        out = new_blk(N, C, H, W)
+        B.small_scale_shift(ctx(), to_blk(x), dev(s), dev(t), out, N, C, H, W, B.RELU if relu else 0)
+        got = from_blk(out, N, C, H, W)
+        assert np.array_equal(got.view(np.int32), ref.view(np.int32))      # a single FMA rounds once, like the oracle
+        assert pad_lanes_are_zero(out, N, C, H, W)
+    buf = to_blk(x)                                                          # in place
+    B.small_scale_shift(ctx(), buf, dev(s), dev(t), buf, N, C, H, W, 0)
+    assert np.array_equal(from_blk(buf, N, C, H, W).view(np.int32), oracle.scale_shift(x, s, t).view(np.int32))
+
+
+@pytest.mark.parametrize("shape,f", [((2, 16, 9, 7), 2), ((1, 40, 5, 5), 3), ((2, 3, 4, 4), 1), ((1, 64, 14, 14), 2), ((3, 33, 1, 6), 4)])
+def test_upsample_nearest_bit_exact(shape, f):
+    N, C, H, W = shape
+    x = rnd(shape, 84)
+    out = new_blk(N, C, H * f, W * f)
+    B.small_upsample_nearest(ctx(), to_blk(x), out, N, C, H, W, f)
+    got = from_blk(out, N, C, H * f, W * f)
+    assert np.array_equal(got.view(np.int32), oracle.upsample_nearest(x, f).view(np.int32))
+    assert pad_lanes_are_zero(out, N, C, H * f, W * f)
+    with pytest.raises(B.SmallError):
+        B.small_upsample_nearest(ctx(), to_blk(x), out, N, C, H, W, 0)
