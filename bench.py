@@ -196,13 +196,30 @@ def reference_arm(args):
     if rank != 0:
         return
     net = configs.NETWORKS[WORKLOAD]()
-    # every step is a bounded sample of the workload, sized so that the whole run stays within a few minutes
-    per_step_s = max(0.05, min(6.0, 150.0 / (args.steps + args.warmup)))
-    rates, n_used, cores, passes = [], 0, 0, 0
+    # every step is a bounded sample of the workload, sized so that the whole run stays within a few minutes:
+    # set-up and the size of the sample are fixed once, a step is `passes` passes over `n_used` images
+    import oracle
+    from oracle import nets
+    params = configs.make_params(net)
+    per_step_s = max(0.02, min(6.0, 100.0 / (args.steps + args.warmup)))
+    probe = 8
+    x = configs.make_input(net, probe)
+    nets.run_net(net, params, x)                            # first call: builds and loads the C oracle
+    t0 = time.perf_counter()
+    nets.run_net(net, params, x)
+    dt = time.perf_counter() - t0
+    n_used = int(max(probe, min(net["batch"], probe * per_step_s / max(dt, 1e-6))))
+    passes = max(1, int(per_step_s / max(dt * n_used / probe, 1e-6)))
+    x = configs.make_input(net, n_used)
+    cores = oracle.num_threads()
+    rates = []
     for i in range(args.warmup + args.steps):
-        ips, n_used, dt, cores, passes = time_oracle_net(net["batch"], target_s=per_step_s)
+        t0 = time.perf_counter()
+        for _ in range(passes):
+            nets.run_net(net, params, x)
+        el = time.perf_counter() - t0
         if i >= args.warmup:
-            rates.append(ips)
+            rates.append(n_used * passes / el)
     value = sum(rates) / len(rates)
     ms = 1e3 * net["batch"] / value                     # one full batch at the sampled rate
     sample = (f"{n_used} of {net['batch']} images per pass, {passes} passes per step (about {per_step_s:.2f} s), "
