@@ -95,6 +95,12 @@ int small_out_size(int I, int F, int stride, int pad_before, int pad_after);
 const char *small_strerror(int status);
 /* Last cudaError_t / CUresult seen by this context (0 if none). */
 int small_last_cuda_error(small_ctx *ctx);
+/* Layer overlap inside small_run_net (on by default; `on` = 0 switches it off).  When on, every layer behind the
+ * first is launched with programmatic stream serialisation: its thread blocks may become resident and set up shared
+ * memory, barriers and tensor memory while the layer in front of it is still draining, and they wait on the device
+ * until that layer has completed before they read or write a tensor.  Results are the same either way.  The paper
+ * has no counterpart. */
+int small_set_layer_overlap(small_ctx *ctx, int on);
 /* Synchronises `stream`, then reads and clears the device status word: *status is SMALL_OK or
  * SMALL_ERR_TIMEOUT (a tensor-core pipeline wait gave up; the affected outputs are undefined). */
 int small_device_status(small_ctx *ctx, int *status, void *stream);

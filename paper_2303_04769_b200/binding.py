@@ -25,7 +25,7 @@ MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
 EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
-    "small_last_cuda_error", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
+    "small_last_cuda_error", "small_set_layer_overlap", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
@@ -71,6 +71,7 @@ def lib():
     L.small_strerror.argtypes = [I]
     L.small_strerror.restype = ctypes.c_char_p
     L.small_last_cuda_error.argtypes = [P]
+    L.small_set_layer_overlap.argtypes = [P, I]
     L.small_device_status.argtypes = [P, ctypes.POINTER(I), P]
     L.small_pack.argtypes = [P, P, P, I, I, I, I, P]
     L.small_unpack.argtypes = [P, P, P, I, I, I, I, P]
@@ -156,6 +157,10 @@ def small_packed_elems(N, C, H, W):
 
 def small_out_size(I, F, stride, pad_before=0, pad_after=0):
     return lib().small_out_size(I, F, stride, pad_before, pad_after)
+
+
+def small_set_layer_overlap(ctx, on):
+    _check(lib().small_set_layer_overlap(ctx, 1 if on else 0), "small_set_layer_overlap")
 
 
 def small_device_status(ctx, stream=None):

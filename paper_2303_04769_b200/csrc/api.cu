@@ -100,6 +100,8 @@ SMALL_API int small_init(int device, small_ctx **out) {
         return SMALL_ERR_CUDA;
     }
     c->encode_tiled = fn;
+    c->overlap = 1;
+    c->dependent = 0;
     *out = c;
     return SMALL_OK;
 }
@@ -113,6 +115,12 @@ SMALL_API int small_shutdown(small_ctx *ctx) {
 }
 
 SMALL_API int small_last_cuda_error(small_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+SMALL_API int small_set_layer_overlap(small_ctx *ctx, int on) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    ctx->overlap = on ? 1 : 0;
+    return SMALL_OK;
+}
 
 SMALL_API int small_device_status(small_ctx *ctx, int *status, void *stream) {
     if (!ctx) return SMALL_ERR_NOT_INIT;

@@ -17,6 +17,8 @@ struct small_ctx {
     void *encode_tiled;      // cuTensorMapEncodeTiled, resolved through the runtime
     int sm_count;
     size_t max_smem_optin;
+    int overlap;             // small_run_net launches every layer after the first as a dependent launch (see launch_kernel)
+    int dependent;           // set by small_run_net while it issues those layers
 };
 
 namespace small {
@@ -43,6 +45,33 @@ static inline int check_launch(small_ctx *ctx) {
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     return SMALL_OK;
 }
+
+// Dependent launches.  Every layer kernel of this library executes grid_dep_sync() before its first access to global
+// memory that an earlier kernel of the stream may have written (or may still read), and nothing it does before that
+// touches such memory; it also executes grid_dep_trigger().  A kernel launched with programmatic stream serialisation
+// may therefore start while the kernel in front of it in the stream is still draining: its blocks become resident as
+// that kernel's blocks leave, set up their shared memory, barriers and tensor memory, and then wait at
+// grid_dep_sync() until the earlier kernel has completed and its writes are visible.  Launched the ordinary way,
+// both instructions do nothing.  Chains stay ordered: a kernel cannot complete before its own grid_dep_sync()
+// returns, so completion of kernel i implies completion of every kernel before it.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dep_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline void launch_kernel(small_ctx *ctx, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->dependent ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+    (void)e;   // picked up by check_launch through cudaGetLastError
+}
+#endif
 
 // Geometry of one windowed layer, validated once on the host and passed to kernels by value.
 struct Geom {

@@ -26,6 +26,7 @@ struct ConvArgs {
 
 template <int PIX, int ST>
 __global__ void __launch_bounds__(256) conv_fp32_kernel(ConvArgs a) {
+    grid_dep_sync();     // no early trigger: see launch_conv_fp32
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int S = ST ? ST : a.S;
@@ -120,7 +121,14 @@ static int launch_variant(small_ctx *ctx, ConvArgs &a, long long blocks, size_t 
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     }
-    kern<<<(unsigned)blocks, 256, smem, st>>>(a);
+    // Always an ordinary launch, and the kernel lets its successor start only as its blocks leave.  Its blocks are small
+    // and many per SM; started beside the big-shared-memory blocks of a persistent kernel in front of it, they would
+    // inherit that kernel's shared-memory / L1 split for the whole launch (measured: the depthwise-separable network
+    // in FP32 mode ran 12 % slower with this kernel as a dependent launch).
+    const int dependent = ctx->dependent;
+    ctx->dependent = 0;
+    launch_kernel(ctx, kern, dim3((unsigned)blocks), dim3(256), smem, st, a);
+    ctx->dependent = dependent;
     return check_launch(ctx);
 }
 

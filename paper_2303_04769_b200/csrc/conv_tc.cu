@@ -356,6 +356,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // everything above touched only shared memory, tensor memory and the layer's own constants (bias, depthwise
+    // filters); from here on the roles read the input tensor and write the output tensor
+    grid_dep_sync();
+    grid_dep_trigger();
 
     // Stages a producer has armed and the parity of each stage's latest fill, kept past the role loops: if any role
     // gave up, the producers wait (bounded) for their copies in flight before the CTA may exit.
@@ -1190,7 +1194,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
-    kern<<<grid, dw ? kThreadsDW : x3 ? kThreadsX3 : kThreads, p.smem_bytes, st>>>(map_a, map_b, map_b_lo, a);
+    launch_kernel(ctx, kern, dim3(grid), dim3(dw ? kThreadsDW : x3 ? kThreadsX3 : kThreads), p.smem_bytes, st, map_a, map_b, map_b_lo, a);
     return check_launch(ctx);
 }
 

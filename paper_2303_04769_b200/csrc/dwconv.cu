@@ -23,6 +23,8 @@ __device__ __forceinline__ void fma4(float4 &a, const float4 &v, const float4 &w
 
 // Generic window / stride: one output pixel x four channels per thread.
 __global__ void __launch_bounds__(256) dwconv_generic_kernel(DwArgs a) {
+    grid_dep_sync();
+    grid_dep_trigger();
     const long long total = a.planes * a.OH * a.OW * 8;
     for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
         int q = (int)(t & 7);
@@ -97,6 +99,8 @@ __global__ void __launch_bounds__(256) dwconv3x3_tma_kernel(const __grid_constan
         failed = 0;
     }
     __syncthreads();
+    grid_dep_sync();
+    grid_dep_trigger();
     const long long first = blockIdx.x, stride = gridDim.x;
     if (threadIdx.x == 0) {
         if (first < a.tiles) issue(first, 0);
@@ -224,13 +228,13 @@ int launch_dwconv(small_ctx *ctx, const float *in, const float *w, const float *
         auto kern = g.S == 1 ? dwconv3x3_tma_kernel<1> : dwconv3x3_tma_kernel<2>;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
-        kern<<<grid, 256, smem, st>>>(map, t);
+        launch_kernel(ctx, kern, dim3(grid), dim3(256), smem, st, map, t);
         return check_launch(ctx);
     }
     long long total = a.planes * g.OH * g.OW * 8;
     long long want = (total + 255) / 256, cap = (long long)ctx->sm_count * 32;
     int grid = (int)(want < cap ? want : cap);
-    dwconv_generic_kernel<<<grid, 256, 0, st>>>(a);
+    launch_kernel(ctx, dwconv_generic_kernel, dim3(grid), dim3(256), 0, st, a);
     return check_launch(ctx);
 }
 

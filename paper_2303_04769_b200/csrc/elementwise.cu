@@ -9,6 +9,8 @@ __device__ __forceinline__ float4 relu4(float4 v) { return make_float4(relu1(v.x
 
 template <int UNROLL>
 __global__ void __launch_bounds__(256) relu_kernel(const float4 *__restrict__ in, float4 *__restrict__ out, size_t n4) {
+    grid_dep_sync();
+    grid_dep_trigger();
     size_t stride = (size_t)gridDim.x * blockDim.x;
     size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     for (; i + (UNROLL - 1) * stride < n4; i += UNROLL * stride) {
@@ -24,6 +26,8 @@ __global__ void __launch_bounds__(256) relu_kernel(const float4 *__restrict__ in
 template <int UNROLL>
 __global__ void __launch_bounds__(256) add_kernel(const float4 *__restrict__ a, const float4 *__restrict__ b,
                                                   float4 *__restrict__ out, size_t n4, bool relu) {
+    grid_dep_sync();
+    grid_dep_trigger();
     size_t stride = (size_t)gridDim.x * blockDim.x;
     size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
     for (; i + (UNROLL - 1) * stride < n4; i += UNROLL * stride) {
@@ -108,8 +112,8 @@ int launch_relu(small_ctx *ctx, const float *in, float *out, size_t n, cudaStrea
     size_t n4 = n / 4;   // a blocked tensor is a whole number of 32-float lines
     const float4 *i4 = reinterpret_cast<const float4 *>(in);
     float4 *o4 = reinterpret_cast<float4 *>(out);
-    if (is_large(n4)) relu_kernel<2><<<stream_grid(ctx, n4, 2, 4), 256, 0, st>>>(i4, o4, n4);
-    else relu_kernel<8><<<stream_grid(ctx, n4, 8, 8), 256, 0, st>>>(i4, o4, n4);
+    if (is_large(n4)) launch_kernel(ctx, relu_kernel<2>, dim3((unsigned)(stream_grid(ctx, n4, 2, 4))), dim3(256), 0, st, i4, o4, n4);
+    else launch_kernel(ctx, relu_kernel<8>, dim3((unsigned)(stream_grid(ctx, n4, 8, 8))), dim3(256), 0, st, i4, o4, n4);
     return check_launch(ctx);
 }
 
@@ -117,8 +121,8 @@ int launch_add(small_ctx *ctx, const float *a, const float *b, float *out, size_
     size_t n4 = n / 4;
     const float4 *a4 = reinterpret_cast<const float4 *>(a), *b4 = reinterpret_cast<const float4 *>(b);
     float4 *o4 = reinterpret_cast<float4 *>(out);
-    if (is_large(n4)) add_kernel<2><<<stream_grid(ctx, n4, 2, 4), 256, 0, st>>>(a4, b4, o4, n4, relu);
-    else add_kernel<4><<<stream_grid(ctx, n4, 4, 8), 256, 0, st>>>(a4, b4, o4, n4, relu);
+    if (is_large(n4)) launch_kernel(ctx, add_kernel<2>, dim3((unsigned)(stream_grid(ctx, n4, 2, 4))), dim3(256), 0, st, a4, b4, o4, n4, relu);
+    else launch_kernel(ctx, add_kernel<4>, dim3((unsigned)(stream_grid(ctx, n4, 4, 8))), dim3(256), 0, st, a4, b4, o4, n4, relu);
     return check_launch(ctx);
 }
 

@@ -7,6 +7,8 @@ namespace small {
 __global__ void __launch_bounds__(256) fc_kernel(const float *__restrict__ in, const float *__restrict__ w,
                                                  const float *__restrict__ bias, float *__restrict__ out,
                                                  int N, int JB, int K, int KB, bool relu) {
+    grid_dep_sync();
+    grid_dep_trigger();
     const int lane = threadIdx.x & 31;
     const long long warps = (long long)N * KB;
     for (long long wid = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5; wid < warps;
@@ -31,7 +33,7 @@ int launch_fc(small_ctx *ctx, const float *in, const float *w, const float *bias
     int JB = blocks_of(J), KB = blocks_of(K);
     long long warps = (long long)N * KB;
     long long want = (warps + 7) / 8, cap = (long long)ctx->sm_count * 16;
-    fc_kernel<<<(int)(want < cap ? want : cap), 256, 0, st>>>(in, w, bias, out, N, JB, K, KB, relu);
+    launch_kernel(ctx, fc_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(256), 0, st, in, w, bias, out, N, JB, K, KB, relu);
     return check_launch(ctx);
 }
 

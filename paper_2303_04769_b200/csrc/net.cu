@@ -116,6 +116,8 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
     for (int i = 0; i < n_layers; ++i) {
         const small_layer &L = layers[i];
         int s = SMALL_OK;
+        // every layer behind the first may start its set-up while the layer in front of it drains (see launch_kernel)
+        ctx->dependent = ctx->overlap && i > 0;
         switch (L.op) {
             case SMALL_OP_CONV:
                 s = small_conv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
@@ -143,6 +145,7 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
                                       L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
                 break;
         }
+        ctx->dependent = 0;
         if (s != SMALL_OK) return s;
     }
     return SMALL_OK;

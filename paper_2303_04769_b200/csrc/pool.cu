@@ -14,6 +14,8 @@ struct PoolArgs {
 
 template <bool MAX, bool IDX>
 __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a) {
+    grid_dep_sync();
+    grid_dep_trigger();
     const long long total = a.planes * a.OH * a.OW * 8;
     for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
         int q = (int)(t & 7);
@@ -69,6 +71,8 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a) {
 // so this is a pure stream.  Two output pixels per thread = eight independent 128-bit loads in flight.
 __global__ void __launch_bounds__(256) maxpool2x2_kernel(const float4 *__restrict__ in, float4 *__restrict__ out, long long planes,
                                                          int H, int W, int OH, int OW, int C, int CB) {
+    grid_dep_sync();
+    grid_dep_trigger();
     const long long total = planes * OH * OW * 8, stride = (long long)gridDim.x * blockDim.x;
     for (long long t0 = blockIdx.x * (long long)blockDim.x + threadIdx.x; t0 < total; t0 += 2 * stride) {
         float4 v[2][4];
@@ -117,6 +121,8 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const float4 *__restric
 // beyond rounding (average) or not at all (maximum), and indices are not produced here.
 template <bool MAX>
 __global__ void __launch_bounds__(256) pool_window_kernel(PoolArgs a) {
+    grid_dep_sync();
+    grid_dep_trigger();
     const int lane = threadIdx.x & 31, q = lane & 7, sub = lane >> 3;
     const long long warps = a.planes * a.OH * a.OW;
     for (long long wid = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5; wid < warps; wid += ((long long)gridDim.x * blockDim.x) >> 5) {
@@ -163,7 +169,7 @@ int launch_pool(small_ctx *ctx, const float *in, float *out, int32_t *idx, const
     int grid = (int)(want < cap ? want : cap);
     if (mode == SMALL_POOL_MAX && !idx && g.FH == 2 && g.FW == 2 && g.S == 2 && !(g.pt | g.pb | g.pl | g.pr)) {
         long long w2 = (total + 511) / 512, cap2 = (long long)ctx->sm_count * 8;
-        maxpool2x2_kernel<<<(int)(w2 < cap2 ? w2 : cap2), 256, 0, st>>>(reinterpret_cast<const float4 *>(in), reinterpret_cast<float4 *>(out),
+        launch_kernel(ctx, maxpool2x2_kernel, dim3((unsigned)((int)(w2 < cap2 ? w2 : cap2))), dim3(256), 0, st, reinterpret_cast<const float4 *>(in), reinterpret_cast<float4 *>(out),
                                                                      a.planes, g.H, g.W, g.OH, g.OW, g.C, g.CB);
         return check_launch(ctx);
     }
@@ -171,15 +177,15 @@ int launch_pool(small_ctx *ctx, const float *in, float *out, int32_t *idx, const
         const long long warps = a.planes * g.OH * g.OW;
         long long wb = (warps + 7) / 8, capb = (long long)ctx->sm_count * 16;
         const int gridb = (int)(wb < capb ? wb : capb);
-        if (mode == SMALL_POOL_MAX) pool_window_kernel<true><<<gridb, 256, 0, st>>>(a);
-        else pool_window_kernel<false><<<gridb, 256, 0, st>>>(a);
+        if (mode == SMALL_POOL_MAX) launch_kernel(ctx, pool_window_kernel<true>, dim3((unsigned)(gridb)), dim3(256), 0, st, a);
+        else launch_kernel(ctx, pool_window_kernel<false>, dim3((unsigned)(gridb)), dim3(256), 0, st, a);
         return check_launch(ctx);
     }
     if (mode == SMALL_POOL_MAX) {
-        if (idx) pool_kernel<true, true><<<grid, 256, 0, st>>>(a);
-        else pool_kernel<true, false><<<grid, 256, 0, st>>>(a);
+        if (idx) launch_kernel(ctx, pool_kernel<true, true>, dim3((unsigned)(grid)), dim3(256), 0, st, a);
+        else launch_kernel(ctx, pool_kernel<true, false>, dim3((unsigned)(grid)), dim3(256), 0, st, a);
     } else {
-        pool_kernel<false, false><<<grid, 256, 0, st>>>(a);
+        launch_kernel(ctx, pool_kernel<false, false>, dim3((unsigned)(grid)), dim3(256), 0, st, a);
     }
     return check_launch(ctx);
 }

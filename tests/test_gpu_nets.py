@@ -47,6 +47,35 @@ def test_network_matches_oracle_layer_by_layer(name, batch, math):
     assert B.small_device_status(ctx()) == 0
 
 
+@pytest.mark.parametrize("name,batch", [("residual_cnn", 96), ("dwsep_cnn", 24), ("kws_cnn", 200), ("autoencoder_fc", 1500)])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "3xtf32"])
+def test_layer_overlap_changes_no_bit(name, batch, math):
+    """Layers launched as dependent launches (the default) give exactly the tensor that fully serialised launches
+    give, run after run, eagerly and replayed from a CUDA graph: a layer that read or wrote a tensor before the layer
+    in front of it had finished would show up here.  The batch is large enough for several tiles per SM."""
+    net = configs.NETWORKS[name](batch=batch)
+    params = configs.make_params(net)
+    in_blk = to_blk(configs.make_input(net, batch))
+    try:
+        B.small_set_layer_overlap(ctx(), 0)
+        want = Net(ctx(), net, params, batch=batch, math=math).run(in_blk).clone()
+        B.small_set_layer_overlap(ctx(), 1)
+        gnet = Net(ctx(), net, params, batch=batch, math=math)
+        for _ in range(3):
+            assert torch.equal(gnet.run(in_blk), want)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            out = gnet.run(in_blk)
+        for _ in range(5):
+            out.fill_(float("nan"))
+            g.replay()
+            assert torch.equal(out, want)
+    finally:
+        B.small_set_layer_overlap(ctx(), 1)
+    assert B.small_device_status(ctx()) == 0
+
+
 def test_run_net_host_end_to_end():
     net = configs.residual_cnn(batch=8)
     params = configs.make_params(net)
