@@ -79,6 +79,7 @@ struct TcPlan {
     uint32_t raw_stage_bytes; int dw_Hb, dw_Wb, dw_rows;   // fused depthwise: halo tile per (tile, channel block)
     int x_packed;        // 3xTF32 with one channel block of <= 16 channels: hi in lanes [0, h), lo in [h, 2h) of each row
     int x3;              // 3xTF32: stages hold both halves, three MMAs per K step
+    int x3_wide;         // 3xTF32, pixels on M, at most 64 filters: two MMAs per K step, the first over both filter halves
     double taps_eff;     // taps per block that exist (a stride-2 view has empty ones)
     int ks_last;         // K steps (8 channels each) of the last channel block that hold real channels
     uint32_t a_stage_bytes, b_stage_bytes, smem_bytes;
@@ -103,6 +104,7 @@ struct TcArgs {
     int dw_s, dw_Wb, dw_Hb, dw_pt, dw_pl, dw_relu, dw_rows, dw_C;   // stride, halo box, pads, ReLU, strip rows per image
     uint32_t raw_stage_bytes, raw_box_bytes;
     int x_packed;              // 3xTF32, at most 16 channels: the residual sits in the unused lanes of the same row
+    int x3_wide;               // 3xTF32, pixels on M: x_hi meets [w_hi; w_lo] in one MMA of twice the filters (see the issue loop)
     uint32_t x_lo_off;         // 3xTF32: 16-byte units from a strip's TF32 part to its residual
     int relu, accumulate;
 };
@@ -459,6 +461,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t row_wrap = (uint32_t)(a.Wq - a.FW + 1) * 8u;     // tap offset step from the end of a window row
         // N of the MMA: pixels of a slot (filters on M), or the filters of the tile (pixels on M)
         const uint32_t idesc = instr_desc(PM ? a.w_rows : a.n_slot);
+        const uint32_t idesc_wide = instr_desc(PM ? 2 * a.w_rows : a.n_slot);   // x3_wide: both filter halves on N
+        const bool wide = X3 && PM && a.x3_wide;
         // strip offset (in 16-byte units) of each MMA chain of a tile: one per slot or one per 128-pixel chunk
         uint32_t xo[CH];
 #pragma unroll
@@ -509,6 +513,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     } else {
                         // the residual halves sit x_half / w_half (16-byte units) behind the TF32 halves
                         const uint32_t da_lo = da + (PM ? x_half : w_half), db_lo = db + (PM ? w_half : x_half);
+                        if (PM && wide) {
+                            // columns [0, w) of the chunk: x_hi w_hi + x_lo w_hi; columns [w, 2w): x_hi w_lo
+#pragma unroll
+                            for (int k = 0; k < KS; ++k) {
+                                mma_tf32(acc[c] + r_col, da + 2u * k, db + 2u * k, kDescHi, idesc_wide, k == 0 ? first : 1u);
+                                mma_tf32(acc[c] + r_col, da_lo + 2u * k, db + 2u * k, kDescHi, idesc, 1u);
+                            }
+                        } else
 #pragma unroll
                         for (int k = 0; k < KS; ++k) {
                             mma_tf32(acc[c] + r_col, da_lo + 2u * k, db + 2u * k, kDescHi, idesc, k == 0 ? first : 1u);   // small terms first
@@ -715,6 +727,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int jj = 0; jj * 32 < a.w_rows; ++jj) {
                             float v[32];
                             tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx) + (uint32_t)c * sw + jj * 32u, v);
+                            if (X3 && a.x3_wide) {     // the x_hi w_lo products of the same filters, w_rows columns on
+                                float v2[32];
+                                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kSlotPx) + (uint32_t)c * sw + (uint32_t)a.w_rows + jj * 32u, v2);
+#pragma unroll
+                                for (int e = 0; e < 32; ++e) v[e] += v2[e];
+                            }
                             const int kbj = kb_tile + jj;
                             if (!ok || kbj >= a.KB) continue;
                             float *dst = a.out + ((((size_t)n * a.KB + kbj) * a.OH + oh) * a.OW + ow) * 32;
@@ -829,7 +847,13 @@ TcPlan make_plan_with(const Geom &g, size_t max_smem, int max_px, int pixel_m, i
         if (group_k > p.w_tile) return p;
         p.w_tile = group_k; p.w_rows = group_k; p.n_tiles = Kp / group_k;
     }
-    p.cps = !pixel_m ? 1 : p.w_rows <= 64 ? 4 : p.w_rows <= 128 ? 2 : 1;
+    // 3xTF32 with pixels on M and few filters: the residual filter rows lie directly behind the TF32 rows in a stage, so
+    // one MMA of N = 2 x filters forms x_hi w_hi and x_hi w_lo side by side in tensor memory (an MMA below N = 128 costs
+    // the pipe the same 50 cycles whatever N is); a second MMA adds x_lo w_hi, and the epilogue adds the two column
+    // groups.  Two MMAs per K step instead of three.
+    p.x3_wide = (x3 && pixel_m && p.w_rows <= 64) ? 1 : 0;
+    const int acc_cols = p.x3_wide ? 2 * p.w_rows : p.w_rows;      // tensor-memory columns of one 128-pixel chunk
+    p.cps = !pixel_m ? 1 : acc_cols <= 64 ? 4 : acc_cols <= 128 ? 2 : 1;
     p.ks_last = (g.C - (g.CB - 1) * 32 + 7) / 8;
     if (pixel_m && max_px > kSlots * p.cps * 128) return p;       // more pixels than the accumulator slots hold
     p.racc = racc;
@@ -954,6 +978,7 @@ double plan_cost(const TcPlan &p, const Geom &g, int sms) {
         const double chunks = (double)(long long)((avg_px + 127.0) / 128.0);
         slots = p.px_tile > p.cps * 128 ? 2 : 1;
         mma = taps * ksteps * chunks * (p.w_rows / 2.0 > 48.0 ? p.w_rows / 2.0 : 48.0);
+        if (p.x3_wide) mma = taps * ksteps * chunks * ((p.w_rows > 48.0 ? p.w_rows : 48.0) + 48.0) / 3.0;   // x 3 below
         epi = avg_px * 1.2 * (p.w_rows / 32.0) + 300.0 * chunks;
     } else {
         slots = p.px_tile > kSlotPx / p.racc ? 2 : 1;
@@ -1166,6 +1191,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.a_stages = p.a_stages; a.pixel_m = p.pixel_m; a.w_tile = p.w_tile; a.cps = p.cps; a.b_stage_bytes = p.b_stage_bytes;
     a.a_stage_bytes = p.a_stage_bytes; a.a_half = p.a_half; a.b_half = p.b_half; a.racc = p.racc;
     a.x_packed = p.x_packed;
+    a.x3_wide = p.x3_wide;
     a.x_lo_off = p.x_packed ? 2u * (uint32_t)p.ks_last : (p.a_half >> 4);   // packed: the residual starts h = 8 ks_last lanes on
     a.a_box_bytes = (uint32_t)p.strip_px * 128u;
     a.b_resident = p.b_resident; a.ks_last = p.ks_last;
