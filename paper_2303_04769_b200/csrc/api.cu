@@ -277,6 +277,7 @@ SMALL_API int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, 
                                              int pt, int pb, int pl, int pr) {
     Geom g;
     if (make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr) != SMALL_OK) return 0;
+    if (conv_thin_supported(g)) return 0;      // a reduction of a few dozen terms: CUDA cores in every math mode
     return conv_tc_supported(g) ? 1 : 0;
 }
 
@@ -294,6 +295,8 @@ SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, cons
         return SMALL_ERR_OVERLAP;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     bool relu = flags & SMALL_RELU, acc = flags & SMALL_ACCUMULATE;
+    // at most four input channels: no dense contraction to give the tensor cores; FP32 FMAs meet every mode's tolerance
+    if (conv_thin_supported(g)) return launch_conv_thin(ctx, in, w, bias, out, g, relu, acc, st);
     // the tensor-core epilogue may store 32 bytes per thread: an output that is only 16-byte aligned takes the FP32 kernel
     if (math != SMALL_MATH_FP32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
         const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);

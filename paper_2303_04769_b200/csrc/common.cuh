@@ -100,6 +100,10 @@ int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, f
 // (Kg filters per group, groups S_C channels apart); span = 0: full reduction over all channel blocks
 int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
                      bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
+// at most four input channels, 3 x 3 (strides 1, 2) or the 10 x 4 stride-2 window: FP32 FMAs with the filters in registers
+bool conv_thin_supported(const Geom &);
+int launch_conv_thin(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
+                     bool relu, bool accumulate, cudaStream_t);
 int group_conv_span(int C, int F_C, int S_C, int Kg);      // channel blocks a filter block of a group convolution needs
 int launch_pack_group_conv_weights(small_ctx *, const float *w, float *wb, int C, int F_C, int S_C, int Kg, int FH, int FW, cudaStream_t);
 // tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32

@@ -212,7 +212,8 @@ CONV_TC_CASES = [  # N, C, K, H, W, FH, FW, pad  (stride 1: the shapes the tenso
     (2, 64, 64, 56, 56, 1, 1, (0, 0, 0, 0)),
     (23, 512, 512, 7, 7, 1, 1, (0, 0, 0, 0)),
     (3, 64, 64, 25, 5, 1, 1, (0, 0, 0, 0)),
-    (2, 3, 16, 32, 32, 3, 3, (1, 1, 1, 1)),        # few input channels: the rest of the block is zero
+    (2, 5, 16, 32, 32, 3, 3, (1, 1, 1, 1)),        # few input channels: the rest of the block is zero
+    (2, 3, 16, 32, 32, 3, 3, (1, 1, 1, 1)),        # at most four: the register-filter CUDA-core kernel in every mode
     (2, 70, 45, 9, 11, 3, 3, (1, 1, 1, 1)),        # ragged channel counts
     (2, 33, 200, 17, 19, 5, 3, (2, 1, 0, 2)),      # asymmetric pads, rectangular window, ragged filter tile
     (1, 40, 40, 17, 17, 2, 2, (0, 1, 1, 0)),
@@ -258,8 +259,8 @@ CONV_TC_STRIDE2_CASES = [  # N, C, K, H, W, FH, FW, pad  (stride 2: read as a st
     (3, 16, 32, 32, 32, 3, 3, (1, 1, 1, 1)),       # the residual network's downsampling convolutions
     (3, 16, 32, 32, 32, 1, 1, (0, 0, 0, 0)),       # and its 1x1 shortcut: a single phase plane
     (2, 32, 64, 16, 16, 3, 3, (1, 1, 1, 1)),
-    (2, 3, 8, 96, 96, 3, 3, (1, 1, 1, 1)),         # depthwise-separable stem
-    (5, 1, 64, 49, 10, 10, 4, (4, 5, 1, 1)),       # keyword-spotting stem: tall window, odd height, asymmetric pads
+    (2, 5, 8, 96, 96, 3, 3, (1, 1, 1, 1)),         # the depthwise-separable stem's shape with five channels
+    (5, 5, 64, 49, 10, 10, 4, (4, 5, 1, 1)),       # the keyword-spotting stem's: tall window, odd height, asymmetric pads
     (2, 70, 45, 17, 19, 3, 3, (0, 1, 1, 0)),       # odd planes, ragged channels, pads on one side only
     (2, 40, 40, 15, 15, 2, 2, (0, 0, 0, 0)),       # window = stride: every phase plane has one tap
     (3, 64, 64, 9, 9, 5, 5, (2, 2, 2, 2)),
@@ -302,12 +303,12 @@ CONV_3XTF32_CASES = [  # N, C, K, H, W, FH, FW, stride, pad
     (19, 512, 512, 7, 7, 3, 3, 1, (1, 1, 1, 1)),      # ... or 4 accumulators
     (19, 512, 512, 7, 7, 1, 1, 1, (0, 0, 0, 0)),
     (2, 64, 64, 56, 56, 1, 1, 1, (0, 0, 0, 0)),
-    (2, 3, 16, 32, 32, 3, 3, 1, (1, 1, 1, 1)),
+    (2, 5, 16, 32, 32, 3, 3, 1, (1, 1, 1, 1)),
     (2, 70, 45, 9, 11, 3, 3, 1, (1, 1, 1, 1)),
     (2, 33, 200, 17, 19, 5, 3, 1, (2, 1, 0, 2)),
     (3, 16, 32, 32, 32, 3, 3, 2, (1, 1, 1, 1)),
     (3, 16, 32, 32, 32, 1, 1, 2, (0, 0, 0, 0)),
-    (5, 1, 64, 49, 10, 10, 4, 2, (4, 5, 1, 1)),
+    (5, 5, 64, 49, 10, 10, 4, 2, (4, 5, 1, 1)),
 ]
 
 
