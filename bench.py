@@ -1,6 +1,6 @@
 """Benchmark of the SMaLL layer set on B200.
 
-python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--math fp32|tf32|3xtf32] [--no-sweep]
+python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--math fp32|tf32|3xtf32] [--no-sweep] [--no-overlap]
 
 One step = one pass of the 8-layer residual CNN (batch 256 per GPU) through small_run_net, inputs resident in HBM.
 The JSON line also carries the end-to-end figure from host buffers (small_run_net_host), the per-kernel roofline
@@ -34,10 +34,10 @@ TOL = {"fp32": 1e-5, "tf32": 2e-3, "3xtf32": 1e-5}
 # this file's network step, averaged over the kernel's launches in one step).  It is reported only while the kernel's
 # source still has the hash it had when the counters were taken.
 TRAFFIC = {
-    "conv_3xtf32_tensor": {"bytes_per_launch": 23813802.7, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                           "sha256": "0cc36ed8da753741e573f7b9eab712a91bc26890e190c2df8c14310d21e7959f"},
-    "conv_tf32_tensor": {"bytes_per_launch": 23752590.2, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                         "sha256": "0cc36ed8da753741e573f7b9eab712a91bc26890e190c2df8c14310d21e7959f"},
+    "conv_3xtf32_tensor": {"bytes_per_launch": 22487360.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                           "sha256": "f595f2741c1c6048b793322fcf73f336380423e953e0f9ed42e9bc5ac75f3efb"},
+    "conv_tf32_tensor": {"bytes_per_launch": 22427168.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                         "sha256": "f595f2741c1c6048b793322fcf73f336380423e953e0f9ed42e9bc5ac75f3efb"},
 }
 
 
@@ -253,6 +253,8 @@ def gpu_main(args):
     if world > 1:
         dist.barrier()
     ctx = B.small_init(local)
+    if args.no_overlap:
+        B.small_set_layer_overlap(ctx, False)
     peaks = load_peaks()
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
 
@@ -480,7 +482,8 @@ def gpu_main(args):
             "config": {"workload": f"{WORKLOAD}: 8-layer residual CNN, 3x32x32 input, batch {N} per GPU (configs[1])",
                        "math": args.math, "tolerance_rel_l2": TOL[args.math], "l2": "flushed between steps (256 MB write)",
                        "inputs": f"{R} rotating seeded input sets", "parallelism": f"batch shards x{world}, no collective",
-                       "launch": "small_run_net captured in a CUDA graph per input set and replayed", "eager_ms_per_step": ms_eager},
+                       "launch": "small_run_net captured in a CUDA graph per input set and replayed", "eager_ms_per_step": ms_eager,
+                       "layer_overlap": not args.no_overlap},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * N * c * h * w, "d2h_bytes_per_step": 4 * N * oc * oh * ow,
                     "ms_per_step": ms_e2e},
             "gpu_launches": len(gnet.layer_rows) * args.steps,
@@ -666,6 +669,8 @@ def main():
                     help="arithmetic of the convolutions; the default keeps FP32-level accuracy (1e-5) on the tensor cores")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="launch every layer fully serialised (small_set_layer_overlap off): for profiler captures and comparisons")
     ap.add_argument("--layer", default=None, help="KIND:C:HW[:BATCH] - run one sweep layer only (for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:
