@@ -26,8 +26,12 @@ struct ThinArgs {
     bool relu, accumulate;
 };
 
+// Threads per block: four warps.  A block loads a tile, then computes on it, with nothing in flight meanwhile, so
+// memory-level parallelism comes from many small blocks per SM being at different points of that cycle.
+constexpr int kThinThreads = 128;
+
 template <int C, int FH, int FW, int S, int PIX, int KPT>
-__global__ void __launch_bounds__(256) conv_thin_kernel(const ThinArgs a) {
+__global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs a) {
     extern __shared__ __align__(16) float tile[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int SEG = (PIX - 1) * S + FW, SEG2 = (SEG + 1) / 2;
@@ -64,24 +68,41 @@ __global__ void __launch_bounds__(256) conv_thin_kernel(const ThinArgs a) {
         const int ih0 = oh0 * S - a.pt;
         const int rows = (th - 1) * S + FH;
         __syncthreads();                       // the previous tile is no longer read
-        for (int e = threadIdx.x; e < imgs * rows * a.pitch; e += 256) {
-            const int img = e / (rows * a.pitch), rc = e - img * rows * a.pitch;
-            const int r = rc / a.pitch, c = rc - r * a.pitch;
-            const int gh = ih0 + r, gw = c - a.pl;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (gh >= 0 && gh < a.H && gw >= 0 && gw < a.W) {
-                const float *p = a.in + (((size_t)(n0 + img) * a.H + gh) * a.W + gw) * 32;    // one channel block
-                if (C == 1) v.x = *p; else v = *reinterpret_cast<const float4 *>(p);
+        // four pixels per thread and step: the loads are issued together, then stored, so that a thread has four
+        // lines in flight instead of one
+        const int total = imgs * rows * a.pitch;
+        for (int e0 = threadIdx.x; e0 < total; e0 += 4 * kThinThreads) {
+            float4 v[4];
+            int at[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e = e0 + u * kThinThreads;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                at[u] = -1;
+                if (e < total) {
+                    const int img = e / (rows * a.pitch), rc = e - img * rows * a.pitch;
+                    const int r = rc / a.pitch, c = rc - r * a.pitch;
+                    const int gh = ih0 + r, gw = c - a.pl;
+                    at[u] = img * C * a.plane + r * a.pitch + c;
+                    if (gh >= 0 && gh < a.H && gw >= 0 && gw < a.W) {
+                        const float *p = a.in + (((size_t)(n0 + img) * a.H + gh) * a.W + gw) * 32;    // one channel block
+                        if (C == 1) v[u].x = __ldg(p); else v[u] = __ldg(reinterpret_cast<const float4 *>(p));
+                    }
+                }
             }
-            float *dst = tile + (size_t)img * C * a.plane + r * a.pitch + c;
-            dst[0] = v.x;
-            if (C > 1) dst[a.plane] = v.y;
-            if (C > 2) dst[2 * a.plane] = v.z;
-            if (C > 3) dst[3 * a.plane] = v.w;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (at[u] < 0) continue;
+                float *dst = tile + at[u];
+                dst[0] = v[u].x;
+                if (C > 1) dst[a.plane] = v[u].y;
+                if (C > 2) dst[2 * a.plane] = v[u].z;
+                if (C > 3) dst[3 * a.plane] = v[u].w;
+            }
         }
         __syncthreads();
         const int items = imgs * th * a.groups;              // (image, output row, column group)
-        for (int it = warp; it < items; it += 8) {
+        for (int it = warp; it < items; it += kThinThreads / 32) {
             const int img = it / (th * a.groups), rg = it - img * th * a.groups;
             const int r = rg / a.groups, cg = rg - r * a.groups;
             float acc[PIX][KPT];
@@ -193,7 +214,7 @@ int launch_conv_thin(small_ctx *ctx, const float *in, const float *w, const floa
     auto tile_bytes = [&](int nb, int th) { return (size_t)nb * g.C * ((th - 1) * g.S + g.FH) * a.pitch * sizeof(float); };
     // CTAs that run at once: the grid is that many (or fewer), each walking the tile list
     int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, budget) != cudaSuccess || per_sm < 1) per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThinThreads, budget / 2) != cudaSuccess || per_sm < 1) per_sm = 1;
     const long long cap = (long long)per_sm * ctx->sm_count;
     // output rows per tile: the whole plane if it fits, halved while that leaves the GPU short of tiles
     a.TH = g.OH;
@@ -218,7 +239,7 @@ int launch_conv_thin(small_ctx *ctx, const float *in, const float *w, const floa
     long long gx_ll = cap / a.kgroups;
     if (gx_ll < 1) gx_ll = 1;
     const unsigned gx = (unsigned)(a.tiles < gx_ll ? a.tiles : gx_ll);
-    launch_kernel(ctx, kern, dim3(gx, (unsigned)a.kgroups), dim3(256), smem, st, a);
+    launch_kernel(ctx, kern, dim3(gx, (unsigned)a.kgroups), dim3(kThinThreads), smem, st, a);
     return check_launch(ctx);
 }
 
