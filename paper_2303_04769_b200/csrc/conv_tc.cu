@@ -683,12 +683,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         *src = h;
                     }
                 } else
-                for (int i = tid; i < n4; i += 128) {
-                    const uint4 v = hi[i];
-                    const uint4 h = make_uint4(v.x & 0xffffe000u, v.y & 0xffffe000u, v.z & 0xffffe000u, v.w & 0xffffe000u);
-                    lo[i] = make_float4(__uint_as_float(v.x) - __uint_as_float(h.x), __uint_as_float(v.y) - __uint_as_float(h.y),
-                                        __uint_as_float(v.z) - __uint_as_float(h.z), __uint_as_float(v.w) - __uint_as_float(h.w));
-                    hi[i] = h;
+                {
+                    // four vectors per step, loads first: one warp per scheduler has nothing else to hide their latency
+                    auto split1 = [&](int i, const uint4 v) {
+                        const uint4 h = make_uint4(v.x & 0xffffe000u, v.y & 0xffffe000u, v.z & 0xffffe000u, v.w & 0xffffe000u);
+                        lo[i] = make_float4(__uint_as_float(v.x) - __uint_as_float(h.x), __uint_as_float(v.y) - __uint_as_float(h.y),
+                                            __uint_as_float(v.z) - __uint_as_float(h.z), __uint_as_float(v.w) - __uint_as_float(h.w));
+                        hi[i] = h;
+                    };
+                    int i = tid;
+                    for (; i + 3 * 128 < n4; i += 4 * 128) {
+                        const uint4 v0 = hi[i], v1 = hi[i + 128], v2 = hi[i + 256], v3 = hi[i + 384];
+                        split1(i, v0); split1(i + 128, v1); split1(i + 256, v2); split1(i + 384, v3);
+                    }
+                    for (; i < n4; i += 128) split1(i, hi[i]);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these writes are read by the tensor core
                 mbar_arrive(bar_a_split + 8 * s);
