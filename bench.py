@@ -34,10 +34,10 @@ TOL = {"fp32": 1e-5, "tf32": 2e-3, "3xtf32": 1e-5}
 # this file's network step, averaged over the kernel's launches in one step).  It is reported only while the kernel's
 # source still has the hash it had when the counters were taken.
 TRAFFIC = {
-    "conv_3xtf32_tensor": {"bytes_per_launch": 22487360.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                           "sha256": "f595f2741c1c6048b793322fcf73f336380423e953e0f9ed42e9bc5ac75f3efb"},
-    "conv_tf32_tensor": {"bytes_per_launch": 22427168.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                         "sha256": "f595f2741c1c6048b793322fcf73f336380423e953e0f9ed42e9bc5ac75f3efb"},
+    "conv_3xtf32_tensor": {"bytes_per_launch": 22474912.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                           "sha256": "56f83a2606504907c5bad7c2a578e13d07d365bfe95bc1a36b6202336994f7ca"},
+    "conv_tf32_tensor": {"bytes_per_launch": 22428480.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                         "sha256": "56f83a2606504907c5bad7c2a578e13d07d365bfe95bc1a36b6202336994f7ca"},
 }
 
 
