@@ -744,12 +744,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             const int kbj = kb_tile + jj;
                             if (!ok || kbj >= a.KB) continue;
                             float *dst = a.out + ((((size_t)n * a.KB + kbj) * a.OH + oh) * a.OW + ow) * 32;
-                            const float *bs = bias_s + kbj * 32;
+                            const float4 *bs = reinterpret_cast<const float4 *>(bias_s + kbj * 32);   // 16-byte aligned: two loads per eight filters
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 float r[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) r[e] = v[8 * i + e] + bs[8 * i + e];
+                                const float4 b0 = bs[2 * i], b1 = bs[2 * i + 1];
+                                r[0] = v[8 * i + 0] + b0.x; r[1] = v[8 * i + 1] + b0.y; r[2] = v[8 * i + 2] + b0.z; r[3] = v[8 * i + 3] + b0.w;
+                                r[4] = v[8 * i + 4] + b1.x; r[5] = v[8 * i + 5] + b1.y; r[6] = v[8 * i + 6] + b1.z; r[7] = v[8 * i + 7] + b1.w;
                                 if (a.accumulate) {
                                     float o[8];
                                     ld_global_v8(dst + 8 * i, o);
