@@ -34,10 +34,10 @@ TOL = {"fp32": 1e-5, "tf32": 2e-3, "3xtf32": 1e-5}
 # this file's network step, averaged over the kernel's launches in one step).  It is reported only while the kernel's
 # source still has the hash it had when the counters were taken.
 TRAFFIC = {
-    "conv_3xtf32_tensor": {"bytes_per_launch": 22474912.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                           "sha256": "56f83a2606504907c5bad7c2a578e13d07d365bfe95bc1a36b6202336994f7ca"},
-    "conv_tf32_tensor": {"bytes_per_launch": 22428480.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                         "sha256": "56f83a2606504907c5bad7c2a578e13d07d365bfe95bc1a36b6202336994f7ca"},
+    "conv_3xtf32_tensor": {"bytes_per_launch": 22471040.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                           "sha256": "3788f28a029a03005913b9f8e2f18eb4681d617500595f75edd934977a8ef8f7"},
+    "conv_tf32_tensor": {"bytes_per_launch": 22413408.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                         "sha256": "3788f28a029a03005913b9f8e2f18eb4681d617500595f75edd934977a8ef8f7"},
 }
 
 
