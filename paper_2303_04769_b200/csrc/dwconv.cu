@@ -68,6 +68,7 @@ struct Dw3Args {
     const float *w; const float *bias; float *out; int *status;
     int N, C, CB, OH, OW, pt, pl;
     int nn, TR, Hb, Wb, strips, groups;    // groups = ceil(N / nn)
+    int segs, rps;                         // a column's TR rows are walked by `segs` threads, `rps` rows each
     long long tiles;
     uint32_t stage_bytes;
     bool relu;
@@ -135,17 +136,21 @@ __global__ void __launch_bounds__(256) dwconv3x3_tma_kernel(const __grid_constan
                 if (cbase + 3 < a.C) bias4.w = a.bias[cbase + 3];
             }
             const int oh0 = strip * a.TR, rows = min(a.TR, a.OH - oh0);
-            for (int c = threadIdx.x >> 3; c < cols; c += 32) {
+            // unit = (row segment, column): narrow tiles (few columns) split each column's rows over several threads so
+            // that all 32 column slots of the block have work
+            for (int u = threadIdx.x >> 3; u < cols * a.segs; u += 32) {
+                const int seg = u / cols, c = u - seg * cols;
                 const int img = c / a.OW, ow = c - img * a.OW;
                 const int n = grp * a.nn + img;
-                if (n >= a.N) continue;
-                const float4 *col = tile + ((size_t)img * a.Hb * a.Wb + ow * ST) * 8 + q;     // window's top-left pixel
-                float4 *dst = reinterpret_cast<float4 *>(a.out) + ((((size_t)n * a.CB + cb) * a.OH + oh0) * a.OW + ow) * 8 + q;
+                const int i0 = seg * a.rps, i1 = min(rows, i0 + a.rps);
+                if (n >= a.N || i0 >= i1) continue;
+                const float4 *col = tile + ((size_t)img * a.Hb * a.Wb + (size_t)i0 * ST * a.Wb + ow * ST) * 8 + q;     // window's top-left pixel
+                float4 *dst = reinterpret_cast<float4 *>(a.out) + ((((size_t)n * a.CB + cb) * a.OH + oh0 + i0) * a.OW + ow) * 8 + q;
                 float4 r0[3], r1[3], r2[3];
 #pragma unroll
                 for (int y = 0; y < 3; ++y) { r0[y] = col[y * 8]; r1[y] = col[(a.Wb + y) * 8]; }
                 const float4 *next = col + 2 * a.Wb * 8;
-                for (int i = 0; i < rows; ++i) {
+                for (int i = i0; i < i1; ++i) {
 #pragma unroll
                     for (int y = 0; y < 3; ++y) r2[y] = next[y * 8];
                     float4 acc = bias4;
@@ -164,7 +169,7 @@ __global__ void __launch_bounds__(256) dwconv3x3_tma_kernel(const __grid_constan
                     } else {
 #pragma unroll
                         for (int y = 0; y < 3; ++y) r0[y] = r2[y];
-                        if (i + 1 < rows) {
+                        if (i + 1 < i1) {
 #pragma unroll
                             for (int y = 0; y < 3; ++y) r1[y] = next[(a.Wb + y) * 8];
                         }
@@ -208,6 +213,12 @@ static bool plan_dw3(const Geom &g, int sms, Dw3Args &a) {
         a.Hb = (a.TR - 1) * S + 3;
     }
     a.groups = ceil_div(g.N, a.nn);
+    // 256 threads = 32 column slots x 8 lane groups; a tile with fewer columns splits its rows (at least 3 per thread)
+    const int cols = a.nn * g.OW;
+    a.segs = cols >= 32 ? 1 : 32 / cols;
+    if (a.segs > a.TR / 3) a.segs = a.TR / 3 > 0 ? a.TR / 3 : 1;
+    a.rps = ceil_div(a.TR, a.segs);
+    a.segs = ceil_div(a.TR, a.rps);
     a.tiles = (long long)a.groups * g.CB * a.strips;
     a.stage_bytes = (uint32_t)((size_t)a.nn * a.Hb * row_bytes);
     return true;
