@@ -1,5 +1,9 @@
 // Full reduction (paper Section 3.2 item 5): the fully connected layer on blocked [N][J][1][1] -> [N][K][1][1].
-// One warp per (image, block of 32 outputs); the lane is the output channel, as in the convolution kernels.
+// The lane is the output channel, as in the convolution kernels.  Two mappings of the (image, block of 32 outputs)
+// units: one thread block per unit, its eight warps sharing out the input's channel blocks, so that a long reduction
+// (a classifier head behind a wide last layer) is eight short chains combined through shared memory instead of one
+// long one; and, when there are units enough to fill the GPU many times over, one warp per unit with no block-wide
+// synchronisation.
 #include "common.cuh"
 
 namespace small {
@@ -9,18 +13,51 @@ __global__ void __launch_bounds__(256) fc_kernel(const float *__restrict__ in, c
                                                  int N, int JB, int K, int KB, bool relu) {
     grid_dep_sync();
     grid_dep_trigger();
+    __shared__ float part[8][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long units = (long long)N * KB;
+    for (long long u = blockIdx.x; u < units; u += gridDim.x) {
+        const int kb = (int)(u % KB);
+        const long long n = u / KB;
+        const float *x = in + n * JB * 32;
+        const float *wt = w + (size_t)kb * JB * 32 * 32 + lane;
+        float acc = 0.0f;
+        for (int jb = warp; jb < JB; jb += 8) {
+            const float xv = x[jb * 32 + lane];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc = fmaf(__shfl_sync(0xffffffffu, xv, j), wt[(jb * 32 + j) * 32], acc);
+        }
+        part[warp][lane] = acc;
+        __syncthreads();
+        if (warp == 0) {
+            const int k = kb * 32 + lane;
+            float v = (bias && k < K) ? bias[k] : 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v += part[i][lane];
+            if (relu) v = v > 0.f ? v : 0.f;
+            out[u * 32 + lane] = k < K ? v : 0.0f;
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(256) fc_warp_kernel(const float *__restrict__ in, const float *__restrict__ w,
+                                                      const float *__restrict__ bias, float *__restrict__ out,
+                                                      int N, int JB, int K, int KB, bool relu) {
+    grid_dep_sync();
+    grid_dep_trigger();
     const int lane = threadIdx.x & 31;
     const long long warps = (long long)N * KB;
     for (long long wid = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5; wid < warps;
          wid += ((long long)gridDim.x * blockDim.x) >> 5) {
-        int kb = (int)(wid % KB);
-        long long n = wid / KB;
-        int k = kb * 32 + lane;
+        const int kb = (int)(wid % KB);
+        const long long n = wid / KB;
+        const int k = kb * 32 + lane;
         float acc = (bias && k < K) ? bias[k] : 0.0f;
         const float *x = in + n * JB * 32;
         const float *wt = w + (size_t)kb * JB * 32 * 32 + lane;
         for (int jb = 0; jb < JB; ++jb) {
-            float xv = x[jb * 32 + lane];
+            const float xv = x[jb * 32 + lane];
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc = fmaf(__shfl_sync(0xffffffffu, xv, j), wt[(jb * 32 + j) * 32], acc);
         }
@@ -31,9 +68,13 @@ __global__ void __launch_bounds__(256) fc_kernel(const float *__restrict__ in, c
 
 int launch_fc(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, int N, int J, int K, bool relu, cudaStream_t st) {
     int JB = blocks_of(J), KB = blocks_of(K);
-    long long warps = (long long)N * KB;
-    long long want = (warps + 7) / 8, cap = (long long)ctx->sm_count * 16;
-    launch_kernel(ctx, fc_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(256), 0, st, in, w, bias, out, N, JB, K, KB, relu);
+    long long units = (long long)N * KB, cap = (long long)ctx->sm_count * 8;
+    if (units >= 64LL * ctx->sm_count) {      // every SM gets 64 units or more: a warp each
+        long long want = (units + 7) / 8, capw = (long long)ctx->sm_count * 16;
+        launch_kernel(ctx, fc_warp_kernel, dim3((unsigned)(want < capw ? want : capw)), dim3(256), 0, st, in, w, bias, out, N, JB, K, KB, relu);
+        return check_launch(ctx);
+    }
+    launch_kernel(ctx, fc_kernel, dim3((unsigned)(units < cap ? units : cap)), dim3(256), 0, st, in, w, bias, out, N, JB, K, KB, relu);
     return check_launch(ctx);
 }
 

@@ -139,9 +139,11 @@ class Net:
                 d.op = B.OP_POOL
                 d.pool_mode = B.POOL_MAX if L["pool"] == "max" else B.POOL_AVG
                 wb = None
-            elif L["op"] == "fc" and self.math != B.MATH["fp32"] and h == 1 and wd == 1:
+            elif L["op"] == "fc" and self.math != B.MATH["fp32"] and h == 1 and wd == 1 and 2 * self.N * L["C"] * L["K"] >= 4e6:
                 # a full reduction over a 1x1 plane is a 1x1 convolution whose pixels are the images: in the
-                # tensor-core modes it runs on the convolution kernel (same arithmetic, same blocked buffers)
+                # tensor-core modes it runs on the convolution kernel (same arithmetic, same blocked buffers).  A
+                # classifier head of a megaflop or so stays on the FP32 kernel (3 us; the tensor-core kernel's set-up
+                # alone costs more).
                 d.op = B.OP_CONV
                 d.FH = d.FW = 1
                 flags |= self.math
