@@ -35,6 +35,27 @@ def test_residual_cnn_batch_256_sampled_images(math):
         assert rel_l2(got[n], ref[j]) <= 8 * TOL[math], n
 
 
+@pytest.mark.parametrize("name,sample", [("kws_cnn", [0, 6, 7, 511, 1021, 1023]), ("dwsep_cnn", [0, 31, 63]),
+                                         ("autoencoder_fc", [0, 255, 256, 4095])])
+@pytest.mark.parametrize("math", ["3xtf32", "tf32", "fp32"])
+def test_other_networks_full_batch_sampled_images(name, sample, math):
+    """The other network workloads the benchmark reports, at their full batch and with the benchmark's layer
+    fusion: images from the first, a middle and the ragged last tile against the oracle."""
+    net = configs.NETWORKS[name]()
+    N = net["batch"]
+    params = configs.make_params(net)
+    x = configs.make_input(net, N)
+    gnet = Net(ctx(), net, params, math=math)
+    out = gnet.run(to_blk(x))
+    oc, oh, ow = gnet.out_shape
+    got = from_blk(out, N, oc, oh, ow)
+    assert B.small_device_status(ctx()) == 0
+    ref = nets.run_net(net, params, x[sample])["out"]
+    assert rel_l2(got[sample], ref) <= 4 * TOL[math]
+    for j, n in enumerate(sample):
+        assert rel_l2(got[n], ref[j]) <= 8 * TOL[math], n
+
+
 SWEEP = [(C, HW) for C, HW in configs.SWEEP_SIZES]
 
 
