@@ -168,9 +168,10 @@ def whole_job_throughput(units_local, ms_local, world, device=None):
 
 
 # ------------------------------------------------------------------------------------------- CPU oracle legs
-def time_oracle_net(batch_cap, target_s=12.0):
+def time_oracle_net(batch_cap, target_s=12.0, f32acc=False):
     """The oracle as it stands on the host cores: a bounded sample of the workload (at most the full batch per pass,
-    whole passes repeated until about target_s seconds of CPU work are done)."""
+    whole passes repeated until about target_s seconds of CPU work are done).  f32acc: the convolutions' sums in a
+    float accumulator instead of double (the same loops; a second, fairer CPU figure - parity always uses double)."""
     import oracle
     from oracle import nets
     net = configs.NETWORKS[WORKLOAD]()
@@ -178,14 +179,14 @@ def time_oracle_net(batch_cap, target_s=12.0):
     probe = 8
     x = configs.make_input(net, probe)
     t0 = time.perf_counter()
-    nets.run_net(net, params, x)
+    nets.run_net(net, params, x, f32acc=f32acc)
     dt = time.perf_counter() - t0
     n = int(max(probe, min(batch_cap, probe * target_s / max(dt, 1e-6))))
     x = configs.make_input(net, n)
     passes, total = 0, 0.0
     while passes == 0 or (total < target_s and passes < 64):
         t0 = time.perf_counter()
-        nets.run_net(net, params, x)
+        nets.run_net(net, params, x, f32acc=f32acc)
         total += time.perf_counter() - t0
         passes += 1
     return n * passes / total, n, total, oracle.num_threads(), passes
@@ -357,9 +358,9 @@ def gpu_main(args):
         fl, by = layer_work(row, N, L.get("accumulate", False))
         kern = row["op"]
         if row["op"] == "conv":
-            tc = args.math != "fp32" and B.small_conv2d_uses_tensor_cores(N, row["C"], row["K"], row["H"], row["W"], row["FH"], row["FW"],
-                                                                           row["stride"], row["pad"])
-            kern = f"conv_{args.math}_tensor" if tc else "conv_fp32_cuda_core"
+            path = B.small_conv2d_path(ctx, N, row["C"], row["K"], row["H"], row["W"], row["FH"], row["FW"], row["stride"], row["pad"],
+                                       B.MATH[args.math])
+            kern = f"conv_{args.math}_tensor" if path == 3 else "conv_fp32_cuda_core"
         layer_table.append({"layer": row["name"], "kernel": kern, "us": round(tmed * 1e3, 2), "gflops": round(fl / tmed / 1e6, 1),
                             "gbs": round(by / tmed / 1e6, 1)})
         k = by_kernel.setdefault(kern, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
@@ -473,6 +474,9 @@ def gpu_main(args):
         ips, n_used, dt, cores, passes = time_oracle_net(N)
         cpu = {"value": ips, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"{n_used} of {N} images per pass, {passes} passes, {dt:.1f} s of CPU work, double accumulation, OpenMP"}
+        ips32, n32, dt32, _, passes32 = time_oracle_net(N, target_s=6.0, f32acc=True)
+        cpu["float_accumulator"] = {"value": ips32, "unit": UNIT,
+                                    "sample": f"{n32} of {N} images per pass, {passes32} passes, {dt32:.1f} s of CPU work, the same loops with a float accumulator"}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -535,9 +539,8 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
             B.small_pack_conv_weights(ctx, w, wb, C, C, F, F, B.MATH_3XTF32)
             fl = 2.0 * N * HW * HW * C * C * F * F
             by = 4.0 * (2 * N * C * HW * HW + C * C * F * F + C)
-            uses_tc = B.small_conv2d_uses_tensor_cores(N, C, C, HW, HW, F, F, 1, pad)
             for mode in ("fp32", "tf32", "3xtf32"):
-                if mode != "fp32" and not uses_tc:
+                if mode != "fp32" and B.small_conv2d_path(ctx, N, C, C, HW, HW, F, F, 1, pad, B.MATH[mode]) != 3:
                     continue
                 def call(mode=mode):
                     a, o = rot()

@@ -101,6 +101,17 @@ int small_last_cuda_error(small_ctx *ctx);
  * until that layer has completed before they read or write a tensor.  Results are the same either way.  The paper
  * has no counterpart. */
 int small_set_layer_overlap(small_ctx *ctx, int on);
+/* Kernel family of the full channel reductions under the tensor-core math modes.  AUTO (the default): per layer,
+ * whichever of the tensor-core kernel and the register-tiled FP32 kernel is the faster one for its channel counts
+ * (FP32 FMAs meet every mode's tolerance); TENSOR / CUDA_CORES force one family wherever it takes the shape.  For
+ * measurements and comparisons; results stay within the mode's tolerance either way.  The paper has no counterpart. */
+enum { SMALL_CONV_PATH_AUTO = 0, SMALL_CONV_PATH_TENSOR = 1, SMALL_CONV_PATH_CUDA_CORES = 2 };
+int small_set_conv_path(small_ctx *ctx, int path);
+/* Which kernel small_conv2d runs for this shape and math mode (with a 32-byte aligned output) under the context's
+ * path setting: 0 = few-input-channel kernel (network stems), 1 = register-tiled FP32 kernel, 2 = general FP32 kernel,
+ * 3 = tensor-core kernel; -1 for invalid arguments. */
+int small_conv2d_path(small_ctx *ctx, int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                      int pad_t, int pad_b, int pad_l, int pad_r, unsigned math);
 /* Synchronises `stream`, then reads and clears the device status word: *status is SMALL_OK or
  * SMALL_ERR_TIMEOUT (a tensor-core pipeline wait gave up; the affected outputs are undefined). */
 int small_device_status(small_ctx *ctx, int *status, void *stream);
@@ -188,7 +199,7 @@ int small_dwpw_conv2d(small_ctx *ctx, const float *in, const float *dw_w_blk, co
                       int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
 /* 1 if small_dwpw_conv2d runs this shape as one fused kernel under the given tensor-core math mode, else 0. */
 int small_dwpw_fused(int N, int C, int K, int H, int W, int stride, int pad_t, int pad_b, int pad_l, int pad_r, unsigned math);
-/* 1 if small_conv2d would run this shape on the tensor cores under SMALL_MATH_TF32, else 0. */
+/* 1 if small_conv2d would run this shape on the tensor cores under SMALL_MATH_TF32 (automatic path), else 0. */
 int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
                                    int pad_t, int pad_b, int pad_l, int pad_r);
 
@@ -280,19 +291,22 @@ int small_run_net_host(small_ctx *ctx, const small_layer *layers, int n_layers, 
 
 /* ---- for callers that cannot allocate device memory (the paper has no counterpart to this entry point) ---- */
 
-/* Size in bytes (32 MiB) of the workspace array built into the library image.  Every GPU that loads the library
- * holds that much device memory until the process exits. */
+/* Size in bytes (32 MiB) of the workspace array built into the library image.  A GPU holds that much device memory
+ * from small_init on that device (which loads the library's device code and looks the array up) until the process
+ * exits. */
 size_t small_static_workspace_bytes(void);
 /* small_run_net with the intermediate buffers taken from that built-in array instead of a caller workspace, for
- * callers that have no device memory to give and may not allocate any: a process whose device memory was handed
- * in full to another allocator, or a request path on which an allocation's possible device-wide synchronisation
- * is not acceptable.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine); the
- * caller still passes the blocked input and output.  Arguments, validation and results are those of
- * small_run_net.  Extra errors: SMALL_ERR_WORKSPACE when small_net_workspace_bytes(layers, n_layers, N) exceeds
- * small_static_workspace_bytes() (nothing is launched; use small_run_net with your own workspace, or a smaller
- * batch); SMALL_ERR_UNSUPPORTED for a device index of 64 or more.
- * First call on a device: looks up the array's device address (made with that device current, restored
- * afterwards).  Make that first call before starting any stream capture.
+ * callers that have no device memory to give and may not allocate any: a process whose device memory is handed
+ * to another allocator after start-up, or a request path on which an allocation's possible device-wide
+ * synchronisation is not acceptable.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library
+ * routine); the array's memory is taken earlier, when small_init loads the library on the device, so create the
+ * context before the device's memory is given away, and before any stream capture.  (The first launch of a kernel
+ * variant may still make the driver load that kernel's code; run the network once through either entry point
+ * beforehand if even that must stay off the request path.)  The caller still passes the blocked input and output.
+ * Arguments, validation and results are those of small_run_net.  Extra errors: SMALL_ERR_WORKSPACE when
+ * small_net_workspace_bytes(layers, n_layers, N) exceeds small_static_workspace_bytes() (nothing is launched; use
+ * small_run_net with your own workspace, or a smaller batch); SMALL_ERR_INVALID_ARG when the current CUDA device
+ * is not the context's device.
  * Sharing: all calls on a device use the same array, and it keeps what the last call left there.  No call
  * depends on that content (each layer overwrites its whole output before it is read), but two calls whose work
  * overlaps on the GPU - different streams, or one stream per thread - race on the array: order them, e.g. by

@@ -63,7 +63,7 @@ def lib():
         L.so_scale_shift.argtypes = [_f32p, _f32p, _f32p, _f32p, I, I, I, I, I]
         L.so_upsample_nearest.argtypes = [_f32p, _f32p, I, I, I, I, I]
         L.so_fc.argtypes = [_f32p, _f32p, _f32p, _f32p] + [I] * 4
-        L.so_abstract_layer.argtypes = [_f32p, _f32p, _f32p] + [I] * 15 + [ctypes.c_double]
+        L.so_abstract_layer.argtypes = [_f32p, _f32p, _f32p] + [I] * 11 + [ctypes.c_double]
         L.so_abstract_layer.restype = I
         L.so_num_threads.restype = I
         _lib = L
@@ -230,8 +230,8 @@ def fc(x, w, bias=None, relu=False):
     return out
 
 
-def abstract_layer(x, w, F_H, F_W, F_C, S_H, S_W, S_C, K, G_b=1, K_b=1, F_Cb=1, O_Wb=1, op="fma", init=0.0):
-    """Algorithm 1 on one image x[C][H][W]; w is [G][K][F_C][F_H][F_W] or None (op='max')."""
+def abstract_layer(x, w, F_H, F_W, F_C, S_H, S_W, S_C, K, op="fma", init=0.0):
+    """The abstract layer of Section 3.1 on one image x[C][H][W]; w is [G][K][F_C][F_H][F_W] or None (op='max')."""
     x, xp = _f(x)
     I_C, I_H, I_W = x.shape
     G = groups(I_C, F_C, S_C)
@@ -242,7 +242,7 @@ def abstract_layer(x, w, F_H, F_W, F_C, S_H, S_W, S_C, K, G_b=1, K_b=1, F_Cb=1, 
         assert w.shape == (G, K, F_C, F_H, F_W), (w.shape, (G, K, F_C, F_H, F_W))
     out = np.empty((out_channels(K, G), O_H, O_W), dtype=np.float32)
     rc = lib().so_abstract_layer(xp, wp, out.ctypes.data_as(_f32p), I_C, I_H, I_W, F_H, F_W, F_C,
-                                 S_H, S_W, S_C, K, G_b, K_b, F_Cb, O_Wb, 0 if op == "fma" else 1, float(init))
+                                 S_H, S_W, S_C, K, 0 if op == "fma" else 1, float(init))
     if rc != 0:
         raise ValueError(f"abstract layer rejected the parameters (code {rc})")
     return out

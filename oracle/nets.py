@@ -10,10 +10,13 @@ import numpy as np
 from . import conv2d, dwconv2d, fc, pool2d, out_size
 
 
-def run_net(net, params, x, keep_all=True, f32acc=False):
+def run_net(net, params, x, keep_all=True, f32acc=False, init=None):
     """x: [N][C][H][W] float32.  Returns dict name -> NCHW array ('out' is the result;
-    an FC result is [N][K][1][1])."""
+    an FC result is [N][K][1][1]).  init: named tensors that exist before the first layer
+    (the target of an accumulating layer when a sub-list of a network is run)."""
     t = {"in": np.ascontiguousarray(x, dtype=np.float32)}
+    if init:
+        t.update({k: np.ascontiguousarray(v, dtype=np.float32) for k, v in init.items()})
     for layer, (w, b) in zip(net["layers"], params):
         src = t[layer["src"]]
         op = layer["op"]

@@ -16,9 +16,8 @@
  * Two independent statements of the arithmetic live here on purpose:
  *   - so_conv2d / so_dwconv2d / so_pool2d / so_relu / so_scale_shift / so_upsample_nearest / so_fc: the per-output
  *     definitions of Section 3.2 (classes of layers);
- *   - so_abstract_layer: Algorithm 1 (the abstract layer loop nest) with its
- *     blocking parameters, taken in the paper's loop order, for any
- *     (F_H, F_W, F_C, S_H, S_W, S_C, K, G) of Section 3.1 and Table 1.
+ *   - so_abstract_layer: the abstract layer of Section 3.1 itself, element by element, for any
+ *     (F_H, F_W, F_C, S_H, S_W, S_C, K, G) - the one definition that Table 1 specialises into the classes.
  * The tests check each against the other, and both against brute force,
  * library routines and closed forms.
  *
@@ -270,83 +269,40 @@ SO_EXPORT void so_fc(const float *in, const float *w, const float *bias, float *
         }
 }
 
-/* ---- Algorithm 1: the abstract layer loop nest, for one image, in the paper's loop order.
+/* ---- The abstract layer of Section 3.1, for one image, element by element.
  *
- * Section 3.1: the window F_H x F_W x F_C slides with strides S_H, S_W over the plane and S_C over
- * channels; G = (I_C - F_C)/S_C + 1 groups, K filters per group, O_C = K*G.  Output channel g*K + k
- * reduces input channels g*S_C .. g*S_C + F_C - 1 with filter W[g][k] (Section 3.1.3: the filter
- * tensor is F_H x F_W x F_C x K x G; stored here as [G][K][F_C][F_H][F_W]).  No padding: this is the
- * paper's definition as printed.
- *
- * Blocking (Section 4.1): g in steps of G_b, k in steps of K_b, the channel reduction in steps of
- * F_Cb, output columns in steps of O_Wb; the innermost six loops are the kernel, which updates an
- * O_Wb x G_b x K_b tile in three phases (Section 4.2.1): LOAD the tile, COMPUTE, STORE it back.
- * The first F_C block starts the tile at `init` (0 for FMA layers, -inf for max pooling, 0 for ReLU);
- * later blocks pick up the stored partial result.
- *
- * op 0: FMA  (tile += I * W)        op 1: MAX (tile = max(tile, I), W unused, may be NULL)
- * The running tile is kept in double; `out` is float and receives the final values only. */
+ * Section 3.1.2: a window of F_H x F_W x F_C input elements slides with strides S_H, S_W over the plane and S_C over
+ * the channels, which gives G = (I_C - F_C)/S_C + 1 channel positions ("groups") and O_H x O_W plane positions; at
+ * every position K filters are applied, so O_C = K*G.  Output element (g*K + k, oh, ow) is the reduction of the input
+ * window whose corner is (g*S_C, oh*S_H, ow*S_W) - with the matching elements of filter W[g][k] when the reduction
+ * is a sum of products (Section 3.1.3: the filter tensor is F_H x F_W x F_C x K x G; stored here as
+ * [G][K][F_C][F_H][F_W]).  Table 1 gives the layer classes as settings of (F_H, F_W, F_C, K, G) and Table 2 the
+ * reduction of each layer: op 0 = sum of products (FMA), op 1 = maximum (W unused, may be NULL).  No padding: this is
+ * the paper's definition as printed.  `init` is what the reduction starts from (0 for sums, -inf for max pooling, 0
+ * for ReLU).  The sum is carried in double and rounded once. */
 SO_EXPORT int so_abstract_layer(const float *in, const float *w, float *out,
                                 int I_C, int I_H, int I_W,
                                 int F_H, int F_W, int F_C, int S_H, int S_W, int S_C, int K,
-                                int G_b, int K_b, int F_Cb, int O_Wb, int op, double init) {
-    if (F_C < 1 || S_C < 1 || (I_C - F_C) % S_C != 0) return -1;
+                                int op, double init) {
+    if (F_C < 1 || S_C < 1 || I_C < F_C || (I_C - F_C) % S_C != 0 || K < 1) return -1;
     int G = so_groups(I_C, F_C, S_C);
     int O_H = so_out_size(I_H, F_H, S_H, 0, 0), O_W = so_out_size(I_W, F_W, S_W, 0, 0);
-    int O_C = so_out_channels(K, G);
     if (O_H < 1 || O_W < 1 || G < 1) return -1;
-    if (G_b < 1 || K_b < 1 || F_Cb < 1 || O_Wb < 1) return -1;
-    long osz = (long)O_C * O_H * O_W;
-    double *partial = (double *)malloc(sizeof(double) * (size_t)osz); /* O between F_C blocks */
-    double *tile = (double *)malloc(sizeof(double) * (size_t)O_Wb * G_b * K_b);
-    if (!partial || !tile) { free(partial); free(tile); return -2; }
-
-    for (int g = 0; g < G; g += G_b)
-        for (int k = 0; k < K; k += K_b)
-            for (int i = 0; i < F_C; i += F_Cb)
-                for (int j = 0; j < O_H; ++j)
-                    for (int l = 0; l < O_W; l += O_Wb) {
-                        int nl = O_W - l < O_Wb ? O_W - l : O_Wb;
-                        int ng = G - g < G_b ? G - g : G_b;
-                        int nk = K - k < K_b ? K - k : K_b;
-                        int ni = F_C - i < F_Cb ? F_C - i : F_Cb;
-                        /* LOAD phase */
-                        for (int ll = 0; ll < nl; ++ll)
-                            for (int gg = 0; gg < ng; ++gg)
-                                for (int kk = 0; kk < nk; ++kk) {
-                                    long oc = (long)(g + gg) * K + (k + kk);
-                                    tile[((long)ll * G_b + gg) * K_b + kk] =
-                                        i == 0 ? init : partial[(oc * O_H + j) * O_W + (l + ll)];
-                                }
-                        /* COMPUTE phase: the kernel loops */
+    if (op == 0 && !w) return -1;
+    for (int g = 0; g < G; ++g)
+        for (int k = 0; k < K; ++k)
+            for (int oh = 0; oh < O_H; ++oh)
+                for (int ow = 0; ow < O_W; ++ow) {
+                    double r = init;
+                    for (int c = 0; c < F_C; ++c)
                         for (int x = 0; x < F_H; ++x)
-                            for (int y = 0; y < F_W; ++y)
-                                for (int ii = 0; ii < ni; ++ii)
-                                    for (int ll = 0; ll < nl; ++ll)
-                                        for (int gg = 0; gg < ng; ++gg)
-                                            for (int kk = 0; kk < nk; ++kk) {
-                                                int c = (g + gg) * S_C + (i + ii);
-                                                int ih = j * S_H + x, iw = (l + ll) * S_W + y;
-                                                double v = (double)in[((long)c * I_H + ih) * I_W + iw];
-                                                double *t = &tile[((long)ll * G_b + gg) * K_b + kk];
-                                                if (op == 0) {
-                                                    long wi = (((((long)(g + gg) * K + (k + kk)) * F_C + (i + ii)) * F_H + x) * F_W + y);
-                                                    *t += v * (double)w[wi];
-                                                } else {
-                                                    if (v > *t) *t = v;
-                                                }
-                                            }
-                        /* STORE phase */
-                        for (int ll = 0; ll < nl; ++ll)
-                            for (int gg = 0; gg < ng; ++gg)
-                                for (int kk = 0; kk < nk; ++kk) {
-                                    long oc = (long)(g + gg) * K + (k + kk);
-                                    partial[(oc * O_H + j) * O_W + (l + ll)] = tile[((long)ll * G_b + gg) * K_b + kk];
-                                }
-                    }
-    for (long o = 0; o < osz; ++o) out[o] = (float)partial[o];
-    free(partial);
-    free(tile);
+                            for (int y = 0; y < F_W; ++y) {
+                                double v = (double)in[((long)(g * S_C + c) * I_H + (oh * S_H + x)) * I_W + (ow * S_W + y)];
+                                if (op == 0) r += v * (double)w[((((long)g * K + k) * F_C + c) * F_H + x) * F_W + y];
+                                else if (v > r) r = v;
+                            }
+                    out[((long)(g * K + k) * O_H + oh) * O_W + ow] = (float)r;
+                }
     return 0;
 }
 

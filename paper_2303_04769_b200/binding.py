@@ -25,7 +25,7 @@ MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
 EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
-    "small_last_cuda_error", "small_set_layer_overlap", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
+    "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_conv2d_path", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
@@ -73,6 +73,8 @@ def lib():
     L.small_last_cuda_error.argtypes = [P]
     L.small_set_layer_overlap.argtypes = [P, I]
     L.small_device_status.argtypes = [P, ctypes.POINTER(I), P]
+    L.small_set_conv_path.argtypes = [P, I]
+    L.small_conv2d_path.argtypes = [P] + [I] * 12 + [U]
     L.small_pack.argtypes = [P, P, P, I, I, I, I, P]
     L.small_unpack.argtypes = [P, P, P, I, I, I, I, P]
     L.small_conv_weight_elems.argtypes = [I, I, I, I, U]
@@ -161,6 +163,19 @@ def small_out_size(I, F, stride, pad_before=0, pad_after=0):
 
 def small_set_layer_overlap(ctx, on):
     _check(lib().small_set_layer_overlap(ctx, 1 if on else 0), "small_set_layer_overlap")
+
+
+CONV_PATH = {"auto": 0, "tensor": 1, "cuda_cores": 2}
+CONV_KERNEL = {0: "conv_thin", 1: "conv_direct", 2: "conv_fp32", 3: "conv_tc"}
+
+
+def small_set_conv_path(ctx, path):
+    _check(lib().small_set_conv_path(ctx, CONV_PATH[path] if isinstance(path, str) else path), "small_set_conv_path")
+
+
+def small_conv2d_path(ctx, N, C, K, H, W, FH, FW, stride, pad, math):
+    pt, pb, pl, pr = pad
+    return int(lib().small_conv2d_path(ctx, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr, math))
 
 
 def small_device_status(ctx, stream=None):

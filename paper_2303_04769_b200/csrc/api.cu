@@ -100,8 +100,15 @@ SMALL_API int small_init(int device, small_ctx **out) {
         return SMALL_ERR_CUDA;
     }
     c->encode_tiled = fn;
+    c->static_workspace = nullptr;
+    if (resolve_static_workspace(c) != SMALL_OK) {      // loads the library's device code here, not inside a later call
+        cudaFree(block);
+        delete c;
+        return SMALL_ERR_CUDA;
+    }
     c->overlap = 1;
     c->dependent = 0;
+    c->conv_path = SMALL_CONV_PATH_AUTO;
     *out = c;
     return SMALL_OK;
 }
@@ -119,6 +126,13 @@ SMALL_API int small_last_cuda_error(small_ctx *ctx) { return ctx ? ctx->last_cud
 SMALL_API int small_set_layer_overlap(small_ctx *ctx, int on) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     ctx->overlap = on ? 1 : 0;
+    return SMALL_OK;
+}
+
+SMALL_API int small_set_conv_path(small_ctx *ctx, int path) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (path != SMALL_CONV_PATH_AUTO && path != SMALL_CONV_PATH_TENSOR && path != SMALL_CONV_PATH_CUDA_CORES) return SMALL_ERR_INVALID_ARG;
+    ctx->conv_path = path;
     return SMALL_OK;
 }
 
@@ -273,12 +287,42 @@ SMALL_API int small_pack_fc_weights(small_ctx *ctx, const float *w, float *wb, i
 }
 
 // ---- layers ----
+// Which kernel family a full channel reduction takes under a tensor-core math mode.  The tensor-core kernel's MMAs are
+// 128 x N x 8 with N = the layer's filters: with few channels each still occupies the pipe for its floor of 40 to 50
+// cycles, and a launch carries some microseconds of pipeline set-up and drain.  The register-tiled FP32 kernel (whose
+// result meets every mode's tolerance) has neither cost but sustains about half the FP32 FMA rate.  Measured on the
+// residual network's layers at batch 256 (tensor cores TF32 / 3xTF32 against CUDA cores, microseconds): 1x1 stride 2
+// 16->32: 9.9 / 13.6 against 8.8; 3x3 stride 2 16->32: 20.1 / 29.5 against 25.3; 3x3 16->16: 25.7 / 39.3 against 44.4;
+// 1x1 stride 2 32->64: 8.1 / 9.0 against 11.0.  Hence: CUDA cores for C * K <= 512 when the window is 1 x 1, or when the
+// mode is 3xTF32 and the stride 2 (the stride-2 view spends two or three MMAs per product on four phase planes).
+static bool prefer_cuda_cores(const small_ctx *ctx, const Geom &g, unsigned math) {
+    if (ctx && ctx->conv_path == SMALL_CONV_PATH_TENSOR) return false;
+    if (ctx && ctx->conv_path == SMALL_CONV_PATH_CUDA_CORES) return true;
+    if ((long long)g.C * g.K > 512) return false;
+    return g.FH * g.FW == 1 || (math == SMALL_MATH_3XTF32 && g.S == 2);
+}
+
+static int conv2d_path(const small_ctx *ctx, const Geom &g, unsigned math, bool out_aligned32) {
+    if (conv_thin_supported(g)) return 0;          // a reduction of a few dozen terms: CUDA cores in every math mode
+    const bool direct = conv_direct_supported(g);
+    if (math == SMALL_MATH_FP32) return direct ? 1 : 2;
+    const bool tc = out_aligned32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32);
+    if (tc && !(direct && prefer_cuda_cores(ctx, g, math))) return 3;
+    return direct ? 1 : 2;
+}
+
 SMALL_API int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
                                              int pt, int pb, int pl, int pr) {
     Geom g;
     if (make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr) != SMALL_OK) return 0;
-    if (conv_thin_supported(g)) return 0;      // a reduction of a few dozen terms: CUDA cores in every math mode
-    return conv_tc_supported(g) ? 1 : 0;
+    return conv2d_path(nullptr, g, SMALL_MATH_TF32, true) == 3 ? 1 : 0;
+}
+
+SMALL_API int small_conv2d_path(small_ctx *ctx, int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                                int pt, int pb, int pl, int pr, unsigned math) {
+    Geom g;
+    if (!ctx || !math_valid(math) || make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr) != SMALL_OK) return -1;
+    return conv2d_path(ctx, g, math, true);
 }
 
 SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
@@ -295,15 +339,17 @@ SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, cons
         return SMALL_ERR_OVERLAP;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     bool relu = flags & SMALL_RELU, acc = flags & SMALL_ACCUMULATE;
-    // at most four input channels: no dense contraction to give the tensor cores; FP32 FMAs meet every mode's tolerance
-    if (conv_thin_supported(g)) return launch_conv_thin(ctx, in, w, bias, out, g, relu, acc, st);
-    // the tensor-core epilogue may store 32 bytes per thread: an output that is only 16-byte aligned takes the FP32 kernel
-    if (math != SMALL_MATH_FP32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
-        const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);
-        const float *w_lo = w_hi + conv_w_tc_elems(C, K, FH, FW);
-        return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, relu, acc, math, st);
+    // the tensor-core epilogue may store 32 bytes per thread: an output that is only 16-byte aligned takes a CUDA-core kernel
+    switch (conv2d_path(ctx, g, math, (reinterpret_cast<uintptr_t>(out) & 31u) == 0)) {
+        case 0: return launch_conv_thin(ctx, in, w, bias, out, g, relu, acc, st);
+        case 1: return launch_conv_direct(ctx, in, w, bias, out, g, relu, acc, st);
+        case 3: {
+            const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);
+            const float *w_lo = w_hi + conv_w_tc_elems(C, K, FH, FW);
+            return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, relu, acc, math, st);
+        }
+        default: return launch_conv_fp32(ctx, in, w, bias, out, g, relu, acc, st);
     }
-    return launch_conv_fp32(ctx, in, w, bias, out, g, relu, acc, st);
 }
 
 SMALL_API int small_dwconv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,

@@ -19,6 +19,8 @@ struct small_ctx {
     size_t max_smem_optin;
     int overlap;             // small_run_net launches every layer after the first as a dependent launch (see launch_kernel)
     int dependent;           // set by small_run_net while it issues those layers
+    void *static_workspace;  // device address of the library's built-in workspace array on this device (net_static.cu)
+    int conv_path;           // SMALL_CONV_PATH_*: automatic, or one kernel family forced where it takes the shape
 };
 
 namespace small {
@@ -82,6 +84,8 @@ struct Geom {
 // Fills g and returns SMALL_OK, or the status that describes what is wrong.
 int make_geom(Geom &g, int N, int C, int K, int H, int W, int FH, int FW, int S, int pt, int pb, int pl, int pr);
 
+int resolve_static_workspace(small_ctx *);   // net_static.cu; called by small_init with the context's device current
+
 // ---- kernel launchers (each in its own .cu); all return a small_status ----
 int launch_pack(small_ctx *, const float *nchw, float *blk, int N, int C, int H, int W, cudaStream_t);
 int launch_unpack(small_ctx *, const float *blk, float *nchw, int N, int C, int H, int W, cudaStream_t);
@@ -100,6 +104,10 @@ int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, f
 // (Kg filters per group, groups S_C channels apart); span = 0: full reduction over all channel blocks
 int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
                      bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
+// register-tiled FP32 kernel: windows 1 or 3 wide, strides 1 and 2 (group convolutions as launch_conv_fp32 takes them)
+bool conv_direct_supported(const Geom &, int span = 0, int Kg = 0, int S_C = 0);
+int launch_conv_direct(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
+                       bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
 // at most four input channels, 3 x 3 (strides 1, 2) or the 10 x 4 stride-2 window: FP32 FMAs with the filters in registers
 bool conv_thin_supported(const Geom &);
 int launch_conv_thin(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,

@@ -122,7 +122,7 @@ class Net:
                 dims[L["dst"]] = (L["C"], oh, ow)
                 dims[nxt["dst"]] = (nxt["K"], oh, ow)
                 self.layer_rows.append(dict(name=L["name"] + "+" + nxt["name"], op="dwpw", C=L["C"], K=nxt["K"], H=h, W=wd, FH=3, FW=3,
-                                            stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=nxt["dst"], upto=li + 2))
+                                            stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=nxt["dst"], first=li, upto=li + 2))
                 descs.append(d)
                 skip = True
                 continue
@@ -163,7 +163,7 @@ class Net:
             self.keep += [wb, bt, wt]
             dims[L["dst"]] = (L["K"], oh, ow)
             self.layer_rows.append(dict(name=L["name"], op=L["op"], C=L["C"], K=L["K"], H=h, W=wd, FH=fh, FW=fw,
-                                        stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=L["dst"], upto=li + 1))
+                                        stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=L["dst"], first=li, upto=li + 1))
             descs.append(d)
         torch.cuda.synchronize()
         self.dims = dims

@@ -7,7 +7,7 @@ import torch
 import oracle
 import synth
 from paper_2303_04769_b200 import binding as B
-from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_l2, pad_lanes_are_zero
+from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_err, pad_lanes_are_zero, conv_path
 
 pytestmark = pytest.mark.gpu
 
@@ -31,8 +31,11 @@ def _cases(count, seed):
     return out
 
 
+@pytest.mark.parametrize("path", ["tensor", "cuda_cores"])
 @pytest.mark.parametrize("case", _cases(48, 20230304))
-def test_random_geometry_tf32_and_3xtf32(case):
+def test_random_geometry_tf32_and_3xtf32(case, path):
+    """Each geometry with the tensor-core kernel forced wherever it takes the shape, and with the register-tiled
+    CUDA-core kernel forced wherever that one does (the automatic choice between them is by channel counts)."""
     N, C, K, H, W, FH, FW, S, pad = case
     x = synth.uniform((N, C, H, W), -1.0, 1.0, 61, seed=99)
     w = synth.uniform((K, C, FH, FW), -1.0, 1.0, 62, seed=99)
@@ -44,8 +47,9 @@ def test_random_geometry_tf32_and_3xtf32(case):
     bx = to_blk(x)
     for math, tol in (("tf32", 2e-3), ("3xtf32", 1e-5)):
         out = new_blk(N, K, OH, OW)
-        B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH[math])
+        with conv_path(path):
+            B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH[math])
         assert B.small_device_status(ctx()) == 0
-        err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+        err = rel_err(from_blk(out, N, K, OH, OW), ref)
         assert err <= tol, (math, err)
         assert pad_lanes_are_zero(out, N, K, OH, OW)

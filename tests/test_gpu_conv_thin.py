@@ -7,7 +7,7 @@ import torch
 import oracle
 import synth
 from paper_2303_04769_b200 import binding as B
-from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_l2, pad_lanes_are_zero
+from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_err, pad_lanes_are_zero
 
 pytestmark = pytest.mark.gpu
 
@@ -43,16 +43,16 @@ def test_thin_conv_matches_oracle(case, math):
     OH, OW = ref.shape[2:]
     out = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | math)
-    assert rel_l2(from_blk(out, N, K, OH, OW), ref) <= 1e-5      # FP32 arithmetic whatever the mode allows
+    assert rel_err(from_blk(out, N, K, OH, OW), ref) <= 1e-5      # FP32 arithmetic whatever the mode allows
     assert pad_lanes_are_zero(out, N, K, OH, OW)
     # no bias, no ReLU
     B.small_conv2d(ctx(), bx, wb, None, out, N, C, K, H, W, FH, FW, S, pad, math)
-    assert rel_l2(from_blk(out, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad)) <= 1e-5
+    assert rel_err(from_blk(out, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad)) <= 1e-5
     # accumulate onto an existing tensor, then ReLU
     prev = rnd((N, K, OH, OW), 64)
     acc = to_blk(prev)
     B.small_conv2d(ctx(), bx, wb, dev(b), acc, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.ACCUMULATE | math)
-    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, b, S, pad, relu=True, accumulate_into=prev)) <= 1e-5
+    assert rel_err(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, b, S, pad, relu=True, accumulate_into=prev)) <= 1e-5
     assert pad_lanes_are_zero(acc, N, K, OH, OW)
     assert B.small_device_status(ctx()) == 0
 

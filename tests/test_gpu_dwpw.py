@@ -6,7 +6,7 @@ import torch
 import oracle
 import synth
 from paper_2303_04769_b200 import binding as B
-from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_l2, pad_lanes_are_zero
+from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_err, pad_lanes_are_zero
 
 pytestmark = pytest.mark.gpu
 
@@ -47,7 +47,7 @@ def test_dwpw_matches_the_two_layers(case, math):
     B.small_dwpw_conv2d(ctx(), to_blk(x), wdb, dev(bd), wpb, dev(bp), out, None if fused else scratch,
                         N, C, K, H, W, S, pad, B.RELU | B.RELU_MID | B.MATH[math])
     assert B.small_device_status(ctx()) == 0
-    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    err = rel_err(from_blk(out, N, K, OH, OW), ref)
     assert err <= {"tf32": 2e-3, "3xtf32": 1e-5, "fp32": 1e-5}[math], err
     assert pad_lanes_are_zero(out, N, K, OH, OW)
     if math != "fp32":

@@ -8,7 +8,7 @@ import torch
 import oracle
 import synth
 from paper_2303_04769_b200 import binding as B
-from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_l2, pad_lanes_are_zero
+from gpu_util import ctx, dev, to_blk, from_blk, new_blk, rel_err, pad_lanes_are_zero, conv_path, runs_on_tensor_cores
 
 pytestmark = pytest.mark.gpu
 TOL_FP32 = 1e-5
@@ -87,7 +87,7 @@ def test_avg_pool(case):
     OH, OW = ref.shape[2:]
     out = new_blk(N, C, OH, OW)
     B.small_pool2d(ctx(), to_blk(x), out, None, N, C, H, W, FH, FW, S, pad, B.POOL_AVG)
-    assert rel_l2(from_blk(out, N, C, OH, OW), ref) <= 2e-6
+    assert rel_err(from_blk(out, N, C, OH, OW), ref) <= 2e-6
     assert pad_lanes_are_zero(out, N, C, OH, OW)
 
 
@@ -117,11 +117,11 @@ def test_depthwise(case, relu):
     B.small_pack_dw_weights(ctx(), dev(w), wb, C, FH, FW)
     out = new_blk(N, C, OH, OW)
     B.small_dwconv2d(ctx(), to_blk(x), wb, dev(b), out, N, C, H, W, FH, FW, S, pad, B.RELU if relu else 0)
-    assert rel_l2(from_blk(out, N, C, OH, OW), ref) <= TOL_FP32
+    assert rel_err(from_blk(out, N, C, OH, OW), ref) <= TOL_FP32
     assert pad_lanes_are_zero(out, N, C, OH, OW)
     if not relu:
         B.small_dwconv2d(ctx(), to_blk(x), wb, None, out, N, C, H, W, FH, FW, S, pad, 0)
-        assert rel_l2(from_blk(out, N, C, OH, OW), oracle.dwconv2d(x, w, None, S, pad)) <= TOL_FP32
+        assert rel_err(from_blk(out, N, C, OH, OW), oracle.dwconv2d(x, w, None, S, pad)) <= TOL_FP32
 
 
 CONV_CASES = [  # N, C, K, H, W, FH, FW, S, pad
@@ -153,16 +153,16 @@ def test_conv_fp32(case):
     OH, OW = ref.shape[2:]
     out = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH_FP32)
-    assert rel_l2(from_blk(out, N, K, OH, OW), ref) <= TOL_FP32
+    assert rel_err(from_blk(out, N, K, OH, OW), ref) <= TOL_FP32
     assert pad_lanes_are_zero(out, N, K, OH, OW)
     # no bias, no ReLU
     B.small_conv2d(ctx(), bx, wb, None, out, N, C, K, H, W, FH, FW, S, pad, 0)
-    assert rel_l2(from_blk(out, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad)) <= TOL_FP32
+    assert rel_err(from_blk(out, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad)) <= TOL_FP32
     # accumulate onto an existing tensor (the residual join), then ReLU
     prev = rnd((N, K, OH, OW), 12)
     acc = to_blk(prev)
     B.small_conv2d(ctx(), bx, wb, dev(b), acc, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.ACCUMULATE)
-    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, b, S, pad, relu=True, accumulate_into=prev)) <= TOL_FP32
+    assert rel_err(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, b, S, pad, relu=True, accumulate_into=prev)) <= TOL_FP32
     assert pad_lanes_are_zero(acc, N, K, OH, OW)
 
 
@@ -173,10 +173,10 @@ def test_fc(N, J, K):
     B.small_pack_fc_weights(ctx(), dev(w), wb, J, K)
     out = new_blk(N, K, 1, 1)
     B.small_fc(ctx(), to_blk(x), wb, dev(b), out, N, J, K, 0)
-    assert rel_l2(from_blk(out, N, K, 1, 1).reshape(N, K), oracle.fc(x, w, b)) <= TOL_FP32
+    assert rel_err(from_blk(out, N, K, 1, 1).reshape(N, K), oracle.fc(x, w, b)) <= TOL_FP32
     assert pad_lanes_are_zero(out, N, K, 1, 1)
     B.small_fc(ctx(), to_blk(x), wb, None, out, N, J, K, B.RELU)
-    assert rel_l2(from_blk(out, N, K, 1, 1).reshape(N, K), oracle.fc(x, w, None, relu=True)) <= TOL_FP32
+    assert rel_err(from_blk(out, N, K, 1, 1).reshape(N, K), oracle.fc(x, w, None, relu=True)) <= TOL_FP32
 
 
 def test_argument_errors_launch_nothing():
@@ -225,6 +225,15 @@ CONV_TC_CASES = [  # N, C, K, H, W, FH, FW, pad  (stride 1: the shapes the tenso
 ]
 
 
+@pytest.fixture
+def tensor_path():
+    """The tests below are about the tensor-core kernel: they force it wherever it takes the shape (the automatic
+    choice hands layers with few channels to the CUDA-core kernel)."""
+    with conv_path("tensor"):
+        yield
+
+
+@pytest.mark.usefixtures("tensor_path")
 @pytest.mark.parametrize("case", CONV_TC_CASES)
 def test_conv_tf32_tensor_cores(case):
     N, C, K, H, W, FH, FW, pad = case
@@ -234,12 +243,12 @@ def test_conv_tf32_tensor_cores(case):
     bx = to_blk(x)
     ref = oracle.conv2d(x, w, b, 1, pad, relu=True)
     OH, OW = ref.shape[2:]
-    uses = B.small_conv2d_uses_tensor_cores(N, C, K, H, W, FH, FW, 1, pad)
+    uses = runs_on_tensor_cores(N, C, K, H, W, FH, FW, 1, pad)
     if W > 255:
         assert not uses      # the padded row must fit a 256-pixel TMA box (very wide rows may also exceed shared memory)
     out = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, 1, pad, B.RELU | B.MATH_TF32)
-    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    err = rel_err(from_blk(out, N, K, OH, OW), ref)
     assert B.small_device_status(ctx()) == 0
     assert err <= 2e-3, err
     if uses:
@@ -248,7 +257,7 @@ def test_conv_tf32_tensor_cores(case):
     prev = rnd((N, K, OH, OW), 19)
     acc = to_blk(prev)
     B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, 1, pad, B.ACCUMULATE | B.MATH_TF32)
-    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, 1, pad, accumulate_into=prev)) <= 2e-3
+    assert rel_err(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, 1, pad, accumulate_into=prev)) <= 2e-3
     # deterministic: the same launch twice gives the same bits
     out2 = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out2, N, C, K, H, W, FH, FW, 1, pad, B.RELU | B.MATH_TF32)
@@ -269,6 +278,7 @@ CONV_TC_STRIDE2_CASES = [  # N, C, K, H, W, FH, FW, pad  (stride 2: read as a st
 ]
 
 
+@pytest.mark.usefixtures("tensor_path")
 @pytest.mark.parametrize("case", CONV_TC_STRIDE2_CASES)
 def test_conv_tf32_tensor_cores_stride2(case):
     N, C, K, H, W, FH, FW, pad = case
@@ -278,21 +288,21 @@ def test_conv_tf32_tensor_cores_stride2(case):
     bx = to_blk(x)
     ref = oracle.conv2d(x, w, b, 2, pad, relu=True)
     OH, OW = ref.shape[2:]
-    assert B.small_conv2d_uses_tensor_cores(N, C, K, H, W, FH, FW, 2, pad)
+    assert runs_on_tensor_cores(N, C, K, H, W, FH, FW, 2, pad)
     out = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, 2, pad, B.RELU | B.MATH_TF32)
-    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    err = rel_err(from_blk(out, N, K, OH, OW), ref)
     assert B.small_device_status(ctx()) == 0
     assert 1e-7 < err <= 2e-3, err
     assert pad_lanes_are_zero(out, N, K, OH, OW)
     prev = rnd((N, K, OH, OW), 29)
     acc = to_blk(prev)
     B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, 2, pad, B.ACCUMULATE | B.MATH_TF32)
-    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, 2, pad, accumulate_into=prev)) <= 2e-3
+    assert rel_err(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, 2, pad, accumulate_into=prev)) <= 2e-3
     # the FP32 mode of the same layer stays within its own bound
     out32 = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out32, N, C, K, H, W, FH, FW, 2, pad, B.RELU | B.MATH_FP32)
-    assert rel_l2(from_blk(out32, N, K, OH, OW), ref) <= 1e-5
+    assert rel_err(from_blk(out32, N, K, OH, OW), ref) <= 1e-5
 
 
 CONV_3XTF32_CASES = [  # N, C, K, H, W, FH, FW, stride, pad
@@ -312,6 +322,7 @@ CONV_3XTF32_CASES = [  # N, C, K, H, W, FH, FW, stride, pad
 ]
 
 
+@pytest.mark.usefixtures("tensor_path")
 @pytest.mark.parametrize("case", CONV_3XTF32_CASES)
 def test_conv_3xtf32_tensor_cores(case):
     """3xTF32: TF32 part and residual of both operands, three MMAs per K step, FP32-level accuracy."""
@@ -325,7 +336,7 @@ def test_conv_3xtf32_tensor_cores(case):
     out = new_blk(N, K, OH, OW)
     B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH_3XTF32)
     assert B.small_device_status(ctx()) == 0
-    err = rel_l2(from_blk(out, N, K, OH, OW), ref)
+    err = rel_err(from_blk(out, N, K, OH, OW), ref)
     assert err <= 1e-5, err
     assert pad_lanes_are_zero(out, N, K, OH, OW)
     # not the CUDA-core kernel under another name: the same layer in FP32 mode sums in another order
@@ -335,7 +346,7 @@ def test_conv_3xtf32_tensor_cores(case):
     prev = rnd((N, K, OH, OW), 39)
     acc = to_blk(prev)
     B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, S, pad, B.ACCUMULATE | B.MATH_3XTF32)
-    assert rel_l2(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad, accumulate_into=prev)) <= 1e-5
+    assert rel_err(from_blk(acc, N, K, OH, OW), oracle.conv2d(x, w, None, S, pad, accumulate_into=prev)) <= 1e-5
 
 
 def test_tf32_issue_probe():

@@ -265,29 +265,51 @@ def test_relu_invariants():
     np.testing.assert_array_equal(r, np.maximum(x, 0) + 0.0)
 
 
-# ---------------------------------------------------------------- Algorithm 1 vs the definitions
-@pytest.mark.parametrize("blocking", [(1, 1, 1, 1), (1, 2, 3, 4), (1, 16, 2, 6), (1, 3, 5, 100)])
-def test_abstract_layer_as_convolution(blocking):
-    # Table 1 row 4: F_C = I_C, K = O_C, G = 1; result independent of the blocking parameters
-    G_b, K_b, F_Cb, O_Wb = blocking
+def test_float_accumulator_variant_is_exact_on_integers_and_within_the_rounding_bound():
+    """so_conv2d_f32acc (timed as a second CPU baseline, never used for parity): on small integers every partial sum is
+    an integer below 2^24, so float accumulation is exact and must equal the double version bit for bit - including
+    padding, stride, bias, accumulate and ReLU; on general data it may differ from the double version by at most the
+    forward error bound of a recursive float sum, n * 2^-24 * sum |terms| (Higham, Accuracy and Stability, Section 4.2)."""
+    rng = np.random.RandomState(7)
+    xi = rng.randint(-8, 9, size=(2, 5, 9, 8)).astype(np.float32)
+    wi = rng.randint(-4, 5, size=(6, 5, 3, 2)).astype(np.float32)
+    bi = rng.randint(-9, 10, size=(6,)).astype(np.float32)
+    for S, pad in [(1, (0, 0, 0, 0)), (2, (1, 2, 0, 1)), (1, (2, 1, 1, 0))]:
+        a = oracle.conv2d(xi, wi, bi, S, pad, relu=True)
+        b = oracle.conv2d(xi, wi, bi, S, pad, relu=True, f32acc=True)
+        np.testing.assert_array_equal(a.view(np.int32), b.view(np.int32))
+        prev = rng.randint(-20, 21, size=a.shape).astype(np.float32)
+        np.testing.assert_array_equal(oracle.conv2d(xi, wi, bi, S, pad, accumulate_into=prev),
+                                      oracle.conv2d(xi, wi, bi, S, pad, accumulate_into=prev, f32acc=True))
+    x, w, b = rnd((2, 7, 10, 9), 71), rnd((4, 7, 3, 3), 72), rnd((4,), 73)
+    d = oracle.conv2d(x, w, b, 1, (1, 1, 1, 1)).astype(np.float64)
+    f = oracle.conv2d(x, w, b, 1, (1, 1, 1, 1), f32acc=True).astype(np.float64)
+    n_terms = 7 * 9 + 1
+    mag = oracle.conv2d(np.abs(x), np.abs(w), np.abs(b), 1, (1, 1, 1, 1)).astype(np.float64)   # sum of |terms|
+    assert np.all(np.abs(f - d) <= (n_terms + 1) * 2.0 ** -24 * mag)
+    assert np.any(f != d)          # and it really is another accumulator, not the double routine again
+
+
+# ---------------------------------------------------------------- the abstract layer vs the layer classes
+def test_abstract_layer_as_convolution():
+    # Table 1 row 4: F_C = I_C, K = O_C, G = 1
     x = rnd((1, 5, 8, 9), 35)
     w = rnd((6, 5, 3, 2), 36)
     for S in (1, 2):
-        got = oracle.abstract_layer(x[0], w.reshape(1, 6, 5, 3, 2), 3, 2, 5, S, S, 1, 6, G_b, K_b, F_Cb, O_Wb)
+        got = oracle.abstract_layer(x[0], w.reshape(1, 6, 5, 3, 2), 3, 2, 5, S, S, 1, 6)
         np.testing.assert_array_max_ulp(got, oracle.conv2d(x, w, None, S)[0], maxulp=1)
 
 
-@pytest.mark.parametrize("G_b,O_Wb", [(1, 1), (4, 3), (16, 6)])
-def test_abstract_layer_as_depthwise_and_pool_and_relu(G_b, O_Wb):
+def test_abstract_layer_as_depthwise_and_pool_and_relu():
     # Table 1 row 2: F_C = 1, K = 1, G = I_C.  Table 2: depthwise = FMA, max pool = Max, ReLU = Max.
     x = rnd((1, 7, 8, 9), 37)
     w = rnd((7, 3, 3), 38)
-    got = oracle.abstract_layer(x[0], w.reshape(7, 1, 1, 3, 3), 3, 3, 1, 2, 2, 1, 1, G_b, 1, 1, O_Wb)
+    got = oracle.abstract_layer(x[0], w.reshape(7, 1, 1, 3, 3), 3, 3, 1, 2, 2, 1, 1)
     np.testing.assert_array_max_ulp(got, oracle.dwconv2d(x, w, None, 2)[0], maxulp=1)
-    got = oracle.abstract_layer(x[0], None, 2, 2, 1, 2, 2, 1, 1, G_b, 1, 1, O_Wb, op="max", init=-np.inf)
+    got = oracle.abstract_layer(x[0], None, 2, 2, 1, 2, 2, 1, 1, op="max", init=-np.inf)
     np.testing.assert_array_equal(got, oracle.pool2d(x, 2, 2, 2)[0])
-    # Table 1 row 1 (single element): ReLU is the Max kernel over a 1x1x1 window started at zero
-    got = oracle.abstract_layer(x[0], None, 1, 1, 1, 1, 1, 1, 1, G_b, 1, 1, O_Wb, op="max", init=0.0)
+    # Table 1 row 1 (single element): ReLU is the Max reduction over a 1x1x1 window started at zero
+    got = oracle.abstract_layer(x[0], None, 1, 1, 1, 1, 1, 1, 1, op="max", init=0.0)
     np.testing.assert_array_equal(got, oracle.relu(x)[0])
 
 
@@ -295,18 +317,30 @@ def test_abstract_layer_figure1_group_convolution():
     # Figure 1's shape: two overlapping groups of three filters over four channels each
     x = rnd((1, 6, 6, 7), 39)
     w = rnd((2, 3, 4, 3, 3), 40)
-    got = oracle.abstract_layer(x[0], w, 3, 3, 4, 1, 1, 2, 3, G_b=2, K_b=2, F_Cb=3, O_Wb=4)
+    got = oracle.abstract_layer(x[0], w, 3, 3, 4, 1, 1, 2, 3)
     assert got.shape[0] == GOLD["fig1_OC"]
     for g in range(2):
         ref = oracle.conv2d(x[:, 2 * g:2 * g + 4], w[g])[0]
         np.testing.assert_array_max_ulp(got[3 * g:3 * g + 3], ref, maxulp=1)
+    # brute force, written a second time with the indices in another order: output channel oc = g*K + k
+    xd, wd = x[0].astype(np.float64), w.astype(np.float64)
+    for oc, oh, ow in [(0, 0, 0), (2, 3, 4), (3, 0, 1), (5, 3, 4)]:
+        g, k = divmod(oc, 3)
+        want = sum(xd[g * 2 + c, oh + a, ow + b] * wd[g, k, c, a, b] for c in range(4) for a in range(3) for b in range(3))
+        assert abs(float(got[oc, oh, ow]) - want) <= 4e-7 * max(1.0, abs(want))
 
 
 def test_abstract_layer_full_reduction_is_fc():
     x = rnd((1, 4, 3, 5), 41)
     w = rnd((6, 60), 42)
-    got = oracle.abstract_layer(x[0], w.reshape(1, 6, 4, 3, 5), 3, 5, 4, 1, 1, 1, 6, 1, 4, 2, 1)
+    got = oracle.abstract_layer(x[0], w.reshape(1, 6, 4, 3, 5), 3, 5, 4, 1, 1, 1, 6)
     np.testing.assert_array_max_ulp(got.reshape(6), oracle.fc(x, w)[0], maxulp=1)
+
+
+def test_abstract_layer_rejects_windows_that_do_not_tile_the_channels():
+    x = rnd((1, 6, 4, 4), 44)
+    with pytest.raises(ValueError):
+        oracle.abstract_layer(x[0], None, 1, 1, 4, 1, 1, 3, 1, op="max")       # (6 - 4) % 3 != 0
 
 
 # ---------------------------------------------------------------- layout
