@@ -66,6 +66,15 @@ def lib():
         L.so_abstract_layer.argtypes = [_f32p, _f32p, _f32p] + [I] * 11 + [ctypes.c_double]
         L.so_abstract_layer.restype = I
         L.so_num_threads.restype = I
+        _u8p = ctypes.POINTER(ctypes.c_uint8)
+        L.so_requantize.argtypes = [I] * 5
+        L.so_requantize.restype = I
+        L.so_q_conv2d.argtypes = [_u8p, _u8p, _i32p, _u8p] + [I] * 18
+        L.so_q_dwconv2d.argtypes = [_u8p, _u8p, _i32p, _u8p] + [I] * 17
+        L.so_q_maxpool2d.argtypes = [_u8p, _u8p] + [I] * 12
+        L.so_q_relu.argtypes = [_u8p, _u8p, ctypes.c_long, I]
+        L.so_model_memory_q_mib.argtypes = [ctypes.c_long] * 3
+        L.so_model_memory_q_mib.restype = ctypes.c_double
         _lib = L
     return _lib
 
@@ -246,3 +255,75 @@ def abstract_layer(x, w, F_H, F_W, F_C, S_H, S_W, S_C, K, op="fma", init=0.0):
     if rc != 0:
         raise ValueError(f"abstract layer rejected the parameters (code {rc})")
     return out
+
+
+# ---- quantised layers: uint8 tensors (NCHW), int32 accumulation, one requantisation per output ----
+_u8p = ctypes.POINTER(ctypes.c_uint8)
+
+
+def _u8(a):
+    a = np.ascontiguousarray(a, dtype=np.uint8)
+    return a, a.ctypes.data_as(_u8p)
+
+
+def requantize(acc, mult, shift, z_out, lo=0) -> int:
+    """clamp(z_out + floor((acc * mult + 2^(shift-1)) / 2^shift), lo, 255)."""
+    return int(lib().so_requantize(int(acc), int(mult), int(shift), int(z_out), int(lo)))
+
+
+def q_conv2d(x, w, bias, stride, pad, z_in, z_w, z_out, mult, shift, relu=False):
+    x, xp = _u8(x)
+    w, wp = _u8(w)
+    N, C, H, W = x.shape
+    K, C2, FH, FW = w.shape
+    assert C2 == C
+    pt, pb, pl, pr = pad
+    OH, OW = out_size(H, FH, stride, pt, pb), out_size(W, FW, stride, pl, pr)
+    assert OH > 0 and OW > 0
+    bp = None
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.int32)
+        bp = bias.ctypes.data_as(_i32p)
+    out = np.empty((N, K, OH, OW), dtype=np.uint8)
+    lib().so_q_conv2d(xp, wp, bp, out.ctypes.data_as(_u8p), N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr,
+                      z_in, z_w, z_out, mult, shift, int(relu))
+    return out
+
+
+def q_dwconv2d(x, w, bias, stride, pad, z_in, z_w, z_out, mult, shift, relu=False):
+    x, xp = _u8(x)
+    w, wp = _u8(w)
+    N, C, H, W = x.shape
+    C2, FH, FW = w.shape
+    assert C2 == C
+    pt, pb, pl, pr = pad
+    OH, OW = out_size(H, FH, stride, pt, pb), out_size(W, FW, stride, pl, pr)
+    bp = None
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.int32)
+        bp = bias.ctypes.data_as(_i32p)
+    out = np.empty((N, C, OH, OW), dtype=np.uint8)
+    lib().so_q_dwconv2d(xp, wp, bp, out.ctypes.data_as(_u8p), N, C, H, W, FH, FW, stride, pt, pb, pl, pr,
+                        z_in, z_w, z_out, mult, shift, int(relu))
+    return out
+
+
+def q_maxpool2d(x, FH, FW, stride, pad=(0, 0, 0, 0), z=0):
+    x, xp = _u8(x)
+    N, C, H, W = x.shape
+    pt, pb, pl, pr = pad
+    OH, OW = out_size(H, FH, stride, pt, pb), out_size(W, FW, stride, pl, pr)
+    out = np.empty((N, C, OH, OW), dtype=np.uint8)
+    lib().so_q_maxpool2d(xp, out.ctypes.data_as(_u8p), N, C, H, W, FH, FW, stride, pt, pb, pl, pr, z)
+    return out
+
+
+def q_relu(x, z):
+    x, xp = _u8(x)
+    out = np.empty_like(x)
+    lib().so_q_relu(xp, out.ctypes.data_as(_u8p), x.size, z)
+    return out
+
+
+def model_memory_q_mib(params, intermediates, largest_plane) -> float:
+    return float(lib().so_model_memory_q_mib(params, intermediates, largest_plane))

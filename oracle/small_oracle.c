@@ -21,6 +21,9 @@
  * The tests check each against the other, and both against brute force,
  * library routines and closed forms.
  *
+ *   - so_q_*: the quantised (uint8 data, int32 accumulation) forms of the same definitions; the requantisation
+ *     step is a reading of this build (the paper fixes only the types), stated above so_requantize.
+ *
  * Parity unpinned: nothing (every exported routine has at least one pin in
  * tests/test_oracle_*.py).  Accuracy of trained networks is not computed here.
  */
@@ -304,6 +307,113 @@ SO_EXPORT int so_abstract_layer(const float *in, const float *w, float *out,
                     out[((long)(g * K + k) * O_H + oh) * O_W + ow] = (float)r;
                 }
     return 0;
+}
+
+/* ======================================================================================================
+ * Quantised inference (Section 5.1: "quantized to integer (unsigned 8 bit)"; Section 5.3: "input and output values
+ * are uint8, accumulations to the partial result are in int32"; Section 5.5).  The paper fixes the types and says
+ * no more; the reading taken here is the usual affine one: a tensor's real value is scale * (q - zero_point), with
+ * one (scale, zero_point) per tensor.  A layer then is exact integer arithmetic:
+ *     acc  = bias[k] + sum (q_in - z_in) * (q_w - z_w)                       (int32; padded positions are real zeros,
+ *                                                                             i.e. q_in = z_in: they add nothing)
+ *     q_out = clamp(z_out + round_half_up(acc * mult / 2^shift), lo, 255)    (one rounding; 64-bit product)
+ * where mult / 2^shift (0 <= mult < 2^31, 1 <= shift <= 62) stands for scale_in * scale_w / scale_out and bias is in
+ * units of scale_in * scale_w; lo = z_out when ReLU is fused (real 0 maps to z_out), else 0.
+ * round_half_up(a / 2^s) = floor((a + 2^(s-1)) / 2^s): an arithmetic right shift after the addition. */
+SO_EXPORT int so_requantize(int acc, int mult, int shift, int z_out, int lo) {
+    int64_t prod = (int64_t)acc * (int64_t)mult;
+    int64_t r = (prod + ((int64_t)1 << (shift - 1))) >> shift;      /* >> of a negative value: arithmetic (gcc) */
+    int64_t q = (int64_t)z_out + r;
+    if (q < lo) q = lo;
+    if (q > 255) q = 255;
+    return (int)q;
+}
+
+/* Full channel reduction on uint8 (Table 1 row 4), NCHW, filters [K][C][FH][FW] uint8, bias int32 (or NULL). */
+SO_EXPORT void so_q_conv2d(const uint8_t *in, const uint8_t *w, const int32_t *bias, uint8_t *out,
+                           int N, int C, int K, int H, int W, int FH, int FW, int S,
+                           int pt, int pb, int pl, int pr,
+                           int z_in, int z_w, int z_out, int mult, int shift, int relu) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k)
+            for (int oh = 0; oh < OH; ++oh)
+                for (int ow = 0; ow < OW; ++ow) {
+                    int32_t acc = bias ? bias[k] : 0;
+                    for (int c = 0; c < C; ++c)
+                        for (int x = 0; x < FH; ++x) {
+                            int ih = oh * S + x - pt;
+                            if (ih < 0 || ih >= H) continue;
+                            for (int y = 0; y < FW; ++y) {
+                                int iw = ow * S + y - pl;
+                                if (iw < 0 || iw >= W) continue;
+                                acc += ((int32_t)in[(((long)n * C + c) * H + ih) * W + iw] - z_in) *
+                                       ((int32_t)w[(((long)k * C + c) * FH + x) * FW + y] - z_w);
+                            }
+                        }
+                    out[(((long)n * K + k) * OH + oh) * OW + ow] = (uint8_t)so_requantize(acc, mult, shift, z_out, relu ? z_out : 0);
+                }
+}
+
+/* Single channel reduction with weights on uint8 (Table 1 row 2): depthwise, filters [C][FH][FW]. */
+SO_EXPORT void so_q_dwconv2d(const uint8_t *in, const uint8_t *w, const int32_t *bias, uint8_t *out,
+                             int N, int C, int H, int W, int FH, int FW, int S,
+                             int pt, int pb, int pl, int pr,
+                             int z_in, int z_w, int z_out, int mult, int shift, int relu) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int oh = 0; oh < OH; ++oh)
+                for (int ow = 0; ow < OW; ++ow) {
+                    int32_t acc = bias ? bias[c] : 0;
+                    for (int x = 0; x < FH; ++x) {
+                        int ih = oh * S + x - pt;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int y = 0; y < FW; ++y) {
+                            int iw = ow * S + y - pl;
+                            if (iw < 0 || iw >= W) continue;
+                            acc += ((int32_t)in[(((long)n * C + c) * H + ih) * W + iw] - z_in) *
+                                   ((int32_t)w[((long)c * FH + x) * FW + y] - z_w);
+                        }
+                    }
+                    out[(((long)n * C + c) * OH + oh) * OW + ow] = (uint8_t)so_requantize(acc, mult, shift, z_out, relu ? z_out : 0);
+                }
+}
+
+/* Max pooling on uint8 (Table 2: Max): order-preserving under the affine map, so it is the maximum of the bytes;
+ * padded positions are ignored; a window that lies wholly in the pad gives the zero point. */
+SO_EXPORT void so_q_maxpool2d(const uint8_t *in, uint8_t *out, int N, int C, int H, int W, int FH, int FW, int S,
+                              int pt, int pb, int pl, int pr, int z) {
+    int OH = so_out_size(H, FH, S, pt, pb), OW = so_out_size(W, FW, S, pl, pr);
+    for (long nc = 0; nc < (long)N * C; ++nc)
+        for (int oh = 0; oh < OH; ++oh)
+            for (int ow = 0; ow < OW; ++ow) {
+                int best = -1;
+                for (int x = 0; x < FH; ++x) {
+                    int ih = oh * S + x - pt;
+                    if (ih < 0 || ih >= H) continue;
+                    for (int y = 0; y < FW; ++y) {
+                        int iw = ow * S + y - pl;
+                        if (iw < 0 || iw >= W) continue;
+                        int v = in[(nc * H + ih) * W + iw];
+                        if (v > best) best = v;
+                    }
+                }
+                out[(nc * OH + oh) * OW + ow] = (uint8_t)(best < 0 ? z : best);
+            }
+}
+
+/* ReLU on uint8 (Table 2: Max with zero): real 0 is the zero point. */
+SO_EXPORT void so_q_relu(const uint8_t *in, uint8_t *out, long n, int z) {
+    for (long i = 0; i < n; ++i) out[i] = in[i] > z ? in[i] : (uint8_t)z;
+}
+
+/* Section 5.3, quantised models: parameters + intermediates (one byte each) + 4 bytes x the largest H x W plane of
+ * any intermediate (the int32 accumulators), in MiB. */
+SO_EXPORT double so_model_memory_q_mib(long params, long intermediates, long largest_plane) {
+    return ((double)params + (double)intermediates + 4.0 * (double)largest_plane) / 1048576.0;
 }
 
 SO_EXPORT int so_num_threads(void) {

@@ -304,7 +304,9 @@ static bool prefer_cuda_cores(const small_ctx *ctx, const Geom &g, unsigned math
 
 static int conv2d_path(const small_ctx *ctx, const Geom &g, unsigned math, bool out_aligned32) {
     if (conv_thin_supported(g)) return 0;          // a reduction of a few dozen terms: CUDA cores in every math mode
-    const bool direct = conv_direct_supported(g);
+    bool direct = conv_direct_supported(g);
+    // the register-tiled kernel computes runs of 8 output columns: planes narrower than 4 columns leave it mostly idle
+    if (direct && g.OW < 4 && !(ctx && ctx->conv_path == SMALL_CONV_PATH_CUDA_CORES)) direct = false;
     if (math == SMALL_MATH_FP32) return direct ? 1 : 2;
     const bool tc = out_aligned32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32);
     if (tc && !(direct && prefer_cuda_cores(ctx, g, math))) return 3;
