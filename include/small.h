@@ -243,6 +243,45 @@ int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N,
 int small_fc(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
              int N, int J, int K, unsigned flags, void *stream);
 
+/* ---- quantised inference (Section 5.1: "quantized to integer (unsigned 8 bit)"; Section 5.3: uint8 values, int32
+ * accumulation; Section 5.5) -------------------------------------------------------------------------------------
+ * The same blocked layout with one byte per channel: uint8[N][ceil(C/32)][H][W][32], pad lanes 0.  A tensor's real
+ * value is scale * (q - zero_point), one (scale, zero_point) per tensor; the paper fixes only the types, the affine
+ * form and the rounding below are this library's reading.  A weighted layer is exact integer arithmetic:
+ *     acc   = bias[k] + sum (q_in - z_in) * (q_w - z_w)                      (int32; padding = real zeros = z_in)
+ *     q_out = clamp(z_out + floor((acc * mult + 2^(shift-1)) / 2^shift), lo, 255)        (64-bit product, one rounding)
+ * mult / 2^shift (0 <= mult < 2^31, 1 <= shift <= 62) stands for scale_in * scale_w / scale_out; bias: int32 in
+ * units of scale_in * scale_w, or NULL; lo = z_out with SMALL_RELU (the only flag), else 0.  C * FH * FW must not
+ * exceed 33000 so that the sums stay inside 32 bits (SMALL_ERR_SHAPE).  Results are bit-exact against that
+ * definition.  Errors otherwise as the float layers. */
+size_t small_q_packed_bytes(int N, int C, int H, int W);      /* bytes of a blocked uint8 tensor */
+/* NCHW uint8[N][C][H][W] <-> blocked; byte moves. */
+int small_q_pack(small_ctx *ctx, const uint8_t *nchw, uint8_t *blk, int N, int C, int H, int W, void *stream);
+int small_q_unpack(small_ctx *ctx, const uint8_t *blk, uint8_t *nchw, int N, int C, int H, int W, void *stream);
+size_t small_q_conv_weight_bytes(int C, int K, int FH, int FW);
+/* w_kcrs: device uint8[K][C][FH][FW]; w_blk: device, 16-byte aligned, small_q_conv_weight_bytes bytes (private layout). */
+int small_q_pack_conv_weights(small_ctx *ctx, const uint8_t *w_kcrs, void *w_blk, int C, int K, int FH, int FW, void *stream);
+/* Full channel reduction on uint8 (Table 1 row 4): standard and 1x1 convolution; with H = W = FH = FW = 1 a fully
+ * connected layer.  Windows 1 or 3 wide of any height, stride 1 or 2, any padding (else SMALL_ERR_UNSUPPORTED). */
+int small_q_conv2d(small_ctx *ctx, const uint8_t *in, const void *w_blk, const int32_t *bias, uint8_t *out,
+                   int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                   int pad_t, int pad_b, int pad_l, int pad_r,
+                   int z_in, int z_w, int z_out, int mult, int shift, unsigned flags, void *stream);
+size_t small_q_dw_weight_bytes(int C, int FH, int FW);
+/* w_crs: device uint8[C][FH][FW]. */
+int small_q_pack_dw_weights(small_ctx *ctx, const uint8_t *w_crs, uint8_t *w_blk, int C, int FH, int FW, void *stream);
+/* Single channel reduction with weights on uint8 (Table 1 row 2): depthwise convolution, any window and stride. */
+int small_q_dwconv2d(small_ctx *ctx, const uint8_t *in, const uint8_t *w_blk, const int32_t *bias, uint8_t *out,
+                     int N, int C, int H, int W, int FH, int FW, int stride,
+                     int pad_t, int pad_b, int pad_l, int pad_r,
+                     int z_in, int z_w, int z_out, int mult, int shift, unsigned flags, void *stream);
+/* Max pooling on uint8 (Table 2: Max): the maximum of the bytes (the affine map keeps order); padded positions are
+ * ignored, a window wholly in the padding gives z (the tensor's zero point). */
+int small_q_maxpool2d(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, int C, int H, int W, int FH, int FW,
+                      int stride, int pad_t, int pad_b, int pad_l, int pad_r, int z, void *stream);
+/* ReLU on uint8 (Table 2: Max with zero): out = max(in, z), real zero being the zero point z.  out may equal in. */
+int small_q_relu(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, int C, int H, int W, int z, void *stream);
+
 /* ---- networks (Section 5.3: layers share intermediate buffers; Section 5.4: end-to-end inference) -- */
 
 enum { SMALL_OP_CONV = 0, SMALL_OP_DWCONV = 1, SMALL_OP_POOL = 2, SMALL_OP_RELU = 3, SMALL_OP_ADD = 4, SMALL_OP_FC = 5,

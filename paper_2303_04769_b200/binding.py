@@ -31,6 +31,8 @@ EXPORTS = [
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
     "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
+    "small_q_packed_bytes", "small_q_pack", "small_q_unpack", "small_q_conv_weight_bytes", "small_q_pack_conv_weights", "small_q_conv2d",
+    "small_q_dw_weight_bytes", "small_q_pack_dw_weights", "small_q_dwconv2d", "small_q_maxpool2d", "small_q_relu",
 ]
 
 
@@ -112,6 +114,20 @@ def lib():
     L.small_static_workspace_bytes.argtypes = []
     L.small_static_workspace_bytes.restype = Z
     L.small_run_net_static.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, P, P]
+    L.small_q_packed_bytes.argtypes = [I] * 4
+    L.small_q_packed_bytes.restype = Z
+    L.small_q_pack.argtypes = [P, P, P, I, I, I, I, P]
+    L.small_q_unpack.argtypes = [P, P, P, I, I, I, I, P]
+    L.small_q_conv_weight_bytes.argtypes = [I] * 4
+    L.small_q_conv_weight_bytes.restype = Z
+    L.small_q_pack_conv_weights.argtypes = [P, P, P, I, I, I, I, P]
+    L.small_q_conv2d.argtypes = [P, P, P, P, P] + [I] * 17 + [U, P]
+    L.small_q_dw_weight_bytes.argtypes = [I] * 3
+    L.small_q_dw_weight_bytes.restype = Z
+    L.small_q_pack_dw_weights.argtypes = [P, P, P, I, I, I, P]
+    L.small_q_dwconv2d.argtypes = [P, P, P, P, P] + [I] * 16 + [U, P]
+    L.small_q_maxpool2d.argtypes = [P, P, P] + [I] * 12 + [P]
+    L.small_q_relu.argtypes = [P, P, P, I, I, I, I, I, P]
     _lib = L
     return L
 
@@ -326,3 +342,56 @@ def small_measure_tf32_peak(ctx, n=128, iters=4096, stream=None):
     _check(lib().small_measure_tf32_peak(ctx, n, iters, _ptr(cycles), ctypes.byref(tf), ctypes.byref(cpm), _stream(stream)),
            "small_measure_tf32_peak")
     return tf.value, cpm.value
+
+
+# ---- quantised layers (uint8 tensors; qp = (z_in, z_w, z_out, mult, shift)) ----
+
+def small_q_packed_bytes(N, C, H, W):
+    return lib().small_q_packed_bytes(N, C, H, W)
+
+
+def small_q_pack(ctx, nchw, blk, N, C, H, W, stream=None):
+    _check(lib().small_q_pack(ctx, _ptr(nchw), _ptr(blk), N, C, H, W, _stream(stream)), "small_q_pack")
+
+
+def small_q_unpack(ctx, blk, nchw, N, C, H, W, stream=None):
+    _check(lib().small_q_unpack(ctx, _ptr(blk), _ptr(nchw), N, C, H, W, _stream(stream)), "small_q_unpack")
+
+
+def small_q_conv_weight_bytes(C, K, FH, FW):
+    return lib().small_q_conv_weight_bytes(C, K, FH, FW)
+
+
+def small_q_pack_conv_weights(ctx, w_kcrs, w_blk, C, K, FH, FW, stream=None):
+    _check(lib().small_q_pack_conv_weights(ctx, _ptr(w_kcrs), _ptr(w_blk), C, K, FH, FW, _stream(stream)), "small_q_pack_conv_weights")
+
+
+def small_q_conv2d(ctx, inp, w_blk, bias, out, N, C, K, H, W, FH, FW, stride, pad, qp, flags=0, stream=None):
+    pt, pb, pl, pr = pad
+    z_in, z_w, z_out, mult, shift = qp
+    _check(lib().small_q_conv2d(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr,
+                                z_in, z_w, z_out, mult, shift, flags, _stream(stream)), "small_q_conv2d")
+
+
+def small_q_dw_weight_bytes(C, FH, FW):
+    return lib().small_q_dw_weight_bytes(C, FH, FW)
+
+
+def small_q_pack_dw_weights(ctx, w_crs, w_blk, C, FH, FW, stream=None):
+    _check(lib().small_q_pack_dw_weights(ctx, _ptr(w_crs), _ptr(w_blk), C, FH, FW, _stream(stream)), "small_q_pack_dw_weights")
+
+
+def small_q_dwconv2d(ctx, inp, w_blk, bias, out, N, C, H, W, FH, FW, stride, pad, qp, flags=0, stream=None):
+    pt, pb, pl, pr = pad
+    z_in, z_w, z_out, mult, shift = qp
+    _check(lib().small_q_dwconv2d(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, C, H, W, FH, FW, stride, pt, pb, pl, pr,
+                                  z_in, z_w, z_out, mult, shift, flags, _stream(stream)), "small_q_dwconv2d")
+
+
+def small_q_maxpool2d(ctx, inp, out, N, C, H, W, FH, FW, stride, pad, z, stream=None):
+    pt, pb, pl, pr = pad
+    _check(lib().small_q_maxpool2d(ctx, _ptr(inp), _ptr(out), N, C, H, W, FH, FW, stride, pt, pb, pl, pr, z, _stream(stream)), "small_q_maxpool2d")
+
+
+def small_q_relu(ctx, inp, out, N, C, H, W, z, stream=None):
+    _check(lib().small_q_relu(ctx, _ptr(inp), _ptr(out), N, C, H, W, z, _stream(stream)), "small_q_relu")

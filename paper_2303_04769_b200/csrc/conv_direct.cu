@@ -20,6 +20,8 @@
 // differ in the low three bits.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -34,8 +36,12 @@ constexpr int kMaxThreads = 256;
 constexpr int kMaxRegs = 168;     // 12 resident warps per SM
 
 struct DirectArgs {
-    const float *bias; float *out; int *status;
+    const void *bias; void *out; int *status;     // float (quantised form: int32 bias, uint8 output)
     int N, C, K, OH, OW, CB, KB, FH, pt, pl;
+    int H, W;                   // input plane (the quantised epilogue needs the taps that fall inside it)
+    const int *q_tab;           // quantised form: per filter and tap the sum of its weight bytes [K][T], then per filter [K]
+    int zx, zw, zo, mult, shift;   // quantised form: zero points of input, weights and output; requantisation multiplier / 2^shift
+    int cpb;                    // stages per 32-channel block (32 / cch; the quantised form takes a whole block per stage)
     int gw, gw_shift;           // column groups (of 8 pixels) of a unit: 1, 2 or 4
     int TH, NI;                 // output rows per image in a unit, images per unit
     int bands, tiles_w, units;  // row bands per image, column tiles per row, all units of the layer
@@ -51,11 +57,17 @@ struct DirectArgs {
     int relu, accumulate;
 };
 
-__device__ __forceinline__ void lds128(uint32_t addr, float *v) {
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "r"(addr));
+__device__ __forceinline__ void lds128(uint32_t addr, uint32_t *v) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(addr));
 }
 
-template <int FW, int S>
+// Q: the quantised form of the same loop nest (Section 5.5).  A pixel of a channel block is 32 bytes = 8 words of 4
+// channels, so the shared-memory geometry is that of the float form with 8 channels per stage; a word of the input
+// meets a word of 4 channel bytes of a filter in one 4-way dot product with 32-bit accumulation (dp4a) instead of an
+// FMA.  Accumulated are the raw sums of byte products and, per pixel, the sum of the input bytes; the zero points enter
+// in the STORE phase:  sum (x - zx)(w - zw) = sum x w - zw sum x - zx sum_{taps inside the plane} w + taps C zx zw,
+// where pixels outside the plane (TMA's zero fill) take no part, which makes them real zeros.
+template <int FW, int S, bool Q>
 __global__ void __maxnreg__(kMaxRegs)
 conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_w, const DirectArgs a) {
     constexpr int PXH = S == 1 ? 8 : 4;           // pixels per pass over the registers (stride 2: two passes of 4)
@@ -91,9 +103,9 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
     // channel blocks this filter tile reduces over (all of them; a group convolution's filter block reads `span`)
     const int cb0 = a.Kg > 0 ? ((kb0 * 32) / a.Kg * a.S_C) / 32 : 0;
     const int blocks = min(a.span, a.CB - cb0);
-    const int cpb = 32 / a.cch;
+    const int cpb = a.cpb;
     const int last_n = min(32, a.C - (cb0 + blocks - 1) * 32);
-    const int n_chunks = (blocks - 1) * cpb + (last_n + a.cch - 1) / a.cch;
+    const int n_chunks = Q ? blocks : (blocks - 1) * cpb + (last_n + a.cch - 1) / a.cch;
 
     auto issue = [&](int q, int s) {       // one thread: arm the stage's barrier, start its copies
         const int cbj = q / cpb, c0 = (q - cbj * cpb) * a.cch;
@@ -118,11 +130,15 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
     if (threadIdx.x == 0)
         for (int q = 0; q < a.stages - 1 && q < n_chunks; ++q) issue(q, q);
 
-    float acc[kPW][kKQ];
+    typedef typename std::conditional<Q, uint32_t, float>::type AccT;
+    AccT acc[kPW][kKQ];
+    uint32_t sx[Q ? kPW : 1];                     // quantised form: sum of the input bytes each pixel's window has seen
 #pragma unroll
-    for (int p = 0; p < kPW; ++p)
+    for (int p = 0; p < kPW; ++p) {
+        if (Q) sx[Q ? p : 0] = 0u;
 #pragma unroll
-        for (int k = 0; k < kKQ; ++k) acc[p][k] = 0.0f;
+        for (int k = 0; k < kKQ; ++k) acc[p][k] = AccT(0);
+    }
 
     // idle lanes read the box's first run: in bounds, never stored
     const int p_base = img < a.NI ? (img * a.th_in + row * S) * a.cols_box + g * kPW * S : 0;
@@ -144,8 +160,9 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
         __syncwarp();
         if (ok) {
             const int cbj = q / cpb, c0 = (q - cbj * cpb) * a.cch;
-            const int ci_n = min(a.cch, a.C - (cb0 + cbj) * 32 - c0);
-            const int c4_n = (ci_n + 3) >> 2;
+            // 16-byte chunks of a pixel that hold real channels: 4 floats, or 16 channel bytes, each
+            const int lanes_n = min(32, a.C - (cb0 + cbj) * 32);
+            const int c4_n = Q ? (lanes_n + 15) >> 4 : (min(a.cch, lanes_n - c0) + 3) >> 2;
             const uint32_t in_u = base + s * a.stage_bytes + pw * a.unit_bytes;       // shared-window addresses
             const uint32_t w_s = base + s * a.stage_bytes + w_off;
             for (int x = 0; x < a.FH; ++x) {
@@ -161,23 +178,29 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
                         pa[i] = in_u + ((uint32_t)p << pix_shift) + (((uint32_t)(p >> a.sw_shift) & a.sw_mask) << 4);
                     }
                     for (int j = 0; j < c4_n; ++j) {
-                        float v[NINH * 4];
+                        uint32_t v[NINH * 4];
 #pragma unroll
                         for (int i = 0; i < NINH; ++i) lds128(pa[i] ^ ((uint32_t)j << 4), &v[4 * i]);
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) {
 #pragma unroll
                             for (int y = 0; y < FW; ++y) {
-                                float w[8];
+                                uint32_t w[8];
                                 const uint32_t wa = w_s + (uint32_t)(((x * FW + y) * a.cch + 4 * j + cc) * KTb) * 4u;
                                 lds128(wa, &w[0]);
                                 lds128(wa + 16, &w[4]);
 #pragma unroll
                                 for (int p = 0; p < PXH; ++p) {
-                                    const float xv = v[(p * S + y) * 4 + cc];
-                                    float *ac = acc[pass * PXH + p];
+                                    const uint32_t xv = v[(p * S + y) * 4 + cc];
+                                    AccT *ac = acc[pass * PXH + p];
+                                    if (Q) {
+                                        sx[Q ? pass * PXH + p : 0] = __dp4a(xv, 0x01010101u, sx[Q ? pass * PXH + p : 0]);
 #pragma unroll
-                                    for (int k = 0; k < kKQ; ++k) ac[k] = fmaf(xv, w[k], ac[k]);
+                                        for (int k = 0; k < kKQ; ++k) ac[k] = (AccT)__dp4a(xv, w[k], (uint32_t)ac[k]);
+                                    } else {
+#pragma unroll
+                                        for (int k = 0; k < kKQ; ++k) ac[k] = (AccT)fmaf(__uint_as_float(xv), __uint_as_float(w[k]), (float)ac[k]);
+                                    }
                                 }
                             }
                         }
@@ -195,42 +218,91 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
         return;
     }
 
-    // STORE phase: + bias, + the tensor already in `out` (accumulate), ReLU; 32 bytes per pixel and thread.  Lanes of
-    // the last filter block beyond K stay +0: the thread holding the launch's last filter group writes them.
+    // STORE phase.  Lanes of the last filter block beyond K stay zero: the thread holding the launch's last filter group
+    // writes them.
     if (!valid) return;
     const int kq0 = k0 + kw * kKQ;
     const int kb = kq0 >> 5, kl = kq0 & 31;
     if (kb >= a.KB) return;
-    float bv[kKQ];
-#pragma unroll
-    for (int k = 0; k < kKQ; ++k) bv[k] = (a.bias && kq0 + k < a.K) ? a.bias[kq0 + k] : 0.0f;
     const int n = n0 + img, oh = oh0 + row;
     const bool last_group = kq0 + kKQ == a.k_tiles * a.KT;
-    float *dst = a.out + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow0 + g * kPW) * 32 + kl;
+    if constexpr (Q) {
+        // zero points, bias, one requantisation (round half up of the 64-bit product), clamp, 8 bytes per pixel and thread
+        const int T = a.FH * FW;
+        const int *bias = static_cast<const int *>(a.bias);
+        int bv[kKQ], wall[kKQ];
 #pragma unroll
-    for (int p = 0; p < kPW; ++p) {
-        if (ow0 + g * kPW + p >= a.OW) break;
-        float4 *d4 = reinterpret_cast<float4 *>(dst + p * 32);
-        float r[kKQ];
-#pragma unroll
-        for (int k = 0; k < kKQ; ++k) r[k] = acc[p][k] + bv[k];
-        if (a.accumulate) {
-            const float4 o0 = d4[0], o1 = d4[1];
-            r[0] += o0.x; r[1] += o0.y; r[2] += o0.z; r[3] += o0.w;
-            r[4] += o1.x; r[5] += o1.y; r[6] += o1.z; r[7] += o1.w;
+        for (int k = 0; k < kKQ; ++k) {
+            const bool real = kq0 + k < a.K;
+            bv[k] = (bias && real) ? bias[kq0 + k] : 0;
+            wall[k] = real ? a.q_tab[a.K * T + kq0 + k] : 0;
         }
-        if (a.relu) {
+        const int ih0 = oh * a.cs - a.pt;
+        const int x0 = max(0, -ih0), x1 = min(a.FH, a.H - ih0);
+        const int lo = a.relu ? a.zo : 0;
+        uint8_t *dst = static_cast<uint8_t *>(a.out) + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow0 + g * kPW) * 32 + kl;
 #pragma unroll
-            for (int k = 0; k < kKQ; ++k) r[k] = fmaxf(r[k], 0.0f);
-        }
-        if (kq0 + kKQ > a.K) {
+        for (int p = 0; p < kPW; ++p) {
+            const int ow = ow0 + g * kPW + p;
+            if (ow >= a.OW) break;
+            const int iw0 = ow * a.cs - a.pl;
+            const int y0 = max(0, -iw0), y1 = min(FW, a.W - iw0);
+            const int nv = (x1 - x0) * (y1 - y0);                 // taps of this pixel's window that lie inside the plane
+            uint32_t packed[2] = {0u, 0u};
 #pragma unroll
-            for (int k = 0; k < kKQ; ++k) if (kq0 + k >= a.K) r[k] = 0.0f;
+            for (int k = 0; k < kKQ; ++k) {
+                int q = 0;
+                if (kq0 + k < a.K) {
+                    int sw = wall[k];
+                    if (nv != T) {                                // a border pixel: only the taps inside count
+                        sw = 0;
+                        for (int x = x0; x < x1; ++x)
+                            for (int y = y0; y < y1; ++y) sw += a.q_tab[(kq0 + k) * T + x * FW + y];
+                    }
+                    const long long t = (long long)acc[p][k] - (long long)a.zw * (long long)sx[Q ? p : 0] - (long long)a.zx * sw +
+                                        (long long)nv * a.C * a.zx * a.zw + bv[k];
+                    const long long r = (t * (long long)a.mult + (1ll << (a.shift - 1))) >> a.shift;
+                    const long long z = (long long)a.zo + r;
+                    q = (int)(z < lo ? lo : z > 255 ? 255 : z);
+                }
+                packed[k >> 2] |= (uint32_t)q << (8 * (k & 3));
+            }
+            *reinterpret_cast<uint2 *>(dst + p * 32) = make_uint2(packed[0], packed[1]);
+            if (last_group)
+                for (int z = kl + kKQ; z < 32; z += 8) *reinterpret_cast<uint2 *>(dst + p * 32 - kl + z) = make_uint2(0u, 0u);
         }
-        d4[0] = make_float4(r[0], r[1], r[2], r[3]);
-        d4[1] = make_float4(r[4], r[5], r[6], r[7]);
-        if (last_group)
-            for (int z = kl + kKQ; z < 32; z += 4) *reinterpret_cast<float4 *>(dst + p * 32 - kl + z) = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+        // + bias, + the tensor already in `out` (accumulate), ReLU; 32 bytes per pixel and thread
+        const float *bias = static_cast<const float *>(a.bias);
+        float bv[kKQ];
+#pragma unroll
+        for (int k = 0; k < kKQ; ++k) bv[k] = (bias && kq0 + k < a.K) ? bias[kq0 + k] : 0.0f;
+        float *dst = static_cast<float *>(a.out) + ((((size_t)n * a.KB + kb) * a.OH + oh) * a.OW + ow0 + g * kPW) * 32 + kl;
+#pragma unroll
+        for (int p = 0; p < kPW; ++p) {
+            if (ow0 + g * kPW + p >= a.OW) break;
+            float4 *d4 = reinterpret_cast<float4 *>(dst + p * 32);
+            float r[kKQ];
+#pragma unroll
+            for (int k = 0; k < kKQ; ++k) r[k] = (float)acc[p][k] + bv[k];
+            if (a.accumulate) {
+                const float4 o0 = d4[0], o1 = d4[1];
+                r[0] += o0.x; r[1] += o0.y; r[2] += o0.z; r[3] += o0.w;
+                r[4] += o1.x; r[5] += o1.y; r[6] += o1.z; r[7] += o1.w;
+            }
+            if (a.relu) {
+#pragma unroll
+                for (int k = 0; k < kKQ; ++k) r[k] = fmaxf(r[k], 0.0f);
+            }
+            if (kq0 + kKQ > a.K) {
+#pragma unroll
+                for (int k = 0; k < kKQ; ++k) if (kq0 + k >= a.K) r[k] = 0.0f;
+            }
+            d4[0] = make_float4(r[0], r[1], r[2], r[3]);
+            d4[1] = make_float4(r[4], r[5], r[6], r[7]);
+            if (last_group)
+                for (int z = kl + kKQ; z < 32; z += 4) *reinterpret_cast<float4 *>(dst + p * 32 - kl + z) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
     }
 }
 
@@ -241,12 +313,13 @@ size_t round1k(size_t b) { return (b + 1023) & ~(size_t)1023; }
 // Tile shapes.  The unit of a row warp follows from the plane's width; what is chosen is the number of channels per
 // stage (8 or 16) and of units per block: the smallest blocks (finest work granularity over the SMs) that still keep
 // 12 or more warps resident per SM within shared memory.
-DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem) {
+DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem, bool quant = false) {
     DirectPlan best{};
     best.ok = false;
     if ((g.FW != 1 && g.FW != 3) || (g.S != 1 && g.S != 2) || g.FH * g.FW > 256) return best;
     DirectArgs a{};
     a.N = g.N; a.C = g.C; a.K = g.K; a.OH = g.OH; a.OW = g.OW; a.CB = g.CB; a.KB = g.KB; a.FH = g.FH; a.pt = g.pt; a.pl = g.pl;
+    a.H = g.H; a.W = g.W;
     a.span = span > 0 ? span : g.CB; a.Kg = span > 0 ? Kg : 0; a.S_C = S_C;
     a.gw = g.OW <= 8 ? 1 : g.OW <= 16 ? 2 : 4;
     a.gw_shift = a.gw == 1 ? 0 : a.gw == 2 ? 1 : 2;
@@ -269,12 +342,13 @@ DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem
     const int T = g.FH * g.FW;
     const int last_n = g.C - (g.CB - 1) * 32;
     int best_warps = 0;
-    for (int cch = 16; cch >= 8; cch -= 8) {
-        const int n_chunks = ((span > 0 ? span : g.CB) - 1) * (32 / cch) + ceil_div(last_n, cch);
+    // (the quantised form has one geometry: a stage is a whole 32-channel block, 8 words of 4 channel bytes per pixel)
+    for (int cch = quant ? 8 : 16; cch >= 8; cch -= 8) {
+        const int n_chunks = quant ? g.CB : ((span > 0 ? span : g.CB) - 1) * (32 / cch) + ceil_div(last_n, cch);
         for (int pwarps = 1; pwarps * kwarps * 32 <= kMaxThreads; ++pwarps) {
             if (pwarps * kwarps < 2) continue;
             DirectArgs c = a;
-            c.cch = cch; c.pwarps = pwarps;
+            c.cch = cch; c.pwarps = pwarps; c.cpb = quant ? 1 : 32 / cch;
             c.sw_shift = cch == 16 ? 1 : 2; c.sw_mask = cch == 16 ? 3 : 1;
             c.in_box_bytes = (uint32_t)((size_t)a.NI * a.th_in * a.cols_box * cch * 4);
             c.unit_bytes = (uint32_t)round1k(c.in_box_bytes);
@@ -311,39 +385,46 @@ bool conv_direct_supported(const Geom &g, int span, int Kg, int S_C) {
     return plan_direct(g, span, Kg, S_C, 227 * 1024).ok;
 }
 
-int launch_conv_direct(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, const Geom &g,
-                       bool relu, bool accumulate, cudaStream_t st, int span, int Kg, int S_C) {
-    DirectPlan p = plan_direct(g, span, Kg, S_C, ctx->max_smem_optin);
-    if (!p.ok) return SMALL_ERR_UNSUPPORTED;
+namespace {
+
+// Tensor maps and launch shared by the float and the quantised form.  esize: bytes per channel of the activation
+// tensor (4 or 1); the filter tensor is [KB][span][FH*FW][32][32] 4-byte words in both forms (floats [ci][ko], or
+// words of 4 channel bytes [c4][ko] in the first 8 of the 32 rows' worth - see pack_q_conv_w_kernel).
+int launch_direct(small_ctx *ctx, DirectPlan &p, const Geom &g, const void *in, const void *w, bool quant, cudaStream_t st) {
     DirectArgs &a = p.a;
-    a.bias = bias; a.out = out; a.status = ctx->dev_status; a.relu = relu; a.accumulate = accumulate;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_in, map_w;
-    {   // activations [N][CB][H][W][32]: box = cch channels x cols_box x th_in x 1 block x NI images, swizzled
+    {   // activations [N][CB][H][W][32]: box = one stage's channels x cols_box x th_in x 1 block x NI images, swizzled
+        const cuuint64_t px = quant ? 32 : 128;      // bytes per pixel and channel block
         cuuint64_t dims[5] = {32, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.CB, (cuuint64_t)g.N};
-        cuuint64_t strides[4] = {128, (cuuint64_t)g.W * 128, (cuuint64_t)g.H * g.W * 128, (cuuint64_t)g.CB * g.H * g.W * 128};
+        cuuint64_t strides[4] = {px, (cuuint64_t)g.W * px, (cuuint64_t)g.H * g.W * px, (cuuint64_t)g.CB * g.H * g.W * px};
         const cuuint32_t es = (cuuint32_t)a.es;     // element stride 2: a box of 2 cols x 2 rows elements lands as cols x rows pixels
-        cuuint32_t box[5] = {(cuuint32_t)a.cch, (cuuint32_t)a.cols_box * es, (cuuint32_t)a.th_in * es, 1, (cuuint32_t)a.NI};
+        cuuint32_t box[5] = {(cuuint32_t)(quant ? 32 : a.cch), (cuuint32_t)a.cols_box * es, (cuuint32_t)a.th_in * es, 1, (cuuint32_t)a.NI};
         cuuint32_t estr[5] = {1, es, es, 1, 1};
-        CUresult r = encode(&map_in, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float *>(in), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, a.cch == 16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
-    }
-    {   // packed FP32 filters [KB][span][FH*FW][32 ci][32 ko]: box = up to 32 filters x cch channels x all taps
-        const int T = g.FH * g.FW;
-        cuuint64_t dims[4] = {32, 32, (cuuint64_t)T, (cuuint64_t)g.KB * a.span};
-        cuuint64_t strides[3] = {128, 32 * 128, (cuuint64_t)T * 32 * 128};
-        cuuint32_t box[4] = {(cuuint32_t)(a.KT < 32 ? a.KT : 32), (cuuint32_t)a.cch, (cuuint32_t)T, 1};
-        cuuint32_t estr[4] = {1, 1, 1, 1};
-        CUresult r = encode(&map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float *>(w), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CUresult r = encode(&map_in, quant ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<void *>(in), dims,
+                            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            a.cch == 16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
     }
-    void (*kern)(const CUtensorMap, const CUtensorMap, const DirectArgs) =
-        g.FW == 1 ? (g.S / a.es == 1 ? conv_direct_kernel<1, 1> : conv_direct_kernel<1, 2>)
-                  : (g.S == 1 ? conv_direct_kernel<3, 1> : conv_direct_kernel<3, 2>);
+    {   // packed filters: box = up to 32 filters x one stage's channel rows x all taps
+        const int T = g.FH * g.FW;
+        const cuuint64_t rows = quant ? 8 : 32;      // words per filter, tap and channel block
+        cuuint64_t dims[4] = {32, rows, (cuuint64_t)T, (cuuint64_t)g.KB * a.span};
+        cuuint64_t strides[3] = {128, rows * 128, (cuuint64_t)T * rows * 128};
+        cuuint32_t box[4] = {(cuuint32_t)(a.KT < 32 ? a.KT : 32), (cuuint32_t)a.cch, (cuuint32_t)T, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        CUresult r = encode(&map_w, quant ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void *>(w), dims,
+                            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
+    }
+    const int S = g.S / a.es;
+    void (*kern)(const CUtensorMap, const CUtensorMap, const DirectArgs);
+    if (quant) kern = g.FW == 1 ? (S == 1 ? conv_direct_kernel<1, 1, true> : conv_direct_kernel<1, 2, true>)
+                                : (S == 1 ? conv_direct_kernel<3, 1, true> : conv_direct_kernel<3, 2, true>);
+    else kern = g.FW == 1 ? (S == 1 ? conv_direct_kernel<1, 1, false> : conv_direct_kernel<1, 2, false>)
+                          : (S == 1 ? conv_direct_kernel<3, 1, false> : conv_direct_kernel<3, 2, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
@@ -353,6 +434,29 @@ int launch_conv_direct(small_ctx *ctx, const float *in, const float *w, const fl
     launch_kernel(ctx, kern, dim3((unsigned)p.blocks), dim3(p.threads), p.smem, st, map_in, map_w, a);
     ctx->dependent = dependent;
     return check_launch(ctx);
+}
+
+}  // namespace
+
+int launch_conv_direct(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, const Geom &g,
+                       bool relu, bool accumulate, cudaStream_t st, int span, int Kg, int S_C) {
+    DirectPlan p = plan_direct(g, span, Kg, S_C, ctx->max_smem_optin);
+    if (!p.ok) return SMALL_ERR_UNSUPPORTED;
+    DirectArgs &a = p.a;
+    a.bias = bias; a.out = out; a.status = ctx->dev_status; a.relu = relu; a.accumulate = accumulate;
+    return launch_direct(ctx, p, g, in, w, false, st);
+}
+
+bool q_conv_supported(const Geom &g) { return plan_direct(g, 0, 0, 0, 227 * 1024, true).ok; }
+
+int launch_q_conv(small_ctx *ctx, const uint8_t *in, const uint32_t *w_words, const int *tables, const int *bias, uint8_t *out,
+                  const Geom &g, bool relu, int zx, int zw, int zo, int mult, int shift, cudaStream_t st) {
+    DirectPlan p = plan_direct(g, 0, 0, 0, ctx->max_smem_optin, true);
+    if (!p.ok) return SMALL_ERR_UNSUPPORTED;
+    DirectArgs &a = p.a;
+    a.bias = bias; a.out = out; a.status = ctx->dev_status; a.relu = relu; a.accumulate = 0;
+    a.q_tab = tables; a.zx = zx; a.zw = zw; a.zo = zo; a.mult = mult; a.shift = shift;
+    return launch_direct(ctx, p, g, in, w_words, true, st);
 }
 
 }  // namespace small
