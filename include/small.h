@@ -199,6 +199,21 @@ int small_dwpw_conv2d(small_ctx *ctx, const float *in, const float *dw_w_blk, co
                       int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
 /* 1 if small_dwpw_conv2d runs this shape as one fused kernel under the given tensor-core math mode, else 0. */
 int small_dwpw_fused(int N, int C, int K, int H, int W, int stride, int pad_t, int pad_b, int pad_l, int pad_r, unsigned math);
+/* Abstract fused layer (Section 6): convolution (+ bias, + ReLU with SMALL_RELU) followed by a 2 x 2 stride-2 max pool
+ * (no padding; an odd last row or column is dropped, as Section 3.1.2's size rule says), as one layer:
+ *   out[n,k,i,j] = max over the 2 x 2 block (2i.., 2j..) of act(conv(in)[n,k,.,.] + bias[k])
+ * in: blocked [N][C][H][W]; out: blocked [N][K][OH/2][OW/2] with OH, OW the convolution's output size.  Shapes
+ * small_conv_maxpool_fused accepts (windows 1 or 3 wide, stride 1 or 2, an even number of convolution rows per tile) run
+ * as ONE kernel whose STORE phase pools in registers and by one warp shuffle, so the convolution's output never reaches
+ * memory; it computes FP32 FMAs on the CUDA cores in every math mode (within each mode's tolerance).  Other shapes run the
+ * two layers through `scratch` (device, small_packed_elems(N, K, OH, OW) floats; may be NULL when the fused kernel runs -
+ * SMALL_ERR_WORKSPACE if it is needed and NULL).  flags: SMALL_RELU | one SMALL_MATH_*.  Errors as small_conv2d; SHAPE
+ * also when the convolution's output has fewer than 2 rows or columns. */
+int small_conv_maxpool2d(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out, float *scratch,
+                         int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                         int pad_t, int pad_b, int pad_l, int pad_r, unsigned flags, void *stream);
+/* 1 if small_conv_maxpool2d runs this shape as one fused kernel, else 0. */
+int small_conv_maxpool_fused(int N, int C, int K, int H, int W, int FH, int FW, int stride, int pad_t, int pad_b, int pad_l, int pad_r);
 /* 1 if small_conv2d would run this shape on the tensor cores under SMALL_MATH_TF32 (automatic path), else 0. */
 int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, int FH, int FW, int stride,
                                    int pad_t, int pad_b, int pad_l, int pad_r);
@@ -285,7 +300,9 @@ int small_q_relu(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, int C, 
 /* ---- networks (Section 5.3: layers share intermediate buffers; Section 5.4: end-to-end inference) -- */
 
 enum { SMALL_OP_CONV = 0, SMALL_OP_DWCONV = 1, SMALL_OP_POOL = 2, SMALL_OP_RELU = 3, SMALL_OP_ADD = 4, SMALL_OP_FC = 5,
-       SMALL_OP_DWPW = 6 };  /* depthwise 3x3 then 1x1 convolution as one fused layer (small_dwpw_conv2d) */
+       SMALL_OP_DWPW = 6,     /* depthwise 3x3 then 1x1 convolution as one fused layer (small_dwpw_conv2d) */
+       SMALL_OP_CONVPOOL = 7 }; /* convolution then 2x2 stride-2 max pool as one fused layer (small_conv_maxpool2d); the shape
+                                 * must be one small_conv_maxpool_fused accepts */
 enum { SMALL_SLOT_INPUT = -1, SMALL_SLOT_OUTPUT = -2 }; /* the caller's in_blk / out_blk */
 
 typedef struct small_layer {

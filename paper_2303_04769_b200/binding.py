@@ -19,7 +19,7 @@ OK = 0
 RELU, ACCUMULATE, RELU_MID = 1, 2, 4
 MATH_FP32, MATH_TF32, MATH_3XTF32 = 0 << 4, 1 << 4, 2 << 4
 POOL_MAX, POOL_AVG = 0, 1
-OP_CONV, OP_DWCONV, OP_POOL, OP_RELU, OP_ADD, OP_FC, OP_DWPW = range(7)
+OP_CONV, OP_DWCONV, OP_POOL, OP_RELU, OP_ADD, OP_FC, OP_DWPW, OP_CONVPOOL = range(8)
 SLOT_INPUT, SLOT_OUTPUT = -1, -2
 MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
@@ -27,7 +27,7 @@ EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
     "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_conv2d_path", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
-    "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
+    "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_conv_maxpool2d", "small_conv_maxpool_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
     "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
@@ -89,6 +89,8 @@ def lib():
     L.small_group_conv2d.argtypes = [P, P, P, P, P] + [I] * 14 + [U, P]
     L.small_dwpw_conv2d.argtypes = [P] * 8 + [I] * 10 + [U, P]
     L.small_dwpw_fused.argtypes = [I] * 10 + [U]
+    L.small_conv_maxpool2d.argtypes = [P] * 6 + [I] * 12 + [U, P]
+    L.small_conv_maxpool_fused.argtypes = [I] * 12
     L.small_dw_weight_elems.argtypes = [I, I, I]
     L.small_dw_weight_elems.restype = Z
     L.small_pack_dw_weights.argtypes = [P, P, P, I, I, I, P]
@@ -266,6 +268,17 @@ def small_dwpw_conv2d(ctx, inp, dw_w_blk, dw_bias, pw_w_blk, pw_bias, out, scrat
 def small_dwpw_fused(N, C, K, H, W, stride, pad, math):
     pt, pb, pl, pr = pad
     return bool(lib().small_dwpw_fused(N, C, K, H, W, stride, pt, pb, pl, pr, math))
+
+
+def small_conv_maxpool2d(ctx, inp, w_blk, bias, out, scratch, N, C, K, H, W, FH, FW, stride, pad, flags=0, stream=None):
+    pt, pb, pl, pr = pad
+    _check(lib().small_conv_maxpool2d(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), _ptr(scratch), N, C, K, H, W, FH, FW, stride,
+                                      pt, pb, pl, pr, flags, _stream(stream)), "small_conv_maxpool2d")
+
+
+def small_conv_maxpool_fused(N, C, K, H, W, FH, FW, stride, pad):
+    pt, pb, pl, pr = pad
+    return bool(lib().small_conv_maxpool_fused(N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr))
 
 
 def small_conv2d_uses_tensor_cores(N, C, K, H, W, FH, FW, stride, pad):

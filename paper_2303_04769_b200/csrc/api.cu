@@ -354,6 +354,36 @@ SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, cons
     }
 }
 
+// ---- fused convolution -> 2 x 2 stride-2 max pool
+SMALL_API int small_conv_maxpool_fused(int N, int C, int K, int H, int W, int FH, int FW, int stride, int pt, int pb, int pl, int pr) {
+    Geom g;
+    if (make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr) != SMALL_OK) return 0;
+    return conv_direct_pool_supported(g) ? 1 : 0;
+}
+
+SMALL_API int small_conv_maxpool2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, float *scratch,
+                                   int N, int C, int K, int H, int W, int FH, int FW, int stride,
+                                   int pt, int pb, int pl, int pr, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    if (!math_valid(math_of(flags))) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, w, out}, {bias, scratch})) return s;
+    Geom g;
+    if (int s = make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr)) return s;
+    if (g.OH < 2 || g.OW < 2) return SMALL_ERR_SHAPE;                  // the pool's output would be empty
+    const size_t in_b = sizeof(float) * packed_elems(N, C, H, W), out_b = sizeof(float) * packed_elems(N, K, g.OH / 2, g.OW / 2);
+    if (ranges_overlap(in, in_b, out, out_b)) return SMALL_ERR_OVERLAP;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // one kernel: the register-tiled FP32 kernel pools in its STORE phase (FP32 FMAs meet every math mode's tolerance)
+    if (conv_direct_pool_supported(g)) return launch_conv_direct_pool(ctx, in, w, bias, out, g, flags & SMALL_RELU, st);
+    // the two layers one after the other, through the caller's scratch tensor
+    if (!scratch) return SMALL_ERR_WORKSPACE;
+    const size_t mid_b = sizeof(float) * packed_elems(N, K, g.OH, g.OW);
+    if (ranges_overlap(scratch, mid_b, in, in_b) || ranges_overlap(scratch, mid_b, out, out_b)) return SMALL_ERR_OVERLAP;
+    if (int s = small_conv2d(ctx, in, w, bias, scratch, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr, flags, stream)) return s;
+    return small_pool2d(ctx, scratch, out, nullptr, N, K, g.OH, g.OW, 2, 2, 2, 0, 0, 0, 0, SMALL_POOL_MAX, stream);
+}
+
 SMALL_API int small_dwconv2d(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
                              int N, int C, int H, int W, int FH, int FW, int stride,
                              int pt, int pb, int pl, int pr, unsigned flags, void *stream) {

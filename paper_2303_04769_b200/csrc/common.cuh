@@ -108,6 +108,9 @@ int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *
 bool conv_direct_supported(const Geom &, int span = 0, int Kg = 0, int S_C = 0);
 int launch_conv_direct(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
                        bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
+// the same kernel with a 2 x 2 stride-2 max pool taken in its STORE phase: out is [N][K][OH/2][OW/2]
+bool conv_direct_pool_supported(const Geom &);
+int launch_conv_direct_pool(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
 // at most four input channels, 3 x 3 (strides 1, 2) or the 10 x 4 stride-2 window: FP32 FMAs with the filters in registers
 bool conv_thin_supported(const Geom &);
 int launch_conv_thin(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,

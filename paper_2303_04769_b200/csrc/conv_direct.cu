@@ -55,6 +55,7 @@ struct DirectArgs {
     uint32_t unit_bytes, in_box_bytes, w_bytes, w_box_bytes, stage_bytes;
     int span, Kg, S_C;          // group convolution: channel blocks a filter block reads, filters per group, channel step
     int relu, accumulate;
+    int pool;                   // fused 2 x 2 stride-2 max pool behind the layer (float form): out is [N][K][OH/2][OW/2]
 };
 
 __device__ __forceinline__ void lds128(uint32_t addr, uint32_t *v) {
@@ -220,12 +221,46 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
 
     // STORE phase.  Lanes of the last filter block beyond K stay zero: the thread holding the launch's last filter group
     // writes them.
-    if (!valid) return;
     const int kq0 = k0 + kw * kKQ;
     const int kb = kq0 >> 5, kl = kq0 & 31;
-    if (kb >= a.KB) return;
+    if (kb >= a.KB) return;                       // the same for a whole warp
     const int n = n0 + img, oh = oh0 + row;
     const bool last_group = kq0 + kKQ == a.k_tiles * a.KT;
+    if (!Q && a.pool) {
+        // Abstract fused layer (Section 6): the 2 x 2 stride-2 max pool behind the convolution is taken in the STORE
+        // phase.  A thread holds 8 adjacent columns of one row: column pairs are reduced in its registers; rows 2i and
+        // 2i + 1 sit in neighbouring lanes (a unit has an even number of rows per image), so the row pair is one
+        // shuffle; the even row's lane stores 4 pooled pixels.  All lanes take part in the shuffles.
+        const float *bias = static_cast<const float *>(a.bias);
+        float bv[kKQ];
+#pragma unroll
+        for (int k = 0; k < kKQ; ++k) bv[k] = (bias && kq0 + k < a.K) ? bias[kq0 + k] : 0.0f;
+        const int PH = a.OH >> 1, PW = a.OW >> 1;
+        const int prow = oh >> 1, pcol0 = (ow0 + g * kPW) >> 1;
+        const bool store_lane = valid && !(oh & 1) && prow < PH;
+        float *dst = static_cast<float *>(a.out) + ((((size_t)(valid ? n : 0) * a.KB + kb) * PH + (store_lane ? prow : 0)) * PW + pcol0) * 32 + kl;
+#pragma unroll
+        for (int pp = 0; pp < kPW / 2; ++pp) {
+            float m[kKQ];
+#pragma unroll
+            for (int k = 0; k < kKQ; ++k) {
+                float r0 = (float)acc[2 * pp][k] + bv[k], r1 = (float)acc[2 * pp + 1][k] + bv[k];
+                if (a.relu) { r0 = fmaxf(r0, 0.0f); r1 = fmaxf(r1, 0.0f); }
+                m[k] = fmaxf(r0, r1);
+                m[k] = fmaxf(m[k], __shfl_xor_sync(0xffffffffu, m[k], 1));
+                if (kq0 + k >= a.K) m[k] = 0.0f;
+            }
+            if (store_lane && pcol0 + pp < PW) {
+                float4 *d4 = reinterpret_cast<float4 *>(dst + pp * 32);
+                d4[0] = make_float4(m[0], m[1], m[2], m[3]);
+                d4[1] = make_float4(m[4], m[5], m[6], m[7]);
+                if (last_group)
+                    for (int z = kl + kKQ; z < 32; z += 4) *reinterpret_cast<float4 *>(dst + pp * 32 - kl + z) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        return;
+    }
+    if (!valid) return;
     if constexpr (Q) {
         // zero points, bias, one requantisation (round half up of the 64-bit product), clamp, 8 bytes per pixel and thread
         const int T = a.FH * FW;
@@ -313,7 +348,7 @@ size_t round1k(size_t b) { return (b + 1023) & ~(size_t)1023; }
 // Tile shapes.  The unit of a row warp follows from the plane's width; what is chosen is the number of channels per
 // stage (8 or 16) and of units per block: the smallest blocks (finest work granularity over the SMs) that still keep
 // 12 or more warps resident per SM within shared memory.
-DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem, bool quant = false) {
+DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem, bool quant = false, bool pool = false) {
     DirectPlan best{};
     best.ok = false;
     if ((g.FW != 1 && g.FW != 3) || (g.S != 1 && g.S != 2) || g.FH * g.FW > 256) return best;
@@ -327,6 +362,8 @@ DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem
     const int rows_u = 32 / a.gw;
     if (g.OH <= rows_u) { a.TH = g.OH; a.NI = rows_u / g.OH; a.bands = 1; if (a.NI > g.N) a.NI = g.N; }
     else { a.TH = rows_u; a.NI = 1; a.bands = ceil_div(g.OH, rows_u); }
+    if (pool && ((a.TH & 1) || g.OH < 2 || g.OW < 2 || quant || span > 0)) return best;   // row pairs must share a unit
+    a.pool = pool ? 1 : 0;
     const long long units = (long long)ceil_div(g.N, a.NI) * a.bands * a.tiles_w;
     if (units > 0x3fffffffLL) return best;
     a.units = (int)units;
@@ -444,6 +481,17 @@ int launch_conv_direct(small_ctx *ctx, const float *in, const float *w, const fl
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     DirectArgs &a = p.a;
     a.bias = bias; a.out = out; a.status = ctx->dev_status; a.relu = relu; a.accumulate = accumulate;
+    return launch_direct(ctx, p, g, in, w, false, st);
+}
+
+bool conv_direct_pool_supported(const Geom &g) { return plan_direct(g, 0, 0, 0, 227 * 1024, false, true).ok; }
+
+int launch_conv_direct_pool(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, const Geom &g,
+                            bool relu, cudaStream_t st) {
+    DirectPlan p = plan_direct(g, 0, 0, 0, ctx->max_smem_optin, false, true);
+    if (!p.ok) return SMALL_ERR_UNSUPPORTED;
+    DirectArgs &a = p.a;
+    a.bias = bias; a.out = out; a.status = ctx->dev_status; a.relu = relu; a.accumulate = 0;
     return launch_direct(ctx, p, g, in, w, false, st);
 }
 

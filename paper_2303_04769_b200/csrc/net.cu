@@ -36,6 +36,10 @@ static bool layer_out_shape(const small_layer &L, int N, int &oc, int &oh, int &
         case SMALL_OP_DWPW:
             if (L.K < 1 || make_geom(g, N, L.C, L.C, L.H, L.W, 3, 3, L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r)) return false;
             oc = L.K; oh = g.OH; ow = g.OW; return true;
+        case SMALL_OP_CONVPOOL:
+            if (make_geom(g, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r)) return false;
+            if (g.OH < 2 || g.OW < 2) return false;
+            oc = L.K; oh = g.OH / 2; ow = g.OW / 2; return true;
         default: return false;
     }
 }
@@ -96,7 +100,10 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
     // validate every layer before the first launch: weights present where needed, flags known
     for (int i = 0; i < n_layers; ++i) {
         const small_layer &L = layers[i];
-        bool weighted = L.op == SMALL_OP_CONV || L.op == SMALL_OP_DWCONV || L.op == SMALL_OP_FC || L.op == SMALL_OP_DWPW;
+        bool weighted = L.op == SMALL_OP_CONV || L.op == SMALL_OP_DWCONV || L.op == SMALL_OP_FC || L.op == SMALL_OP_DWPW || L.op == SMALL_OP_CONVPOOL;
+        if (L.op == SMALL_OP_CONVPOOL &&
+            !small_conv_maxpool_fused(N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r))
+            return SMALL_ERR_UNSUPPORTED;         // a network has no scratch tensor for the unfused form
         if (L.op == SMALL_OP_DWPW) {
             if (!L.w_blk2 || !aligned16(L.w_blk2) || (L.bias2 && !aligned16(L.bias2))) return SMALL_ERR_INVALID_ARG;
             if (!small_dwpw_fused(N, L.C, L.K, L.H, L.W, L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags & SMALL_MATH_MASK))
@@ -107,6 +114,7 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
         unsigned allowed = L.op == SMALL_OP_CONV ? (SMALL_RELU | SMALL_ACCUMULATE | SMALL_MATH_MASK)
                          : (L.op == SMALL_OP_DWCONV || L.op == SMALL_OP_FC) ? (SMALL_RELU | SMALL_MATH_MASK)
                          : L.op == SMALL_OP_DWPW ? (SMALL_RELU | SMALL_RELU_MID | SMALL_MATH_MASK)
+                         : L.op == SMALL_OP_CONVPOOL ? (SMALL_RELU | SMALL_MATH_MASK)
                          : L.op == SMALL_OP_ADD ? SMALL_RELU : 0u;
         if (L.flags & ~allowed) return SMALL_ERR_INVALID_ARG;
         if ((L.flags & SMALL_MATH_MASK) == SMALL_MATH_MASK) return SMALL_ERR_INVALID_ARG;
@@ -139,6 +147,10 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
                 break;
             case SMALL_OP_FC:
                 s = small_fc(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.flags, stream);
+                break;
+            case SMALL_OP_CONVPOOL:
+                s = small_conv_maxpool2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), nullptr, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
+                                         L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
                 break;
             case SMALL_OP_DWPW:
                 s = small_dwpw_conv2d(ctx, rd(L.src), L.w_blk, L.bias, L.w_blk2, L.bias2, wr(L.dst), nullptr, N, L.C, L.K, L.H, L.W,

@@ -41,7 +41,7 @@ FUSE_DWPW_MAX_BYTES = 24 << 20
 class Net:
     """A network resident on the device: packed filters, descriptors and workspace."""
 
-    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda", fuse_dwpw=True):
+    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda", fuse_dwpw=True, fuse_convpool=True):
         self.ctx = ctx
         self.N = net["batch"] if batch is None else batch
         self.in_shape = tuple(net["input"])
@@ -56,6 +56,7 @@ class Net:
             uses[L["src"]] = uses.get(L["src"], 0) + 1
         shape = {"in": self.in_shape}
         fused_at = set()
+        pool_at = set()           # convolutions whose 2x2 stride-2 max pool is taken in the convolution's STORE phase
         for li, L in enumerate(layers_in):
             c, h, wd = shape[L["src"]]
             fh, fw = (h, wd) if (L["op"] == "pool" and L["FH"] == 0) else (L["FH"], L["FW"])
@@ -70,11 +71,16 @@ class Net:
                     and (fuse_dwpw == "all" or 4 * B.small_packed_elems(self.N, L["C"], oh, ow) <= FUSE_DWPW_MAX_BYTES)
                     and B.small_dwpw_fused(self.N, L["C"], nxt["K"], h, wd, L["stride"], L["pad"], self.math)):
                 fused_at.add(li)
+            if (fuse_convpool and (li - 1) not in fused_at and (li - 1) not in pool_at and L["op"] == "conv" and not L.get("accumulate")
+                    and nxt is not None and nxt["op"] == "pool" and nxt["src"] == L["dst"] and uses.get(L["dst"], 0) == 1
+                    and nxt["pool"] == "max" and nxt["FH"] == 2 and nxt["FW"] == 2 and nxt["stride"] == 2 and tuple(nxt["pad"]) == (0, 0, 0, 0)
+                    and B.small_conv_maxpool_fused(self.N, L["C"], L["K"], h, wd, fh, fw, L["stride"], L["pad"])):
+                pool_at.add(li)
         eff = []
         for li, L in enumerate(layers_in):
-            if li - 1 in fused_at:
+            if li - 1 in fused_at or li - 1 in pool_at:
                 continue
-            eff.append(dict(L, dst=layers_in[li + 1]["dst"]) if li in fused_at else L)
+            eff.append(dict(L, dst=layers_in[li + 1]["dst"]) if (li in fused_at or li in pool_at) else L)
         slot_of, _ = assign_slots(eff)
         self.slot_of = slot_of
         dims = {"in": self.in_shape}
@@ -123,6 +129,24 @@ class Net:
                 dims[nxt["dst"]] = (nxt["K"], oh, ow)
                 self.layer_rows.append(dict(name=L["name"] + "+" + nxt["name"], op="dwpw", C=L["C"], K=nxt["K"], H=h, W=wd, FH=3, FW=3,
                                             stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=nxt["dst"], first=li, upto=li + 2))
+                descs.append(d)
+                skip = True
+                continue
+            if li in pool_at:
+                # convolution -> 2x2 stride-2 max pool as one fused layer
+                d.op = B.OP_CONVPOOL
+                d.dst = slot_of[nxt["dst"]]
+                flags |= self.math
+                wb = torch.empty(B.small_conv_weight_elems(L["C"], L["K"], fh, fw, B.MATH["fp32"]), device=device)
+                B.small_pack_conv_weights(ctx, wt, wb, L["C"], L["K"], fh, fw, B.MATH["fp32"])
+                d.flags = flags
+                d.w_blk = wb.data_ptr()
+                d.bias = None if bt is None else bt.data_ptr()
+                self.keep += [wb, bt, wt]
+                dims[L["dst"]] = (L["K"], oh, ow)
+                dims[nxt["dst"]] = (L["K"], oh // 2, ow // 2)
+                self.layer_rows.append(dict(name=L["name"] + "+" + nxt["name"], op="convpool", C=L["C"], K=L["K"], H=h, W=wd, FH=fh, FW=fw,
+                                            stride=L["stride"], pad=L["pad"], OH=oh // 2, OW=ow // 2, dst=nxt["dst"], first=li, upto=li + 2))
                 descs.append(d)
                 skip = True
                 continue
@@ -216,6 +240,8 @@ class Net:
         elif L.op == B.OP_DWPW:
             B.small_dwpw_conv2d(self.ctx, src, L.w_blk, L.bias, L.w_blk2, L.bias2, dst, None, N, L.C, L.K, L.H, L.W, L.stride, pad,
                                 L.flags, stream)
+        elif L.op == B.OP_CONVPOOL:
+            B.small_conv_maxpool2d(self.ctx, src, L.w_blk, L.bias, dst, None, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride, pad, L.flags, stream)
         else:
             raise ValueError(L.op)
 
