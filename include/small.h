@@ -101,6 +101,15 @@ int small_last_cuda_error(small_ctx *ctx);
  * until that layer has completed before they read or write a tensor.  Results are the same either way.  The paper
  * has no counterpart. */
 int small_set_layer_overlap(small_ctx *ctx, int on);
+/* Limit, in polls, of every bounded device-side wait (default 2^22: seconds, with the polls' back-off); at least 16.
+ * A wait that runs out makes its kernel record SMALL_ERR_TIMEOUT, let its copies in flight land, free its tensor memory
+ * and return; the affected outputs are undefined and later calls work normally.  The paper has no counterpart. */
+int small_set_wait_limit(small_ctx *ctx, unsigned polls);
+/* Runs the give-up-and-return path on purpose, harmlessly: one small kernel waits - with the context's limit and the wait
+ * routine of the layer kernels - on a barrier that nothing arms (no copy is in flight), records SMALL_ERR_TIMEOUT and
+ * returns.  Lower the limit first (a few hundred polls) or the call takes seconds.  small_device_status then reads
+ * SMALL_ERR_TIMEOUT once and the context works as before. */
+int small_selftest_wait_timeout(small_ctx *ctx, void *stream);
 /* Kernel family of the full channel reductions under the tensor-core math modes.  AUTO (the default): per layer,
  * whichever of the tensor-core kernel and the register-tiled FP32 kernel is the faster one for its channel counts
  * (FP32 FMAs meet every mode's tolerance); TENSOR / CUDA_CORES force one family wherever it takes the shape.  For

@@ -25,7 +25,7 @@ MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
 EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
-    "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_conv2d_path", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
+    "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_conv2d_path", "small_set_wait_limit", "small_selftest_wait_timeout", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_conv_maxpool2d", "small_conv_maxpool_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
@@ -76,6 +76,8 @@ def lib():
     L.small_set_layer_overlap.argtypes = [P, I]
     L.small_device_status.argtypes = [P, ctypes.POINTER(I), P]
     L.small_set_conv_path.argtypes = [P, I]
+    L.small_set_wait_limit.argtypes = [P, U]
+    L.small_selftest_wait_timeout.argtypes = [P, P]
     L.small_conv2d_path.argtypes = [P] + [I] * 12 + [U]
     L.small_pack.argtypes = [P, P, P, I, I, I, I, P]
     L.small_unpack.argtypes = [P, P, P, I, I, I, I, P]
@@ -189,6 +191,14 @@ CONV_KERNEL = {0: "conv_thin", 1: "conv_direct", 2: "conv_fp32", 3: "conv_tc"}
 
 def small_set_conv_path(ctx, path):
     _check(lib().small_set_conv_path(ctx, CONV_PATH[path] if isinstance(path, str) else path), "small_set_conv_path")
+
+
+def small_set_wait_limit(ctx, polls):
+    _check(lib().small_set_wait_limit(ctx, polls), "small_set_wait_limit")
+
+
+def small_selftest_wait_timeout(ctx, stream=None):
+    _check(lib().small_selftest_wait_timeout(ctx, _stream(stream)), "small_selftest_wait_timeout")
 
 
 def small_conv2d_path(ctx, N, C, K, H, W, FH, FW, stride, pad, math):

@@ -101,6 +101,7 @@ SMALL_API int small_init(int device, small_ctx **out) {
     }
     c->encode_tiled = fn;
     c->static_workspace = nullptr;
+    c->wait_iters = 1u << 22;     // with the polls' nanosleep back-off: seconds
     if (resolve_static_workspace(c) != SMALL_OK) {      // loads the library's device code here, not inside a later call
         cudaFree(block);
         delete c;
@@ -126,6 +127,13 @@ SMALL_API int small_last_cuda_error(small_ctx *ctx) { return ctx ? ctx->last_cud
 SMALL_API int small_set_layer_overlap(small_ctx *ctx, int on) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     ctx->overlap = on ? 1 : 0;
+    return SMALL_OK;
+}
+
+SMALL_API int small_set_wait_limit(small_ctx *ctx, unsigned polls) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (polls < 16u) return SMALL_ERR_INVALID_ARG;
+    ctx->wait_iters = polls;
     return SMALL_OK;
 }
 

@@ -19,6 +19,7 @@ struct small_ctx {
     size_t max_smem_optin;
     int overlap;             // small_run_net launches every layer after the first as a dependent launch (see launch_kernel)
     int dependent;           // set by small_run_net while it issues those layers
+    unsigned wait_iters;     // limit (polls) of every bounded device-side wait; small_set_wait_limit
     void *static_workspace;  // device address of the library's built-in workspace array on this device (net_static.cu)
     int conv_path;           // SMALL_CONV_PATH_*: automatic, or one kernel family forced where it takes the shape
 };

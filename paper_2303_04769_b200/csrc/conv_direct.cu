@@ -55,6 +55,7 @@ struct DirectArgs {
     uint32_t unit_bytes, in_box_bytes, w_bytes, w_box_bytes, stage_bytes;
     int span, Kg, S_C;          // group convolution: channel blocks a filter block reads, filters per group, channel step
     int relu, accumulate;
+    uint32_t wait_iters;        // limit of the bounded waits (polls)
     int pool;                   // fused 2 x 2 stride-2 max pool behind the layer (float form): out is [N][K][OH/2][OW/2]
 };
 
@@ -155,7 +156,7 @@ conv_direct_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_cons
             issue(q + a.stages - 1, sn);          // the stage read in the previous iteration, released by its __syncthreads
         }
         int ok = 1;
-        if (lane == 0) ok = sm100::mbar_wait(bar0 + 8 * s, phase) ? 1 : 0;
+        if (lane == 0) ok = sm100::mbar_wait(bar0 + 8 * s, phase, a.wait_iters) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) { failed = 1; atomicExch(a.status, (int)SMALL_ERR_TIMEOUT); }
         __syncwarp();
@@ -412,9 +413,7 @@ DirectPlan plan_direct(const Geom &g, int span, int Kg, int S_C, size_t max_smem
     return best;
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using sm100::EncodeTiledFn;
 
 }  // namespace
 
@@ -429,6 +428,7 @@ namespace {
 // words of 4 channel bytes [c4][ko] in the first 8 of the 32 rows' worth - see pack_q_conv_w_kernel).
 int launch_direct(small_ctx *ctx, DirectPlan &p, const Geom &g, const void *in, const void *w, bool quant, cudaStream_t st) {
     DirectArgs &a = p.a;
+    a.wait_iters = ctx->wait_iters;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     CUtensorMap map_in, map_w;
     {   // activations [N][CB][H][W][32]: box = one stage's channels x cols_box x th_in x 1 block x NI images, swizzled

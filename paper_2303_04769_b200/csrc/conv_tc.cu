@@ -41,10 +41,13 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace small {
 
 namespace {
+
+using namespace sm100;
 
 constexpr int kThreads = 256;            // roles of the TF32 kernel; the 3xTF32 kernel adds four splitting warps
 constexpr int kThreadsX3 = 384;
@@ -54,7 +57,6 @@ constexpr int kSlotPx = 256;           // pixels per slot = the MMA's largest N
 constexpr int kFilterTile = 128;       // filters per tile = the MMA's M
 constexpr int kMaxAStages = 6;         // input strips in flight (at least 2; as many as shared memory allows)
 constexpr int kMaxBStages = 8;
-constexpr uint32_t kWaitIters = 1u << 22;   // bounded wait: polls back off with nanosleep, so this is seconds
 constexpr int kRawStages = 2;           // fused depthwise: halo tiles in flight
 constexpr int kCtrlBarrierBytes = 24 * kMaxAStages + 16 * kMaxBStages + 16 * kSlots + 16 * kRawStages;   // all mbarriers
 constexpr int kTapTabEntries = 4 * 64;   // original tap of every (phase plane, view tap), -1 where the view tap has none
@@ -107,137 +109,8 @@ struct TcArgs {
     int x3_wide;               // 3xTF32, pixels on M: x_hi meets [w_hi; w_lo] in one MMA of twice the filters (see the issue loop)
     uint32_t x_lo_off;         // 3xTF32: 16-byte units from a strip's TF32 part to its residual
     int relu, accumulate;
+    uint32_t wait_iters;       // limit of every bounded wait (polls)
 };
-
-// ---------------------------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the limit ran out or another role already gave up (abort flag set).  After a few
-// immediate retries the poll backs off with nanosleep so that waiting roles leave shared-memory bandwidth to the
-// tensor core, which reads its operands from the same shared memory.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
-    for (uint32_t it = 0; it < kWaitIters; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it >= 4) __nanosleep(it < 64 ? 40 : 400);
-        if ((it & 63u) == 63u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicExch(status, (int)SMALL_ERR_TIMEOUT);
-    return false;
-}
-// One lane waits for the whole warp (all 32 lanes must call this together).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, FP32 accumulate, M = 128, N from the instruction descriptor, K = 8.
-// The two 64-bit shared-memory descriptors arrive as (low word, shared high word): only the low word changes between
-// MMAs, which keeps the single issuing thread's instruction count per MMA small.
-__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 da, {%1, %3};\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The mbarrier receives one arrival when every MMA issued so far by this thread has finished.
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows 128 bytes apart, groups of 8 rows 1024
-// bytes apart.  Low word: start address >> 4 (bits 0-13) and the leading byte offset (bits 16-29, unused with this
-// swizzle).  High word: stride byte offset 1024 >> 4 (bits 32-45), descriptor version 1 (bit 46), swizzle mode 2 =
-// 128 bytes (bits 61-63).  The tensor core, like TMA, takes the swizzle phase from the absolute shared-memory address
-// (bits 7-9 select the XOR applied to the 16-byte chunk index), so a start that is not on a 1024-byte boundary - every
-// shifted tap - reads the strip exactly as TMA wrote it and the base-offset field (bits 49-51) stays 0 (checked on
-// the device: a non-zero value permutes the chunks).  Advancing by n bytes adds n >> 4 to the low word.
-constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
-
-// Instruction descriptor: FP32 accumulator, TF32 A and B, both K-major, M = 128, N = n (a multiple of 16, <= 256).
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// 256-bit global accesses (32-byte aligned addresses).
-__device__ __forceinline__ void st_global_v8(float *p, const float *v) {
-    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
-}
-__device__ __forceinline__ void ld_global_v8(const float *p, float *v) {
-    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p) : "memory");
-}
-
-// Predicated global accesses as single instructions, so that the epilogue's unrolled loops stay free of branches.
-__device__ __forceinline__ void st_global_if(float *p, float v, uint32_t flag) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v), "r"(flag) : "memory");
-}
-__device__ __forceinline__ float ld_global_if(const float *p, uint32_t flag) {
-    float v = 0.0f;
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p ld.global.f32 %0, [%1];\n\t}" : "+f"(v) : "l"(p), "r"(flag) : "memory");
-    return v;
-}
 
 // ---------------------------------------------------------------------------------------------- kernel
 // One tile: `px` pixels starting at flattened index q0 of image n0 (nn == 1) or of the strip of images n0.. (nn > 1),
@@ -381,7 +254,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
                 const Tile tl = decode_tile(a, t);
                 for (int cb = 0; cb < a.CBr; ++cb) {
-                    if (wrapped) alive = mbar_wait(bar_raw_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                    if (wrapped) alive = mbar_wait(bar_raw_empty + 8 * s, phase ^ 1u, abort_flag, a.status, a.wait_iters);
                     if (!alive) break;
                     mbar_expect_tx(bar_raw_full + 8 * s, a.raw_box_bytes);
                     tma_load_5d(raw_base + s * a.raw_stage_bytes, &map_a, bar_raw_full + 8 * s, 0, -a.dw_pl, tl.row0 * a.dw_s - a.dw_pt, cb, tl.n0);
@@ -399,7 +272,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int p = 0; p < a.n_phase && alive; ++p) {
                 const int ph = (a.phase_bits >> (2 * p)) & 1, pw = (a.phase_bits >> (2 * p + 1)) & 1;
                 for (int cb = 0; cb < a.CBr; ++cb) {
-                    if (wrapped) alive = mbar_wait(bar_a_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                    if (wrapped) alive = mbar_wait(bar_a_empty + 8 * s, phase ^ 1u, abort_flag, a.status, a.wait_iters);
                     if (!alive) break;
                     mbar_expect_tx(bar_a_full + 8 * s, a.a_box_bytes);
                     tma_load_5d(a_base + s * a.a_stage_bytes, &map_a, bar_a_full + 8 * s, 0, c1 + pw, c2 + ph, cb + tl.n_tile * a.cb_group, tl.n0);
@@ -438,7 +311,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int tap = 0; tap < T; ++tap) {
                             const int orig = tap_tab[p * T + tap];
                             if (orig < 0) continue;
-                            if (wrapped) alive = mbar_wait(bar_b_empty + 8 * s, phase ^ 1u, abort_flag, a.status);
+                            if (wrapped) alive = mbar_wait(bar_b_empty + 8 * s, phase ^ 1u, abort_flag, a.status, a.wait_iters);
                             if (!alive) break;
                             mbar_expect_tx(bar_b_full + 8 * s, X3 ? 2u * box_bytes : box_bytes);
                             tma_load_4d(b_base + s * kBStageBytes, &map_b, bar_b_full + 8 * s, 0, row, orig, cb);
@@ -467,7 +340,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t xo[CH];
 #pragma unroll
         for (int c = 0; c < CH; ++c) xo[c] = (uint32_t)(c * (PM ? 128 : a.n_slot)) * 8u;
-        if (a.b_resident) alive = mbar_wait(bar_b_full, 0, abort_flag, a.status);
+        if (a.b_resident) alive = mbar_wait(bar_b_full, 0, abort_flag, a.status, a.wait_iters);
 
         // all taps of one channel block with KS K-steps each; straight-line MMA issue
         // bit t set: view tap t of the phase plane exists (all of them for stride 1); kept in a register so that the
@@ -494,7 +367,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (a.b_resident) {
                     w_lo = w_res; w_res += b_step;
                 } else {
-                    alive = mbar_wait(bar_b_full + 8 * sb, pb, abort_flag, a.status);
+                    alive = mbar_wait(bar_b_full + 8 * sb, pb, abort_flag, a.status, a.wait_iters);
                     if (!alive) return;
                     w_lo = smem_desc_lo(b_base + sb * kBStageBytes);
                 }
@@ -542,7 +415,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // the previous content of the slots this tile takes must have left tensor memory
             for (int j = 0; j < a.slots && alive; ++j) {
                 const uint32_t u = slot_uses + j;
-                if (u >= kSlots) alive = mbar_wait(bar_slot_free + 8 * (u % kSlots), (u / kSlots - 1) & 1, abort_flag, a.status);
+                if (u >= kSlots) alive = mbar_wait(bar_slot_free + 8 * (u % kSlots), (u / kSlots - 1) & 1, abort_flag, a.status, a.wait_iters);
             }
             if (!alive) break;
             tc_fence_after();
@@ -560,7 +433,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int cb = 0, plane = 0;
             unsigned long long taps = mask0;
             for (int blk = 0; blk < a.CB && alive; ++blk) {       // blocks = phase planes x real channel blocks
-                alive = mbar_wait(((X3 || DW) ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status);   // once split / computed
+                alive = mbar_wait(((X3 || DW) ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status, a.wait_iters);   // once split / computed
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
                 if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, r_sel, started, w_res);
@@ -586,8 +459,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int px_img = a.dw_rows * a.OW;                     // strip pixels per image (row pitch = OW: a 1x1 view)
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x)
             for (int cb = 0; cb < a.CBr; ++cb) {
-                alive = mbar_wait_warp(bar_raw_full + 8 * r, pr, abort_flag, a.status);
-                if (alive && wrapped) alive = mbar_wait_warp(bar_a_empty + 8 * s, ps ^ 1u, abort_flag, a.status);
+                alive = mbar_wait_warp(bar_raw_full + 8 * r, pr, abort_flag, a.status, a.wait_iters);
+                if (alive && wrapped) alive = mbar_wait_warp(bar_a_empty + 8 * s, ps ^ 1u, abort_flag, a.status, a.wait_iters);
                 if (!alive) break;
                 const float4 *raw = reinterpret_cast<const float4 *>(base_ptr + (raw_base - base) + (size_t)r * a.raw_stage_bytes);
                 float4 *hi = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes);
@@ -661,7 +534,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int n4 = (a.strip_px + a.tail_px) * 8;          // 16-byte vectors of the strip and its zero tail
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x)
             for (int blk = 0; blk < a.CB; ++blk) {
-                alive = mbar_wait_warp(bar_a_full + 8 * s, phase, abort_flag, a.status);
+                alive = mbar_wait_warp(bar_a_full + 8 * s, phase, abort_flag, a.status, a.wait_iters);
                 if (!alive) break;
                 uint4 *hi = reinterpret_cast<uint4 *>(base_ptr + (size_t)s * a.a_stage_bytes);
                 float4 *lo = reinterpret_cast<float4 *>(base_ptr + (size_t)s * a.a_stage_bytes + a.a_half);
@@ -716,7 +589,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool lane_real = k < a.K;
             for (int j = 0; j < tl.slots && alive; ++j) {
                 const uint32_t u = slot_uses + j, s = u % kSlots;
-                alive = mbar_wait_warp(bar_slot_full + 8 * s, (u / kSlots) & 1, abort_flag, a.status);
+                alive = mbar_wait_warp(bar_slot_full + 8 * s, (u / kSlots) & 1, abort_flag, a.status, a.wait_iters);
                 if (!alive) break;
                 tc_fence_after();
                 const int px_here = min(tl.n_slot, tl.px - j * tl.n_slot);      // real pixels in this slot
@@ -823,7 +696,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (*abort_flag && armed_mask) {   // a role gave up: let the copies that are still in flight land before the CTA exits
         for (int st = 0; st < 32; ++st)
             if (armed_mask >> st & 1u)
-                for (uint32_t it = 0; it < kWaitIters && !mbar_try_wait(drain_bar + 8 * st, armed_parity >> st & 1u); ++it) __nanosleep(200);
+                for (uint32_t it = 0; it < a.wait_iters && !mbar_try_wait(drain_bar + 8 * st, armed_parity >> st & 1u); ++it) __nanosleep(200);
     }
     __syncthreads();
     if (warp == 1) {
@@ -1068,10 +941,6 @@ TcKernel pick_kernel(int chains, int ks, bool pixel_m, bool masked, bool x3, boo
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 }  // namespace
 
 // A 1x1 window without padding never looks at a neighbour, so the plane may be viewed with any row length that
@@ -1222,7 +1091,7 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
         chains = a.slots;
     }
     const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
-    a.relu = relu; a.accumulate = accumulate;
+    a.relu = relu; a.accumulate = accumulate; a.wait_iters = ctx->wait_iters;
     const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3, dw != nullptr);
     if (!kern) return SMALL_ERR_UNSUPPORTED;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);

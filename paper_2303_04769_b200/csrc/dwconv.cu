@@ -71,6 +71,7 @@ struct Dw3Args {
     int segs, rps;                         // a column's TR rows are walked by `segs` threads, `rps` rows each
     long long tiles;
     uint32_t stage_bytes;
+    uint32_t wait_iters;                   // limit of the bounded waits (polls)
     bool relu;
 };
 
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(256) dwconv3x3_tma_kernel(const __grid_constan
         const int s = it & 1;
         // one lane per warp polls, the rest wait at the shuffle
         int ok = 1;
-        if ((threadIdx.x & 31) == 0) ok = sm100::mbar_wait(bar0 + 8 * s, (it >> 1) & 1) ? 1 : 0;
+        if ((threadIdx.x & 31) == 0) ok = sm100::mbar_wait(bar0 + 8 * s, (it >> 1) & 1, a.wait_iters) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) { failed = 1; atomicExch(a.status, (int)SMALL_ERR_TIMEOUT); }
         const int strip = (int)(t % a.strips);
@@ -228,7 +229,7 @@ int launch_dwconv(small_ctx *ctx, const float *in, const float *w, const float *
     DwArgs a{in, w, bias, out, g.H, g.W, g.FH, g.FW, g.S, g.pt, g.pl, g.OH, g.OW, g.C, g.CB, (long long)g.N * g.CB, relu};
     Dw3Args t{};
     if (g.FH == 3 && g.FW == 3 && (g.S == 1 || g.S == 2) && plan_dw3(g, ctx->sm_count, t)) {
-        t.w = w; t.bias = bias; t.out = out; t.status = ctx->dev_status;
+        t.w = w; t.bias = bias; t.out = out; t.status = ctx->dev_status; t.wait_iters = ctx->wait_iters;
         t.N = g.N; t.C = g.C; t.CB = g.CB; t.OH = g.OH; t.OW = g.OW; t.pt = g.pt; t.pl = g.pl; t.relu = relu;
         CUtensorMap map;
         CUresult r = sm100::encode_blocked_map(ctx->encode_tiled, &map, in, g.N, g.CB, g.H, g.W, t.Wb, t.Hb, t.nn);

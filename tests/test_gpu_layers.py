@@ -389,3 +389,31 @@ def test_upsample_nearest_bit_exact(shape, f):
     assert pad_lanes_are_zero(out, N, C, H * f, W * f)
     with pytest.raises(B.SmallError):
         B.small_upsample_nearest(ctx(), to_blk(x), out, N, C, H, W, 0)
+
+
+def test_bounded_wait_runs_out_records_timeout_and_the_context_stays_usable():
+    """The give-up-and-return path of the device-side waits: with the limit lowered to a few hundred polls, a kernel that
+    waits on a barrier nothing arms returns by itself, the status word reads SMALL_ERR_TIMEOUT once, and ordinary calls
+    (tensor-core, TMA-fed CUDA-core and depthwise kernels, which use the same wait routine and limit) work as before."""
+    c = ctx()
+    assert B.small_device_status(c) == 0
+    try:
+        B.small_set_wait_limit(c, 300)
+        B.small_selftest_wait_timeout(c)
+        torch.cuda.synchronize()                       # the kernel returned: nothing hangs, nothing traps
+        assert B.small_device_status(c) == 8           # SMALL_ERR_TIMEOUT
+        assert B.small_device_status(c) == 0           # read once, then clear
+    finally:
+        B.small_set_wait_limit(c, 1 << 22)
+    with pytest.raises(B.SmallError):
+        B.small_set_wait_limit(c, 3)
+    N, C, K, H, W = 2, 64, 64, 14, 14
+    x, w, b = rnd((N, C, H, W), 81), rnd((K, C, 3, 3), 82), rnd((K,), 83)
+    wb = torch.empty(B.small_conv_weight_elems(C, K, 3, 3, B.MATH_3XTF32), device="cuda")
+    B.small_pack_conv_weights(c, dev(w), wb, C, K, 3, 3, B.MATH_3XTF32)
+    ref = oracle.conv2d(x, w, b, 1, (1, 1, 1, 1), relu=True)
+    for math, tol in (("fp32", 1e-5), ("tf32", 2e-3), ("3xtf32", 1e-5)):
+        out = new_blk(N, K, H, W)
+        B.small_conv2d(c, to_blk(x), wb, dev(b), out, N, C, K, H, W, 3, 3, 1, (1, 1, 1, 1), B.RELU | B.MATH[math])
+        assert rel_err(from_blk(out, N, K, H, W), ref) <= tol
+    assert B.small_device_status(c) == 0
