@@ -444,7 +444,7 @@ def gpu_main(args):
                 with torch.cuda.graph(wg):
                     wn.run(wblk)
                 wms = timed(lambda i: wg.replay(), min(args.steps, 100), 5)
-                res[m] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms, "launches": len(wn.layer_rows)}
+                res[m] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms, "launches": wn.launches()}
                 del wg, wn
                 if m != "fp32":     # the same network with every depthwise and 1x1 layer launched on its own
                     wn = Net(ctx, wnet, wparams, math=m, device=dev, fuse_dwpw=False)
@@ -454,7 +454,7 @@ def gpu_main(args):
                     with torch.cuda.graph(wg):
                         wn.run(wblk)
                     wms = timed(lambda i: wg.replay(), min(args.steps, 100), 5)
-                    res[m + "_unfused"] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms, "launches": len(wn.layer_rows)}
+                    res[m + "_unfused"] = {"value": wN / (wms * 1e-3), "unit": UNIT, "ms_per_step": wms, "launches": wn.launches()}
                     del wg, wn
             other_workloads[wname] = {"batch": wN, "layers": len(wnet["layers"]), "modes": res}
             del wx, wblk
@@ -467,8 +467,20 @@ def gpu_main(args):
             tf, cpm = B.small_measure_tf32_peak(ctx, n, 4096)
             probe[f"n{n}"] = {"tflops": round(tf, 1), "cycles_per_mma": round(cpm, 1)}
 
-    sweep = None if (args.no_sweep or world > 1) else run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch)
+    sweep = None if (args.no_sweep or world > 1) else run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch, probe["n256"]["tflops"] if probe else None)
 
+    if sweep:
+        # the sweep's targets in the retained part of the line: per layer kind and mode the smallest fraction of roofline
+        mins, mins_probe = {}, {}
+        for r in sweep["rows"]:
+            if "frac" not in r or r["layer"].startswith("groupconv") or "fused" in r["layer"]:
+                continue
+            key = r["layer"] if r["layer"] in ("dw3x3", "maxpool2x2", "relu") else f'{r["layer"]}_{r["mode"]}'
+            mins[key] = min(mins.get(key, 9.9), r["frac"])
+            if "frac_vs_measured_tf32" in r:
+                mins_probe[key] = min(mins_probe.get(key, 9.9), r["frac_vs_measured_tf32"])
+        roofline["sweep_min_frac"] = mins
+        roofline["sweep_min_frac_vs_measured_tf32"] = mins_probe
     cpu = None
     if world == 1 and not args.no_cpu:
         ips, n_used, dt, cores, passes = time_oracle_net(N)
@@ -490,7 +502,7 @@ def gpu_main(args):
                        "layer_overlap": not args.no_overlap},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * N * c * h * w, "d2h_bytes_per_step": 4 * N * oc * oh * ow,
                     "ms_per_step": ms_e2e},
-            "gpu_launches": len(gnet.layer_rows) * args.steps,
+            "gpu_launches": gnet.launches() * args.steps,
             "clocks": clocks, "roofline": roofline, "other_math_modes": other_modes, "tf32_issue_probe": probe, "other_workloads": other_workloads, "cpu_baseline": cpu, "device_status": status,
             "kernels": {k: {"launches_per_step": v["launches"], "ms": round(v["ms"], 4),
                             "share": round(v["ms"] / sum(x["ms"] for x in by_kernel.values()), 3)} for k, v in by_kernel.items()},
@@ -502,7 +514,7 @@ def gpu_main(args):
     B.small_shutdown(ctx)
 
 
-def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
+def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch, tf32_probe_tflops=None):
     """GPU-scale layer sweep, batch 128: each layer timed alone over rotating buffer sets that together exceed L2;
     GFLOP/s, GB/s and the fraction of the layer's roofline = max(FLOPs / peak of its math mode, bytes / HBM)."""
     import synth
@@ -510,7 +522,8 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
     rows = []
     for C, HW in configs.SWEEP_SIZES:
         elems = B.small_packed_elems(N, C, HW, HW)
-        sets = max(2, min(6, int((1 << 30) // (8 * elems)) or 2))   # in + out per set, about 1 GB in total
+        sets = max(2, min(48, -(-(1 << 30) // (8 * elems))))         # in + out per set: 1 GiB or more in rotation at every size
+        INNER = max(10, sets)                                        # launches per timed graph: every set once or more
         host = synth.uniform((N, C, HW, HW), -1.0, 1.0, 500 + C)
         nchw = torch.from_numpy(host).to(dev)
         ins, outs = [], []
@@ -524,14 +537,32 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
         state = {"i": 0}
 
         def rot():
+            if state.get("warm"):                # the L2-warm figure: the same buffers in every launch
+                return ins[0], outs[0]
             state["i"] = (state["i"] + 1) % sets
             return ins[state["i"]], outs[state["i"]]
 
-        def record(kind, mode, fl, by, tmin, tmed, bound_mode):
-            t_roof = max(fl / (mode_peak_tflops(bound_mode, peaks, sm_count) * 1e12) if fl and bound_mode else 0.0, by / (peaks["hbm_gbs"] * 1e9))
-            rows.append({"layer": kind, "C": C, "HW": HW, "mode": mode, "us_min": round(tmin * 1e3, 2), "us_med": round(tmed * 1e3, 2),
-                         "gflops": round(fl / tmed / 1e6, 1), "gbs": round(by / tmed / 1e6, 1),
-                         "roofline_us": round(t_roof * 1e6, 2), "frac": round(t_roof / (tmed * 1e-3), 4)})
+        def warm_us(fn, inner=10):
+            """The same launch on one fixed buffer set (its tensors may stay in the 126 MB L2): reported apart, labelled."""
+            state["warm"] = True
+            try:
+                return round(time_launch(fn, reps=10, warm=2, inner=inner)[1] * 1e3, 2)
+            finally:
+                state["warm"] = False
+
+        def record(kind, mode, fl, by, tmin, tmed, bound_mode, us_warm=None):
+            t_hbm = by / (peaks["hbm_gbs"] * 1e9)
+            t_roof = max(fl / (mode_peak_tflops(bound_mode, peaks, sm_count) * 1e12) if fl and bound_mode else 0.0, t_hbm)
+            row = {"layer": kind, "C": C, "HW": HW, "mode": mode, "us_min": round(tmin * 1e3, 2), "us_med": round(tmed * 1e3, 2),
+                   "gflops": round(fl / tmed / 1e6, 1), "gbs": round(by / tmed / 1e6, 1),
+                   "roofline_us": round(t_roof * 1e6, 2), "frac": round(t_roof / (tmed * 1e-3), 4)}
+            if bound_mode in ("tf32", "3xtf32") and tf32_probe_tflops:
+                # the same fraction against the library's own measured TF32 issue rate (a third of it for 3xTF32)
+                pk = tf32_probe_tflops / (3.0 if bound_mode == "3xtf32" else 1.0)
+                row["frac_vs_measured_tf32"] = round(max(fl / (pk * 1e12), t_hbm) / (tmed * 1e-3), 4)
+            if us_warm is not None:
+                row["us_l2_warm"] = us_warm
+            rows.append(row)
 
         for F, pad, kind in ((3, (1, 1, 1, 1), "conv3x3"), (1, (0, 0, 0, 0), "conv1x1")):
             w = torch.from_numpy(synth.uniform((C, C, F, F), -1.0, 1.0, 700 + C + F)).to(dev)
@@ -546,8 +577,8 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
                     a, o = rot()
                     B.small_conv2d(ctx, a, wb, bias, o, N, C, C, HW, HW, F, F, 1, pad, B.RELU | B.MATH[mode])
                 slow = mode == "fp32" and F == 3
-                tmin, tmed = time_launch(call, reps=5 if slow else 20, warm=2, inner=1 if slow else 10)
-                record(kind, mode, fl, by, tmin, tmed, mode)
+                tmin, tmed = time_launch(call, reps=5 if slow else 20, warm=2, inner=2 if slow else INNER)
+                record(kind, mode, fl, by, tmin, tmed, mode, None if slow else warm_us(call))
             del w, wb
         # group convolution, groups of 32 channels with 32 filters each (G = C / 32): block-diagonal filters on the FP32 kernel,
         # one filter tile per group on the tensor-core kernel
@@ -560,7 +591,7 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
             def gc(mode=mode):
                 a, o = rot()
                 B.small_group_conv2d(ctx, a, wgb, bias, o, N, C, 32, 32, 32, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU | B.MATH[mode])
-            tmin, tmed = time_launch(gc, reps=10, warm=2, inner=4 if mode == "fp32" else 10)
+            tmin, tmed = time_launch(gc, reps=10, warm=2, inner=4 if mode == "fp32" else INNER)
             record(f"groupconv3x3_g{G}", mode, 2.0 * N * HW * HW * C * 32 * 9, 4.0 * (2 * N * C * HW * HW + C * 32 * 9 + C), tmin, tmed, mode)
         del wg, wgb
         wdw = torch.from_numpy(synth.uniform((C, 3, 3), -1.0, 1.0, 800 + C)).to(dev)
@@ -576,31 +607,51 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch):
             def fz(mode=mode):
                 a, o = rot()
                 B.small_dwpw_conv2d(ctx, a, wdb, bias, wpb, bias, o, None, N, C, C, HW, HW, 1, (1, 1, 1, 1), B.RELU | B.RELU_MID | B.MATH[mode])
-            tmin, tmed = time_launch(fz, inner=10)
+            tmin, tmed = time_launch(fz, inner=INNER)
             record("dw3x3+conv1x1_fused", mode, 2.0 * N * HW * HW * C * (9 + C), 4.0 * (2 * N * C * HW * HW + C * C + 12 * C), tmin, tmed, mode)
         del wpw, wpb
 
         def dw():
             a, o = rot()
             B.small_dwconv2d(ctx, a, wdb, bias, o, N, C, HW, HW, 3, 3, 1, (1, 1, 1, 1), B.RELU)
-        tmin, tmed = time_launch(dw, inner=10)
-        record("dw3x3", "fp32", 2.0 * N * HW * HW * C * 9, 4.0 * (2 * N * C * HW * HW + 10 * C), tmin, tmed, None)
+        tmin, tmed = time_launch(dw, inner=INNER)
+        record("dw3x3", "fp32", 2.0 * N * HW * HW * C * 9, 4.0 * (2 * N * C * HW * HW + 10 * C), tmin, tmed, None, warm_us(dw))
         OHW = (HW - 2) // 2 + 1
 
         def mp():
             a, o = rot()
             B.small_pool2d(ctx, a, o, None, N, C, HW, HW, 2, 2, 2, (0, 0, 0, 0), B.POOL_MAX)
-        tmin, tmed = time_launch(mp, inner=10)
-        record("maxpool2x2", "fp32", 0.0, 4.0 * N * C * (HW * HW + OHW * OHW), tmin, tmed, None)
+        tmin, tmed = time_launch(mp, inner=INNER)
+        record("maxpool2x2", "fp32", 0.0, 4.0 * N * C * (HW * HW + OHW * OHW), tmin, tmed, None, warm_us(mp))
 
         def rl():
             a, o = rot()
             B.small_relu(ctx, a, o, N, C, HW, HW)
-        tmin, tmed = time_launch(rl, inner=10)
-        record("relu", "fp32", 0.0, 8.0 * N * C * HW * HW, tmin, tmed, None)
+        tmin, tmed = time_launch(rl, inner=INNER)
+        record("relu", "fp32", 0.0, 8.0 * N * C * HW * HW, tmin, tmed, None, warm_us(rl))
+        # the quantised form of the two convolutions (uint8 tensors, int32 accumulation): operations per second and bytes
+        qin = [torch.randint(0, 256, (elems,), dtype=torch.uint8, device=dev) for _ in range(min(sets, 8))]
+        qout = [torch.empty(elems, dtype=torch.uint8, device=dev) for _ in range(min(sets, 8))]
+        for F, pad, kind in ((3, (1, 1, 1, 1), "qconv3x3"), (1, (0, 0, 0, 0), "qconv1x1")):
+            qw = torch.randint(0, 256, (C, C, F, F), dtype=torch.uint8, device=dev)
+            qwb = torch.empty(B.small_q_conv_weight_bytes(C, C, F, F), dtype=torch.uint8, device=dev)
+            B.small_q_pack_conv_weights(ctx, qw, qwb, C, C, F, F)
+            qs = {"i": 0}
+
+            def qc(F=F, pad=pad):
+                qs["i"] = (qs["i"] + 1) % len(qin)
+                B.small_q_conv2d(ctx, qin[qs["i"]], qwb, None, qout[qs["i"]], N, C, C, HW, HW, F, F, 1, pad, (128, 128, 128, 1 << 20, 40), B.RELU)
+            tmin, tmed = time_launch(qc, reps=5, warm=2, inner=4)
+            ops, qby = 2.0 * N * HW * HW * C * C * F * F, 1.0 * (2 * N * C * HW * HW + C * C * F * F) + 4.0 * C
+            rows.append({"layer": kind, "C": C, "HW": HW, "mode": "uint8", "us_min": round(tmin * 1e3, 2), "us_med": round(tmed * 1e3, 2),
+                         "gops": round(ops / tmed / 1e6, 1), "gbs": round(qby / tmed / 1e6, 1)})
+            del qw, qwb
+        del qin, qout
         del ins, outs
         torch.cuda.empty_cache()
-    return {"batch": N, "buffers": "rotating input/output sets of about 1 GB per size (larger than L2)", "rows": rows}
+    return {"batch": N, "buffers": "every launch of a timed graph reads and writes its own input/output set, 1 GiB or more in rotation at "
+                                   "every size (L2 is 126 MB); us_l2_warm: the same launch on one fixed set, for comparison only",
+            "rows": rows}
 
 
 def single_layer(args):

@@ -160,9 +160,9 @@ int small_pack_group_conv_weights(small_ctx *ctx, const float *w_gkcrs, float *w
 size_t small_dw_weight_elems(int C, int FH, int FW);
 /* w_crs: device float[C][FH][FW] (one filter per channel: Table 1, single channel reduction). */
 int small_pack_dw_weights(small_ctx *ctx, const float *w_crs, float *w_blk, int C, int FH, int FW, void *stream);
-size_t small_fc_weight_elems(int J, int K);
+size_t small_fc_weight_elems(int J, int K, unsigned math);
 /* w_kj: device float[K][J]. */
-int small_pack_fc_weights(small_ctx *ctx, const float *w_kj, float *w_blk, int J, int K, void *stream);
+int small_pack_fc_weights(small_ctx *ctx, const float *w_kj, float *w_blk, int J, int K, unsigned math, void *stream);
 
 /* ---- layers -------------------------------------------------------------------------------- */
 
@@ -263,7 +263,9 @@ int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N,
 /* Full reduction (Section 3.2 item 5; Table 1 row 5): out[n,k] = bias[k] + sum_j in[n,j] * w[k,j].
  * in: blocked [N][J][1][1]; out: blocked [N][K][1][1].  (A full reduction over an H x W plane is
  * small_conv2d with FH = H, FW = W, as long as that window fits the kernel's shared-memory tile.)
- * flags: SMALL_RELU (a math mode is accepted and ignored). */
+ * flags: SMALL_RELU | one SMALL_MATH_*.  Under a tensor-core math mode (with filters packed for it) a layer of 4 MFLOP
+ * or more runs on the tensor-core kernel as a 1x1 convolution whose pixels are the images; smaller ones (classifier
+ * heads) and SMALL_MATH_FP32 run FP32 FMAs on the CUDA cores. */
 int small_fc(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
              int N, int J, int K, unsigned flags, void *stream);
 
@@ -306,6 +308,9 @@ int small_q_maxpool2d(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, in
 /* ReLU on uint8 (Table 2: Max with zero): out = max(in, z), real zero being the zero point z.  out may equal in. */
 int small_q_relu(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, int C, int H, int W, int z, void *stream);
 
+/* 1 if small_fc runs this layer on the tensor cores under the given math mode, else 0. */
+int small_fc_uses_tensor_cores(int N, int J, int K, unsigned math);
+
 /* ---- networks (Section 5.3: layers share intermediate buffers; Section 5.4: end-to-end inference) -- */
 
 enum { SMALL_OP_CONV = 0, SMALL_OP_DWCONV = 1, SMALL_OP_POOL = 2, SMALL_OP_RELU = 3, SMALL_OP_ADD = 4, SMALL_OP_FC = 5,
@@ -331,6 +336,19 @@ typedef struct small_layer {
     const float *bias2;     /* DWPW: bias of the 1x1 convolution or NULL */
 } small_layer;
 
+/* Abstract fused layers (Section 6) inside small_run_net.  The caller describes plain layers; the runner itself runs
+ * two neighbouring layers as one fused layer when the first one's result is read by the second one only (no later layer
+ * reads that slot before it is written again), the pair's output slot differs from its input slot, and the fused kernel
+ * takes the shape: a depthwise 3x3 and the 1x1 convolution behind it under a tensor-core math mode (SMALL_FUSE_DWPW: only
+ * where the intermediate tensor is at most 24 MB, where fusing was measured to pay; SMALL_FUSE_DWPW_ALWAYS: wherever the
+ * kernel takes the shape), and a convolution and the 2x2 stride-2 max pool behind it (SMALL_FUSE_CONVPOOL).  The skipped
+ * intermediate tensor is then not written.  Default: SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL; 0 runs every layer on its own.
+ * Results stay within each math mode's tolerance either way. */
+enum { SMALL_FUSE_DWPW = 1u, SMALL_FUSE_DWPW_ALWAYS = 2u, SMALL_FUSE_CONVPOOL = 4u };
+int small_set_net_fusion(small_ctx *ctx, unsigned mask);
+/* Number of kernel launches small_run_net makes for these layers at batch N under the context's fusion setting (one per
+ * layer or fused pair); -1 for invalid arguments. */
+int small_net_launches(small_ctx *ctx, const small_layer *layers, int n_layers, int N);
 /* Bytes of workspace for `layers` at batch N: slot s is as large as the largest tensor any layer reads
  * from or writes to it, rounded up to 256 bytes; slots are laid out back to back.  0 on invalid input. */
 size_t small_net_workspace_bytes(const small_layer *layers, int n_layers, int N);

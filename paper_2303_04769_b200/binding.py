@@ -28,8 +28,8 @@ EXPORTS = [
     "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_conv2d_path", "small_set_wait_limit", "small_selftest_wait_timeout", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_conv_maxpool2d", "small_conv_maxpool_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
-    "small_pack_fc_weights", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
-    "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net",
+    "small_pack_fc_weights", "small_fc_uses_tensor_cores", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
+    "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net", "small_set_net_fusion", "small_net_launches",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
     "small_q_packed_bytes", "small_q_pack", "small_q_unpack", "small_q_conv_weight_bytes", "small_q_pack_conv_weights", "small_q_conv2d",
     "small_q_dw_weight_bytes", "small_q_pack_dw_weights", "small_q_dwconv2d", "small_q_maxpool2d", "small_q_relu",
@@ -96,9 +96,10 @@ def lib():
     L.small_dw_weight_elems.argtypes = [I, I, I]
     L.small_dw_weight_elems.restype = Z
     L.small_pack_dw_weights.argtypes = [P, P, P, I, I, I, P]
-    L.small_fc_weight_elems.argtypes = [I, I]
+    L.small_fc_weight_elems.argtypes = [I, I, U]
     L.small_fc_weight_elems.restype = Z
-    L.small_pack_fc_weights.argtypes = [P, P, P, I, I, P]
+    L.small_pack_fc_weights.argtypes = [P, P, P, I, I, U, P]
+    L.small_fc_uses_tensor_cores.argtypes = [I, I, I, U]
     L.small_conv2d.argtypes = [P, P, P, P, P] + [I] * 12 + [U, P]
     L.small_conv2d_uses_tensor_cores.argtypes = [I] * 12
     L.small_dwconv2d.argtypes = [P, P, P, P, P] + [I] * 11 + [U, P]
@@ -111,6 +112,8 @@ def lib():
     L.small_net_workspace_bytes.argtypes = [ctypes.POINTER(small_layer), I, I]
     L.small_net_workspace_bytes.restype = Z
     L.small_run_net.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, P, P, Z, P]
+    L.small_set_net_fusion.argtypes = [P, U]
+    L.small_net_launches.argtypes = [P, ctypes.POINTER(small_layer), I, I]
     L.small_net_host_staging_bytes.argtypes = [I] * 7
     L.small_net_host_staging_bytes.restype = Z
     L.small_run_net_host.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, I, I, I, P, I, I, I, P, Z, P]
@@ -236,12 +239,16 @@ def small_pack_dw_weights(ctx, w_crs, w_blk, C, FH, FW, stream=None):
     _check(lib().small_pack_dw_weights(ctx, _ptr(w_crs), _ptr(w_blk), C, FH, FW, _stream(stream)), "small_pack_dw_weights")
 
 
-def small_fc_weight_elems(J, K):
-    return lib().small_fc_weight_elems(J, K)
+def small_fc_weight_elems(J, K, math=MATH_FP32):
+    return lib().small_fc_weight_elems(J, K, math)
 
 
-def small_pack_fc_weights(ctx, w_kj, w_blk, J, K, stream=None):
-    _check(lib().small_pack_fc_weights(ctx, _ptr(w_kj), _ptr(w_blk), J, K, _stream(stream)), "small_pack_fc_weights")
+def small_fc_uses_tensor_cores(N, J, K, math):
+    return bool(lib().small_fc_uses_tensor_cores(N, J, K, math))
+
+
+def small_pack_fc_weights(ctx, w_kj, w_blk, J, K, math=MATH_FP32, stream=None):
+    _check(lib().small_pack_fc_weights(ctx, _ptr(w_kj), _ptr(w_blk), J, K, math, _stream(stream)), "small_pack_fc_weights")
 
 
 def small_conv2d(ctx, inp, w_blk, bias, out, N, C, K, H, W, FH, FW, stride, pad, flags=0, stream=None):
@@ -326,6 +333,18 @@ def small_add(ctx, a, b, out, N, C, H, W, flags=0, stream=None):
 
 def small_fc(ctx, inp, w_blk, bias, out, N, J, K, flags=0, stream=None):
     _check(lib().small_fc(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, J, K, flags, _stream(stream)), "small_fc")
+
+
+FUSE_DWPW, FUSE_DWPW_ALWAYS, FUSE_CONVPOOL = 1, 2, 4
+FUSE_DEFAULT = FUSE_DWPW | FUSE_CONVPOOL
+
+
+def small_set_net_fusion(ctx, mask):
+    _check(lib().small_set_net_fusion(ctx, mask), "small_set_net_fusion")
+
+
+def small_net_launches(ctx, layers, N):
+    return int(lib().small_net_launches(ctx, layers, len(layers), N))
 
 
 def small_net_workspace_bytes(layers, N):

@@ -101,6 +101,7 @@ SMALL_API int small_init(int device, small_ctx **out) {
     }
     c->encode_tiled = fn;
     c->static_workspace = nullptr;
+    c->tc_cache = nullptr;
     c->wait_iters = 1u << 22;     // with the polls' nanosleep back-off: seconds
     if (resolve_static_workspace(c) != SMALL_OK) {      // loads the library's device code here, not inside a later call
         cudaFree(block);
@@ -110,6 +111,7 @@ SMALL_API int small_init(int device, small_ctx **out) {
     c->overlap = 1;
     c->dependent = 0;
     c->conv_path = SMALL_CONV_PATH_AUTO;
+    c->net_fusion = SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL;
     *out = c;
     return SMALL_OK;
 }
@@ -118,6 +120,7 @@ SMALL_API int small_shutdown(small_ctx *ctx) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     cudaSetDevice(ctx->device);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    free_tc_cache(ctx);
     delete ctx;
     return SMALL_OK;
 }
@@ -281,17 +284,14 @@ SMALL_API int small_pack_dw_weights(small_ctx *ctx, const float *w, float *wb, i
     return launch_pack_dw_weights(ctx, w, wb, C, FH, FW, static_cast<cudaStream_t>(stream));
 }
 
-SMALL_API size_t small_fc_weight_elems(int J, int K) {
-    if (J < 1 || K < 1) return 0;
-    return (size_t)blocks_of(K) * blocks_of(J) * SMALL_CB * SMALL_CB;
+// A fully-connected layer's filters [K][J] are a 1x1 convolution's [K][C = J][1][1], and the packed FP32 section of the
+// two is the same array; the tensor-core sections come with the math mode the buffer is packed for.
+SMALL_API size_t small_fc_weight_elems(int J, int K, unsigned math) {
+    return small_conv_weight_elems(J, K, 1, 1, math);
 }
 
-SMALL_API int small_pack_fc_weights(small_ctx *ctx, const float *w, float *wb, int J, int K, void *stream) {
-    if (!ctx) return SMALL_ERR_NOT_INIT;
-    if (int s = check_ptrs({w, wb})) return s;
-    if (J < 1 || K < 1) return SMALL_ERR_SHAPE;
-    if (ranges_overlap(w, sizeof(float) * (size_t)K * J, wb, sizeof(float) * small_fc_weight_elems(J, K))) return SMALL_ERR_OVERLAP;
-    return launch_pack_fc_weights(ctx, w, wb, J, K, static_cast<cudaStream_t>(stream));
+SMALL_API int small_pack_fc_weights(small_ctx *ctx, const float *w, float *wb, int J, int K, unsigned math, void *stream) {
+    return small_pack_conv_weights(ctx, w, wb, J, K, 1, 1, math, stream);
 }
 
 // ---- layers ----
@@ -514,13 +514,36 @@ SMALL_API int small_add(small_ctx *ctx, const float *a, const float *b, float *o
     return launch_add(ctx, a, b, out, n, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
 }
 
+// Above this much work a full reduction under a tensor-core math mode runs on the tensor-core kernel as a 1x1
+// convolution over a 1x1 plane (the images are the pixels); below it the CUDA-core kernel's 3 microseconds win over the
+// tensor-core kernel's set-up (measured on the classifier heads and the autoencoder's layers).
+static const double kFcTensorCoreFlops = 4e6;
+
+SMALL_API int small_fc_uses_tensor_cores(int N, int J, int K, unsigned math) {
+    if (math != SMALL_MATH_TF32 && math != SMALL_MATH_3XTF32) return 0;
+    if (2.0 * N * J * K < kFcTensorCoreFlops) return 0;
+    Geom g;
+    if (make_geom(g, N, J, K, 1, 1, 1, 1, 1, 0, 0, 0, 0) != SMALL_OK) return 0;
+    return conv_tc_supported(g, math == SMALL_MATH_3XTF32) ? 1 : 0;
+}
+
 SMALL_API int small_fc(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out,
                        int N, int J, int K, unsigned flags, void *stream) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     if (flags & ~(SMALL_RELU | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
-    if (!math_valid(math_of(flags))) return SMALL_ERR_INVALID_ARG;
+    const unsigned math = math_of(flags);
+    if (!math_valid(math)) return SMALL_ERR_INVALID_ARG;
     if (int s = check_ptrs({in, w, out}, {bias})) return s;
     if (N < 1 || J < 1 || K < 1 || (long long)N * blocks_of(J) > (1ll << 30) || (long long)N * blocks_of(K) > (1ll << 30)) return SMALL_ERR_SHAPE;
     if (ranges_overlap(in, sizeof(float) * packed_elems(N, J, 1, 1), out, sizeof(float) * packed_elems(N, K, 1, 1))) return SMALL_ERR_OVERLAP;
-    return launch_fc(ctx, in, w, bias, out, N, J, K, flags & SMALL_RELU, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (small_fc_uses_tensor_cores(N, J, K, math) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0 &&
+        ctx->conv_path != SMALL_CONV_PATH_CUDA_CORES) {
+        Geom g;
+        make_geom(g, N, J, K, 1, 1, 1, 1, 1, 0, 0, 0, 0);
+        const float *w_hi = w + conv_w_fp32_elems(J, K, 1, 1);
+        const float *w_lo = w_hi + conv_w_tc_elems(J, K, 1, 1);
+        return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, flags & SMALL_RELU, false, math, st);
+    }
+    return launch_fc(ctx, in, w, bias, out, N, J, K, flags & SMALL_RELU, st);
 }

@@ -20,7 +20,9 @@ struct small_ctx {
     int overlap;             // small_run_net launches every layer after the first as a dependent launch (see launch_kernel)
     int dependent;           // set by small_run_net while it issues those layers
     unsigned wait_iters;     // limit (polls) of every bounded device-side wait; small_set_wait_limit
+    void *tc_cache;          // finished launches of the tensor-core kernel by (shape, mode, tensors); conv_tc.cu
     void *static_workspace;  // device address of the library's built-in workspace array on this device (net_static.cu)
+    unsigned net_fusion;     // SMALL_FUSE_*: which neighbouring layers small_run_net runs as one fused layer
     int conv_path;           // SMALL_CONV_PATH_*: automatic, or one kernel family forced where it takes the shape
 };
 
@@ -85,6 +87,7 @@ struct Geom {
 // Fills g and returns SMALL_OK, or the status that describes what is wrong.
 int make_geom(Geom &g, int N, int C, int K, int H, int W, int FH, int FW, int S, int pt, int pb, int pl, int pr);
 
+void free_tc_cache(small_ctx *);             // conv_tc.cu
 int resolve_static_workspace(small_ctx *);   // net_static.cu; called by small_init with the context's device current
 
 // ---- kernel launchers (each in its own .cu); all return a small_status ----
@@ -92,7 +95,6 @@ int launch_pack(small_ctx *, const float *nchw, float *blk, int N, int C, int H,
 int launch_unpack(small_ctx *, const float *blk, float *nchw, int N, int C, int H, int W, cudaStream_t);
 int launch_pack_conv_weights(small_ctx *, const float *w, float *wb, int C, int K, int FH, int FW, unsigned math, cudaStream_t);
 int launch_pack_dw_weights(small_ctx *, const float *w, float *wb, int C, int FH, int FW, cudaStream_t);
-int launch_pack_fc_weights(small_ctx *, const float *w, float *wb, int J, int K, cudaStream_t);
 int launch_relu(small_ctx *, const float *in, float *out, size_t n, cudaStream_t);
 int launch_add(small_ctx *, const float *a, const float *b, float *out, size_t n, bool relu, cudaStream_t);
 int launch_scale_shift(small_ctx *, const float *in, const float *scale, const float *shift, float *out, int N, int C, int H, int W,

@@ -38,7 +38,10 @@
 // word, lets its in-flight copies land, frees tensor memory and returns.
 #include <cuda.h>
 
+#include <mutex>
+#include <string>
 #include <type_traits>
+#include <unordered_map>
 
 #include "common.cuh"
 #include "sm100.cuh"
@@ -1000,7 +1003,7 @@ static bool make_virt(const Geom &g_in, Virt &v, bool keep_rows = false) {
 }
 
 // groups > 1: g describes one group's channels (C = F_C) and all the filters (K = groups * filters per group)
-bool conv_tc_supported(const Geom &g, bool x3, int groups, const DwFuse *dw) {
+static bool conv_tc_supported_uncached(const Geom &g, bool x3, int groups, const DwFuse *dw) {
     Virt v;
     if (!make_virt(g, v, dw != nullptr)) return false;
     if (dw) return groups == 1 && make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, false, 0, dw).ok;
@@ -1009,10 +1012,76 @@ bool conv_tc_supported(const Geom &g, bool x3, int groups, const DwFuse *dw) {
     return make_plan(v.g, 227 * 1024, 148, false, v.S, v.taps_eff, x3, v.CBr == 1 && g.C <= 16).ok;
 }
 
+// Planning a layer walks two orientations x eight tile sizes; its answers depend on the shape alone, so they are kept:
+// whether the kernel takes a shape (process-wide), and per context the finished launch of a (shape, mode, pointers)
+// combination - plan, tensor maps, arguments, kernel - so that a repeated call only launches.
+namespace {
+
+template <typename T>
+void key_add(std::string &k, const T &v) { k.append(reinterpret_cast<const char *>(&v), sizeof(T)); }
+
+std::string shape_key(const Geom &g, bool x3, int groups, const DwFuse *dw) {
+    std::string k;
+    const int f[] = {g.N, g.C, g.K, g.H, g.W, g.FH, g.FW, g.S, g.pt, g.pb, g.pl, g.pr, x3 ? 1 : 0, groups, dw ? 1 : 0,
+                     dw ? dw->C : 0, dw ? dw->H : 0, dw ? dw->W : 0, dw ? dw->s : 0, dw ? dw->pt : 0, dw ? dw->pl : 0};
+    key_add(k, f);
+    return k;
+}
+
+struct TcLaunch {
+    CUtensorMap map_a, map_b, map_b_lo;
+    TcArgs a;
+    TcKernel kern;
+    unsigned grid, threads;
+    uint32_t smem;
+};
+typedef std::unordered_map<std::string, TcLaunch> TcCache;
+
+}  // namespace
+
+bool conv_tc_supported(const Geom &g, bool x3, int groups, const DwFuse *dw) {
+    static std::mutex mu;
+    static std::unordered_map<std::string, bool> known;
+    const std::string key = shape_key(g, x3, groups, dw);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = known.find(key);
+        if (it != known.end()) return it->second;
+    }
+    const bool ok = conv_tc_supported_uncached(g, x3, groups, dw);
+    std::lock_guard<std::mutex> lock(mu);
+    if (known.size() > 65536) known.clear();
+    known[key] = ok;
+    return ok;
+}
+
+void free_tc_cache(small_ctx *ctx) {
+    delete static_cast<TcCache *>(ctx->tc_cache);
+    ctx->tc_cache = nullptr;
+}
+
 int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &g_in, bool relu, bool accumulate, unsigned mode, cudaStream_t st, int groups, const DwFuse *dw) {
     const bool x3 = mode == SMALL_MATH_3XTF32;
     if (x3 && !w_lo) return SMALL_ERR_INVALID_ARG;
+    // a launch seen before (same shape, mode, flags and tensors): everything is ready
+    std::string key = shape_key(g_in, x3, groups, dw);
+    {
+        const void *ptrs[] = {in, w_hi, w_lo, bias, out, dw ? dw->w : nullptr, dw ? dw->bias : nullptr};
+        const unsigned misc[] = {relu ? 1u : 0u, accumulate ? 1u : 0u, mode, dw ? (unsigned)dw->relu : 0u, ctx->wait_iters};
+        key_add(key, ptrs);
+        key_add(key, misc);
+    }
+    if (!ctx->tc_cache) ctx->tc_cache = new TcCache();
+    TcCache &cache = *static_cast<TcCache *>(ctx->tc_cache);
+    {
+        auto it = cache.find(key);
+        if (it != cache.end()) {
+            const TcLaunch &L = it->second;
+            launch_kernel(ctx, L.kern, dim3(L.grid), dim3(L.threads), L.smem, st, L.map_a, L.map_b, L.map_b_lo, L.a);
+            return check_launch(ctx);
+        }
+    }
     Virt v;
     if (!make_virt(g_in, v, dw != nullptr)) return SMALL_ERR_UNSUPPORTED;
     const Geom &g = v.g;
@@ -1094,11 +1163,16 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
     a.relu = relu; a.accumulate = accumulate; a.wait_iters = ctx->wait_iters;
     const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3, dw != nullptr);
     if (!kern) return SMALL_ERR_UNSUPPORTED;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    // the attribute belongs to the kernel instance, which other layers share: always the device's limit, so that a
+    // launch kept in the cache never finds it lowered by a later layer with a smaller tile
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->max_smem_optin);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);   // persistent: one CTA per SM
-    launch_kernel(ctx, kern, dim3(grid), dim3(dw ? kThreadsDW : x3 ? kThreadsX3 : kThreads), p.smem_bytes, st, map_a, map_b, map_b_lo, a);
+    const unsigned threads = dw ? kThreadsDW : x3 ? kThreadsX3 : kThreads;
+    if (cache.size() >= 4096) cache.clear();
+    cache[key] = TcLaunch{map_a, map_b, map_b_lo, a, kern, grid, threads, p.smem_bytes};
+    launch_kernel(ctx, kern, dim3(grid), dim3(threads), p.smem_bytes, st, map_a, map_b, map_b_lo, a);
     return check_launch(ctx);
 }
 

@@ -157,16 +157,6 @@ __global__ void pack_dw_w_kernel(const float *__restrict__ w, float *__restrict_
 }
 
 // Fully connected: [KB][JB*32 j][32 ko], ko fastest.
-__global__ void pack_fc_w_kernel(const float *__restrict__ w, float *__restrict__ wb, int J, int K, size_t total) {
-    int Jp = ((J + 31) / 32) * 32;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        int ko = (int)(i % 32);
-        int j = (int)((i / 32) % Jp);
-        int kb = (int)(i / 32 / Jp);
-        int k = kb * 32 + ko;
-        wb[i] = (k < K && j < J) ? w[(size_t)k * J + j] : 0.0f;
-    }
-}
 
 static int flat_grid(small_ctx *ctx, size_t total) {
     size_t b = (total + 255) / 256, cap = (size_t)ctx->sm_count * 8;
@@ -235,12 +225,6 @@ int launch_pack_group_conv_weights(small_ctx *ctx, const float *w, float *wb, in
 int launch_pack_dw_weights(small_ctx *ctx, const float *w, float *wb, int C, int FH, int FW, cudaStream_t st) {
     size_t total = (size_t)blocks_of(C) * FH * FW * 32;
     pack_dw_w_kernel<<<flat_grid(ctx, total), 256, 0, st>>>(w, wb, C, FH * FW, total);
-    return check_launch(ctx);
-}
-
-int launch_pack_fc_weights(small_ctx *ctx, const float *w, float *wb, int J, int K, cudaStream_t st) {
-    size_t total = (size_t)blocks_of(K) * blocks_of(J) * 32 * 32;
-    pack_fc_w_kernel<<<flat_grid(ctx, total), 256, 0, st>>>(w, wb, J, K, total);
     return check_launch(ctx);
 }
 

@@ -69,9 +69,69 @@ static bool plan_slots(const small_layer *layers, int n_layers, int N, SlotPlan 
     return true;
 }
 
+// ---- abstract fused layers (Section 6) chosen by the runner itself: the caller describes plain layers.
+// A layer's result may stay on chip when the next layer is its only reader: nothing after that reads the slot before
+// it is written again, and the pair's output slot is not the pair's input slot.
+static bool slot_dead_after(const small_layer *layers, int n_layers, int from, int slot) {
+    for (int j = from; j < n_layers; ++j) {
+        const small_layer &L = layers[j];
+        if (L.src == slot || (L.op == SMALL_OP_ADD && L.src2 == slot)) return false;
+        if (L.dst == slot) return !((L.flags & SMALL_ACCUMULATE) && L.op == SMALL_OP_CONV);
+    }
+    return true;
+}
+
+// Fusing a depthwise 3x3 with the 1x1 convolution behind it pays where the two separate launches are short (measured:
+// a few percent on the depthwise-separable network at batch 64, a loss on large intermediate tensors, where the fused
+// kernel's eight depthwise warps per SM cannot keep up with two full-size kernels); above this size of the
+// intermediate tensor the pair runs as two layers unless SMALL_FUSE_DWPW_ALWAYS is set.
+static const size_t kFuseDwpwMaxBytes = 24u << 20;
+
+// 0: layer i runs on its own; SMALL_OP_DWPW / SMALL_OP_CONVPOOL: layers i and i + 1 run as that fused layer
+static int fused_pair(const small_ctx *ctx, const small_layer *layers, int n_layers, int i, int N) {
+    if (i + 1 >= n_layers) return 0;
+    const small_layer &A = layers[i], &Bn = layers[i + 1];
+    if (A.dst < 0 || Bn.src != A.dst || Bn.dst == A.src || Bn.dst == A.dst) return 0;
+    if (!slot_dead_after(layers, n_layers, i + 2, A.dst)) return 0;
+    Geom g;
+    if (A.op == SMALL_OP_DWCONV && Bn.op == SMALL_OP_CONV && (ctx->net_fusion & (SMALL_FUSE_DWPW | SMALL_FUSE_DWPW_ALWAYS))) {
+        const unsigned math = Bn.flags & SMALL_MATH_MASK;
+        if (A.FH != 3 || A.FW != 3 || Bn.FH != 1 || Bn.FW != 1 || Bn.stride != 1 || (Bn.pad_t | Bn.pad_b | Bn.pad_l | Bn.pad_r)) return 0;
+        if ((Bn.flags & SMALL_ACCUMULATE) || Bn.C != A.C || math == SMALL_MATH_FP32) return 0;
+        if (make_geom(g, N, A.C, A.C, A.H, A.W, 3, 3, A.stride, A.pad_t, A.pad_b, A.pad_l, A.pad_r)) return 0;
+        if (Bn.H != g.OH || Bn.W != g.OW) return 0;
+        if (!(ctx->net_fusion & SMALL_FUSE_DWPW_ALWAYS) && sizeof(float) * packed_elems(N, A.C, g.OH, g.OW) > kFuseDwpwMaxBytes) return 0;
+        return small_dwpw_fused(N, A.C, Bn.K, A.H, A.W, A.stride, A.pad_t, A.pad_b, A.pad_l, A.pad_r, math) ? SMALL_OP_DWPW : 0;
+    }
+    if (A.op == SMALL_OP_CONV && Bn.op == SMALL_OP_POOL && (ctx->net_fusion & SMALL_FUSE_CONVPOOL)) {
+        if ((A.flags & SMALL_ACCUMULATE) || Bn.pool_mode != SMALL_POOL_MAX || Bn.FH != 2 || Bn.FW != 2 || Bn.stride != 2 ||
+            (Bn.pad_t | Bn.pad_b | Bn.pad_l | Bn.pad_r) || Bn.C != A.K)
+            return 0;
+        if (make_geom(g, N, A.C, A.K, A.H, A.W, A.FH, A.FW, A.stride, A.pad_t, A.pad_b, A.pad_l, A.pad_r)) return 0;
+        if (Bn.H != g.OH || Bn.W != g.OW) return 0;
+        return small_conv_maxpool_fused(N, A.C, A.K, A.H, A.W, A.FH, A.FW, A.stride, A.pad_t, A.pad_b, A.pad_l, A.pad_r) ? SMALL_OP_CONVPOOL : 0;
+    }
+    return 0;
+}
+
 }  // namespace small
 
 using namespace small;
+
+SMALL_API int small_set_net_fusion(small_ctx *ctx, unsigned mask) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (mask & ~(unsigned)(SMALL_FUSE_DWPW | SMALL_FUSE_DWPW_ALWAYS | SMALL_FUSE_CONVPOOL)) return SMALL_ERR_INVALID_ARG;
+    ctx->net_fusion = mask;
+    return SMALL_OK;
+}
+
+SMALL_API int small_net_launches(small_ctx *ctx, const small_layer *layers, int n_layers, int N) {
+    if (!ctx || !layers || n_layers < 1 || N < 1) return -1;
+    int launches = 0;
+    for (int i = 0; i < n_layers; ++i, ++launches)
+        if (fused_pair(ctx, layers, n_layers, i, N)) ++i;
+    return launches;
+}
 
 SMALL_API size_t small_net_workspace_bytes(const small_layer *layers, int n_layers, int N) {
     SlotPlan plan;
@@ -126,6 +186,21 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
         int s = SMALL_OK;
         // every layer behind the first may start its set-up while the layer in front of it drains (see launch_kernel)
         ctx->dependent = ctx->overlap && i > 0;
+        if (const int fused = fused_pair(ctx, layers, n_layers, i, N)) {
+            const small_layer &Nx = layers[i + 1];
+            if (fused == SMALL_OP_DWPW) {
+                const unsigned fl = ((L.flags & SMALL_RELU) ? SMALL_RELU_MID : 0u) | (Nx.flags & (SMALL_RELU | SMALL_MATH_MASK));
+                s = small_dwpw_conv2d(ctx, rd(L.src), L.w_blk, L.bias, Nx.w_blk, Nx.bias, wr(Nx.dst), nullptr, N, L.C, Nx.K, L.H, L.W,
+                                      L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r, fl, stream);
+            } else {
+                s = small_conv_maxpool2d(ctx, rd(L.src), L.w_blk, L.bias, wr(Nx.dst), nullptr, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
+                                         L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
+            }
+            ctx->dependent = 0;
+            if (s != SMALL_OK) return s;
+            ++i;
+            continue;
+        }
         switch (L.op) {
             case SMALL_OP_CONV:
                 s = small_conv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,

@@ -9,14 +9,16 @@ from . import binding as B
 
 
 def assign_slots(layers):
-    """Greedy slot reuse by liveness: a tensor's slot is free again after its last reader; a layer never writes
-    the slot it reads (only accumulate updates its destination in place).  'in' / 'out' are the caller's."""
+    """Greedy slot reuse by liveness: a tensor's slot is free again one layer after its last reader (so the output of the
+    layer behind it never lands on it: the library may run those two layers as one fused layer, which must not write the
+    tensor it reads); a layer never writes the slot it reads (only accumulate updates its destination in place).
+    'in' / 'out' are the caller's."""
     last_use = {}
     for i, L in enumerate(layers):
         last_use[L["src"]] = i
         if L.get("accumulate"):
             last_use[L["dst"]] = i
-    slot_of, free, n_slots = {"in": B.SLOT_INPUT, "out": B.SLOT_OUTPUT}, [], 0
+    slot_of, free, pending, n_slots = {"in": B.SLOT_INPUT, "out": B.SLOT_OUTPUT}, [], [], 0
     for i, L in enumerate(layers):
         dst = L["dst"]
         if dst not in slot_of:
@@ -25,72 +27,36 @@ def assign_slots(layers):
             else:
                 slot_of[dst] = n_slots
                 n_slots += 1
+        free += pending                       # slots whose last reader was the previous layer
+        pending = []
         name = L["src"]
         if last_use.get(name) == i and slot_of.get(name, -1) >= 0 and name != dst:
-            free.append(slot_of[name])
+            pending.append(slot_of[name])
     return slot_of, n_slots
 
 
-# Fusing a depthwise 3x3 with the 1x1 convolution behind it pays where the two separate launches are short (measured:
-# a few percent on the depthwise-separable network at batch 64, a loss on large intermediate tensors, where the fused
-# kernel's eight depthwise warps per SM cannot keep up with two full-size kernels); above this size of the
-# intermediate tensor the pair runs as two layers.  fuse_dwpw="all" fuses every pair the kernel takes, False none.
-FUSE_DWPW_MAX_BYTES = 24 << 20
-
-
 class Net:
-    """A network resident on the device: packed filters, descriptors and workspace."""
+    """A network resident on the device: packed filters, plain layer descriptors and workspace.  Which neighbouring
+    layers run as one fused layer is the library's decision inside small_run_net; fuse_dwpw (True: where it pays, "all":
+    wherever the fused kernel takes the shape, False: never) and fuse_convpool only select the library's fusion setting
+    for this network's runs."""
 
     def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda", fuse_dwpw=True, fuse_convpool=True):
         self.ctx = ctx
         self.N = net["batch"] if batch is None else batch
         self.in_shape = tuple(net["input"])
         self.math = B.MATH[math]
+        self.fusion = ((B.FUSE_DWPW_ALWAYS if fuse_dwpw == "all" else B.FUSE_DWPW if fuse_dwpw else 0)
+                       | (B.FUSE_CONVPOOL if fuse_convpool else 0))
         self.keep = []            # device tensors the descriptors point into
         self._offsets = None
-        # which depthwise 3x3 -> 1x1 pairs run as one fused layer (tensor-core modes, shapes the fused kernel takes, the
-        # depthwise result used by nothing else); slots are then assigned over the layers as they will run
         layers_in = net["layers"]
-        uses = {}
-        for L in layers_in:
-            uses[L["src"]] = uses.get(L["src"], 0) + 1
-        shape = {"in": self.in_shape}
-        fused_at = set()
-        pool_at = set()           # convolutions whose 2x2 stride-2 max pool is taken in the convolution's STORE phase
-        for li, L in enumerate(layers_in):
-            c, h, wd = shape[L["src"]]
-            fh, fw = (h, wd) if (L["op"] == "pool" and L["FH"] == 0) else (L["FH"], L["FW"])
-            pt, pb, pl, pr = L["pad"]
-            oh, ow = (1, 1) if L["op"] == "fc" else (B.small_out_size(h, fh, L["stride"], pt, pb), B.small_out_size(wd, fw, L["stride"], pl, pr))
-            shape[L["dst"]] = (L["K"], oh, ow)
-            nxt = layers_in[li + 1] if li + 1 < len(layers_in) else None
-            if (fuse_dwpw and self.math != B.MATH["fp32"] and (li - 1) not in fused_at and L["op"] == "dwconv" and fh == 3 and fw == 3
-                    and nxt is not None and nxt["op"] == "conv" and nxt["src"] == L["dst"] and uses.get(L["dst"], 0) == 1
-                    and nxt["FH"] == 1 and nxt["FW"] == 1 and nxt["stride"] == 1 and tuple(nxt["pad"]) == (0, 0, 0, 0)
-                    and not nxt.get("accumulate")
-                    and (fuse_dwpw == "all" or 4 * B.small_packed_elems(self.N, L["C"], oh, ow) <= FUSE_DWPW_MAX_BYTES)
-                    and B.small_dwpw_fused(self.N, L["C"], nxt["K"], h, wd, L["stride"], L["pad"], self.math)):
-                fused_at.add(li)
-            if (fuse_convpool and (li - 1) not in fused_at and (li - 1) not in pool_at and L["op"] == "conv" and not L.get("accumulate")
-                    and nxt is not None and nxt["op"] == "pool" and nxt["src"] == L["dst"] and uses.get(L["dst"], 0) == 1
-                    and nxt["pool"] == "max" and nxt["FH"] == 2 and nxt["FW"] == 2 and nxt["stride"] == 2 and tuple(nxt["pad"]) == (0, 0, 0, 0)
-                    and B.small_conv_maxpool_fused(self.N, L["C"], L["K"], h, wd, fh, fw, L["stride"], L["pad"])):
-                pool_at.add(li)
-        eff = []
-        for li, L in enumerate(layers_in):
-            if li - 1 in fused_at or li - 1 in pool_at:
-                continue
-            eff.append(dict(L, dst=layers_in[li + 1]["dst"]) if (li in fused_at or li in pool_at) else L)
-        slot_of, _ = assign_slots(eff)
+        slot_of, _ = assign_slots(layers_in)
         self.slot_of = slot_of
         dims = {"in": self.in_shape}
         descs = []
         self.layer_rows = []
-        skip = False
         for li, (L, (w, b)) in enumerate(zip(layers_in, params)):
-            if skip:            # the 1x1 convolution already folded into the previous (fused) descriptor
-                skip = False
-                continue
             c, h, wd = dims[L["src"]]
             fh, fw = L["FH"], L["FW"]
             if L["op"] == "pool" and fh == 0:
@@ -104,52 +70,6 @@ class Net:
             wt = None if w is None else torch.from_numpy(w).to(device)
             bt = None if b is None else torch.from_numpy(b).to(device)
             oh, ow = B.small_out_size(h, fh, L["stride"], pt, pb), B.small_out_size(wd, fw, L["stride"], pl, pr)
-            nxt = layers_in[li + 1] if li + 1 < len(layers_in) else None
-            if li in fused_at:
-                # depthwise 3x3 -> 1x1 as one fused layer: the depthwise result stays in shared memory
-                w2, b2 = params[li + 1]
-                d.op = B.OP_DWPW
-                d.K = nxt["K"]
-                d.dst = slot_of[nxt["dst"]]
-                flags = (B.RELU_MID if L["relu"] else 0) | (B.RELU if nxt["relu"] else 0) | self.math
-                wb = torch.empty(B.small_dw_weight_elems(L["C"], 3, 3), device=device)
-                B.small_pack_dw_weights(ctx, wt, wb, L["C"], 3, 3)
-                wt2 = torch.from_numpy(w2).to(device)
-                bt2 = None if b2 is None else torch.from_numpy(b2).to(device)
-                wb2 = torch.empty(B.small_conv_weight_elems(L["C"], nxt["K"], 1, 1, self.math), device=device)
-                B.small_pack_conv_weights(ctx, wt2, wb2, L["C"], nxt["K"], 1, 1, self.math)
-                d.w_blk2 = wb2.data_ptr()
-                d.bias2 = None if bt2 is None else bt2.data_ptr()
-                self.keep += [wt2, bt2, wb2]
-                d.flags = flags
-                d.w_blk = wb.data_ptr()
-                d.bias = None if bt is None else bt.data_ptr()
-                self.keep += [wb, bt, wt]
-                dims[L["dst"]] = (L["C"], oh, ow)
-                dims[nxt["dst"]] = (nxt["K"], oh, ow)
-                self.layer_rows.append(dict(name=L["name"] + "+" + nxt["name"], op="dwpw", C=L["C"], K=nxt["K"], H=h, W=wd, FH=3, FW=3,
-                                            stride=L["stride"], pad=L["pad"], OH=oh, OW=ow, dst=nxt["dst"], first=li, upto=li + 2))
-                descs.append(d)
-                skip = True
-                continue
-            if li in pool_at:
-                # convolution -> 2x2 stride-2 max pool as one fused layer
-                d.op = B.OP_CONVPOOL
-                d.dst = slot_of[nxt["dst"]]
-                flags |= self.math
-                wb = torch.empty(B.small_conv_weight_elems(L["C"], L["K"], fh, fw, B.MATH["fp32"]), device=device)
-                B.small_pack_conv_weights(ctx, wt, wb, L["C"], L["K"], fh, fw, B.MATH["fp32"])
-                d.flags = flags
-                d.w_blk = wb.data_ptr()
-                d.bias = None if bt is None else bt.data_ptr()
-                self.keep += [wb, bt, wt]
-                dims[L["dst"]] = (L["K"], oh, ow)
-                dims[nxt["dst"]] = (L["K"], oh // 2, ow // 2)
-                self.layer_rows.append(dict(name=L["name"] + "+" + nxt["name"], op="convpool", C=L["C"], K=L["K"], H=h, W=wd, FH=fh, FW=fw,
-                                            stride=L["stride"], pad=L["pad"], OH=oh // 2, OW=ow // 2, dst=nxt["dst"], first=li, upto=li + 2))
-                descs.append(d)
-                skip = True
-                continue
             if L["op"] == "conv":
                 d.op = B.OP_CONV
                 flags |= self.math
@@ -163,21 +83,11 @@ class Net:
                 d.op = B.OP_POOL
                 d.pool_mode = B.POOL_MAX if L["pool"] == "max" else B.POOL_AVG
                 wb = None
-            elif L["op"] == "fc" and self.math != B.MATH["fp32"] and h == 1 and wd == 1 and 2 * self.N * L["C"] * L["K"] >= 4e6:
-                # a full reduction over a 1x1 plane is a 1x1 convolution whose pixels are the images: in the
-                # tensor-core modes it runs on the convolution kernel (same arithmetic, same blocked buffers).  A
-                # classifier head of a megaflop or so stays on the FP32 kernel (3 us; the tensor-core kernel's set-up
-                # alone costs more).
-                d.op = B.OP_CONV
-                d.FH = d.FW = 1
-                flags |= self.math
-                wb = torch.empty(B.small_conv_weight_elems(L["C"], L["K"], 1, 1, self.math), device=device)
-                B.small_pack_conv_weights(ctx, wt.reshape(L["K"], L["C"], 1, 1).contiguous(), wb, L["C"], L["K"], 1, 1, self.math)
-                oh = ow = 1
             elif L["op"] == "fc":
                 d.op = B.OP_FC
-                wb = torch.empty(B.small_fc_weight_elems(L["C"], L["K"]), device=device)
-                B.small_pack_fc_weights(ctx, wt, wb, L["C"], L["K"])
+                flags |= self.math
+                wb = torch.empty(B.small_fc_weight_elems(L["C"], L["K"], self.math), device=device)
+                B.small_pack_fc_weights(ctx, wt, wb, L["C"], L["K"], self.math)
                 oh = ow = 1
             else:
                 raise ValueError(L["op"])
@@ -201,18 +111,34 @@ class Net:
         assert self.workspace.data_ptr() % 256 == 0
         self.out_blk = torch.empty(B.small_packed_elems(self.N, oc, oh, ow), device=device)
 
+    def launches(self):
+        """Kernel launches of one run under this network's fusion setting."""
+        B.small_set_net_fusion(self.ctx, self.fusion)
+        try:
+            return B.small_net_launches(self.ctx, self.layers, self.N)
+        finally:
+            B.small_set_net_fusion(self.ctx, B.FUSE_DEFAULT)
+
     def run(self, in_blk, out_blk=None, stream=None, n_layers=None):
         """Runs all layers (or the first n_layers, to inspect an intermediate)."""
         out_blk = self.out_blk if out_blk is None else out_blk
         layers = self.layers if n_layers is None else (B.small_layer * n_layers)(*self.layers[:n_layers])
-        B.small_run_net(self.ctx, layers, self.N, in_blk, out_blk, self.workspace, self.ws_bytes, stream)
+        B.small_set_net_fusion(self.ctx, self.fusion)
+        try:
+            B.small_run_net(self.ctx, layers, self.N, in_blk, out_blk, self.workspace, self.ws_bytes, stream)
+        finally:
+            B.small_set_net_fusion(self.ctx, B.FUSE_DEFAULT)
         return out_blk
 
     def run_host(self, in_host, out_host, stream=None):
         c, h, w = self.in_shape
         oc, oh, ow = self.out_shape
-        B.small_run_net_host(self.ctx, self.layers, self.N, in_host, c, h, w, out_host, oc, oh, ow,
-                             self.workspace, self.ws_bytes + self.stage_bytes, stream)
+        B.small_set_net_fusion(self.ctx, self.fusion)
+        try:
+            B.small_run_net_host(self.ctx, self.layers, self.N, in_host, c, h, w, out_host, oc, oh, ow,
+                                 self.workspace, self.ws_bytes + self.stage_bytes, stream)
+        finally:
+            B.small_set_net_fusion(self.ctx, B.FUSE_DEFAULT)
 
     def slot_ptr(self, slot, in_blk, out_blk):
         if slot == B.SLOT_INPUT:

@@ -55,6 +55,7 @@ def test_weight_sizes(lib):
     assert B.small_conv_weight_elems(3, 16, 3, 3, 3 << 4) == 0
     assert B.small_dw_weight_elems(70, 3, 3) == 3 * 9 * 32
     assert B.small_fc_weight_elems(64, 10) == 2 * 32 * 32
+    assert B.small_fc_weight_elems(64, 10, B.MATH_3XTF32) == 3 * 2 * 32 * 32
     assert B.small_fc_weight_elems(0, 10) == 0
 
 
@@ -97,7 +98,9 @@ def test_workspace_plan_matches_memory_model(lib):
     # no layer reads and writes the same slot unless it accumulates into it
     for L in net["layers"]:
         assert slot_of[L["src"]] != slot_of[L["dst"]]
-    assert assign_slots(configs.dwsep_cnn()["layers"])[1] == 2
+    # a chain needs three: a slot is reused two layers on, so that a pair of layers run as one fused layer never
+    # writes the tensor it reads
+    assert assign_slots(configs.dwsep_cnn()["layers"])[1] == 3
     # descriptors -> bytes: one conv 16->16 on 32x32 at N=2 from slot 0 to slot 1
     L = B.small_layer()
     L.op, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride = B.OP_CONV, 16, 16, 32, 32, 3, 3, 1

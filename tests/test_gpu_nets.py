@@ -96,6 +96,43 @@ def test_layer_overlap_changes_no_bit(name, batch, math):
     assert B.small_device_status(ctx()) == 0
 
 
+def test_the_runner_fuses_plain_descriptors_itself():
+    """Plain layer descriptors through the C ABI: small_run_net decides which neighbours run as one fused layer.  The launch
+    counts it reports follow the fusion setting, and the results stay the same within the mode's tolerance."""
+    c = ctx()
+    net = configs.dwsep_cnn(batch=2)
+    params = configs.make_params(net)
+    x = configs.make_input(net, 2)
+    ref = nets.run_net(net, params, x)["out"]
+    gnet = Net(c, net, params, batch=2, math="tf32")
+    n_layers = len(gnet.layers)
+    assert n_layers == len(net["layers"]) == 29          # every descriptor is a plain layer
+    in_blk = to_blk(x)
+    counts = {}
+    for mask in (0, B.FUSE_DWPW, B.FUSE_DWPW | B.FUSE_DWPW_ALWAYS, B.FUSE_DEFAULT):
+        B.small_set_net_fusion(c, mask)
+        try:
+            counts[mask] = B.small_net_launches(c, gnet.layers, 2)
+            out = torch.full_like(gnet.out_blk, float("nan"))
+            B.small_run_net(c, gnet.layers, 2, in_blk, out, gnet.workspace, gnet.ws_bytes)
+        finally:
+            B.small_set_net_fusion(c, B.FUSE_DEFAULT)
+        assert rel_err(from_blk(out, 2, 2, 1, 1), ref) <= net_tol("dwsep_cnn", "tf32")
+    assert counts[0] == 29
+    assert counts[B.FUSE_DWPW] == counts[B.FUSE_DEFAULT] == 29 - 13        # all thirteen depthwise / 1x1 pairs at this batch
+    assert counts[B.FUSE_DWPW | B.FUSE_DWPW_ALWAYS] == 16
+    # in FP32 mode nothing of this network fuses; the single-convolution workload is one launch in every mode
+    assert Net(c, net, params, batch=2, math="fp32").launches() == 29
+    one = configs.single_conv_pool()
+    assert Net(c, one, configs.make_params(one), math="3xtf32").launches() == 1
+    assert Net(c, one, configs.make_params(one), math="3xtf32", fuse_convpool=False).launches() == 2
+    # a full reduction under a tensor-core mode is routed by the library, not by the caller
+    assert B.small_fc_uses_tensor_cores(4096, 128, 128, B.MATH_TF32) and not B.small_fc_uses_tensor_cores(256, 64, 10, B.MATH_TF32)
+    with pytest.raises(B.SmallError):
+        B.small_set_net_fusion(c, 8)
+    assert B.small_device_status(c) == 0
+
+
 def test_run_net_host_end_to_end():
     net = configs.residual_cnn(batch=8)
     params = configs.make_params(net)
