@@ -101,6 +101,12 @@ int small_last_cuda_error(small_ctx *ctx);
  * until that layer has completed before they read or write a tensor.  Results are the same either way.  The paper
  * has no counterpart. */
 int small_set_layer_overlap(small_ctx *ctx, int on);
+/* Branch overlap inside small_run_net (on by default; `on` = 0 switches it off).  When on, two neighbouring layers of the
+ * list that share no tensor except as readers - a residual stage's convolution and its shortcut convolution - run at the
+ * same time: the second one on a stream of the context's own (created in small_init), forked from and joined to the
+ * caller's stream by events, which a stream capture records as a fork and a join.  Results are the same either way.  The
+ * paper has no counterpart (its layers are consecutive calls). */
+int small_set_branch_overlap(small_ctx *ctx, int on);
 /* Limit, in polls, of every bounded device-side wait (default 2^22: seconds, with the polls' back-off); at least 16.
  * A wait that runs out makes its kernel record SMALL_ERR_TIMEOUT, let its copies in flight land, free its tensor memory
  * and return; the affected outputs are undefined and later calls work normally.  The paper has no counterpart. */
@@ -112,9 +118,10 @@ int small_set_wait_limit(small_ctx *ctx, unsigned polls);
 int small_selftest_wait_timeout(small_ctx *ctx, void *stream);
 /* Kernel family of the full channel reductions under the tensor-core math modes.  AUTO (the default): per layer,
  * whichever of the tensor-core kernel and the register-tiled FP32 kernel is the faster one for its channel counts
- * (FP32 FMAs meet every mode's tolerance); TENSOR / CUDA_CORES force one family wherever it takes the shape.  For
+ * (FP32 FMAs meet every mode's tolerance); TENSOR / CUDA_CORES force one family wherever it takes the shape, GENERAL the
+ * general FP32 kernel (any window and stride) everywhere except the network stems.  For
  * measurements and comparisons; results stay within the mode's tolerance either way.  The paper has no counterpart. */
-enum { SMALL_CONV_PATH_AUTO = 0, SMALL_CONV_PATH_TENSOR = 1, SMALL_CONV_PATH_CUDA_CORES = 2 };
+enum { SMALL_CONV_PATH_AUTO = 0, SMALL_CONV_PATH_TENSOR = 1, SMALL_CONV_PATH_CUDA_CORES = 2, SMALL_CONV_PATH_GENERAL = 3 };
 int small_set_conv_path(small_ctx *ctx, int path);
 /* Which kernel small_conv2d runs for this shape and math mode (with a 32-byte aligned output) under the context's
  * path setting: 0 = few-input-channel kernel (network stems), 1 = register-tiled FP32 kernel, 2 = general FP32 kernel,

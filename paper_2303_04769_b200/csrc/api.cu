@@ -112,6 +112,16 @@ SMALL_API int small_init(int device, small_ctx **out) {
     c->dependent = 0;
     c->conv_path = SMALL_CONV_PATH_AUTO;
     c->net_fusion = SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL;
+    c->branch_overlap = 1;
+    c->side_stream = c->ev_fork = c->ev_join = nullptr;
+    {
+        cudaStream_t side;
+        cudaEvent_t f, j;
+        if (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) == cudaSuccess) c->side_stream = side;
+        if (cudaEventCreateWithFlags(&f, cudaEventDisableTiming) == cudaSuccess) c->ev_fork = f;
+        if (cudaEventCreateWithFlags(&j, cudaEventDisableTiming) == cudaSuccess) c->ev_join = j;
+        if (!c->side_stream || !c->ev_fork || !c->ev_join) c->branch_overlap = 0;
+    }
     *out = c;
     return SMALL_OK;
 }
@@ -121,6 +131,9 @@ SMALL_API int small_shutdown(small_ctx *ctx) {
     cudaSetDevice(ctx->device);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     free_tc_cache(ctx);
+    if (ctx->ev_fork) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_fork));
+    if (ctx->ev_join) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_join));
+    if (ctx->side_stream) cudaStreamDestroy(static_cast<cudaStream_t>(ctx->side_stream));
     delete ctx;
     return SMALL_OK;
 }
@@ -140,9 +153,15 @@ SMALL_API int small_set_wait_limit(small_ctx *ctx, unsigned polls) {
     return SMALL_OK;
 }
 
+SMALL_API int small_set_branch_overlap(small_ctx *ctx, int on) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    ctx->branch_overlap = (on && ctx->side_stream && ctx->ev_fork && ctx->ev_join) ? 1 : 0;
+    return SMALL_OK;
+}
+
 SMALL_API int small_set_conv_path(small_ctx *ctx, int path) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
-    if (path != SMALL_CONV_PATH_AUTO && path != SMALL_CONV_PATH_TENSOR && path != SMALL_CONV_PATH_CUDA_CORES) return SMALL_ERR_INVALID_ARG;
+    if (path < SMALL_CONV_PATH_AUTO || path > SMALL_CONV_PATH_GENERAL) return SMALL_ERR_INVALID_ARG;
     ctx->conv_path = path;
     return SMALL_OK;
 }
@@ -312,9 +331,14 @@ static bool prefer_cuda_cores(const small_ctx *ctx, const Geom &g, unsigned math
 
 static int conv2d_path(const small_ctx *ctx, const Geom &g, unsigned math, bool out_aligned32) {
     if (conv_thin_supported(g)) return 0;          // a reduction of a few dozen terms: CUDA cores in every math mode
+    if (ctx && ctx->conv_path == SMALL_CONV_PATH_GENERAL) return 2;
     bool direct = conv_direct_supported(g);
-    // the register-tiled kernel computes runs of 8 output columns: planes narrower than 4 columns leave it mostly idle
-    if (direct && g.OW < 4 && !(ctx && ctx->conv_path == SMALL_CONV_PATH_CUDA_CORES)) direct = false;
+    // the register-tiled kernel computes runs of 8 output columns per thread and 256 to 2048 outputs x 8 to 64 filters per
+    // thread block: planes narrower than 4 columns leave it mostly idle, and a layer that gives it fewer blocks than half
+    // the SMs runs faster on the general kernel's many small blocks (measured on the depthwise-separable network)
+    if (direct && !(ctx && ctx->conv_path == SMALL_CONV_PATH_CUDA_CORES) &&
+        (g.OW < 4 || conv_direct_blocks(g) < (ctx ? ctx->sm_count : 148) / 2))
+        direct = false;
     if (math == SMALL_MATH_FP32) return direct ? 1 : 2;
     const bool tc = out_aligned32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32);
     if (tc && !(direct && prefer_cuda_cores(ctx, g, math))) return 3;

@@ -22,6 +22,8 @@ struct small_ctx {
     unsigned wait_iters;     // limit (polls) of every bounded device-side wait; small_set_wait_limit
     void *tc_cache;          // finished launches of the tensor-core kernel by (shape, mode, tensors); conv_tc.cu
     void *static_workspace;  // device address of the library's built-in workspace array on this device (net_static.cu)
+    int branch_overlap;      // small_run_net runs independent neighbouring layers side by side (side stream)
+    void *side_stream, *ev_fork, *ev_join;   // cudaStream_t / cudaEvent_t of that
     unsigned net_fusion;     // SMALL_FUSE_*: which neighbouring layers small_run_net runs as one fused layer
     int conv_path;           // SMALL_CONV_PATH_*: automatic, or one kernel family forced where it takes the shape
 };
@@ -109,6 +111,7 @@ int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *
                      bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
 // register-tiled FP32 kernel: windows 1 or 3 wide, strides 1 and 2 (group convolutions as launch_conv_fp32 takes them)
 bool conv_direct_supported(const Geom &, int span = 0, int Kg = 0, int S_C = 0);
+long long conv_direct_blocks(const Geom &);     // thread blocks its plan launches (0: shape not taken)
 int launch_conv_direct(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
                        bool relu, bool accumulate, cudaStream_t, int span = 0, int Kg = 0, int S_C = 0);
 // the same kernel with a 2 x 2 stride-2 max pool taken in its STORE phase: out is [N][K][OH/2][OW/2]

@@ -421,6 +421,11 @@ bool conv_direct_supported(const Geom &g, int span, int Kg, int S_C) {
     return plan_direct(g, span, Kg, S_C, 227 * 1024).ok;
 }
 
+long long conv_direct_blocks(const Geom &g) {
+    const DirectPlan p = plan_direct(g, 0, 0, 0, 227 * 1024);
+    return p.ok ? p.blocks : 0;
+}
+
 namespace {
 
 // Tensor maps and launch shared by the float and the quantised form.  esize: bytes per channel of the activation

@@ -87,6 +87,15 @@ static bool slot_dead_after(const small_layer *layers, int n_layers, int from, i
 // intermediate tensor the pair runs as two layers unless SMALL_FUSE_DWPW_ALWAYS is set.
 static const size_t kFuseDwpwMaxBytes = 24u << 20;
 
+// Two layers may run at the same time when neither writes a tensor the other one reads or writes.
+static bool independent(const small_layer &A, const small_layer &Bn) {
+    auto reads = [](const small_layer &L, int slot) {
+        return L.src == slot || (L.op == SMALL_OP_ADD && L.src2 == slot) || ((L.flags & SMALL_ACCUMULATE) && L.op == SMALL_OP_CONV && L.dst == slot);
+    };
+    if (A.dst == Bn.dst || reads(Bn, A.dst) || reads(A, Bn.dst)) return false;
+    return A.dst != SMALL_SLOT_INPUT && Bn.dst != SMALL_SLOT_INPUT;
+}
+
 // 0: layer i runs on its own; SMALL_OP_DWPW / SMALL_OP_CONVPOOL: layers i and i + 1 run as that fused layer
 static int fused_pair(const small_ctx *ctx, const small_layer *layers, int n_layers, int i, int N) {
     if (i + 1 >= n_layers) return 0;
@@ -181,11 +190,39 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
         if (L.op == SMALL_OP_POOL && L.pool_mode != SMALL_POOL_MAX && L.pool_mode != SMALL_POOL_AVG) return SMALL_ERR_INVALID_ARG;
         if (L.src == L.dst && L.op != SMALL_OP_RELU && L.op != SMALL_OP_ADD) return SMALL_ERR_OVERLAP;
     }
+    auto run_one = [&](const small_layer &L, void *strm) -> int {
+        switch (L.op) {
+            case SMALL_OP_CONV:
+                return small_conv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
+                                 L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, strm);
+            case SMALL_OP_DWCONV:
+                return small_dwconv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.H, L.W, L.FH, L.FW, L.stride,
+                                   L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, strm);
+            case SMALL_OP_POOL:
+                return small_pool2d(ctx, rd(L.src), wr(L.dst), nullptr, N, L.C, L.H, L.W, L.FH, L.FW, L.stride,
+                                 L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.pool_mode, strm);
+            case SMALL_OP_RELU:
+                return small_relu(ctx, rd(L.src), wr(L.dst), N, L.C, L.H, L.W, strm);
+            case SMALL_OP_ADD:
+                return small_add(ctx, rd(L.src), rd(L.src2), wr(L.dst), N, L.C, L.H, L.W, L.flags, strm);
+            case SMALL_OP_FC:
+                return small_fc(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.flags, strm);
+            case SMALL_OP_CONVPOOL:
+                return small_conv_maxpool2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), nullptr, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
+                                         L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, strm);
+            case SMALL_OP_DWPW:
+                return small_dwpw_conv2d(ctx, rd(L.src), L.w_blk, L.bias, L.w_blk2, L.bias2, wr(L.dst), nullptr, N, L.C, L.K, L.H, L.W,
+                                      L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, strm);
+        }
+        return SMALL_ERR_INVALID_ARG;
+    };
+    bool after_join = false;
     for (int i = 0; i < n_layers; ++i) {
         const small_layer &L = layers[i];
         int s = SMALL_OK;
         // every layer behind the first may start its set-up while the layer in front of it drains (see launch_kernel)
-        ctx->dependent = ctx->overlap && i > 0;
+        ctx->dependent = ctx->overlap && i > 0 && !after_join;
+        after_join = false;
         if (const int fused = fused_pair(ctx, layers, n_layers, i, N)) {
             const small_layer &Nx = layers[i + 1];
             if (fused == SMALL_OP_DWPW) {
@@ -201,37 +238,28 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
             ++i;
             continue;
         }
-        switch (L.op) {
-            case SMALL_OP_CONV:
-                s = small_conv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
-                                 L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
-                break;
-            case SMALL_OP_DWCONV:
-                s = small_dwconv2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.H, L.W, L.FH, L.FW, L.stride,
-                                   L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
-                break;
-            case SMALL_OP_POOL:
-                s = small_pool2d(ctx, rd(L.src), wr(L.dst), nullptr, N, L.C, L.H, L.W, L.FH, L.FW, L.stride,
-                                 L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.pool_mode, stream);
-                break;
-            case SMALL_OP_RELU:
-                s = small_relu(ctx, rd(L.src), wr(L.dst), N, L.C, L.H, L.W, stream);
-                break;
-            case SMALL_OP_ADD:
-                s = small_add(ctx, rd(L.src), rd(L.src2), wr(L.dst), N, L.C, L.H, L.W, L.flags, stream);
-                break;
-            case SMALL_OP_FC:
-                s = small_fc(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), N, L.C, L.K, L.flags, stream);
-                break;
-            case SMALL_OP_CONVPOOL:
-                s = small_conv_maxpool2d(ctx, rd(L.src), L.w_blk, L.bias, wr(L.dst), nullptr, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
-                                         L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
-                break;
-            case SMALL_OP_DWPW:
-                s = small_dwpw_conv2d(ctx, rd(L.src), L.w_blk, L.bias, L.w_blk2, L.bias2, wr(L.dst), nullptr, N, L.C, L.K, L.H, L.W,
-                                      L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);
-                break;
+        // Two neighbouring layers that touch no common tensor except as readers (a residual stage's convolution and its
+        // shortcut) run side by side: the second one on the context's side stream, forked from and joined to the caller's
+        // stream by events, so that a short layer hides behind a long one.  Both are ordinary launches, and so is the
+        // layer behind the join.
+        if (ctx->branch_overlap && ctx->side_stream && i + 1 < n_layers && independent(L, layers[i + 1]) &&
+            !fused_pair(ctx, layers, n_layers, i + 1, N)) {
+            cudaStream_t main_st = static_cast<cudaStream_t>(stream), side = static_cast<cudaStream_t>(ctx->side_stream);
+            cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(ctx->ev_fork), main_st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(side, static_cast<cudaEvent_t>(ctx->ev_fork), 0);
+            if (e != cudaSuccess) { ctx->last_cuda = (int)e; ctx->dependent = 0; return SMALL_ERR_CUDA; }
+            s = run_one(L, stream);
+            ctx->dependent = 0;
+            if (s == SMALL_OK) s = run_one(layers[i + 1], ctx->side_stream);
+            e = cudaEventRecord(static_cast<cudaEvent_t>(ctx->ev_join), side);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(main_st, static_cast<cudaEvent_t>(ctx->ev_join), 0);
+            if (s != SMALL_OK) return s;
+            if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
+            ++i;
+            after_join = true;
+            continue;
         }
+        s = run_one(L, stream);
         ctx->dependent = 0;
         if (s != SMALL_OK) return s;
     }

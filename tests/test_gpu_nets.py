@@ -96,6 +96,34 @@ def test_layer_overlap_changes_no_bit(name, batch, math):
     assert B.small_device_status(ctx()) == 0
 
 
+@pytest.mark.parametrize("math", ["fp32", "tf32", "3xtf32"])
+def test_branch_overlap_changes_no_bit(math):
+    """A residual stage's shortcut convolution runs on the context's side stream next to the stage's first convolution:
+    the result must be the one that strictly consecutive launches give, eagerly and replayed from a CUDA graph."""
+    batch = 96
+    net = configs.residual_cnn(batch=batch)
+    params = configs.make_params(net)
+    in_blk = to_blk(configs.make_input(net, batch))
+    gnet = Net(ctx(), net, params, batch=batch, math=math)
+    try:
+        B.small_set_branch_overlap(ctx(), 0)
+        want = gnet.run(in_blk).clone()
+        B.small_set_branch_overlap(ctx(), 1)
+        for _ in range(3):
+            assert torch.equal(gnet.run(in_blk), want)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            out = gnet.run(in_blk)
+        for _ in range(5):
+            out.fill_(float("nan"))
+            g.replay()
+            assert torch.equal(out, want)
+    finally:
+        B.small_set_branch_overlap(ctx(), 1)
+    assert B.small_device_status(ctx()) == 0
+
+
 def test_the_runner_fuses_plain_descriptors_itself():
     """Plain layer descriptors through the C ABI: small_run_net decides which neighbours run as one fused layer.  The launch
     counts it reports follow the fusion setting, and the results stay the same within the mode's tolerance."""
