@@ -367,13 +367,16 @@ int small_run_net(small_ctx *ctx, const small_layer *layers, int n_layers, int N
                   const float *in_blk, float *out_blk, void *workspace, size_t workspace_bytes, void *stream);
 
 /* Extra device bytes small_run_net_host needs beyond small_net_workspace_bytes: staging for the NCHW
- * input and output and their blocked forms. */
+ * input (twice) and output and their blocked forms. */
 size_t small_net_host_staging_bytes(int N, int C, int H, int W, int outC, int outH, int outW);
 /* End-to-end convenience: in_nchw_host (HOST, float[N][C][H][W]) is copied to the device, packed, run
  * through the layers, unpacked and copied to out_nchw_host (HOST, float[N][outC][outH][outW]).  Pinned
  * host memory makes the copies asynchronous.  workspace: device, 256-byte aligned, at least
  * small_net_workspace_bytes + small_net_host_staging_bytes.  Returns after enqueuing; synchronise
- * `stream` before reading the result. */
+ * `stream` before reading the result, and keep in_nchw_host unchanged until then.
+ * The input copy runs on a stream of the context's own into one of two staging areas of the workspace, so that with
+ * back-to-back calls on one workspace the copy of a call's input overlaps the layers of the call before it; the caller's
+ * stream waits for the copy by an event.  (While `stream` is being captured the copy stays on `stream`.) */
 int small_run_net_host(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
                        const float *in_nchw_host, int C, int H, int W,
                        float *out_nchw_host, int outC, int outH, int outW,

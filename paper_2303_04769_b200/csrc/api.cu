@@ -121,6 +121,15 @@ SMALL_API int small_init(int device, small_ctx **out) {
         if (cudaEventCreateWithFlags(&f, cudaEventDisableTiming) == cudaSuccess) c->ev_fork = f;
         if (cudaEventCreateWithFlags(&j, cudaEventDisableTiming) == cudaSuccess) c->ev_join = j;
         if (!c->side_stream || !c->ev_fork || !c->ev_join) c->branch_overlap = 0;
+        c->copy_stream = nullptr; c->host_ws = nullptr; c->host_parity = 0; c->host_used[0] = c->host_used[1] = 0;
+        cudaStream_t cs;
+        bool ok = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; i < 2; ++i) {
+            cudaEvent_t a = nullptr, b = nullptr;
+            ok = ok && cudaEventCreateWithFlags(&a, cudaEventDisableTiming) == cudaSuccess && cudaEventCreateWithFlags(&b, cudaEventDisableTiming) == cudaSuccess;
+            c->ev_h2d[i] = a; c->ev_pack[i] = b;
+        }
+        if (ok) c->copy_stream = cs;
     }
     *out = c;
     return SMALL_OK;
@@ -134,6 +143,11 @@ SMALL_API int small_shutdown(small_ctx *ctx) {
     if (ctx->ev_fork) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_fork));
     if (ctx->ev_join) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_join));
     if (ctx->side_stream) cudaStreamDestroy(static_cast<cudaStream_t>(ctx->side_stream));
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->ev_h2d[i]) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_h2d[i]));
+        if (ctx->ev_pack[i]) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_pack[i]));
+    }
+    if (ctx->copy_stream) cudaStreamDestroy(static_cast<cudaStream_t>(ctx->copy_stream));
     delete ctx;
     return SMALL_OK;
 }

@@ -24,6 +24,8 @@ struct small_ctx {
     void *static_workspace;  // device address of the library's built-in workspace array on this device (net_static.cu)
     int branch_overlap;      // small_run_net runs independent neighbouring layers side by side (side stream)
     void *side_stream, *ev_fork, *ev_join;   // cudaStream_t / cudaEvent_t of that
+    void *copy_stream, *ev_h2d[2], *ev_pack[2];   // small_run_net_host: input copies on their own stream, two staging areas
+    void *host_ws; int host_parity, host_used[2];
     unsigned net_fusion;     // SMALL_FUSE_*: which neighbouring layers small_run_net runs as one fused layer
     int conv_path;           // SMALL_CONV_PATH_*: automatic, or one kernel family forced where it takes the shape
 };
@@ -119,8 +121,9 @@ bool conv_direct_pool_supported(const Geom &);
 int launch_conv_direct_pool(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
 // at most four input channels, 3 x 3 (strides 1, 2) or the 10 x 4 stride-2 window: FP32 FMAs with the filters in registers
 bool conv_thin_supported(const Geom &);
+// nchw_in: `in` is the NCHW tensor float[N][C][H][W] instead of the blocked one (used at a network's edge)
 int launch_conv_thin(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,
-                     bool relu, bool accumulate, cudaStream_t);
+                     bool relu, bool accumulate, cudaStream_t, bool nchw_in = false);
 int group_conv_span(int C, int F_C, int S_C, int Kg);      // channel blocks a filter block of a group convolution needs
 int launch_pack_group_conv_weights(small_ctx *, const float *w, float *wb, int C, int F_C, int S_C, int Kg, int FH, int FW, cudaStream_t);
 // tensor-core implicit GEMM; mode is SMALL_MATH_TF32 or SMALL_MATH_3XTF32

@@ -24,6 +24,7 @@ struct ThinArgs {
     int rows, pitch, plane;                  // shared tile: rows x pitch floats per (image, channel); plane = rows * pitch
     long long tiles;
     bool relu, accumulate;
+    bool nchw;                               // the input is the NCHW tensor float[N][C][H][W] itself (the network's edge)
 };
 
 // Threads per block: four warps.  A block loads a tile, then computes on it, with nothing in flight meanwhile, so
@@ -85,8 +86,17 @@ __global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs 
                     const int gh = ih0 + r, gw = c - a.pl;
                     at[u] = img * C * a.plane + r * a.pitch + c;
                     if (gh >= 0 && gh < a.H && gw >= 0 && gw < a.W) {
-                        const float *p = a.in + (((size_t)(n0 + img) * a.H + gh) * a.W + gw) * 32;    // one channel block
-                        if (C == 1) v[u].x = __ldg(p); else v[u] = __ldg(reinterpret_cast<const float4 *>(p));
+                        if (a.nchw) {       // planes of the NCHW tensor: the same values land at the same places of the tile
+                            const size_t hw = (size_t)a.H * a.W;
+                            const float *p = a.in + ((size_t)(n0 + img) * C * a.H + gh) * a.W + gw;
+                            v[u].x = __ldg(p);
+                            if (C > 1) v[u].y = __ldg(p + hw);
+                            if (C > 2) v[u].z = __ldg(p + 2 * hw);
+                            if (C > 3) v[u].w = __ldg(p + 3 * hw);
+                        } else {
+                            const float *p = a.in + (((size_t)(n0 + img) * a.H + gh) * a.W + gw) * 32;    // one channel block
+                            if (C == 1) v[u].x = __ldg(p); else v[u] = __ldg(reinterpret_cast<const float4 *>(p));
+                        }
                     }
                 }
             }
@@ -194,12 +204,12 @@ bool conv_thin_supported(const Geom &g) {
 }
 
 int launch_conv_thin(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, const Geom &g,
-                     bool relu, bool accumulate, cudaStream_t st) {
+                     bool relu, bool accumulate, cudaStream_t st, bool nchw_in) {
     if (!conv_thin_supported(g)) return SMALL_ERR_UNSUPPORTED;
     ThinArgs a{};
     a.in = in; a.w = w; a.bias = bias; a.out = out;
     a.N = g.N; a.K = g.K; a.KB = g.KB; a.H = g.H; a.W = g.W; a.OH = g.OH; a.OW = g.OW; a.pt = g.pt; a.pl = g.pl;
-    a.relu = relu; a.accumulate = accumulate;
+    a.relu = relu; a.accumulate = accumulate; a.nchw = nchw_in;
     const int pix = thin_pix(g);
     const int kpt = g.KB >= 2 ? 2 : 1;
     a.groups = ceil_div(g.OW, pix);

@@ -148,8 +148,17 @@ SMALL_API size_t small_net_workspace_bytes(const small_layer *layers, int n_laye
     return plan.total;
 }
 
+static int run_layers(small_ctx *ctx, const small_layer *layers, int n_layers, int from, int N,
+                      const float *in_blk, float *out_blk, void *workspace, size_t workspace_bytes, void *stream);
+
 SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
                             const float *in_blk, float *out_blk, void *workspace, size_t workspace_bytes, void *stream) {
+    return run_layers(ctx, layers, n_layers, 0, N, in_blk, out_blk, workspace, workspace_bytes, stream);
+}
+
+// Validates the whole list, then runs layers from .. n_layers - 1.
+static int run_layers(small_ctx *ctx, const small_layer *layers, int n_layers, int from, int N,
+                      const float *in_blk, float *out_blk, void *workspace, size_t workspace_bytes, void *stream) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     if (!layers || !in_blk || !out_blk) return SMALL_ERR_INVALID_ARG;
     if (!aligned16(in_blk) || !aligned16(out_blk) || (workspace && ((uintptr_t)workspace & 255u))) return SMALL_ERR_ALIGN;
@@ -217,7 +226,7 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
         return SMALL_ERR_INVALID_ARG;
     };
     bool after_join = false;
-    for (int i = 0; i < n_layers; ++i) {
+    for (int i = from; i < n_layers; ++i) {
         const small_layer &L = layers[i];
         int s = SMALL_OK;
         // every layer behind the first may start its set-up while the layer in front of it drains (see launch_kernel)
@@ -268,10 +277,15 @@ SMALL_API int small_run_net(small_ctx *ctx, const small_layer *layers, int n_lay
 
 SMALL_API size_t small_net_host_staging_bytes(int N, int C, int H, int W, int outC, int outH, int outW) {
     if (N < 1 || C < 1 || H < 1 || W < 1 || outC < 1 || outH < 1 || outW < 1) return 0;
-    return round256(sizeof(float) * (size_t)N * C * H * W) + round256(sizeof(float) * packed_elems(N, C, H, W)) +
+    return 2 * round256(sizeof(float) * (size_t)N * C * H * W) + round256(sizeof(float) * packed_elems(N, C, H, W)) +
            round256(sizeof(float) * packed_elems(N, outC, outH, outW)) + round256(sizeof(float) * (size_t)N * outC * outH * outW);
 }
 
+// The host-buffer call keeps the copy engine busy next to the SMs: the NCHW input goes to one of two staging areas on
+// the context's copy stream, so the copy of call i + 1 runs while the layers of call i are still computing on the caller's
+// stream; the caller's stream waits for its own input by an event, and a staging area is not overwritten before the
+// pack that read it last has finished.  Everything else (pack, layers, unpack, the result's copy back) stays in order on
+// the caller's stream.  While the caller's stream is being captured, the input copy stays on that stream.
 SMALL_API int small_run_net_host(small_ctx *ctx, const small_layer *layers, int n_layers, int N,
                                  const float *in_host, int C, int H, int W,
                                  float *out_host, int outC, int outH, int outW,
@@ -293,14 +307,63 @@ SMALL_API int small_run_net_host(small_ctx *ctx, const small_layer *layers, int 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char *p = static_cast<char *>(workspace) + net_b;
     size_t in_nchw_b = sizeof(float) * (size_t)N * C * H * W, out_nchw_b = sizeof(float) * (size_t)N * outC * outH * outW;
-    float *d_in_nchw = reinterpret_cast<float *>(p); p += round256(in_nchw_b);
+    float *d_in_nchw[2];
+    d_in_nchw[0] = reinterpret_cast<float *>(p); p += round256(in_nchw_b);
+    d_in_nchw[1] = reinterpret_cast<float *>(p); p += round256(in_nchw_b);
     float *d_in_blk = reinterpret_cast<float *>(p); p += round256(sizeof(float) * packed_elems(N, C, H, W));
     float *d_out_blk = reinterpret_cast<float *>(p); p += round256(sizeof(float) * packed_elems(N, outC, outH, outW));
     float *d_out_nchw = reinterpret_cast<float *>(p);
-    cudaError_t e = cudaMemcpyAsync(d_in_nchw, in_host, in_nchw_b, cudaMemcpyHostToDevice, st);
+    cudaError_t e = cudaSuccess;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(st, &cap);
+    const bool piped = ctx->copy_stream && cap == cudaStreamCaptureStatusNone;
+    int par = 0;
+    if (piped) {
+        if (ctx->host_ws != workspace) { ctx->host_ws = workspace; ctx->host_parity = 0; ctx->host_used[0] = ctx->host_used[1] = 0; }
+        par = ctx->host_parity;
+        cudaStream_t cs = static_cast<cudaStream_t>(ctx->copy_stream);
+        if (ctx->host_used[par]) e = cudaStreamWaitEvent(cs, static_cast<cudaEvent_t>(ctx->ev_pack[par]), 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d_in_nchw[par], in_host, in_nchw_b, cudaMemcpyHostToDevice, cs);
+        if (e == cudaSuccess) e = cudaEventRecord(static_cast<cudaEvent_t>(ctx->ev_h2d[par]), cs);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(ctx->ev_h2d[par]), 0);
+    } else {
+        e = cudaMemcpyAsync(d_in_nchw[0], in_host, in_nchw_b, cudaMemcpyHostToDevice, st);
+    }
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
-    if (int s = small_pack(ctx, d_in_nchw, d_in_blk, N, C, H, W, stream)) return s;
-    if (int s = small_run_net(ctx, layers, n_layers, N, d_in_blk, d_out_blk, workspace, net_b, stream)) return s;
+    // A first layer with at most four input channels (an image, a spectrogram) reads the NCHW tensor itself: its kernel
+    // gathers the real channels into shared memory either way, so the blocked copy of the input - 32 lanes for one to four
+    // channels - is never made.  The values and their order of summation are those of the blocked path.
+    int first = 0;
+    {
+        const small_layer &L0 = layers[0];
+        Geom g0;
+        bool later_reads_input = false;
+        for (int i = 1; i < n_layers; ++i)
+            if (layers[i].src == SMALL_SLOT_INPUT || (layers[i].op == SMALL_OP_ADD && layers[i].src2 == SMALL_SLOT_INPUT)) later_reads_input = true;
+        if (L0.op == SMALL_OP_CONV && L0.src == SMALL_SLOT_INPUT && L0.dst >= 0 && !(L0.flags & SMALL_ACCUMULATE) && !later_reads_input &&
+            n_layers > 1 && L0.C == C && L0.H == H && L0.W == W && L0.w_blk && aligned16(L0.w_blk) && (!L0.bias || aligned16(L0.bias)) &&
+            !(L0.flags & ~(SMALL_RELU | SMALL_MATH_MASK)) && !fused_pair(ctx, layers, n_layers, 0, N) &&
+            make_geom(g0, N, L0.C, L0.K, L0.H, L0.W, L0.FH, L0.FW, L0.stride, L0.pad_t, L0.pad_b, L0.pad_l, L0.pad_r) == SMALL_OK &&
+            conv_thin_supported(g0)) {
+            SlotPlan plan;
+            plan_slots(layers, n_layers, N, plan);
+            float *dst0 = reinterpret_cast<float *>(static_cast<char *>(workspace) + plan.offset[L0.dst]);
+            if (int s = launch_conv_thin(ctx, d_in_nchw[par], L0.w_blk, L0.bias, dst0, g0, L0.flags & SMALL_RELU, false, st, true)) return s;
+            first = 1;
+        }
+    }
+    if (!first)
+        if (int s = small_pack(ctx, d_in_nchw[par], d_in_blk, N, C, H, W, stream)) return s;
+    if (piped) {
+        e = cudaEventRecord(static_cast<cudaEvent_t>(ctx->ev_pack[par]), st);
+        if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }
+        ctx->host_used[par] = 1;
+        ctx->host_parity = par ^ 1;
+    }
+    if (first) {
+        // the rest of the list over the same slots: its plan must be the whole list's (slot sizes come from all layers)
+        if (int s = run_layers(ctx, layers, n_layers, 1, N, d_in_blk, d_out_blk, workspace, net_b, stream)) return s;
+    } else if (int s = small_run_net(ctx, layers, n_layers, N, d_in_blk, d_out_blk, workspace, net_b, stream)) return s;
     if (int s = small_unpack(ctx, d_out_blk, d_out_nchw, N, outC, outH, outW, stream)) return s;
     e = cudaMemcpyAsync(out_host, d_out_nchw, out_nchw_b, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }

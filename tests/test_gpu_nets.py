@@ -175,6 +175,16 @@ def test_run_net_host_end_to_end():
     # same result as the device-resident call
     got = from_blk(gnet.run(to_blk(x)), 8, 10, 1, 1)
     np.testing.assert_array_equal(got, out_host.numpy())
+    # back-to-back calls: the input copy of a call runs while the call before it computes, through two staging areas;
+    # every call must still see its own input (five calls: each staging area is reused)
+    xs = [configs.make_input(net, 8, seed=100 + i) for i in range(5)]
+    ins = [torch.from_numpy(a).pin_memory() for a in xs]
+    outs = [torch.full((8, 10, 1, 1), float("nan")).pin_memory() for _ in xs]
+    for a, o in zip(ins, outs):
+        gnet.run_host(a, o)
+    torch.cuda.synchronize()
+    for a, o in zip(xs, outs):
+        np.testing.assert_array_equal(o.numpy(), from_blk(gnet.run(to_blk(a)), 8, 10, 1, 1))
 
 
 def test_run_net_rejects_bad_workspace_and_descriptors():
