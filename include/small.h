@@ -315,6 +315,20 @@ int small_q_maxpool2d(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, in
 /* ReLU on uint8 (Table 2: Max with zero): out = max(in, z), real zero being the zero point z.  out may equal in. */
 int small_q_relu(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, int C, int H, int W, int z, void *stream);
 
+/* Abstract fused layer (Section 6) for a chain of full reductions, out = f_L(... f_1(in)), f_i(x) = act_i(W_i x + b_i):
+ * widths[0 .. L] are the channel counts (layer i maps widths[i] to widths[i+1]); w_blk[i] from small_pack_fc_weights(widths[i],
+ * widths[i+1], math); bias: NULL or L pointers (each NULL or widths[i+1] floats); relu[i] != 0 applies max(., 0) after layer i.
+ * in: blocked [N][widths[0]][1][1]; out: blocked [N][widths[L]][1][1], 32-byte aligned for the fused kernel.  flags: one
+ * SMALL_MATH_*.  Chains small_fc_chain_fused accepts (2 to 12 layers; widths[1 .. L-1] at most 128, widths[0] at most 8192,
+ * widths[L] at most 1024; a tensor-core math mode) run as ONE kernel: a thread block keeps 128 images' activations in shared
+ * memory as the tensor cores' operand from the first layer to the last, streams the filters (and the first layer's input
+ * where it is wider than 128), and writes only the final result.  Any other chain runs small_fc layer by layer
+ * through `scratch` (device, 2 * small_packed_elems(N, widest inner width, 1, 1) floats; may be NULL when the fused kernel runs
+ * or L == 1 - SMALL_ERR_WORKSPACE if it is needed and NULL).  All arrays are HOST arrays.  Errors as small_fc. */
+int small_fc_chain(small_ctx *ctx, const float *in, const float *const *w_blk, const float *const *bias, const int *widths,
+                   const int *relu, float *out, float *scratch, int L, int N, unsigned flags, void *stream);
+/* 1 if small_fc_chain runs this chain as one fused kernel under the given math mode, else 0. */
+int small_fc_chain_fused(const int *widths, int L, unsigned math);
 /* 1 if small_fc runs this layer on the tensor cores under the given math mode, else 0. */
 int small_fc_uses_tensor_cores(int N, int J, int K, unsigned math);
 
@@ -348,10 +362,11 @@ typedef struct small_layer {
  * reads that slot before it is written again), the pair's output slot differs from its input slot, and the fused kernel
  * takes the shape: a depthwise 3x3 and the 1x1 convolution behind it under a tensor-core math mode (SMALL_FUSE_DWPW: only
  * where the intermediate tensor is at most 24 MB, where fusing was measured to pay; SMALL_FUSE_DWPW_ALWAYS: wherever the
- * kernel takes the shape), and a convolution and the 2x2 stride-2 max pool behind it (SMALL_FUSE_CONVPOOL).  The skipped
- * intermediate tensor is then not written.  Default: SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL; 0 runs every layer on its own.
+ * kernel takes the shape), a convolution and the 2x2 stride-2 max pool behind it (SMALL_FUSE_CONVPOOL), and a run of 2 to 12
+ * full reductions whose inner widths are at most 128 under a tensor-core math mode (SMALL_FUSE_FC_CHAIN, see small_fc_chain).  The skipped
+ * intermediate tensors are then not written.  Default: all three; 0 runs every layer on its own.
  * Results stay within each math mode's tolerance either way. */
-enum { SMALL_FUSE_DWPW = 1u, SMALL_FUSE_DWPW_ALWAYS = 2u, SMALL_FUSE_CONVPOOL = 4u };
+enum { SMALL_FUSE_DWPW = 1u, SMALL_FUSE_DWPW_ALWAYS = 2u, SMALL_FUSE_CONVPOOL = 4u, SMALL_FUSE_FC_CHAIN = 8u };
 int small_set_net_fusion(small_ctx *ctx, unsigned mask);
 /* Number of kernel launches small_run_net makes for these layers at batch N under the context's fusion setting (one per
  * layer or fused pair); -1 for invalid arguments. */

@@ -28,7 +28,7 @@ EXPORTS = [
     "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_set_branch_overlap", "small_conv2d_path", "small_set_wait_limit", "small_selftest_wait_timeout", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_conv_maxpool2d", "small_conv_maxpool_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
-    "small_pack_fc_weights", "small_fc_uses_tensor_cores", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
+    "small_pack_fc_weights", "small_fc_uses_tensor_cores", "small_fc_chain", "small_fc_chain_fused", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
     "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net", "small_set_net_fusion", "small_net_launches",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
     "small_q_packed_bytes", "small_q_pack", "small_q_unpack", "small_q_conv_weight_bytes", "small_q_pack_conv_weights", "small_q_conv2d",
@@ -101,6 +101,8 @@ def lib():
     L.small_fc_weight_elems.restype = Z
     L.small_pack_fc_weights.argtypes = [P, P, P, I, I, U, P]
     L.small_fc_uses_tensor_cores.argtypes = [I, I, I, U]
+    L.small_fc_chain.argtypes = [P, P, ctypes.POINTER(P), ctypes.POINTER(P), ctypes.POINTER(I), ctypes.POINTER(I), P, P, I, I, U, P]
+    L.small_fc_chain_fused.argtypes = [ctypes.POINTER(I), I, U]
     L.small_conv2d.argtypes = [P, P, P, P, P] + [I] * 12 + [U, P]
     L.small_conv2d_uses_tensor_cores.argtypes = [I] * 12
     L.small_dwconv2d.argtypes = [P, P, P, P, P] + [I] * 11 + [U, P]
@@ -248,6 +250,20 @@ def small_fc_weight_elems(J, K, math=MATH_FP32):
     return lib().small_fc_weight_elems(J, K, math)
 
 
+def small_fc_chain(ctx, inp, w_blks, biases, widths, relu, out, scratch, N, flags=0, stream=None):
+    L = len(w_blks)
+    wp = (ctypes.c_void_p * L)(*[_ptr(w) for w in w_blks])
+    bp = (ctypes.c_void_p * L)(*[_ptr(b) for b in biases]) if biases is not None else None
+    wd = (ctypes.c_int * (L + 1))(*widths)
+    rl = (ctypes.c_int * L)(*[1 if r else 0 for r in relu])
+    _check(lib().small_fc_chain(ctx, _ptr(inp), wp, bp, wd, rl, _ptr(out), _ptr(scratch), L, N, flags, _stream(stream)), "small_fc_chain")
+
+
+def small_fc_chain_fused(widths, math):
+    wd = (ctypes.c_int * len(widths))(*widths)
+    return bool(lib().small_fc_chain_fused(wd, len(widths) - 1, math))
+
+
 def small_fc_uses_tensor_cores(N, J, K, math):
     return bool(lib().small_fc_uses_tensor_cores(N, J, K, math))
 
@@ -340,8 +356,8 @@ def small_fc(ctx, inp, w_blk, bias, out, N, J, K, flags=0, stream=None):
     _check(lib().small_fc(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, J, K, flags, _stream(stream)), "small_fc")
 
 
-FUSE_DWPW, FUSE_DWPW_ALWAYS, FUSE_CONVPOOL = 1, 2, 4
-FUSE_DEFAULT = FUSE_DWPW | FUSE_CONVPOOL
+FUSE_DWPW, FUSE_DWPW_ALWAYS, FUSE_CONVPOOL, FUSE_FC_CHAIN = 1, 2, 4, 8
+FUSE_DEFAULT = FUSE_DWPW | FUSE_CONVPOOL | FUSE_FC_CHAIN
 
 
 def small_set_net_fusion(ctx, mask):

@@ -111,7 +111,7 @@ SMALL_API int small_init(int device, small_ctx **out) {
     c->overlap = 1;
     c->dependent = 0;
     c->conv_path = SMALL_CONV_PATH_AUTO;
-    c->net_fusion = SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL;
+    c->net_fusion = SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL | SMALL_FUSE_FC_CHAIN;
     c->branch_overlap = 1;
     c->side_stream = c->ev_fork = c->ev_join = nullptr;
     {
@@ -584,4 +584,46 @@ SMALL_API int small_fc(small_ctx *ctx, const float *in, const float *w, const fl
         return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, flags & SMALL_RELU, false, math, st);
     }
     return launch_fc(ctx, in, w, bias, out, N, J, K, flags & SMALL_RELU, st);
+}
+
+// ---- a chain of full reductions as one fused kernel
+SMALL_API int small_fc_chain_fused(const int *widths, int L, unsigned math) {
+    if (!widths) return 0;
+    return fc_chain_supported(widths, L, math) ? 1 : 0;
+}
+
+SMALL_API int small_fc_chain(small_ctx *ctx, const float *in, const float *const *w_blk, const float *const *bias, const int *widths,
+                             const int *relu, float *out, float *scratch, int L, int N, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~SMALL_MATH_MASK) return SMALL_ERR_INVALID_ARG;
+    const unsigned math = math_of(flags);
+    if (!math_valid(math) || !w_blk || !widths || !relu || L < 1 || L > 64) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, out}, {scratch})) return s;
+    if (N < 1) return SMALL_ERR_SHAPE;
+    int widest = 0;
+    for (int i = 0; i <= L; ++i) {
+        if (widths[i] < 1) return SMALL_ERR_SHAPE;
+        if (i > 0 && i < L && widths[i] > widest) widest = widths[i];
+    }
+    for (int l = 0; l < L; ++l) {
+        if (!w_blk[l]) return SMALL_ERR_INVALID_ARG;
+        if (!aligned16(w_blk[l]) || (bias && bias[l] && !aligned16(bias[l]))) return SMALL_ERR_ALIGN;
+    }
+    const size_t in_b = sizeof(float) * packed_elems(N, widths[0], 1, 1), out_b = sizeof(float) * packed_elems(N, widths[L], 1, 1);
+    if (ranges_overlap(in, in_b, out, out_b)) return SMALL_ERR_OVERLAP;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (fc_chain_supported(widths, L, math) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0 && ctx->conv_path != SMALL_CONV_PATH_CUDA_CORES)
+        return launch_fc_chain(ctx, in, w_blk, bias, widths, relu, out, L, N, math, st);
+    // layer by layer, through the two halves of the caller's scratch tensor
+    if (L == 1) return small_fc(ctx, in, w_blk[0], bias ? bias[0] : nullptr, out, N, widths[0], widths[1], (relu[0] ? SMALL_RELU : 0u) | math, stream);
+    if (!scratch) return SMALL_ERR_WORKSPACE;
+    const size_t half = packed_elems(N, widest, 1, 1);
+    if (ranges_overlap(scratch, 2 * half * sizeof(float), in, in_b) || ranges_overlap(scratch, 2 * half * sizeof(float), out, out_b)) return SMALL_ERR_OVERLAP;
+    const float *src = in;
+    for (int l = 0; l < L; ++l) {
+        float *dst = l == L - 1 ? out : scratch + (size_t)(l & 1) * half;
+        if (int s = small_fc(ctx, src, w_blk[l], bias ? bias[l] : nullptr, dst, N, widths[l], widths[l + 1], (relu[l] ? SMALL_RELU : 0u) | math, stream)) return s;
+        src = dst;
+    }
+    return SMALL_OK;
 }

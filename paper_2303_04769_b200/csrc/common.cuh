@@ -119,6 +119,10 @@ int launch_conv_direct(small_ctx *, const float *in, const float *w, const float
 // the same kernel with a 2 x 2 stride-2 max pool taken in its STORE phase: out is [N][K][OH/2][OW/2]
 bool conv_direct_pool_supported(const Geom &);
 int launch_conv_direct_pool(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
+// a run of 2 to 8 full reductions of width <= 128 as one tensor-core kernel (fc_chain.cu); widths has L + 1 entries
+bool fc_chain_supported(const int *widths, int L, unsigned math);
+int launch_fc_chain(small_ctx *, const float *in, const float *const *w_blk, const float *const *bias, const int *widths,
+                    const int *relu, float *out, int L, int N, unsigned math, cudaStream_t);
 // at most four input channels, 3 x 3 (strides 1, 2) or the 10 x 4 stride-2 window: FP32 FMAs with the filters in registers
 bool conv_thin_supported(const Geom &);
 // nchw_in: `in` is the NCHW tensor float[N][C][H][W] instead of the blocked one (used at a network's edge)

@@ -123,13 +123,35 @@ static int fused_pair(const small_ctx *ctx, const small_layer *layers, int n_lay
     return 0;
 }
 
+// Length of the run of full reductions starting at layer i that runs as one fused kernel (0: none): each layer reads what
+// the one before it wrote, nothing else reads those intermediates, every width between two layers is at most 128, one
+// tensor-core math mode.
+static int fc_chain_len(const small_ctx *ctx, const small_layer *layers, int n_layers, int i, int N, int *widths) {
+    if (!(ctx->net_fusion & SMALL_FUSE_FC_CHAIN) || layers[i].op != SMALL_OP_FC) return 0;
+    const unsigned math = layers[i].flags & SMALL_MATH_MASK;
+    if (math != SMALL_MATH_TF32 && math != SMALL_MATH_3XTF32) return 0;
+    if (layers[i].C > 8192 || layers[i].K > 128) return 0;       // the first layer's input may be wide, and the last one's output
+    int L = 1;
+    widths[0] = layers[i].C; widths[1] = layers[i].K;
+    while (i + L < n_layers && L < 12) {
+        const small_layer &P = layers[i + L - 1], &Q = layers[i + L];
+        if (Q.op != SMALL_OP_FC || Q.src != P.dst || P.dst < 0 || (Q.flags & SMALL_MATH_MASK) != math || Q.C != P.K || Q.K > 1024 || P.K > 128) break;
+        if (!slot_dead_after(layers, n_layers, i + L + 1, P.dst)) break;
+        if (Q.dst == layers[i].src) break;                      // the run's output must not land on its input
+        widths[L + 1] = Q.K;
+        ++L;
+    }
+    (void)N;
+    return L >= 2 ? L : 0;
+}
+
 }  // namespace small
 
 using namespace small;
 
 SMALL_API int small_set_net_fusion(small_ctx *ctx, unsigned mask) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
-    if (mask & ~(unsigned)(SMALL_FUSE_DWPW | SMALL_FUSE_DWPW_ALWAYS | SMALL_FUSE_CONVPOOL)) return SMALL_ERR_INVALID_ARG;
+    if (mask & ~(unsigned)(SMALL_FUSE_DWPW | SMALL_FUSE_DWPW_ALWAYS | SMALL_FUSE_CONVPOOL | SMALL_FUSE_FC_CHAIN)) return SMALL_ERR_INVALID_ARG;
     ctx->net_fusion = mask;
     return SMALL_OK;
 }
@@ -137,8 +159,11 @@ SMALL_API int small_set_net_fusion(small_ctx *ctx, unsigned mask) {
 SMALL_API int small_net_launches(small_ctx *ctx, const small_layer *layers, int n_layers, int N) {
     if (!ctx || !layers || n_layers < 1 || N < 1) return -1;
     int launches = 0;
-    for (int i = 0; i < n_layers; ++i, ++launches)
-        if (fused_pair(ctx, layers, n_layers, i, N)) ++i;
+    for (int i = 0; i < n_layers; ++i, ++launches) {
+        int widths[13];
+        if (const int L = fc_chain_len(ctx, layers, n_layers, i, N, widths)) i += L - 1;
+        else if (fused_pair(ctx, layers, n_layers, i, N)) ++i;
+    }
     return launches;
 }
 
@@ -232,6 +257,22 @@ static int run_layers(small_ctx *ctx, const small_layer *layers, int n_layers, i
         // every layer behind the first may start its set-up while the layer in front of it drains (see launch_kernel)
         ctx->dependent = ctx->overlap && i > 0 && !after_join;
         after_join = false;
+        {
+            int widths[13];
+            if (const int Lc = fc_chain_len(ctx, layers, n_layers, i, N, widths)) {
+                const float *w[12], *b[12];
+                int relu[12];
+                for (int j = 0; j < Lc; ++j) { w[j] = layers[i + j].w_blk; b[j] = layers[i + j].bias; relu[j] = (layers[i + j].flags & SMALL_RELU) ? 1 : 0; }
+                float *dst = wr(layers[i + Lc - 1].dst);
+                if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+                    s = launch_fc_chain(ctx, rd(L.src), w, b, widths, relu, dst, Lc, N, L.flags & SMALL_MATH_MASK, static_cast<cudaStream_t>(stream));
+                    ctx->dependent = 0;
+                    if (s != SMALL_OK) return s;
+                    i += Lc - 1;
+                    continue;
+                }
+            }
+        }
         if (const int fused = fused_pair(ctx, layers, n_layers, i, N)) {
             const small_layer &Nx = layers[i + 1];
             if (fused == SMALL_OP_DWPW) {

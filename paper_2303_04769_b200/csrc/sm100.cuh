@@ -43,6 +43,11 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
@@ -54,11 +59,13 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 // Bounded wait.  Returns false when the limit ran out or another role already gave up (abort flag set).  After a few
 // immediate retries the poll backs off with nanosleep so that waiting roles leave shared-memory bandwidth to the
-// tensor core, which reads its operands from the same shared memory.
+// tensor core, which reads its operands from the same shared memory.  kFast = polls before the back-off starts: a role
+// on the critical path of a latency-bound kernel takes a large value and so wakes without the sleep's delay.
+template <uint32_t kFast = 4>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, uint32_t limit) {
     for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it >= 4) __nanosleep(it < 64 ? 40 : 400);
+        if (it >= kFast) __nanosleep(it < kFast + 60 ? 40 : 400);
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -66,9 +73,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 // One lane waits for the whole warp (all 32 lanes must call this together).
+template <uint32_t kFast = 4>
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, uint32_t limit) {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, limit) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait<kFast>(bar, parity, abort_flag, status, limit) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 

@@ -157,7 +157,7 @@ def test_the_runner_fuses_plain_descriptors_itself():
     # a full reduction under a tensor-core mode is routed by the library, not by the caller
     assert B.small_fc_uses_tensor_cores(4096, 128, 128, B.MATH_TF32) and not B.small_fc_uses_tensor_cores(256, 64, 10, B.MATH_TF32)
     with pytest.raises(B.SmallError):
-        B.small_set_net_fusion(c, 8)
+        B.small_set_net_fusion(c, 16)
     assert B.small_device_status(c) == 0
 
 
