@@ -320,13 +320,18 @@ int small_q_relu(small_ctx *ctx, const uint8_t *in, uint8_t *out, int N, int C, 
  * widths[i+1], math); bias: NULL or L pointers (each NULL or widths[i+1] floats); relu[i] != 0 applies max(., 0) after layer i.
  * in: blocked [N][widths[0]][1][1]; out: blocked [N][widths[L]][1][1], 32-byte aligned for the fused kernel.  flags: one
  * SMALL_MATH_*.  Chains small_fc_chain_fused accepts (2 to 12 layers; widths[1 .. L-1] at most 128, widths[0] at most 8192,
- * widths[L] at most 1024; a tensor-core math mode) run as ONE kernel: a thread block keeps 128 images' activations in shared
+ * widths[L] at most 1024; a tensor-core math mode) run as ONE kernel: a thread block keeps a tile of images' activations in shared
  * memory as the tensor cores' operand from the first layer to the last, streams the filters (and the first layer's input
  * where it is wider than 128), and writes only the final result.  Any other chain runs small_fc layer by layer
  * through `scratch` (device, 2 * small_packed_elems(N, widest inner width, 1, 1) floats; may be NULL when the fused kernel runs
  * or L == 1 - SMALL_ERR_WORKSPACE if it is needed and NULL).  All arrays are HOST arrays.  Errors as small_fc. */
 int small_fc_chain(small_ctx *ctx, const float *in, const float *const *w_blk, const float *const *bias, const int *widths,
                    const int *relu, float *out, float *scratch, int L, int N, unsigned flags, void *stream);
+/* Images per thread block of the fused kernel: 0 (default) chooses by batch size - 32 while that gives every SM at most
+ * one tile, then 64, then 128 (larger tiles stream the filters fewer times, smaller ones occupy more SMs); 32, 64 or 128
+ * force one (a tile whose shared memory does not fit - a wide first layer with the larger tiles - is halved).
+ * SMALL_ERR_INVALID_ARG for any other value.  Results do not depend on the choice. */
+int small_set_fc_chain_tile(small_ctx *ctx, int images);
 /* 1 if small_fc_chain runs this chain as one fused kernel under the given math mode, else 0. */
 int small_fc_chain_fused(const int *widths, int L, unsigned math);
 /* 1 if small_fc runs this layer on the tensor cores under the given math mode, else 0. */

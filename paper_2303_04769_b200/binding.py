@@ -25,7 +25,7 @@ MATH = {"fp32": MATH_FP32, "tf32": MATH_TF32, "3xtf32": MATH_3XTF32}
 
 EXPORTS = [
     "small_init", "small_shutdown", "small_channel_block", "small_packed_elems", "small_out_size", "small_strerror",
-    "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_set_branch_overlap", "small_conv2d_path", "small_set_wait_limit", "small_selftest_wait_timeout", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
+    "small_last_cuda_error", "small_set_layer_overlap", "small_set_conv_path", "small_set_branch_overlap", "small_conv2d_path", "small_set_wait_limit", "small_set_fc_chain_tile", "small_selftest_wait_timeout", "small_device_status", "small_measure_tf32_peak", "small_pack", "small_unpack", "small_conv_weight_elems",
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_conv_maxpool2d", "small_conv_maxpool_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_fc_uses_tensor_cores", "small_fc_chain", "small_fc_chain_fused", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
@@ -78,6 +78,7 @@ def lib():
     L.small_set_conv_path.argtypes = [P, I]
     L.small_set_branch_overlap.argtypes = [P, I]
     L.small_set_wait_limit.argtypes = [P, U]
+    L.small_set_fc_chain_tile.argtypes = [P, I]
     L.small_selftest_wait_timeout.argtypes = [P, P]
     L.small_conv2d_path.argtypes = [P] + [I] * 12 + [U]
     L.small_pack.argtypes = [P, P, P, I, I, I, I, P]
@@ -201,6 +202,10 @@ def small_set_conv_path(ctx, path):
 
 def small_set_branch_overlap(ctx, on):
     _check(lib().small_set_branch_overlap(ctx, 1 if on else 0), "small_set_branch_overlap")
+
+
+def small_set_fc_chain_tile(ctx, images):
+    _check(lib().small_set_fc_chain_tile(ctx, images), "small_set_fc_chain_tile")
 
 
 def small_set_wait_limit(ctx, polls):

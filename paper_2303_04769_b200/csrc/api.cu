@@ -167,6 +167,13 @@ SMALL_API int small_set_wait_limit(small_ctx *ctx, unsigned polls) {
     return SMALL_OK;
 }
 
+SMALL_API int small_set_fc_chain_tile(small_ctx *ctx, int images) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (images != 0 && images != 32 && images != 64 && images != 128) return SMALL_ERR_INVALID_ARG;
+    ctx->fc_chain_tile = images;
+    return SMALL_OK;
+}
+
 SMALL_API int small_set_branch_overlap(small_ctx *ctx, int on) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
     ctx->branch_overlap = (on && ctx->side_stream && ctx->ev_fork && ctx->ev_join) ? 1 : 0;

@@ -28,6 +28,7 @@ struct small_ctx {
     void *host_ws; int host_parity, host_used[2];
     unsigned net_fusion;     // SMALL_FUSE_*: which neighbouring layers small_run_net runs as one fused layer
     int conv_path;           // SMALL_CONV_PATH_*: automatic, or one kernel family forced where it takes the shape
+    int fc_chain_tile;       // images per thread block of the fused chain of full reductions: 0 = by batch size, else 32, 64 or 128
 };
 
 namespace small {

@@ -28,6 +28,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Non-blocking poll.  try_wait may suspend the thread when the phase is not complete yet, and a suspended thread was
+// measured to come back long after the phase completes (up to the suspension's time limit, about 1.5 us); a spin on
+// test_wait sees the completion within some tens of cycles.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: false when `limit` polls (seconds at the default, with the nanosleep back-off) ran out; the caller
 // records the timeout.
 constexpr uint32_t kDefaultWaitIters = 1u << 22;
@@ -64,7 +76,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 template <uint32_t kFast = 4>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, uint32_t limit) {
     for (uint32_t it = 0; it < limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (kFast > 4 && it < kFast ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if (it >= kFast) __nanosleep(it < kFast + 60 ? 40 : 400);
         if ((it & 63u) == 63u && *abort_flag) return false;
     }

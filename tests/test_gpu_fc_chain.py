@@ -98,3 +98,40 @@ def test_fc_chain_falls_back_and_rejects():
     scratch = torch.empty(2 * B.small_packed_elems(N, 256, 1, 1), device="cuda")
     B.small_fc_chain(ctx(), to_blk(x), wbs, [dev(b) for b in bs], widths, [True, False], out, scratch, N, B.MATH_3XTF32)
     assert rel_err(from_blk(out, N, 128, 1, 1).reshape(N, 128), ref) <= 1e-5
+
+
+@pytest.mark.parametrize("math", ["tf32", "3xtf32"])
+def test_fc_chain_tile_sizes_agree(math):
+    """Every tile size gives the same bits, on a batch that gives the thread blocks of the smallest tile several tiles
+    each (the slots and accumulators are then reused across tiles) and ends in a ragged tile."""
+    widths, N = [200, 128, 16, 300], 32 * 148 * 2 + 37
+    L = len(widths) - 1
+    ws, bs = chain_params(widths, 79)
+    relu = [True, True, False]
+    x = synth.normal((N, widths[0], 1, 1), 0.0, 1.0, 297, 79)
+    ref = x.reshape(N, widths[0])
+    for w, b, r in zip(ws, bs, relu):
+        ref = oracle.fc(ref, w, b, relu=r)
+    wbs = []
+    for i, w in enumerate(ws):
+        wb = torch.empty(B.small_fc_weight_elems(widths[i], widths[i + 1], B.MATH[math]), device="cuda")
+        B.small_pack_fc_weights(ctx(), dev(w), wb, widths[i], widths[i + 1], B.MATH[math])
+        wbs.append(wb)
+    dbs = [dev(b) for b in bs]
+    bx = to_blk(x)
+    outs = []
+    try:
+        for tile in (32, 64, 128, 0):
+            B.small_set_fc_chain_tile(ctx(), tile)
+            out = new_blk(N, widths[-1], 1, 1)
+            B.small_fc_chain(ctx(), bx, wbs, dbs, widths, relu, out, None, N, B.MATH[math])
+            assert B.small_device_status(ctx()) == 0
+            outs.append(out)
+    finally:
+        B.small_set_fc_chain_tile(ctx(), 0)
+    assert rel_err(from_blk(outs[0], N, widths[-1], 1, 1).reshape(N, widths[-1]), ref) <= 2.5 * TOL[math]
+    assert pad_lanes_are_zero(outs[0], N, widths[-1], 1, 1)
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int32), outs[0].view(torch.int32))
+    with pytest.raises(B.SmallError):
+        B.small_set_fc_chain_tile(ctx(), 48)
