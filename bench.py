@@ -34,10 +34,10 @@ TOL = {"fp32": 1e-5, "tf32": 2e-3, "3xtf32": 1e-5}
 # this file's network step, averaged over the kernel's launches in one step).  It is reported only while the kernel's
 # source still has the hash it had when the counters were taken.
 TRAFFIC = {
-    "conv_3xtf32_tensor": {"bytes_per_launch": 22471040.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                           "sha256": "3788f28a029a03005913b9f8e2f18eb4681d617500595f75edd934977a8ef8f7"},
-    "conv_tf32_tensor": {"bytes_per_launch": 22413408.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
-                         "sha256": "3788f28a029a03005913b9f8e2f18eb4681d617500595f75edd934977a8ef8f7"},
+    "conv_3xtf32_tensor": {"bytes_per_launch": 22910037.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                           "sha256": "46edea15c263baabda86068dc7269c4601c27973edc2dd8509505bfd06924f4c"},
+    "conv_tf32_tensor": {"bytes_per_launch": 24391387.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
+                         "sha256": "46edea15c263baabda86068dc7269c4601c27973edc2dd8509505bfd06924f4c"},
 }
 
 
@@ -677,6 +677,38 @@ def run_sweep(ctx, B, torch, dev, peaks, sm_count, time_launch, tf32_probe_tflop
             "rows": rows}
 
 
+def single_network(args, ctx, dev, name, batch):
+    """One of the small networks, a few graph-replayed steps, for profiler captures of its kernels."""
+    import torch
+    from paper_2303_04769_b200 import binding as B
+    from paper_2303_04769_b200.net import Net
+    net = configs.NETWORKS[name]()
+    N = batch or net["batch"]
+    params = configs.make_params(net)
+    x = torch.from_numpy(configs.make_input(net, N)).to(dev)
+    blk = torch.empty(B.small_packed_elems(N, *net["input"]), device=dev)
+    B.small_pack(ctx, x, blk, N, *net["input"])
+    gnet = Net(ctx, net, params, batch=N, math=args.math, device=dev)
+    gnet.run(blk)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        gnet.run(blk)
+    ts = []
+    for i in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        e1.synchronize()
+        if i >= args.warmup:
+            ts.append(e0.elapsed_time(e1))
+    t = statistics.median(ts)
+    flops = sum(2.0 * N * L["C"] * L["K"] for L in net["layers"])
+    print(json.dumps({"network": name, "batch": N, "math": args.math, "launches": gnet.launches(), "us_med": t * 1e3, "us_min": min(ts) * 1e3,
+                      "gflops": flops / t / 1e6, "device_status": B.small_device_status(ctx)}))
+
+
 def single_layer(args):
     """--layer KIND:C:HW[:BATCH]: one sweep layer, a few launches, for profiler captures (ncu -k ... -c ...)."""
     import torch
@@ -687,6 +719,8 @@ def single_layer(args):
     N = int(parts[3]) if len(parts) > 3 else configs.SWEEP_BATCH
     dev = torch.device("cuda", 0)
     ctx = B.small_init(0)
+    if kind == "autoencoder":                  # the fully-connected autoencoder as the runner launches it (C, HW ignored)
+        return single_network(args, ctx, dev, "autoencoder_fc", N if len(parts) > 3 else None)
     elems = B.small_packed_elems(N, C, HW, HW)
     x = torch.empty(elems, device=dev)
     B.small_pack(ctx, torch.from_numpy(synth.uniform((N, C, HW, HW), -1.0, 1.0, 500 + C)).to(dev), x, N, C, HW, HW)
