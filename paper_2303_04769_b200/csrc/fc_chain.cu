@@ -7,10 +7,13 @@
 //                 TMA through a ring of stages (3xTF32: the TF32 part and, 16 KB on, the residual); rows past the layer's
 //                 filter count hold whatever the stage held before and only feed accumulator lanes nobody reads
 //   B operand   = the tile's activations [nt images][32 channels] per channel block, K-major with the 128-byte swizzle,
-//                 resident in shared memory slots 0 .. 3 (3xTF32: the residuals in a second area); the first layer's
-//                 input, which may be wider than 128 channels, streams through all the slots (slot = block mod slots)
+//                 resident in shared memory slots 0 .. 3 (3xTF32: each block's residual rows right behind its TF32 rows);
+//                 the first layer's input, which may be wider than 128 channels, streams through all the slots
 //   accumulator = 128 lanes (filters) x nt columns (images) of tensor memory, 256 / nt of them in rotation, so that a
-//                 last layer wider than 128 filters runs its chunks of 128 back to back while the epilogue drains them
+//                 last layer wider than 128 filters runs its chunks of 128 back to back while the epilogue drains them.
+//                 3xTF32 takes two MMAs per K step for its three products: w_hi against the 2 nt rows [x_hi; x_lo]
+//                 (columns [0, nt) and [nt, 2 nt) of a 2 nt wide accumulator), then w_lo against x_hi into columns
+//                 [0, nt); the epilogue adds the two halves
 //   epilogue    = thread = filter: tensor memory -> registers, + bias, ReLU, and the filter's nt values go straight back
 //                 into the B slots as the next layer's operand (for 3xTF32 split into TF32 part and residual); the last
 //                 layer's values go to global memory, a warp writing one image's 32-channel line per store
@@ -88,8 +91,10 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
     constexpr uint32_t kWStage = X3 ? 2 * kWBlock : kWBlock;
     const int nt = a.nt, n_slots = a.n_slots;
-    const uint32_t slot_bytes = (uint32_t)nt * 128u, x_half = (uint32_t)n_slots * slot_bytes;
-    const uint32_t x_base = base, w_base = base + (X3 ? 2u : 1u) * x_half;
+    // a slot: the tile's nt rows of one channel block; 3xTF32: the residuals' nt rows right behind them, so that one
+    // descriptor of 2 nt rows covers both
+    const uint32_t slot_bytes = (uint32_t)nt * 128u, slot_pitch = X3 ? 2u * slot_bytes : slot_bytes;
+    const uint32_t x_base = base, w_base = base + (uint32_t)n_slots * slot_pitch;
     const uint32_t ctrl = w_base + (uint32_t)a.w_stages * kWStage;
     uint8_t *ctrl_ptr = base_ptr + (ctrl - base);
     const uint32_t bar_w_full = ctrl + kOffWFull, bar_w_empty = ctrl + kOffWEmpty, bar_in = ctrl + kOffInFull, bar_split = ctrl + kOffSplit,
@@ -104,7 +109,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
     const int JB0 = (a.J[0] + 31) >> 5;
     // the last layer may have more than 128 filters: it runs as chunks of 128, each one more pass over the same operand
     const int last_chunks = (a.K[a.L - 1] + 127) >> 7, steps_per_tile = a.L - 1 + last_chunks;
-    const uint32_t nacc_log2 = nt == 32 ? 3u : nt == 64 ? 2u : 1u, nacc = 1u << nacc_log2;     // accumulators in rotation: 256 / nt
+    // accumulators in rotation: 256 columns / (nt, or 2 nt for 3xTF32, whose x_lo products land in a second set of columns)
+    const uint32_t acc_cols = X3 ? 2u * (uint32_t)nt : (uint32_t)nt;
+    const uint32_t nacc_log2 = (nt == 32 ? 3u : nt == 64 ? 2u : 1u) - (X3 ? 1u : 0u), nacc = 1u << nacc_log2;
     // slots, stages and stages per commit are powers of two
     const int ns_log2 = 31 - __clz(n_slots);
     const uint32_t ws_log2 = 31 - __clz(a.w_stages), rel_log2 = 31 - __clz(a.release);
@@ -113,7 +120,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
     auto slot_uses = [&](int slot) -> uint32_t { return slot < JB0 ? (uint32_t)((JB0 - 1 - slot) >> ns_log2) + 1u : 0u; };
     auto group_uses = [&](int sg) -> uint32_t { return 4 * sg < JB0 ? (uint32_t)((JB0 - 1 - 4 * sg) >> ns_log2) + 1u : 0u; };
 
-    if (threadIdx.x == 0) {
+    // Set-up.  TF32: in two halves that meet at named barrier 1 - warp 1 initialises the barriers, arrives and goes straight
+    // to its loads; the other warps fill the bias table, allocate tensor memory and wait there for the barriers to exist
+    // (measured on the ten-layer chain: 39.6 -> 37.8 us).  3xTF32 keeps one block-wide barrier after the set-up: the same
+    // change measured slower there (52.5 -> 57.8 us).
+    if (threadIdx.x == 32) {
         for (int s = 0; s < 8; ++s) {
             mbar_init(bar_w_full + 8 * s, 1); mbar_init(bar_w_empty + 8 * s, 1);
             mbar_init(bar_acc + 8 * s, 1); mbar_init(bar_epi + 8 * s, n_epi_warps);
@@ -125,16 +136,24 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
         *steps_done = 0;
         mbar_fence_init();
     }
-    // filters and biases are no layer's output: they are read ahead of the wait on the launch before this one
-    for (int i = threadIdx.x; i < steps_per_tile * 128; i += blockDim.x) {
-        const int l = min(i >> 7, a.L - 1), k = i - l * 128;
-        bias_s[i] = (a.bias[l] && k < a.K[l]) ? a.bias[l][k] : 0.0f;
+    uint32_t tmem = 0;
+    if (warp == 1 && !X3) {
+        __syncwarp();
+        asm volatile("bar.arrive 1, %0;" ::"r"(blockDim.x) : "memory");
+    } else {
+        // filters and biases are no layer's output: they are read ahead of the wait on the launch before this one
+        const int fillers = X3 ? blockDim.x : blockDim.x - 32;            // every thread, or every thread but warp 1's
+        for (int i = threadIdx.x - (!X3 && warp > 1 ? 32 : 0); i < steps_per_tile * 128; i += fillers) {
+            const int l = min(i >> 7, a.L - 1), k = i - l * 128;
+            bias_s[i] = (a.bias[l] && k < a.K[l]) ? a.bias[l][k] : 0.0f;
+        }
+        if (warp == 0) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), (uint32_t)kTmemCols);
+        tc_fence_before();
+        if (X3) __syncthreads();
+        else asm volatile("bar.sync 1, %0;" ::"r"(blockDim.x) : "memory");
+        tc_fence_after();
+        tmem = *tmem_slot;
     }
-    if (warp == 0) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), (uint32_t)kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
     grid_dep_trigger();
 
     // copies a producer lane started and the parity of each barrier's latest one, kept for the drain after an abort
@@ -177,7 +196,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
                     if (!alive) return;
                     if (!synced) { grid_dep_sync(); synced = true; }
                     mbar_expect_tx(bar_in + 8 * slot, slot_bytes);
-                    tma_load_3d(x_base + slot * slot_bytes, &a.map_in, bar_in + 8 * slot, 0, cb, t * nt);
+                    tma_load_3d(x_base + slot * slot_pitch, &a.map_in, bar_in + 8 * slot, 0, cb, t * nt);
                     in_mask |= 1u << slot;
                     in_par = (in_par & ~(1u << slot)) | ((use & 1u) << slot);
                 }
@@ -199,9 +218,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
         // count is the chain's critical path: descriptors and counters advance by addition, a layer's polls start together.
         bool alive = true;
         uint32_t g = 0, tile_k = 0;                        // g: steps so far; accumulator and its barriers = g mod nacc
-        const uint32_t idesc = instr_desc(nt);
+        const uint32_t idesc = instr_desc(nt), idesc_wide = instr_desc(2 * nt);
         const uint32_t w_desc0 = smem_desc_lo(w_base), x_desc0 = smem_desc_lo(x_base);
-        const uint32_t w_step = kWStage >> 4, x_step = slot_bytes >> 4, x_lo = x_half >> 4, w_lo = kWBlock >> 4;
+        const uint32_t w_step = kWStage >> 4, x_step = slot_pitch >> 4, w_lo = kWBlock >> 4;
         uint32_t sw = 0, pw = 0, wa = w_desc0;             // filter stage in turn, its parity, its descriptor
         uint32_t rel_left = (uint32_t)a.release, rel_bar = bar_w_empty;        // stages until the group in turn goes back
         const int group = min(4, a.w_stages);              // channel blocks whose barriers are polled together
@@ -210,9 +229,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
             for (int k = 0; k < 4; ++k)
                 if (k < ks) {
                     if (X3) {
-                        mma_tf32(acc, wa + 2u * k, xb + x_lo + 2u * k, kDescHi, idesc, started);       // w_hi x_lo
-                        mma_tf32(acc, wa + w_lo + 2u * k, xb + 2u * k, kDescHi, idesc, 1u);            // w_lo x_hi
-                        mma_tf32(acc, wa + 2u * k, xb + 2u * k, kDescHi, idesc, 1u);                   // w_hi x_hi
+                        // columns [0, nt): w_hi x_hi + w_lo x_hi; columns [nt, 2 nt): w_hi x_lo - two MMAs for three products
+                        mma_tf32(acc, wa + 2u * k, xb + 2u * k, kDescHi, idesc_wide, started);
+                        mma_tf32(acc, wa + w_lo + 2u * k, xb + 2u * k, kDescHi, idesc, 1u);
                     } else {
                         mma_tf32(acc, wa + 2u * k, xb + 2u * k, kDescHi, idesc, started);
                     }
@@ -233,34 +252,40 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
                 const int l = min(st, a.L - 1), ch = st - l;
                 const uint32_t ga = g & (nacc - 1u);
                 const int JB = (a.J[l] + 31) >> 5, ks_last = (a.J[l] - (JB - 1) * 32 + 7) >> 3;      // K steps with real channels
-                // the accumulator's previous step has been read out; a new layer's operand is what the epilogue of the step
-                // before wrote
-                // (epilogues finish in order: the second wait covers the first)
-                if (st > 0 && ch == 0)
-                    alive = mbar_wait<kSpin>(bar_epi + 8 * ((g - 1u) & (nacc - 1u)), ((g - 1u) >> nacc_log2) & 1u, abort_flag, a.status, a.wait_iters);
-                else if (g >= nacc)
-                    alive = mbar_wait<kSpin>(bar_epi + 8 * ga, ((g >> nacc_log2) - 1u) & 1u, abort_flag, a.status, a.wait_iters);
-                if (!alive) break;
-                tc_fence_after();                          // once per step: orders the MMAs after the epilogue's reads of the accumulator
-                const uint32_t acc = tmem + ga * (uint32_t)nt;
+                const uint32_t acc = tmem + ga * acc_cols;
                 uint32_t started = 0;
                 for (int cb0 = 0; cb0 < JB && alive; cb0 += group) {
                     const int nb = min(group, JB - cb0);
                     // start the group's polls together, then wait properly for whatever was not there yet
-                    uint32_t ready = 0;
+                    auto poll_group = [&]() {
+                        uint32_t ready = 0;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (j < nb) {
-                            uint32_t sj = sw + j, pj = pw;
-                            if (sj >= (uint32_t)a.w_stages) { sj -= a.w_stages; pj ^= 1u; }
-                            bool ok = mbar_test_wait(bar_w_full + 8 * sj, pj);
-                            if (l == 0) {
-                                const int slot = (cb0 + j) & (n_slots - 1);
-                                const uint32_t use = tile_k * slot_uses(slot) + (uint32_t)((cb0 + j) >> ns_log2);
-                                ok = mbar_test_wait((X3 ? bar_split : bar_in) + 8 * slot, use & 1u) && ok;
+                        for (int j = 0; j < 4; ++j)
+                            if (j < nb) {
+                                uint32_t sj = sw + j, pj = pw;
+                                if (sj >= (uint32_t)a.w_stages) { sj -= a.w_stages; pj ^= 1u; }
+                                bool ok = mbar_test_wait(bar_w_full + 8 * sj, pj);
+                                if (l == 0) {
+                                    const int slot = (cb0 + j) & (n_slots - 1);
+                                    const uint32_t use = tile_k * slot_uses(slot) + (uint32_t)((cb0 + j) >> ns_log2);
+                                    ok = mbar_test_wait((X3 ? bar_split : bar_in) + 8 * slot, use & 1u) && ok;
+                                }
+                                ready |= (ok ? 1u : 0u) << j;
                             }
-                            ready |= (ok ? 1u : 0u) << j;
-                        }
+                        return ready;
+                    };
+                    uint32_t ready = poll_group();
+                    if (cb0 == 0) {
+                        // Only now (the filters' polls are behind us) wait for the epilogue: the accumulator's previous
+                        // step has been read out, and a new layer's operand is what the epilogue of the step before wrote
+                        // (epilogues finish in order: the second wait covers the first).
+                        if (st > 0 && ch == 0)
+                            alive = mbar_wait<kSpin>(bar_epi + 8 * ((g - 1u) & (nacc - 1u)), ((g - 1u) >> nacc_log2) & 1u, abort_flag, a.status, a.wait_iters);
+                        else if (g >= nacc)
+                            alive = mbar_wait<kSpin>(bar_epi + 8 * ga, ((g >> nacc_log2) - 1u) & 1u, abort_flag, a.status, a.wait_iters);
+                        if (!alive) break;
+                        tc_fence_after();                  // once per step: orders the MMAs after the epilogue's reads of the accumulator
+                    }
                     if (l > 0) {
                         uint32_t xb = x_desc0 + (uint32_t)cb0 * x_step;
                         for (int j = 0; j < nb; ++j, xb += x_step) {
@@ -307,12 +332,12 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
                     alive = mbar_wait_warp<kSpin>(bar_in + 8 * slot, use & 1u, abort_flag, a.status, a.wait_iters);
                     if (!alive) break;
                     for (int idx = tid_e; idx < nt * 8; idx += n_epi) {               // 16-byte chunks of the block
-                        float4 *p = reinterpret_cast<float4 *>(x_ptr + (size_t)slot * slot_bytes + (size_t)idx * 16);
+                        float4 *p = reinterpret_cast<float4 *>(x_ptr + (size_t)slot * slot_pitch + (size_t)idx * 16);
                         const float4 v = *p;
                         const float4 h = make_float4(__uint_as_float(__float_as_uint(v.x) & 0xffffe000u), __uint_as_float(__float_as_uint(v.y) & 0xffffe000u),
                                                      __uint_as_float(__float_as_uint(v.z) & 0xffffe000u), __uint_as_float(__float_as_uint(v.w) & 0xffffe000u));
                         *p = h;
-                        *reinterpret_cast<float4 *>(reinterpret_cast<uint8_t *>(p) + x_half) = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+                        *reinterpret_cast<float4 *>(reinterpret_cast<uint8_t *>(p) + slot_bytes) = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
@@ -331,7 +356,13 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
                 if (quarter * 32 < K) {                                               // else: no filter of this step in this warp
                     const int k = quarter * 32 + lane;
                     float v[32];
-                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + ga * (uint32_t)nt + (uint32_t)cg * 32u, v);
+                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + ga * acc_cols + (uint32_t)cg * 32u, v);
+                    if (X3) {                                                         // + the x_lo products
+                        float u[32];
+                        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + ga * acc_cols + (uint32_t)nt + (uint32_t)cg * 32u, u);
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] += u[e];
+                    }
                     const float b = bias_s[st * 128 + k];
                     const bool relu = a.relu[l] != 0, real = k < K;
 #pragma unroll
@@ -342,14 +373,14 @@ __global__ void __launch_bounds__(kMaxThreads, 1) fc_chain_kernel(const __grid_c
                     }
                     if (!last) {
                         // image cg*32 + e, channel k: block `quarter`, row = image, 16-byte chunk (lane / 4) ^ (row & 7)
-                        uint8_t *blk = x_ptr + (size_t)quarter * slot_bytes + (size_t)(cg * 32) * 128 + (lane & 3) * 4;
+                        uint8_t *blk = x_ptr + (size_t)quarter * slot_pitch + (size_t)(cg * 32) * 128 + (lane & 3) * 4;
 #pragma unroll
                         for (int e = 0; e < 32; ++e) {
                             float *dst = reinterpret_cast<float *>(blk + e * 128 + (((lane >> 2) ^ (e & 7)) << 4));
                             if (X3) {
                                 const float h = __uint_as_float(__float_as_uint(v[e]) & 0xffffe000u);
                                 *dst = h;
-                                *reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(dst) + x_half) = v[e] - h;
+                                *reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(dst) + slot_bytes) = v[e] - h;
                             } else {
                                 *dst = v[e];
                             }
