@@ -110,6 +110,7 @@ struct TcArgs {
     uint32_t raw_stage_bytes, raw_box_bytes;
     int x_packed;              // 3xTF32, at most 16 channels: the residual sits in the unused lanes of the same row
     int x3_wide;               // 3xTF32, pixels on M: x_hi meets [w_hi; w_lo] in one MMA of twice the filters (see the issue loop)
+    int alt_tiles;             // one chain per tile: the two MMA threads take alternate tiles (else warp 1 issues everything)
     uint32_t x_lo_off;         // 3xTF32: 16-byte units from a strip's TF32 part to its residual
     int relu, accumulate;
     uint32_t wait_iters;       // limit of every bounded wait (polls)
@@ -185,10 +186,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     float *dw_s_w = reinterpret_cast<float *>(ctrl_ptr + kCtrlBarrierBytes + 16 + (size_t)a.KB * 32 * 4 + kTapTabEntries * sizeof(short));   // [CB][10][32]: 9 taps + bias
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // Tiles with two or more MMA chains split them over two issuing threads (warps 1 and 3, on different schedulers):
-    // issuing a small MMA costs a thread more cycles than the pipe needs to run it.
-    constexpr int kIssuers = CH >= 2 ? 2 : 1;
-    constexpr int kSplit = (CH + 1) / 2;       // chains [0, kSplit) belong to warp 1, the rest to warp 3
+    // Two issuing threads (warps 1 and 3, on different schedulers): issuing a small MMA costs a thread about twice the
+    // cycles the pipe needs to run it.  A tile's MMA chains are split between them; an odd number of chains is split the
+    // other way round on odd tiles (chains [0, kSplit) and [kSplit, CH) on even tiles, [0, CH - kSplit) and the rest on
+    // odd ones), so that both issue the same number of MMAs over two tiles.  With one chain per tile the two threads take
+    // alternate tiles where the MMAs are small enough to be issue-bound (alt_tiles; measured: the 32 -> 32 layer of the
+    // residual CNN 32.4 -> 26.6 us in 3xTF32), else warp 1 issues alone: a second thread that only walks the barriers
+    // cost the TF32 step 6 us.  Both threads walk every tile and every barrier; only the chains they issue for differ.
+    // (TF32 kernels keep the fixed split and the single thread: alternating measured 7 us slower per step there.)
+    const int kIssuers = (CH >= 2 || (X3 && a.alt_tiles)) ? 2 : 1;
+    constexpr int kSplit = (CH + 1) / 2, kOddSplit = X3 ? CH - kSplit : kSplit;      // chains of warp 1 on even / odd tiles
     const int T = a.FH * a.FW;
     const int total_tiles = a.m_tiles * a.n_tiles;
 
@@ -327,8 +334,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if ((warp == 1 || (kIssuers == 2 && warp == 3)) && lane == 0) {
         // ---- MMA issue: this thread's chains are [C0, C1)
-        auto mma_role = [&](auto c0_tag, auto c1_tag) {
-        constexpr int C0 = decltype(c0_tag)::value, C1 = decltype(c1_tag)::value;
+        auto mma_role = [&](auto c0_tag, auto c1_tag, auto d0_tag, auto d1_tag) {
+        constexpr int C0 = decltype(c0_tag)::value, C1 = decltype(c1_tag)::value;       // chains on even tiles
+        constexpr int D0 = decltype(d0_tag)::value, D1 = decltype(d1_tag)::value;       // chains on odd tiles
         bool alive = true;
         uint32_t sa = 0, pa = 0, sb = 0, pb = 0;
         uint32_t slot_uses = 0;                   // slots taken so far; slot j of a tile is (slot_uses + j) % 2
@@ -355,9 +363,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         };
         const unsigned long long mask0 = MASKED ? load_mask(0) : ~0ull;
 
-        auto issue_block = [&](auto ks_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const unsigned long long taps, const uint32_t r_sel, uint32_t &started, uint32_t &w_res) {
+        auto issue_block = [&](auto ks_tag, auto lo_tag, auto hi_tag, const uint32_t x_stage, const uint32_t (&acc)[CH], const unsigned long long taps, const uint32_t r_sel, uint32_t &started, uint32_t &w_res) {
             const uint32_t r_col = r_sel * (uint32_t)(kSlotPx / a.racc);   // this block's accumulator within each slot
-            constexpr int KS = decltype(ks_tag)::value;
+            constexpr int KS = decltype(ks_tag)::value, CL = decltype(lo_tag)::value, CU = decltype(hi_tag)::value;
             uint32_t off = 0;
             int y = 0;
             for (int tap = 0; tap < T; ++tap) {
@@ -378,7 +386,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t first = (started >> r_sel) & 1u;   // 0 for an accumulator's first MMAs of the tile: they overwrite
                 started |= 1u << r_sel;
 #pragma unroll
-                for (int c = C0; c < C1; ++c) {
+                for (int c = CL; c < CU; ++c) {
                     const uint32_t xs = x_lo + xo[c];
                     const uint32_t da = PM ? xs : w_lo, db = PM ? w_lo : xs;
                     if (!X3) {
@@ -413,7 +421,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         };
 
-        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+        bool odd_tile = false;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x, odd_tile = !odd_tile) {
             const Tile tl = decode_tile(a, t);
             // the previous content of the slots this tile takes must have left tensor memory
             for (int j = 0; j < a.slots && alive; ++j) {
@@ -439,8 +448,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 alive = mbar_wait(((X3 || DW) ? bar_a_split : bar_a_full) + 8 * sa, pa, abort_flag, a.status, a.wait_iters);   // once split / computed
                 if (!alive) break;
                 const uint32_t x_stage = smem_desc_lo(a_base + sa * a.a_stage_bytes) + (uint32_t)tl.a0 * 8u;   // 128 bytes per pixel, >> 4
-                if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, x_stage, acc, taps, r_sel, started, w_res);
-                else issue_block(std::integral_constant<int, 4>{}, x_stage, acc, taps, r_sel, started, w_res);
+                if (odd_tile && (D0 != C0 || D1 != C1)) {
+                    if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, d0_tag, d1_tag, x_stage, acc, taps, r_sel, started, w_res);
+                    else issue_block(std::integral_constant<int, 4>{}, d0_tag, d1_tag, x_stage, acc, taps, r_sel, started, w_res);
+                } else {
+                    if (cb == a.CBr - 1) issue_block(std::integral_constant<int, KS_LAST>{}, c0_tag, c1_tag, x_stage, acc, taps, r_sel, started, w_res);
+                    else issue_block(std::integral_constant<int, 4>{}, c0_tag, c1_tag, x_stage, acc, taps, r_sel, started, w_res);
+                }
                 if (++r_sel == (uint32_t)a.racc) r_sel = 0;
                 if (alive) mma_commit(bar_a_empty + 8 * sa);
                 if (++sa == (uint32_t)kAStages) { sa = 0; pa ^= 1u; }
@@ -451,8 +465,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             slot_uses += a.slots;
         }
         };
-        if (kIssuers == 1 || warp == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, kIssuers == 1 ? CH : kSplit>{});
-        else mma_role(std::integral_constant<int, kSplit>{}, std::integral_constant<int, CH>{});
+        if (CH == 1 && kIssuers == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, CH>{},
+                                               std::integral_constant<int, 0>{}, std::integral_constant<int, CH>{});
+        else if (warp == 1) mma_role(std::integral_constant<int, 0>{}, std::integral_constant<int, kSplit>{},
+                                     std::integral_constant<int, 0>{}, std::integral_constant<int, kOddSplit>{});
+        else mma_role(std::integral_constant<int, kSplit>{}, std::integral_constant<int, CH>{},
+                      std::integral_constant<int, kOddSplit>{}, std::integral_constant<int, CH>{});
     } else if (DW && warp >= 8) {
         // ---- fused depthwise 3x3: halo tile -> strip (FMAs, bias, ReLU, 16-byte stores at the swizzled places of the
         // K-major strip the MMAs read).
@@ -1159,6 +1177,8 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
         a.n_slot = ((p.px_tile + a.slots - 1) / a.slots + 15) & ~15;
         chains = a.slots;
     }
+    // the MMA's N: filters of the tile (twice that for x3_wide) or pixels of a slot; up to 128 columns an MMA is issue-bound
+    a.alt_tiles = (x3 && (p.pixel_m ? (p.x3_wide ? 2 : 1) * p.w_rows : a.n_slot) <= 128) ? 1 : 0;
     const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
     a.relu = relu; a.accumulate = accumulate; a.wait_iters = ctx->wait_iters;
     const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3, dw != nullptr);
