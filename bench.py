@@ -380,7 +380,7 @@ def gpu_main(args):
         if row["op"] == "conv":
             path = B.small_conv2d_path(ctx, N, row["C"], row["K"], row["H"], row["W"], row["FH"], row["FW"], row["stride"], row["pad"],
                                        B.MATH[args.math])
-            kern = f"conv_{args.math}_tensor" if path == 3 else "conv_fp32_cuda_core"
+            kern = f"conv_{args.math}_tensor" if path == 3 else f"conv_{args.math}_warp_mma" if path == 4 else "conv_fp32_cuda_core"
         layer_table.append({"layer": row["name"], "kernel": kern, "us": round(tmed * 1e3, 2), "gflops": round(fl / tmed / 1e6, 1),
                             "gbs": round(by / tmed / 1e6, 1)})
         k = by_kernel.setdefault(kern, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})

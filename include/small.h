@@ -118,14 +118,17 @@ int small_set_wait_limit(small_ctx *ctx, unsigned polls);
 int small_selftest_wait_timeout(small_ctx *ctx, void *stream);
 /* Kernel family of the full channel reductions under the tensor-core math modes.  AUTO (the default): per layer,
  * whichever of the tensor-core kernel and the register-tiled FP32 kernel is the faster one for its channel counts
- * (FP32 FMAs meet every mode's tolerance); TENSOR / CUDA_CORES force one family wherever it takes the shape, GENERAL the
- * general FP32 kernel (any window and stride) everywhere except the network stems.  For
+ * (FP32 FMAs meet every mode's tolerance); layers of one channel block and at most 32 filters take the warp-level
+ * tensor-core kernel.  TENSOR (the block-level tensor-core kernel) / CUDA_CORES / WARP_MMA force one family wherever it
+ * takes the shape, GENERAL the general FP32 kernel (any window and stride) everywhere except the network stems.  For
  * measurements and comparisons; results stay within the mode's tolerance either way.  The paper has no counterpart. */
-enum { SMALL_CONV_PATH_AUTO = 0, SMALL_CONV_PATH_TENSOR = 1, SMALL_CONV_PATH_CUDA_CORES = 2, SMALL_CONV_PATH_GENERAL = 3 };
+enum { SMALL_CONV_PATH_AUTO = 0, SMALL_CONV_PATH_TENSOR = 1, SMALL_CONV_PATH_CUDA_CORES = 2, SMALL_CONV_PATH_GENERAL = 3,
+       SMALL_CONV_PATH_WARP_MMA = 4 };
 int small_set_conv_path(small_ctx *ctx, int path);
 /* Which kernel small_conv2d runs for this shape and math mode (with a 32-byte aligned output) under the context's
  * path setting: 0 = few-input-channel kernel (network stems), 1 = register-tiled FP32 kernel, 2 = general FP32 kernel,
- * 3 = tensor-core kernel; -1 for invalid arguments. */
+ * 3 = block-level tensor-core kernel (tcgen05), 4 = warp-level tensor-core kernel (few channels and filters);
+ * -1 for invalid arguments. */
 int small_conv2d_path(small_ctx *ctx, int N, int C, int K, int H, int W, int FH, int FW, int stride,
                       int pad_t, int pad_b, int pad_l, int pad_r, unsigned math);
 /* Synchronises `stream`, then reads and clears the device status word: *status is SMALL_OK or

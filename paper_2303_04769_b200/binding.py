@@ -192,8 +192,8 @@ def small_set_layer_overlap(ctx, on):
     _check(lib().small_set_layer_overlap(ctx, 1 if on else 0), "small_set_layer_overlap")
 
 
-CONV_PATH = {"auto": 0, "tensor": 1, "cuda_cores": 2, "general": 3}
-CONV_KERNEL = {0: "conv_thin", 1: "conv_direct", 2: "conv_fp32", 3: "conv_tc"}
+CONV_PATH = {"auto": 0, "tensor": 1, "cuda_cores": 2, "general": 3, "warp_mma": 4}
+CONV_KERNEL = {0: "conv_thin", 1: "conv_direct", 2: "conv_fp32", 3: "conv_tc", 4: "conv_mma"}
 
 
 def small_set_conv_path(ctx, path):

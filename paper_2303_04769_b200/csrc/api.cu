@@ -182,7 +182,7 @@ SMALL_API int small_set_branch_overlap(small_ctx *ctx, int on) {
 
 SMALL_API int small_set_conv_path(small_ctx *ctx, int path) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
-    if (path < SMALL_CONV_PATH_AUTO || path > SMALL_CONV_PATH_GENERAL) return SMALL_ERR_INVALID_ARG;
+    if (path < SMALL_CONV_PATH_AUTO || path > SMALL_CONV_PATH_WARP_MMA) return SMALL_ERR_INVALID_ARG;
     ctx->conv_path = path;
     return SMALL_OK;
 }
@@ -361,6 +361,15 @@ static int conv2d_path(const small_ctx *ctx, const Geom &g, unsigned math, bool 
         (g.OW < 4 || conv_direct_blocks(g) < (ctx ? ctx->sm_count : 148) / 2))
         direct = false;
     if (math == SMALL_MATH_FP32) return direct ? 1 : 2;
+    // One channel block and at most 32 filters: the warp-level MMA (see conv_mma.cu), which measured faster than both
+    // other families on such layers (residual CNN at batch 256, microseconds, TF32 / 3xTF32, block-level tensor-core
+    // kernel against warp-level: 3x3 16->16 25.3 / 37.4 against 17.3 / 28.7; 3x3 stride 2 16->32 19.9 / 28.3 against
+    // 12.2 / 15.8; 1x1 stride 2 16->32 10.2 / 14.3 against 7.1 / 7.6; 3x3 32->32 on 16x16 planes 15.5 / 27.2 against
+    // 14.8 / 23.9, on 8x8 planes 10.2 / 13.4 against 8.1 / 9.1).
+    if (!(ctx && (ctx->conv_path == SMALL_CONV_PATH_TENSOR || ctx->conv_path == SMALL_CONV_PATH_CUDA_CORES)) &&
+        conv_mma_supported(g, math == SMALL_MATH_3XTF32))
+        return 4;
+    if (ctx && ctx->conv_path == SMALL_CONV_PATH_WARP_MMA) return direct ? 1 : 2;
     const bool tc = out_aligned32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32);
     if (tc && !(direct && prefer_cuda_cores(ctx, g, math))) return 3;
     return direct ? 1 : 2;
@@ -402,6 +411,11 @@ SMALL_API int small_conv2d(small_ctx *ctx, const float *in, const float *w, cons
             const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);
             const float *w_lo = w_hi + conv_w_tc_elems(C, K, FH, FW);
             return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, relu, acc, math, st);
+        }
+        case 4: {
+            const float *w_hi = w + conv_w_fp32_elems(C, K, FH, FW);
+            const float *w_lo = w_hi + conv_w_tc_elems(C, K, FH, FW);
+            return launch_conv_mma(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, relu, acc, math, st);
         }
         default: return launch_conv_fp32(ctx, in, w, bias, out, g, relu, acc, st);
     }
