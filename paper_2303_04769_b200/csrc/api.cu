@@ -361,13 +361,14 @@ static int conv2d_path(const small_ctx *ctx, const Geom &g, unsigned math, bool 
         (g.OW < 4 || conv_direct_blocks(g) < (ctx ? ctx->sm_count : 148) / 2))
         direct = false;
     if (math == SMALL_MATH_FP32) return direct ? 1 : 2;
-    // One channel block and at most 32 filters: the warp-level MMA (see conv_mma.cu), which measured faster than both
+    // One channel block and at most 32 filters (64 with a 1x1 window): the warp-level MMA (see conv_mma.cu), which measured faster than both
     // other families on such layers (residual CNN at batch 256, microseconds, TF32 / 3xTF32, block-level tensor-core
     // kernel against warp-level: 3x3 16->16 25.3 / 37.4 against 17.3 / 28.7; 3x3 stride 2 16->32 19.9 / 28.3 against
     // 12.2 / 15.8; 1x1 stride 2 16->32 10.2 / 14.3 against 7.1 / 7.6; 3x3 32->32 on 16x16 planes 15.5 / 27.2 against
-    // 14.8 / 23.9, on 8x8 planes 10.2 / 13.4 against 8.1 / 9.1).
+    // 14.8 / 23.9, on 8x8 planes 10.2 / 13.4 against 8.1 / 9.1; 1x1 stride 2 32->64 8.3 / 9.8 against 7.1 / 7.7; but 3x3
+    // stride 2 32->64 15.4 / 18.4 against 15.4 / 23.6, so 3x3 layers with more than 32 filters stay where they were).
     if (!(ctx && (ctx->conv_path == SMALL_CONV_PATH_TENSOR || ctx->conv_path == SMALL_CONV_PATH_CUDA_CORES)) &&
-        conv_mma_supported(g, math == SMALL_MATH_3XTF32))
+        ((ctx && ctx->conv_path == SMALL_CONV_PATH_WARP_MMA) || g.K <= 32 || (g.K <= 64 && g.FH * g.FW == 1)) && conv_mma_supported(g, math == SMALL_MATH_3XTF32))
         return 4;
     if (ctx && ctx->conv_path == SMALL_CONV_PATH_WARP_MMA) return direct ? 1 : 2;
     const bool tc = out_aligned32 && conv_tc_supported(g, math == SMALL_MATH_3XTF32);

@@ -1,4 +1,4 @@
-"""GPU parity of the warp-level tensor-core convolution (one channel block, at most 32 filters) against the CPU
+"""GPU parity of the warp-level tensor-core convolution (one channel block; filters in tiles of 32) against the CPU
 oracle, through small_conv2d: TF32 at 2e-3, 3xTF32 at 1e-5, each on the relative L2 error and on every element."""
 import numpy as np
 import pytest
@@ -20,7 +20,7 @@ def rnd(shape, tid, lo=-1.0, hi=1.0):
 
 # (N, C, K, H, W, FH, FW, stride, pads t b l r): the residual network's layers, every fragment shape (planes 12 and more,
 # 6 to 11, under 6 columns wide), ragged widths and heights, several images per tile, bands and column tiles, both row
-# widths of the shared-memory tiles (C <= 16 and C <= 32), 8 / 16 / 32 filters and ragged filter counts, strides 1 and 2,
+# widths of the shared-memory tiles (C <= 16 and C <= 32), 8 / 16 / 32 filters, several filter tiles and ragged filter counts, strides 1 and 2,
 # windows 1x1, 3x3, 5x5, 1x3 and 10x4, asymmetric pads.
 CASES = [
     (3, 16, 16, 32, 32, 3, 3, 1, (1, 1, 1, 1)),
@@ -39,6 +39,10 @@ CASES = [
     (3, 7, 12, 49, 10, 10, 4, 2, (4, 5, 1, 1)),
     (300, 16, 16, 3, 3, 3, 3, 1, (1, 1, 1, 1)),
     (2, 32, 16, 33, 31, 3, 3, 2, (0, 1, 1, 0)),
+    (6, 32, 64, 16, 16, 3, 3, 2, (1, 1, 1, 1)),
+    (6, 32, 64, 16, 16, 1, 1, 2, (0, 0, 0, 0)),
+    (3, 20, 72, 11, 13, 3, 3, 1, (1, 1, 1, 1)),
+    (2, 16, 130, 9, 9, 1, 1, 1, (0, 0, 0, 0)),
 ]
 
 
