@@ -351,6 +351,7 @@ static bool prefer_cuda_cores(const small_ctx *ctx, const Geom &g, unsigned math
 }
 
 static int conv2d_path(const small_ctx *ctx, const Geom &g, unsigned math, bool out_aligned32) {
+    if (ctx && ctx->conv_path == SMALL_CONV_PATH_WARP_MMA && math != SMALL_MATH_FP32 && conv_mma_supported(g, math == SMALL_MATH_3XTF32)) return 4;
     if (conv_thin_supported(g)) return 0;          // a reduction of a few dozen terms: CUDA cores in every math mode
     if (ctx && ctx->conv_path == SMALL_CONV_PATH_GENERAL) return 2;
     bool direct = conv_direct_supported(g);

@@ -58,7 +58,7 @@ MmaPlan plan_mma(const Geom &g, bool x3, size_t max_smem) {
     MmaPlan best{};
     best.ok = false;
     double best_score = 0.0;
-    const int GM = p.NF >= 4 ? 1 : p.NF == 2 ? 2 : 4;      // the kernel computes fragments in groups of GM
+    const int GM = p.NF >= 4 ? 2 : 4;      // the kernel computes fragments in groups of GM
     for (int warps = 2; warps <= 8; warps *= 2)
     for (int mfw = p.MF; mfw >= GM; mfw /= 2) {
         const int F = warps * mfw;

@@ -46,7 +46,7 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
     constexpr uint32_t RB = CW * 4;                 // bytes per pixel / filter row
     constexpr int RSH = CW == 16 ? 6 : 7;
     constexpr int PAIRS = CW / 16;
-    constexpr int GM = NF >= 4 ? 1 : NF == 2 ? 2 : 4;   // pixel fragments whose MMAs are interleaved
+    constexpr int GM = NF >= 4 ? 2 : 4;   // pixel fragments whose MMAs are interleaved
     constexpr int FWU = FWT ? FWT : 1;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;

@@ -43,6 +43,8 @@ CASES = [
     (6, 32, 64, 16, 16, 1, 1, 2, (0, 0, 0, 0)),
     (3, 20, 72, 11, 13, 3, 3, 1, (1, 1, 1, 1)),
     (2, 16, 130, 9, 9, 1, 1, 1, (0, 0, 0, 0)),
+    (4, 3, 16, 32, 32, 3, 3, 1, (1, 1, 1, 1)),
+    (2, 21, 16, 12, 12, 3, 3, 1, (1, 1, 1, 1)),
 ]
 
 
