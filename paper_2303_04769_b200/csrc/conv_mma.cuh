@@ -19,6 +19,8 @@ struct MmaArgs {
     int tiles_w, tiles_h, n_tiles;
     int frags_w, frags_img, frags_tile;   // fragments per fragment row, per image of a tile, per tile (the rest idle)
     int mf_warp;               // fragments per warp actually used (<= MF)
+    int cs;                    // stride of the box origin in the tensor (S of the kernel = stride between the box's pixels:
+                               // 1 when a 1 x 1 window's copy itself skips the pixels a stride leaves out)
     int k_tiles;               // filter tiles of 32 (= KB): thread block b computes tile b % k_tiles of its pixel tiles
     uint32_t in_box_bytes, stage_bytes;
     uint32_t w_box_bytes, w_half_bytes;   // bytes of one filter box (TF32 part or residual) and its 1 KB-rounded place
@@ -72,7 +74,7 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
         int n0, oh0, ow0;
         tile_origin(t, n0, oh0, ow0);
         sm100::mbar_expect_tx(bar_in + 8 * s, a.in_box_bytes);
-        sm100::tma_load_5d(in_s + s * a.stage_bytes, &map_in, bar_in + 8 * s, 0, ow0 * S - a.pl, oh0 * S - a.pt, 0, n0);
+        sm100::tma_load_5d(in_s + s * a.stage_bytes, &map_in, bar_in + 8 * s, 0, ow0 * a.cs - a.pl, oh0 * a.cs - a.pt, 0, n0);
     };
 
     if (threadIdx.x == 0) {
@@ -251,22 +253,47 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
             tile_origin(t, n0, oh0, ow0);
             float *tile_out = a.out + ((((size_t)n0 * a.KB + kt) * a.OH + oh0) * a.OW + ow0) * 32;
             const int n_left = a.N - n0, oh_left = a.OH - oh0, ow_left = a.OW - ow0;
+            uint32_t vmask = 0;                                     // bit 2 m + h: this lane stores that pixel
+#pragma unroll
+            for (int m = 0; m < MF; ++m)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t pk = st_pix[m][h];               // image, row, column of this pixel within the tile
+                    if (pk != 0xffffffffu && (int)(pk >> 20) < n_left && (int)((pk >> 10) & 1023u) < oh_left && (int)(pk & 1023u) < ow_left)
+                        vmask |= 1u << (2 * m + h);
+                }
+            if (a.accumulate) {
+                // the residual join: all loads of the tensor already in `out` first, so that their latencies overlap
+                // (between stores the compiler has to keep them in program order)
+                float2 res[MF][2][NF];
+#pragma unroll
+                for (int m = 0; m < MF; ++m)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int nf = 0; nf < NF; ++nf)
+                            res[m][h][nf] = (vmask >> (2 * m + h) & 1u) ? *reinterpret_cast<const float2 *>(tile_out + st_off[m][h] + 8 * nf)
+                                                                        : make_float2(0.0f, 0.0f);
+#pragma unroll
+                for (int m = 0; m < MF; ++m)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int nf = 0; nf < NF; ++nf) { acc[m][nf][2 * h] += res[m][h][nf].x; acc[m][nf][2 * h + 1] += res[m][h][nf].y; }
+            }
 #pragma unroll
             for (int m = 0; m < MF; ++m) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const uint32_t pk = st_pix[m][h];               // image, row, column of this pixel within the tile
-                    if (pk == 0xffffffffu || (int)(pk >> 20) >= n_left || (int)((pk >> 10) & 1023u) >= oh_left || (int)(pk & 1023u) >= ow_left) continue;
+                    if (!(vmask >> (2 * m + h) & 1u)) continue;
                     float *dst = tile_out + st_off[m][h];
 #pragma unroll
                     for (int nf = 0; nf < NF; ++nf) {
                         float2 r = make_float2(acc[m][nf][2 * h] + bv[nf][0], acc[m][nf][2 * h + 1] + bv[nf][1]);
-                        float2 *d2 = reinterpret_cast<float2 *>(dst + 8 * nf);
-                        if (a.accumulate) { const float2 o = *d2; r.x += o.x; r.y += o.y; }
                         if (a.relu) { r.x = fmaxf(r.x, 0.0f); r.y = fmaxf(r.y, 0.0f); }
                         if (!(k_real >> (2 * nf) & 1u)) r.x = 0.0f;      // pad lanes stay +0
                         if (!(k_real >> (2 * nf + 1) & 1u)) r.y = 0.0f;
-                        *d2 = r;
+                        *reinterpret_cast<float2 *>(dst + 8 * nf) = r;
                     }
 #pragma unroll
                     for (int z = 8 * NF; z < 32; z += 8) *reinterpret_cast<float2 *>(dst + z) = make_float2(0.0f, 0.0f);
