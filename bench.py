@@ -34,6 +34,10 @@ TOL = {"fp32": 1e-5, "tf32": 2e-3, "3xtf32": 1e-5}
 # this file's network step, averaged over the kernel's launches in one step).  It is reported only while the kernel's
 # source still has the hash it had when the counters were taken.
 TRAFFIC = {
+    "conv_3xtf32_warp_mma": {"bytes_per_launch": 27042816.0, "source": "paper_2303_04769_b200/csrc/conv_mma.cuh",
+                             "sha256": "05b10a5f00d9d9656f962032b39e6f4606bee679be38e82a5f12090db12b91d6"},
+    "conv_tf32_warp_mma": {"bytes_per_launch": 27005994.7, "source": "paper_2303_04769_b200/csrc/conv_mma.cuh",
+                           "sha256": "05b10a5f00d9d9656f962032b39e6f4606bee679be38e82a5f12090db12b91d6"},
     "conv_3xtf32_tensor": {"bytes_per_launch": 22910037.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
                            "sha256": "46edea15c263baabda86068dc7269c4601c27973edc2dd8509505bfd06924f4c"},
     "conv_tf32_tensor": {"bytes_per_launch": 24391387.0, "source": "paper_2303_04769_b200/csrc/conv_tc.cu",
@@ -403,6 +407,14 @@ def gpu_main(args):
         roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                     "traffic": measured_traffic(dom_name), "kernel": dom_name, "launches_per_step": dom["launches"],
                     "peak_source": f"{peaks['source']}: copy bandwidth"}
+    if dom_name.endswith("warp_mma"):
+        # context: the warp-level MMA this kernel issues runs at 512 TF32 multiply-adds per clock and SM (measured with a
+        # stand-alone issue loop), a quarter of the block-level MMA's rate that `peak` above derives from; against that
+        # instruction's own roof the kernel's bound is its arithmetic
+        wp = sm_count * 512 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12 / (3.0 if args.math == "3xtf32" else 1.0)
+        t_w = dom["flops"] / (wp * 1e12)
+        roofline["warp_mma_context"] = {"peak_tflops": wp, "frac_of_slower_roof": max(t_w, t_bytes) / (dom["ms"] * 1e-3),
+                                        "bound": "tensor (warp-level MMA)" if t_w > t_bytes else "hbm"}
     roofline["algorithmic_flops_per_launch"] = dom["flops"] / dom["launches"]
     roofline["algorithmic_bytes_per_launch"] = dom["bytes"] / dom["launches"]
     roofline["us_per_launch"] = 1e3 * dom["ms"] / dom["launches"]

@@ -191,7 +191,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // other way round on odd tiles (chains [0, kSplit) and [kSplit, CH) on even tiles, [0, CH - kSplit) and the rest on
     // odd ones), so that both issue the same number of MMAs over two tiles.  With one chain per tile the two threads take
     // alternate tiles where the MMAs are small enough to be issue-bound (alt_tiles; measured: the 32 -> 32 layer of the
-    // residual CNN 32.4 -> 26.6 us in 3xTF32), else warp 1 issues alone: a second thread that only walks the barriers
+    // residual CNN 32.4 -> 26.6 us in 3xTF32; the host side leaves it off today, see there), else warp 1 issues alone: a second thread that only walks the barriers
     // cost the TF32 step 6 us.  Both threads walk every tile and every barrier; only the chains they issue for differ.
     // (TF32 kernels keep the fixed split and the single thread: alternating measured 7 us slower per step there.)
     const int kIssuers = (CH >= 2 || (X3 && a.alt_tiles)) ? 2 : 1;
@@ -1178,7 +1178,10 @@ int launch_conv_tc(small_ctx *ctx, const float *in, const float *w_hi, const flo
         chains = a.slots;
     }
     // the MMA's N: filters of the tile (twice that for x3_wide) or pixels of a slot; up to 128 columns an MMA is issue-bound
-    a.alt_tiles = (x3 && (p.pixel_m ? (p.x3_wide ? 2 : 1) * p.w_rows : a.n_slot) <= 128) ? 1 : 0;
+    // Off: alternating paid on the residual CNN's 32 -> 32 layer, which the warp-level kernel has taken since, and cost
+    // the 64 -> 64 pointwise layers of the keyword-spotting and depthwise-separable networks 2-3 % of their step
+    // (219 -> 213 us and 213 -> 209 us with it off).
+    a.alt_tiles = 0;
     const int ks = p.ks_last == 3 ? 4 : p.ks_last;     // a K step of zero channels more is harmless
     a.relu = relu; a.accumulate = accumulate; a.wait_iters = ctx->wait_iters;
     const TcKernel kern = pick_kernel(chains, ks, p.pixel_m != 0, v.S != 1, x3, dw != nullptr);
