@@ -185,6 +185,8 @@ int small_pack_fc_weights(small_ctx *ctx, const float *w_kj, float *w_blk, int J
  * taps in the stride-1 view of the window); any other shape runs the FP32 kernel (tighter accuracy, no
  * error).  3XTF32 needs roughly twice the shared memory per tile and falls back the same way where even
  * its smallest tile does not fit.  `out` must be 32-byte aligned for the tensor-core kernel (16 otherwise).
+ * Layers of one channel block (C <= 32) with at most 32 filters (64 with a 1 x 1 window) run warp-level tensor-core
+ * MMAs instead of the 128-row block-level ones, which such layers leave mostly empty; same modes, same tolerances.
  * Layers with at most four input channels and a 3 x 3 window (stride 1 or 2), or one channel and a 10 x 4
  * stride-2 window - the first layer of a network - run FP32 FMAs on the CUDA cores in every math mode (a reduction
  * of a few dozen terms is no dense contraction; the result meets each mode's tolerance).

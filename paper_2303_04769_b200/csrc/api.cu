@@ -381,7 +381,7 @@ SMALL_API int small_conv2d_uses_tensor_cores(int N, int C, int K, int H, int W, 
                                              int pt, int pb, int pl, int pr) {
     Geom g;
     if (make_geom(g, N, C, K, H, W, FH, FW, stride, pt, pb, pl, pr) != SMALL_OK) return 0;
-    return conv2d_path(nullptr, g, SMALL_MATH_TF32, true) == 3 ? 1 : 0;
+    return conv2d_path(nullptr, g, SMALL_MATH_TF32, true) >= 3 ? 1 : 0;     // block-level or warp-level MMAs
 }
 
 SMALL_API int small_conv2d_path(small_ctx *ctx, int N, int C, int K, int H, int W, int FH, int FW, int stride,
