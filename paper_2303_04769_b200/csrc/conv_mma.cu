@@ -81,6 +81,11 @@ MmaPlan plan_mma(const Geom &g, bool x3, size_t max_smem) {
         c.frags_tile = c.frags_img * c.NI;
         c.mf_warp = ceil_div(ceil_div(c.frags_tile, warps), GM) * GM;
         if (c.mf_warp > p.MF) continue;
+        // rows shared down the window (see VERT in the kernel): fragments of one row, a 3 x 3 window at stride 1, the
+        // tile's rows dealt to the warps in whole groups of mf_warp, and at most 16 filters (with 32 the filter
+        // fragments of three taps take 96 registers more: 32 -> 32 on 16x16 planes 31.9 us against 23.1 without)
+        c.vert = (p.NF <= 2 && a.fwd_shift == 4 && g.FH == 3 && g.FW == 3 && g.S == 1 && c.NI == 1 && rows_f % c.mf_warp == 0 &&
+                  (rows_f / c.mf_warp) * a.frags_w == warps) ? 1 : 0;
         c.TH = rows_f * frag_h;
         c.Ht = (c.TH - 1) * S + g.FH;
         c.Wt = ((c.TWd - 1) * S + g.FW + 7) & ~7;      // a multiple of 8: see the kernel's ready-made addresses
@@ -93,7 +98,7 @@ MmaPlan plan_mma(const Geom &g, bool x3, size_t max_smem) {
         const size_t smem = 1024 + (size_t)c.w_half_bytes * (x3 ? 2 : 1) + 2 * (size_t)c.stage_bytes;
         if (smem + 1024 > max_smem) continue;
         int per_sm = (int)((225 * 1024) / (smem + 1024));
-        const int reg_warps = p.NF == 4 ? 12 : 16;         // registers: up to 140 (32 filters) or 100 per thread
+        const int reg_warps = p.NF == 4 ? 12 : 16;   // registers per thread: up to 155 (32 filters), else up to 128
         if (per_sm * warps > reg_warps) per_sm = reg_warps / warps;
         if (per_sm < 1) per_sm = 1;
         // resident warps count; idle fragments and few tiles per block cost
@@ -147,8 +152,8 @@ int launch_conv_mma(small_ctx *ctx, const float *in, const float *w_hi, const fl
         if (r != CUDA_SUCCESS) { ctx->last_cuda = (int)r; return SMALL_ERR_CUDA; }
     }
     if (!x3) map_w_lo = map_w;
-    const MmaKernel kern = p.CW == 16 ? (x3 ? pick_mma_16_x3(p.NF, g.FW, g.S / p.es) : pick_mma_16_tf32(p.NF, g.FW, g.S / p.es))
-                                        : (x3 ? pick_mma_32_x3(p.NF, g.FW, g.S / p.es) : pick_mma_32_tf32(p.NF, g.FW, g.S / p.es));
+    const MmaKernel kern = p.CW == 16 ? (x3 ? pick_mma_16_x3(p.NF, g.FW, g.S / p.es, a.vert) : pick_mma_16_tf32(p.NF, g.FW, g.S / p.es, a.vert))
+                                        : (x3 ? pick_mma_32_x3(p.NF, g.FW, g.S / p.es, a.vert) : pick_mma_32_tf32(p.NF, g.FW, g.S / p.es, a.vert));
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->max_smem_optin - 1024);   // the kernel has static shared memory too
     if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SMALL_ERR_CUDA; }

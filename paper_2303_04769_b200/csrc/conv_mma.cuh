@@ -19,6 +19,7 @@ struct MmaArgs {
     int tiles_w, tiles_h, n_tiles;
     int frags_w, frags_img, frags_tile;   // fragments per fragment row, per image of a tile, per tile (the rest idle)
     int mf_warp;               // fragments per warp actually used (<= MF)
+    int vert;                  // a warp's fragments are mf_warp consecutive rows of one column block (see VERT)
     int cs;                    // stride of the box origin in the tensor (S of the kernel = stride between the box's pixels:
                                // 1 when a 1 x 1 window's copy itself skips the pixels a stride leaves out)
     int k_tiles;               // filter tiles of 32 (= KB): thread block b computes tile b % k_tiles of its pixel tiles
@@ -41,7 +42,10 @@ __device__ __forceinline__ void mma_16x8x8(float (&c)[4], const uint32_t *a, con
 // rows and swizzle, layers of at most 16 channels; 32: 128-byte rows); S: stride; X3: 3xTF32; FWT: width of the window
 // (1 or 3; 0: any, at run time).  The halo box is a multiple of 8 pixels wide, so a step down the window leaves a
 // pixel's swizzle phase alone and each lane keeps one ready-made address per window column and fragment.
-template <int NF, int MF, int CW, int S, bool X3, int FWT>
+// VERT (3 x 3 windows at stride 1, fragments of one row): a warp's fragments are consecutive output rows of one column
+// block, so input row r of that block serves the window rows of up to three of them: each input fragment is loaded
+// (and, for 3xTF32, split) once per window column instead of once per tap - half the operand loads and splits.
+template <int NF, int MF, int CW, int S, bool X3, int FWT, bool VERT = false>
 __global__ void __launch_bounds__(256)
 conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_w,
                 const __grid_constant__ CUtensorMap map_w_lo, const MmaArgs a) {
@@ -98,14 +102,27 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
     const int FWD = 1 << a.fwd_shift;
     const int jl = (lane & 7) | (((lane >> 3) & 1) << 3);          // pixel of the fragment this lane addresses
     const int a_chunk = lane >> 4;
+    // fragment m of this warp: image, fragment row and fragment column within the tile; false for an idle one
+    auto frag_of = [&](int m, int &img, int &frow, int &fcol) {
+        if (a.vert) {       // consecutive rows of one column block (one image per tile)
+            img = 0; fcol = warp % a.frags_w; frow = (warp / a.frags_w) * a.mf_warp + m;
+            return m < a.mf_warp && frow * a.frags_w + fcol < a.frags_tile;
+        }
+        const int f = warp * a.mf_warp + m;
+        img = f / a.frags_img;
+        const int rem = f - img * a.frags_img;
+        frow = rem / a.frags_w; fcol = rem - frow * a.frags_w;
+        return m < a.mf_warp && f < a.frags_tile;
+    };
     int p_lane[MF];                                                // its pixel index in the halo box at tap (0, 0)
     uint32_t pre[FWU][MF];                                         // byte offset of its 16 bytes at window column y, row 0
 #pragma unroll
     for (int m = 0; m < MF; ++m) {
-        int f = warp * a.mf_warp + m;
-        if (m >= a.mf_warp || f >= a.frags_tile) f = 0;            // idle fragments read in bounds and store nothing
-        const int img = f / a.frags_img, rem = f - img * a.frags_img;
-        const int frow = rem / a.frags_w, fcol = rem - frow * a.frags_w;
+        int img, frow, fcol;
+        if (!frag_of(m, img, frow, fcol)) {                        // idle fragments read in bounds and store nothing
+            img = 0; fcol = 0;
+            if (!a.vert) frow = 0;                                 // (a vertical warp's rows stay consecutive: all inside the box)
+        }
         const int row = frow * (16 >> a.fwd_shift) + (jl >> a.fwd_shift), col = fcol * FWD + (jl & (FWD - 1));
         p_lane[m] = (img * a.Ht + row * S) * a.Wt + col * S;
 #pragma unroll
@@ -134,11 +151,9 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
     int st_off[MF][2];
 #pragma unroll
     for (int m = 0; m < MF; ++m) {
-        const int f = warp * a.mf_warp + m;
-        const bool used = m < a.mf_warp && f < a.frags_tile;
-        const int ff = used ? f : 0;
-        const int img = ff / a.frags_img, rem = ff - img * a.frags_img;
-        const int frow = rem / a.frags_w, fcol = rem - frow * a.frags_w;
+        int img, frow, fcol;
+        const bool used = frag_of(m, img, frow, fcol);
+        if (!used) { img = 0; frow = 0; fcol = 0; }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int j = (lane >> 2) + 8 * h;
@@ -234,7 +249,61 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
                     }
                 }
             };
-            if (FWT) {
+            if constexpr (VERT) {
+                // window column y: the filter fragments of its three taps, then one pass down the MF + 2 input rows
+#pragma unroll
+                for (int pr = 0; pr < PAIRS; ++pr) {
+#pragma unroll
+                    for (int y = 0; y < 3; ++y) {
+                        uint32_t bh[3][NF][4], bl[X3 ? 3 : 1][X3 ? NF : 1][4];
+#pragma unroll
+                        for (int x = 0; x < 3; ++x)
+#pragma unroll
+                            for (int n = 0; n < NF; ++n) {
+                                const uint32_t wa = ((uint32_t)((x * 3 + y) * NF * 8 + n * 8) * RB + w_lane) ^ ((uint32_t)pr << 6);
+                                ldsm4(w_hi_s + wa, bh[x][n]);
+                                if (X3) ldsm4(w_lo_s + wa, bl[X3 ? x : 0][X3 ? n : 0]);
+                            }
+#pragma unroll
+                        for (int ir = 0; ir < MF + 2; ++ir) {
+                            if (ir >= a.mf_warp + 2) break;
+                            const uint32_t addr = in_t + (uint32_t)(ir * a.Wt) * RB + pre[y][0];
+                            uint32_t ah[2][4], al[2][4];
+#pragma unroll
+                            for (int ks = 0; ks < 2; ++ks) {
+                                uint32_t av[4];
+                                ldsm4(addr ^ ((uint32_t)(4 * pr + 2 * ks) << 4), av);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    ah[ks][e] = X3 ? av[e] & 0xffffe000u : av[e];
+                                    if (X3) al[ks][e] = __float_as_uint(__uint_as_float(av[e]) - __uint_as_float(ah[ks][e]));
+                                }
+                            }
+                            // input row ir is window row x of output row ir - x
+#pragma unroll
+                            for (int ks = 0; ks < 2; ++ks) {
+                                if (X3) {
+#pragma unroll
+                                    for (int x = 0; x < 3; ++x)
+                                        if (ir - x >= 0 && ir - x < MF && ir - x < a.mf_warp)
+#pragma unroll
+                                            for (int n = 0; n < NF; ++n) mma_16x8x8(acc[ir - x < 0 ? 0 : ir - x >= MF ? 0 : ir - x][n], al[ks], &bh[x][n][2 * ks]);
+#pragma unroll
+                                    for (int x = 0; x < 3; ++x)
+                                        if (ir - x >= 0 && ir - x < MF && ir - x < a.mf_warp)
+#pragma unroll
+                                            for (int n = 0; n < NF; ++n) mma_16x8x8(acc[ir - x < 0 ? 0 : ir - x >= MF ? 0 : ir - x][n], ah[ks], &bl[X3 ? x : 0][X3 ? n : 0][2 * ks]);
+                                }
+#pragma unroll
+                                for (int x = 0; x < 3; ++x)
+                                    if (ir - x >= 0 && ir - x < MF && ir - x < a.mf_warp)
+#pragma unroll
+                                        for (int n = 0; n < NF; ++n) mma_16x8x8(acc[ir - x < 0 ? 0 : ir - x >= MF ? 0 : ir - x][n], ah[ks], &bh[x][n][2 * ks]);
+                            }
+                        }
+                    }
+                }
+            } else if (FWT) {
                 for (int dy = 0; dy < a.FH; ++dy) {
                     const uint32_t row_base = in_t + (uint32_t)(dy * a.Wt) * RB;
 #pragma unroll
@@ -312,20 +381,21 @@ conv_mma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constan
 typedef void (*MmaKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const MmaArgs);
 
 // One function per (shared-memory row width, math mode), each in its own translation unit (conv_mma_inst*.cu)
-MmaKernel pick_mma_16_tf32(int NF, int FW, int S);
-MmaKernel pick_mma_16_x3(int NF, int FW, int S);
-MmaKernel pick_mma_32_tf32(int NF, int FW, int S);
-MmaKernel pick_mma_32_x3(int NF, int FW, int S);
+MmaKernel pick_mma_16_tf32(int NF, int FW, int S, bool vert);
+MmaKernel pick_mma_16_x3(int NF, int FW, int S, bool vert);
+MmaKernel pick_mma_32_tf32(int NF, int FW, int S, bool vert);
+MmaKernel pick_mma_32_x3(int NF, int FW, int S, bool vert);
 
 template <int NF, int CW, bool X3, int FWT>
 MmaKernel pick_mma_s(int S) { return S == 1 ? conv_mma_kernel<NF, 4, CW, 1, X3, FWT> : conv_mma_kernel<NF, 4, CW, 2, X3, FWT>; }
 template <int NF, int CW, bool X3>
-MmaKernel pick_mma_fw(int FW, int S) {
+MmaKernel pick_mma_fw(int FW, int S, bool vert) {
+    if (vert && NF <= 2) return conv_mma_kernel<NF <= 2 ? NF : 2, 4, CW, 1, X3, 3, true>;
     return FW == 1 ? pick_mma_s<NF, CW, X3, 1>(S) : FW == 3 ? pick_mma_s<NF, CW, X3, 3>(S) : pick_mma_s<NF, CW, X3, 0>(S);
 }
 template <int CW, bool X3>
-MmaKernel pick_mma_nf(int NF, int FW, int S) {
-    return NF == 1 ? pick_mma_fw<1, CW, X3>(FW, S) : NF == 2 ? pick_mma_fw<2, CW, X3>(FW, S) : pick_mma_fw<4, CW, X3>(FW, S);
+MmaKernel pick_mma_nf(int NF, int FW, int S, bool vert) {
+    return NF == 1 ? pick_mma_fw<1, CW, X3>(FW, S, vert) : NF == 2 ? pick_mma_fw<2, CW, X3>(FW, S, vert) : pick_mma_fw<4, CW, X3>(FW, S, vert);
 }
 
 }  // namespace mma_conv

@@ -4,7 +4,7 @@
 namespace small {
 namespace mma_conv {
 
-MmaKernel pick_mma_32_x3(int NF, int FW, int S) { return pick_mma_nf<32, true>(NF, FW, S); }
+MmaKernel pick_mma_32_x3(int NF, int FW, int S, bool vert) { return pick_mma_nf<32, true>(NF, FW, S, vert); }
 
 }  // namespace mma_conv
 }  // namespace small
