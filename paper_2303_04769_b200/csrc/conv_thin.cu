@@ -25,6 +25,7 @@ struct ThinArgs {
     long long tiles;
     bool relu, accumulate;
     bool nchw;                               // the input is the NCHW tensor float[N][C][H][W] itself (the network's edge)
+    bool half;                               // at most 16 filters: the two halves of a warp take different items (see the kernel)
 };
 
 // Threads per block: four warps.  A block loads a tile, then computes on it, with nothing in flight meanwhile, so
@@ -37,6 +38,9 @@ __global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int SEG = (PIX - 1) * S + FW, SEG2 = (SEG + 1) / 2;
 
+    // With at most 16 filters, lanes 16-31 would hold pad filters: the half-warps then hold the same 16 filters and work
+    // on different items, `fl` being a lane's filter and `sub` its half (measured: 3 -> 16 stem at batch 256 21.9 us before).
+    const int fl = a.half ? (lane & 15) : lane, sub = a.half ? (lane >> 4) : 0, halves = a.half ? 2 : 1;
     // filters of this lane's output channels (the filter group is fixed per CTA: blockIdx.y): [kb][0][x][y][ci][ko]
     const int kg = blockIdx.y;
     float wr[C][FH][FW][KPT];
@@ -49,12 +53,12 @@ __global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs 
             for (int y = 0; y < FW; ++y)
 #pragma unroll
                 for (int c = 0; c < C; ++c)
-                    wr[c][x][y][kp] = kb < a.KB ? __ldg(a.w + ((((size_t)kb * FH + x) * FW + y) * 32 + c) * 32 + lane) : 0.0f;
+                    wr[c][x][y][kp] = kb < a.KB ? __ldg(a.w + ((((size_t)kb * FH + x) * FW + y) * 32 + c) * 32 + fl) : 0.0f;
     }
     float bv[KPT];
 #pragma unroll
     for (int kp = 0; kp < KPT; ++kp) {
-        const int k = (kg * KPT + kp) * 32 + lane;
+        const int k = (kg * KPT + kp) * 32 + fl;
         bv[kp] = (a.bias && k < a.K) ? a.bias[k] : 0.0f;
     }
     grid_dep_sync();       // filters and bias are the layer's own constants; the tensors come next
@@ -112,7 +116,7 @@ __global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs 
         }
         __syncthreads();
         const int items = imgs * th * a.groups;              // (image, output row, column group)
-        for (int it = warp; it < items; it += kThinThreads / 32) {
+        for (int it = warp * halves + sub; it < items; it += halves * (kThinThreads / 32)) {
             const int img = it / (th * a.groups), rg = it - img * th * a.groups;
             const int r = rg / a.groups, cg = rg - r * a.groups;
             float acc[PIX][KPT];
@@ -142,8 +146,8 @@ __global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs 
             for (int kp = 0; kp < KPT; ++kp) {
                 const int kb = kg * KPT + kp;
                 if (kb >= a.KB) break;
-                const bool real = kb * 32 + lane < a.K;           // pad lanes of the last filter block stay +0
-                float *dst = a.out + ((((size_t)(n0 + img) * a.KB + kb) * a.OH + oh) * a.OW + ow0) * 32 + lane;
+                const bool real = kb * 32 + fl < a.K;             // pad lanes of the last filter block stay +0
+                float *dst = a.out + ((((size_t)(n0 + img) * a.KB + kb) * a.OH + oh) * a.OW + ow0) * 32 + fl;
 #pragma unroll
                 for (int p = 0; p < PIX; ++p) {
                     if (ow0 + p < a.OW) {
@@ -151,6 +155,7 @@ __global__ void __launch_bounds__(kThinThreads) conv_thin_kernel(const ThinArgs 
                         if (a.accumulate) v += dst[p * 32];
                         if (a.relu) v = v > 0.f ? v : 0.f;
                         dst[p * 32] = real ? v : 0.0f;
+                        if (a.half) dst[p * 32 + 16] = 0.0f;      // the line's other 16 lanes
                     }
                 }
             }
@@ -210,6 +215,7 @@ int launch_conv_thin(small_ctx *ctx, const float *in, const float *w, const floa
     a.in = in; a.w = w; a.bias = bias; a.out = out;
     a.N = g.N; a.K = g.K; a.KB = g.KB; a.H = g.H; a.W = g.W; a.OH = g.OH; a.OW = g.OW; a.pt = g.pt; a.pl = g.pl;
     a.relu = relu; a.accumulate = accumulate; a.nchw = nchw_in;
+    a.half = g.K <= 16;
     const int pix = thin_pix(g);
     const int kpt = g.KB >= 2 ? 2 : 1;
     a.groups = ceil_div(g.OW, pix);
