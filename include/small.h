@@ -281,6 +281,20 @@ int small_add(small_ctx *ctx, const float *a, const float *b, float *out, int N,
 int small_fc(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out,
              int N, int J, int K, unsigned flags, void *stream);
 
+/* Abstract fused layer (Section 6, "abstract fused layer"): a global average pool - the single channel reduction of
+ * Section 3.2 item 2 over the whole H x W plane, Average in place of Max - and the full reduction (item 5) behind
+ * it, the classifier head of the paper's networks, as one kernel:
+ *   out[n,k] = bias[k] + sum_c w[k,c] * mean_{h,w} in[n,c,h,w]      (the mean rounded to float as the pooling layer stores it)
+ * in: blocked [N][C][H][W]; w_blk: small_pack_fc_weights(J = C, K); out: blocked [N][K][1][1]; flags: SMALL_RELU | one
+ * SMALL_MATH_* (FP32 FMAs on the CUDA cores in every mode: a classifier head is far below the size at which small_fc
+ * takes the tensor cores).  Where small_gap_fc_fused says 0 (a full reduction large enough for the tensor-core route)
+ * the two layers run one after the other through `scratch`, a blocked [N][C][1][1] tensor the caller provides (NULL:
+ * UNSUPPORTED for such shapes).  Errors: NOT_INIT, INVALID_ARG, SHAPE, ALIGN, OVERLAP, UNSUPPORTED. */
+int small_gap_fc(small_ctx *ctx, const float *in, const float *w_blk, const float *bias, float *out, float *scratch,
+                 int N, int C, int H, int W, int K, unsigned flags, void *stream);
+/* 1 if small_gap_fc runs this shape as one fused kernel, else 0. */
+int small_gap_fc_fused(int N, int C, int K, unsigned math);
+
 /* ---- quantised inference (Section 5.1: "quantized to integer (unsigned 8 bit)"; Section 5.3: uint8 values, int32
  * accumulation; Section 5.5) -------------------------------------------------------------------------------------
  * The same blocked layout with one byte per channel: uint8[N][ceil(C/32)][H][W][32], pad lanes 0.  A tensor's real
@@ -376,7 +390,8 @@ typedef struct small_layer {
  * full reductions whose inner widths are at most 128 under a tensor-core math mode (SMALL_FUSE_FC_CHAIN, see small_fc_chain).  The skipped
  * intermediate tensors are then not written.  Default: all three; 0 runs every layer on its own.
  * Results stay within each math mode's tolerance either way. */
-enum { SMALL_FUSE_DWPW = 1u, SMALL_FUSE_DWPW_ALWAYS = 2u, SMALL_FUSE_CONVPOOL = 4u, SMALL_FUSE_FC_CHAIN = 8u };
+enum { SMALL_FUSE_DWPW = 1u, SMALL_FUSE_DWPW_ALWAYS = 2u, SMALL_FUSE_CONVPOOL = 4u, SMALL_FUSE_FC_CHAIN = 8u,
+       SMALL_FUSE_POOLFC = 16u };   /* a global average pool and the full reduction behind it (small_gap_fc) */
 int small_set_net_fusion(small_ctx *ctx, unsigned mask);
 /* Number of kernel launches small_run_net makes for these layers at batch N under the context's fusion setting (one per
  * layer or fused pair); -1 for invalid arguments. */

@@ -29,7 +29,7 @@ EXPORTS = [
     "small_pack_conv_weights", "small_group_count", "small_group_conv_weight_elems", "small_pack_group_conv_weights",
     "small_group_conv2d", "small_dwpw_conv2d", "small_dwpw_fused", "small_conv_maxpool2d", "small_conv_maxpool_fused", "small_dw_weight_elems", "small_pack_dw_weights", "small_fc_weight_elems",
     "small_pack_fc_weights", "small_fc_uses_tensor_cores", "small_fc_chain", "small_fc_chain_fused", "small_conv2d", "small_conv2d_uses_tensor_cores", "small_dwconv2d", "small_pool2d",
-    "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_net_workspace_bytes", "small_run_net", "small_set_net_fusion", "small_net_launches",
+    "small_relu", "small_scale_shift", "small_upsample_nearest", "small_add", "small_fc", "small_gap_fc", "small_gap_fc_fused", "small_net_workspace_bytes", "small_run_net", "small_set_net_fusion", "small_net_launches",
     "small_net_host_staging_bytes", "small_run_net_host", "small_static_workspace_bytes", "small_run_net_static",
     "small_q_packed_bytes", "small_q_pack", "small_q_unpack", "small_q_conv_weight_bytes", "small_q_pack_conv_weights", "small_q_conv2d",
     "small_q_dw_weight_bytes", "small_q_pack_dw_weights", "small_q_dwconv2d", "small_q_maxpool2d", "small_q_relu",
@@ -113,6 +113,8 @@ def lib():
     L.small_scale_shift.argtypes = [P, P, P, P, P, I, I, I, I, U, P]
     L.small_upsample_nearest.argtypes = [P, P, P, I, I, I, I, I, P]
     L.small_fc.argtypes = [P, P, P, P, P, I, I, I, U, P]
+    L.small_gap_fc.argtypes = [P, P, P, P, P, P, I, I, I, I, I, U, P]
+    L.small_gap_fc_fused.argtypes = [I, I, I, U]
     L.small_net_workspace_bytes.argtypes = [ctypes.POINTER(small_layer), I, I]
     L.small_net_workspace_bytes.restype = Z
     L.small_run_net.argtypes = [P, ctypes.POINTER(small_layer), I, I, P, P, P, Z, P]
@@ -361,8 +363,17 @@ def small_fc(ctx, inp, w_blk, bias, out, N, J, K, flags=0, stream=None):
     _check(lib().small_fc(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), N, J, K, flags, _stream(stream)), "small_fc")
 
 
-FUSE_DWPW, FUSE_DWPW_ALWAYS, FUSE_CONVPOOL, FUSE_FC_CHAIN = 1, 2, 4, 8
-FUSE_DEFAULT = FUSE_DWPW | FUSE_CONVPOOL | FUSE_FC_CHAIN
+def small_gap_fc(ctx, inp, w_blk, bias, out, scratch, N, C, H, W, K, flags=0, stream=None):
+    _check(lib().small_gap_fc(ctx, _ptr(inp), _ptr(w_blk), _ptr(bias), _ptr(out), _ptr(scratch), N, C, H, W, K, flags, _stream(stream)),
+           "small_gap_fc")
+
+
+def small_gap_fc_fused(N, C, K, math):
+    return bool(lib().small_gap_fc_fused(N, C, K, math))
+
+
+FUSE_DWPW, FUSE_DWPW_ALWAYS, FUSE_CONVPOOL, FUSE_FC_CHAIN, FUSE_POOLFC = 1, 2, 4, 8, 16
+FUSE_DEFAULT = FUSE_DWPW | FUSE_CONVPOOL | FUSE_FC_CHAIN | FUSE_POOLFC
 
 
 def small_set_net_fusion(ctx, mask):

@@ -111,7 +111,7 @@ SMALL_API int small_init(int device, small_ctx **out) {
     c->overlap = 1;
     c->dependent = 0;
     c->conv_path = SMALL_CONV_PATH_AUTO;
-    c->net_fusion = SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL | SMALL_FUSE_FC_CHAIN;
+    c->net_fusion = SMALL_FUSE_DWPW | SMALL_FUSE_CONVPOOL | SMALL_FUSE_FC_CHAIN | SMALL_FUSE_POOLFC;
     c->branch_overlap = 1;
     c->side_stream = c->ev_fork = c->ev_join = nullptr;
     {
@@ -607,6 +607,37 @@ SMALL_API int small_fc(small_ctx *ctx, const float *in, const float *w, const fl
         return launch_conv_tc(ctx, in, w_hi, math == SMALL_MATH_3XTF32 ? w_lo : nullptr, bias, out, g, flags & SMALL_RELU, false, math, st);
     }
     return launch_fc(ctx, in, w, bias, out, N, J, K, flags & SMALL_RELU, st);
+}
+
+// ---- global average pool -> full reduction as one fused layer
+SMALL_API int small_gap_fc_fused(int N, int C, int K, unsigned math) {
+    if (N < 1 || C < 1 || K < 1 || !math_valid(math)) return 0;
+    if ((size_t)blocks_of(C) * 32 * sizeof(float) > 40 * 1024) return 0;
+    return small_fc_uses_tensor_cores(N, C, K, math) ? 0 : 1;       // large full reductions keep their tensor-core route
+}
+
+SMALL_API int small_gap_fc(small_ctx *ctx, const float *in, const float *w, const float *bias, float *out, float *scratch,
+                           int N, int C, int H, int W, int K, unsigned flags, void *stream) {
+    if (!ctx) return SMALL_ERR_NOT_INIT;
+    if (flags & ~(SMALL_RELU | SMALL_MATH_MASK)) return SMALL_ERR_INVALID_ARG;
+    const unsigned math = math_of(flags);
+    if (!math_valid(math)) return SMALL_ERR_INVALID_ARG;
+    if (int s = check_ptrs({in, w, out}, {bias, scratch})) return s;
+    if (N < 1 || C < 1 || K < 1 || H < 1 || W < 1 || (long long)H * W > (1ll << 24) || (long long)N * blocks_of(C) > (1ll << 30) ||
+        (long long)N * blocks_of(K) > (1ll << 30))
+        return SMALL_ERR_SHAPE;
+    const size_t in_b = sizeof(float) * packed_elems(N, C, H, W), out_b = sizeof(float) * packed_elems(N, K, 1, 1);
+    if (ranges_overlap(in, in_b, out, out_b)) return SMALL_ERR_OVERLAP;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (small_gap_fc_fused(N, C, K, math))
+        return launch_gap_fc(ctx, in, w, bias, out, N, C, H, W, K, flags & SMALL_RELU, st);
+    // the two layers one after the other, through the caller's scratch tensor [N][C][1][1]
+    if (!scratch) return SMALL_ERR_UNSUPPORTED;
+    if (!aligned16(scratch)) return SMALL_ERR_ALIGN;
+    const size_t mid_b = sizeof(float) * packed_elems(N, C, 1, 1);
+    if (ranges_overlap(scratch, mid_b, in, in_b) || ranges_overlap(scratch, mid_b, out, out_b)) return SMALL_ERR_OVERLAP;
+    if (int s = small_pool2d(ctx, in, scratch, nullptr, N, C, H, W, H, W, 1, 0, 0, 0, 0, SMALL_POOL_AVG, stream)) return s;
+    return small_fc(ctx, scratch, w, bias, out, N, C, K, flags, stream);
 }
 
 // ---- a chain of full reductions as one fused kernel

@@ -108,6 +108,9 @@ int launch_upsample_nearest(small_ctx *, const float *in, float *out, int N, int
 int launch_pool(small_ctx *, const float *in, float *out, int32_t *idx, const Geom &, int mode, cudaStream_t);
 int launch_dwconv(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &, bool relu, cudaStream_t);
 int launch_fc(small_ctx *, const float *in, const float *w, const float *bias, float *out, int N, int J, int K, bool relu, cudaStream_t);
+// global average pool over the H x W plane and the full reduction behind it as one kernel; w as launch_fc takes it
+int launch_gap_fc(small_ctx *, const float *in, const float *w, const float *bias, float *out, int N, int C, int H, int W, int K,
+                  bool relu, cudaStream_t);
 // span > 0: group convolution - filter block kb reads `span` channel blocks from that of its first group on
 // (Kg filters per group, groups S_C channels apart); span = 0: full reduction over all channel blocks
 int launch_conv_fp32(small_ctx *, const float *in, const float *w, const float *bias, float *out, const Geom &,

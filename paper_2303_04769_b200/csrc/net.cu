@@ -96,7 +96,8 @@ static bool independent(const small_layer &A, const small_layer &Bn) {
     return A.dst != SMALL_SLOT_INPUT && Bn.dst != SMALL_SLOT_INPUT;
 }
 
-// 0: layer i runs on its own; SMALL_OP_DWPW / SMALL_OP_CONVPOOL: layers i and i + 1 run as that fused layer
+// 0: layer i runs on its own; SMALL_OP_DWPW / SMALL_OP_CONVPOOL / kFusedPoolFc: layers i and i + 1 run as that fused layer
+static const int kFusedPoolFc = 1000;      // (no descriptor op of its own: only the runner forms this pair)
 static int fused_pair(const small_ctx *ctx, const small_layer *layers, int n_layers, int i, int N) {
     if (i + 1 >= n_layers) return 0;
     const small_layer &A = layers[i], &Bn = layers[i + 1];
@@ -119,6 +120,11 @@ static int fused_pair(const small_ctx *ctx, const small_layer *layers, int n_lay
         if (make_geom(g, N, A.C, A.K, A.H, A.W, A.FH, A.FW, A.stride, A.pad_t, A.pad_b, A.pad_l, A.pad_r)) return 0;
         if (Bn.H != g.OH || Bn.W != g.OW) return 0;
         return small_conv_maxpool_fused(N, A.C, A.K, A.H, A.W, A.FH, A.FW, A.stride, A.pad_t, A.pad_b, A.pad_l, A.pad_r) ? SMALL_OP_CONVPOOL : 0;
+    }
+    if (A.op == SMALL_OP_POOL && Bn.op == SMALL_OP_FC && (ctx->net_fusion & SMALL_FUSE_POOLFC)) {
+        // a global average pool (window = plane, no padding) and the full reduction over its channels
+        if (A.pool_mode != SMALL_POOL_AVG || A.FH != A.H || A.FW != A.W || (A.pad_t | A.pad_b | A.pad_l | A.pad_r) || Bn.C != A.C) return 0;
+        return small_gap_fc_fused(N, A.C, Bn.K, Bn.flags & SMALL_MATH_MASK) ? kFusedPoolFc : 0;
     }
     return 0;
 }
@@ -151,7 +157,7 @@ using namespace small;
 
 SMALL_API int small_set_net_fusion(small_ctx *ctx, unsigned mask) {
     if (!ctx) return SMALL_ERR_NOT_INIT;
-    if (mask & ~(unsigned)(SMALL_FUSE_DWPW | SMALL_FUSE_DWPW_ALWAYS | SMALL_FUSE_CONVPOOL | SMALL_FUSE_FC_CHAIN)) return SMALL_ERR_INVALID_ARG;
+    if (mask & ~(unsigned)(SMALL_FUSE_DWPW | SMALL_FUSE_DWPW_ALWAYS | SMALL_FUSE_CONVPOOL | SMALL_FUSE_FC_CHAIN | SMALL_FUSE_POOLFC)) return SMALL_ERR_INVALID_ARG;
     ctx->net_fusion = mask;
     return SMALL_OK;
 }
@@ -279,6 +285,9 @@ static int run_layers(small_ctx *ctx, const small_layer *layers, int n_layers, i
                 const unsigned fl = ((L.flags & SMALL_RELU) ? SMALL_RELU_MID : 0u) | (Nx.flags & (SMALL_RELU | SMALL_MATH_MASK));
                 s = small_dwpw_conv2d(ctx, rd(L.src), L.w_blk, L.bias, Nx.w_blk, Nx.bias, wr(Nx.dst), nullptr, N, L.C, Nx.K, L.H, L.W,
                                       L.stride, L.pad_t, L.pad_b, L.pad_l, L.pad_r, fl, stream);
+            } else if (fused == kFusedPoolFc) {
+                s = small_gap_fc(ctx, rd(L.src), Nx.w_blk, Nx.bias, wr(Nx.dst), nullptr, N, L.C, L.H, L.W, Nx.K,
+                                 Nx.flags & (SMALL_RELU | SMALL_MATH_MASK), stream);
             } else {
                 s = small_conv_maxpool2d(ctx, rd(L.src), L.w_blk, L.bias, wr(Nx.dst), nullptr, N, L.C, L.K, L.H, L.W, L.FH, L.FW, L.stride,
                                          L.pad_t, L.pad_b, L.pad_l, L.pad_r, L.flags, stream);

@@ -41,13 +41,14 @@ class Net:
     wherever the fused kernel takes the shape, False: never) and fuse_convpool only select the library's fusion setting
     for this network's runs."""
 
-    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda", fuse_dwpw=True, fuse_convpool=True, fuse_fc_chain=True):
+    def __init__(self, ctx, net, params, batch=None, math="fp32", device="cuda", fuse_dwpw=True, fuse_convpool=True, fuse_fc_chain=True, fuse_poolfc=True):
         self.ctx = ctx
         self.N = net["batch"] if batch is None else batch
         self.in_shape = tuple(net["input"])
         self.math = B.MATH[math]
         self.fusion = ((B.FUSE_DWPW_ALWAYS if fuse_dwpw == "all" else B.FUSE_DWPW if fuse_dwpw else 0)
-                       | (B.FUSE_CONVPOOL if fuse_convpool else 0) | (B.FUSE_FC_CHAIN if fuse_fc_chain else 0))
+                       | (B.FUSE_CONVPOOL if fuse_convpool else 0) | (B.FUSE_FC_CHAIN if fuse_fc_chain else 0)
+                       | (B.FUSE_POOLFC if fuse_poolfc else 0))
         self.keep = []            # device tensors the descriptors point into
         self._offsets = None
         layers_in = net["layers"]
