@@ -102,6 +102,7 @@ SMALL_API int small_init(int device, small_ctx **out) {
     c->encode_tiled = fn;
     c->static_workspace = nullptr;
     c->tc_cache = nullptr;
+    c->mma_cache = nullptr;
     c->wait_iters = 1u << 22;     // with the polls' nanosleep back-off: seconds
     if (resolve_static_workspace(c) != SMALL_OK) {      // loads the library's device code here, not inside a later call
         cudaFree(block);
@@ -140,6 +141,7 @@ SMALL_API int small_shutdown(small_ctx *ctx) {
     cudaSetDevice(ctx->device);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     free_tc_cache(ctx);
+    free_mma_cache(ctx);
     if (ctx->ev_fork) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_fork));
     if (ctx->ev_join) cudaEventDestroy(static_cast<cudaEvent_t>(ctx->ev_join));
     if (ctx->side_stream) cudaStreamDestroy(static_cast<cudaStream_t>(ctx->side_stream));

@@ -21,6 +21,7 @@ struct small_ctx {
     int dependent;           // set by small_run_net while it issues those layers
     unsigned wait_iters;     // limit (polls) of every bounded device-side wait; small_set_wait_limit
     void *tc_cache;          // finished launches of the tensor-core kernel by (shape, mode, tensors); conv_tc.cu
+    void *mma_cache;         // the same for the warp-level tensor-core kernel; conv_mma.cu
     void *static_workspace;  // device address of the library's built-in workspace array on this device (net_static.cu)
     int branch_overlap;      // small_run_net runs independent neighbouring layers side by side (side stream)
     void *side_stream, *ev_fork, *ev_join;   // cudaStream_t / cudaEvent_t of that
@@ -93,6 +94,7 @@ struct Geom {
 int make_geom(Geom &g, int N, int C, int K, int H, int W, int FH, int FW, int S, int pt, int pb, int pl, int pr);
 
 void free_tc_cache(small_ctx *);             // conv_tc.cu
+void free_mma_cache(small_ctx *);            // conv_mma.cu
 int resolve_static_workspace(small_ctx *);   // net_static.cu; called by small_init with the context's device current
 
 // ---- kernel launchers (each in its own .cu); all return a small_status ----

@@ -21,6 +21,9 @@
 // 3xTF32: x = x_hi + x_lo split in registers after the load, filters arrive split; x_lo w_hi + x_hi w_lo + x_hi w_hi.
 #include <cuda.h>
 
+#include <string>
+#include <unordered_map>
+
 #include "conv_mma.cuh"
 
 namespace small {
@@ -118,10 +121,39 @@ MmaPlan plan_mma(const Geom &g, bool x3, size_t max_smem) {
 
 bool conv_mma_supported(const Geom &g, bool x3) { return plan_mma(g, x3, 227 * 1024).ok; }
 
+// A finished launch - plan, tensor maps, arguments, kernel - is kept per context by (shape, mode, flags, tensors), so that
+// a repeated call (a network step) only launches.
+namespace {
+struct MmaLaunch { CUtensorMap map_in, map_w, map_w_lo; MmaArgs a; MmaKernel kern; unsigned grid, threads; size_t smem; };
+typedef std::unordered_map<std::string, MmaLaunch> MmaCache;
+}  // namespace
+
+void free_mma_cache(small_ctx *ctx) {
+    delete static_cast<MmaCache *>(ctx->mma_cache);
+    ctx->mma_cache = nullptr;
+}
+
 int launch_conv_mma(small_ctx *ctx, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                     const Geom &g, bool relu, bool accumulate, unsigned mode, cudaStream_t st) {
     const bool x3 = mode == SMALL_MATH_3XTF32;
     if (x3 && !w_lo) return SMALL_ERR_INVALID_ARG;
+    std::string key;
+    {
+        const int f[] = {g.N, g.C, g.K, g.H, g.W, g.FH, g.FW, g.S, g.pt, g.pb, g.pl, g.pr, x3 ? 1 : 0, relu ? 1 : 0, accumulate ? 1 : 0, (int)ctx->wait_iters};
+        const void *ptrs[] = {in, w_hi, w_lo, bias, out};
+        key.append(reinterpret_cast<const char *>(f), sizeof(f));
+        key.append(reinterpret_cast<const char *>(ptrs), sizeof(ptrs));
+    }
+    if (!ctx->mma_cache) ctx->mma_cache = new MmaCache();
+    MmaCache &cache = *static_cast<MmaCache *>(ctx->mma_cache);
+    {
+        auto it = cache.find(key);
+        if (it != cache.end()) {
+            const MmaLaunch &L = it->second;
+            launch_kernel(ctx, L.kern, dim3(L.grid), dim3(L.threads), L.smem, st, L.map_in, L.map_w, L.map_w_lo, L.a);
+            return check_launch(ctx);
+        }
+    }
     MmaPlan p = plan_mma(g, x3, ctx->max_smem_optin);
     if (!p.ok) return SMALL_ERR_UNSUPPORTED;
     MmaArgs &a = p.a;
@@ -161,6 +193,8 @@ int launch_conv_mma(small_ctx *ctx, const float *in, const float *w_hi, const fl
     long long slots = (long long)ctx->sm_count * p.per_sm / a.k_tiles;
     if (slots < 1) slots = 1;
     const unsigned grid = (unsigned)((a.n_tiles < slots ? a.n_tiles : slots) * a.k_tiles);
+    if (cache.size() >= 4096) cache.clear();
+    cache[key] = MmaLaunch{map_in, map_w, map_w_lo, a, kern, grid, (unsigned)(32 * p.warps), p.smem};
     launch_kernel(ctx, kern, dim3(grid), dim3(32 * p.warps), p.smem, st, map_in, map_w, map_w_lo, a);
     return check_launch(ctx);
 }
