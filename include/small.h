@@ -387,8 +387,9 @@ typedef struct small_layer {
  * takes the shape: a depthwise 3x3 and the 1x1 convolution behind it under a tensor-core math mode (SMALL_FUSE_DWPW: only
  * where the intermediate tensor is at most 24 MB, where fusing was measured to pay; SMALL_FUSE_DWPW_ALWAYS: wherever the
  * kernel takes the shape), a convolution and the 2x2 stride-2 max pool behind it (SMALL_FUSE_CONVPOOL), and a run of 2 to 12
- * full reductions whose inner widths are at most 128 under a tensor-core math mode (SMALL_FUSE_FC_CHAIN, see small_fc_chain).  The skipped
- * intermediate tensors are then not written.  Default: all three; 0 runs every layer on its own.
+ * full reductions whose inner widths are at most 128 under a tensor-core math mode (SMALL_FUSE_FC_CHAIN, see small_fc_chain), and
+ * a global average pool with the full reduction behind it, in every math mode (SMALL_FUSE_POOLFC, see small_gap_fc).  The skipped
+ * intermediate tensors are then not written.  Default: all four (without DWPW_ALWAYS); 0 runs every layer on its own.
  * Results stay within each math mode's tolerance either way. */
 enum { SMALL_FUSE_DWPW = 1u, SMALL_FUSE_DWPW_ALWAYS = 2u, SMALL_FUSE_CONVPOOL = 4u, SMALL_FUSE_FC_CHAIN = 8u,
        SMALL_FUSE_POOLFC = 16u };   /* a global average pool and the full reduction behind it (small_gap_fc) */
