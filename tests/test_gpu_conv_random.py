@@ -53,3 +53,53 @@ def test_random_geometry_tf32_and_3xtf32(case, path):
         err = rel_err(from_blk(out, N, K, OH, OW), ref)
         assert err <= tol, (math, err)
         assert pad_lanes_are_zero(out, N, K, OH, OW)
+
+
+def _cases_few_channels(count, seed):
+    """Shapes the warp-level tensor-core kernel takes: one channel block, filters in tiles of 32."""
+    rng = np.random.RandomState(seed)
+    out = []
+    while len(out) < count:
+        S = int(rng.choice([1, 1, 2]))
+        FH, FW = (int(v) for v in rng.choice([1, 2, 3, 3, 3, 5], size=2))
+        H, W = int(rng.randint(FH, 45)), int(rng.randint(FW, 80))
+        pad = tuple(int(rng.randint(0, min(3, f))) for f in (FH, FH, FW, FW))
+        C = int(rng.choice([1, 3, 5, 8, 9, 16, 17, 24, 31, 32]))
+        K = int(rng.choice([1, 5, 8, 12, 16, 20, 32, 33, 64, 70, 200]))
+        N = int(rng.choice([1, 2, 3, 5, 9, 40]))
+        if (H + pad[0] + pad[1] - FH) // S + 1 < 1 or (W + pad[2] + pad[3] - FW) // S + 1 < 1:
+            continue
+        if 2.0 * N * H * W * C * K * FH * FW > 6e8:       # keep the oracle quick
+            continue
+        out.append((N, C, K, H, W, FH, FW, S, pad))
+    return out
+
+
+@pytest.mark.parametrize("case", _cases_few_channels(40, 20230305))
+def test_random_geometry_warp_level_kernel(case):
+    """The same comparison with the warp-level kernel forced: its planner picks fragment shapes, bands, column tiles,
+    images per tile, filter tiles and the row-sharing form from the shape; plain and accumulating form."""
+    N, C, K, H, W, FH, FW, S, pad = case
+    x = synth.uniform((N, C, H, W), -1.0, 1.0, 71, seed=98)
+    w = synth.uniform((K, C, FH, FW), -1.0, 1.0, 72, seed=98)
+    b = synth.uniform((K,), -1.0, 1.0, 73, seed=98)
+    wb = torch.empty(B.small_conv_weight_elems(C, K, FH, FW, B.MATH_3XTF32), device="cuda")
+    B.small_pack_conv_weights(ctx(), dev(w), wb, C, K, FH, FW, B.MATH_3XTF32)
+    ref = oracle.conv2d(x, w, b, S, pad, relu=True)
+    OH, OW = ref.shape[2:]
+    prev = synth.uniform((N, K, OH, OW), -1.0, 1.0, 74, seed=98)
+    ref_acc = oracle.conv2d(x, w, None, S, pad, accumulate_into=prev)
+    bx = to_blk(x)
+    with conv_path("warp_mma"):
+        for math, tol in (("tf32", 2e-3), ("3xtf32", 1e-5)):
+            assert B.small_conv2d_path(ctx(), N, C, K, H, W, FH, FW, S, pad, B.MATH[math]) == 4
+            out = new_blk(N, K, OH, OW)
+            B.small_conv2d(ctx(), bx, wb, dev(b), out, N, C, K, H, W, FH, FW, S, pad, B.RELU | B.MATH[math])
+            assert B.small_device_status(ctx()) == 0
+            err = rel_err(from_blk(out, N, K, OH, OW), ref)
+            assert err <= tol, (math, err)
+            assert pad_lanes_are_zero(out, N, K, OH, OW)
+            acc = to_blk(prev)
+            B.small_conv2d(ctx(), bx, wb, None, acc, N, C, K, H, W, FH, FW, S, pad, B.ACCUMULATE | B.MATH[math])
+            err = rel_err(from_blk(acc, N, K, OH, OW), ref_acc)
+            assert err <= tol, (math, "accumulate", err)
