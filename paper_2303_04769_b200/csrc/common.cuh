@@ -145,7 +145,7 @@ struct DwFuse { const float *w; const float *bias; int C, H, W, s, pt, pl, relu;
 bool conv_tc_supported(const Geom &, bool x3 = false, int groups = 1, const DwFuse *dw = nullptr);
 int launch_conv_tc(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,
                    const Geom &, bool relu, bool accumulate, unsigned mode, cudaStream_t, int groups = 1, const DwFuse *dw = nullptr);
-// warp-level tensor-core kernel (conv_mma.cu): one channel block, at most 32 filters, strides 1 and 2; reads the same
+// warp-level tensor-core kernel (conv_mma.cu): one channel block, filters in tiles of 32, strides 1 and 2; reads the same
 // filter sections as launch_conv_tc
 bool conv_mma_supported(const Geom &, bool x3);
 int launch_conv_mma(small_ctx *, const float *in, const float *w_hi, const float *w_lo, const float *bias, float *out,

@@ -1,5 +1,5 @@
-// Full channel reduction for layers with few channels and few filters (at most 32 of each) on the warp-level tensor
-// core instruction (paper Section 3.2 item 4; Algorithms 1 and 2), TF32 and 3xTF32, strides 1 and 2, any window.
+// Full channel reduction for layers with few channels (one channel block, C <= 32; filters in tiles of 32) on the
+// warp-level tensor core instruction (paper Section 3.2 item 4; Algorithms 1 and 2), TF32 and 3xTF32, strides 1 and 2, any window.
 //
 // Why a second tensor-core kernel.  The block-level MMA of conv_tc.cu works on 128 rows and reads both operands from
 // shared memory: whatever its N, one 128 x N x 8 step costs the pipe 40 to 52 cycles, so a layer with 16 filters fills
